@@ -1,0 +1,565 @@
+"""CPU oracle for the layer-parallel training step (TEST INFRASTRUCTURE ONLY).
+
+A plain, slow, fp64 numpy statement of what one step of the paper's
+layer-parallel method computes: AuxNet forward chain (Eq. AV-Net-FP-lambda,
+Algorithm 1 first loop), decoupled module forward (Eq.
+Parallel-ResNet-Feature-Flow), penalty / augmented-Lagrangian local loss with
+its terminal adjoint (Eq. Parallel-ResNet-Gradient-Propagation-Equation, AL
+functional of Section 3), module back-propagation (Eq.
+Parallel-ResNet-Backpropagation), and the SGD / multiplier update (Eq.
+Parallel-ResNet-Multiplier-Update).  Every operator is its textbook definition;
+a matrix product per filter tap is the only library primitive used.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this module.  It shares no code with the CUDA path and imports nothing from it.
+All parts are pinned by tests/test_oracle_*.py (brute force, adjoint
+identities, finite differences, closed forms, the paper's own invariants).
+
+Layout: activations NHWC, convolution weights [C_out, R, S, C_in], linear
+weights [classes, C].  Penalty coefficient: the paper's beta*||.||^2 is written
+(rho/2)*||.||^2, rho = 2*beta.  The multiplier attached to the constraint
+F_k(x_k) = x_{k+1} is the paper's kappa_{k+1}.
+"""
+import numpy as np
+
+F = np.float64
+
+
+# ----------------------------------------------------------------------------
+# operators (definitions)
+# ----------------------------------------------------------------------------
+def out_size(h, r, stride, pad):
+    return (h + 2 * pad - r) // stride + 1
+
+
+def conv_fwd(x, w, stride, pad):
+    """Cross-correlation y[n,oh,ow,co] = sum_{r,s,ci} w[co,r,s,ci] x[n,oh*st+r-p,ow*st+s-p,ci]."""
+    n, h, wd, ci = x.shape
+    co, R, S, ci2 = w.shape
+    assert ci == ci2
+    oh, ow = out_size(h, R, stride, pad), out_size(wd, S, stride, pad)
+    xp = np.zeros((n, h + 2 * pad, wd + 2 * pad, ci), dtype=F)
+    xp[:, pad:pad + h, pad:pad + wd, :] = x
+    y = np.zeros((n * oh * ow, co), dtype=F)
+    for r in range(R):
+        for s in range(S):
+            xs = xp[:, r:r + stride * (oh - 1) + 1:stride, s:s + stride * (ow - 1) + 1:stride, :]
+            y += xs.reshape(-1, ci) @ w[:, r, s, :].T
+    return y.reshape(n, oh, ow, co)
+
+
+def conv_dgrad(dy, w, stride, pad, x_shape):
+    """Gradient of <conv_fwd(x,w), dy> with respect to x."""
+    n, h, wd, ci = x_shape
+    co, R, S, _ = w.shape
+    _, oh, ow, _ = dy.shape
+    dxp = np.zeros((n, h + 2 * pad, wd + 2 * pad, ci), dtype=F)
+    d2 = dy.reshape(-1, co)
+    for r in range(R):
+        for s in range(S):
+            contrib = (d2 @ w[:, r, s, :]).reshape(n, oh, ow, ci)
+            dxp[:, r:r + stride * (oh - 1) + 1:stride, s:s + stride * (ow - 1) + 1:stride, :] += contrib
+    return dxp[:, pad:pad + h, pad:pad + wd, :].copy()
+
+
+def conv_wgrad(x, dy, w_shape, stride, pad):
+    """Gradient of <conv_fwd(x,w), dy> with respect to w."""
+    n, h, wd, ci = x.shape
+    co, R, S, _ = w_shape
+    _, oh, ow, _ = dy.shape
+    xp = np.zeros((n, h + 2 * pad, wd + 2 * pad, ci), dtype=F)
+    xp[:, pad:pad + h, pad:pad + wd, :] = x
+    d2 = dy.reshape(-1, co)
+    dw = np.zeros(w_shape, dtype=F)
+    for r in range(R):
+        for s in range(S):
+            xs = xp[:, r:r + stride * (oh - 1) + 1:stride, s:s + stride * (ow - 1) + 1:stride, :]
+            dw[:, r, s, :] = d2.T @ xs.reshape(-1, ci)
+    return dw
+
+
+def bn_fwd(x, gamma, beta, eps):
+    """Training-mode batch normalisation over (N,H,W) per channel, biased variance."""
+    mean = x.mean(axis=(0, 1, 2))
+    var = ((x - mean) ** 2).mean(axis=(0, 1, 2))
+    rstd = 1.0 / np.sqrt(var + eps)
+    xhat = (x - mean) * rstd
+    return gamma * xhat + beta, (xhat, rstd)
+
+
+def bn_bwd(dy, cache, gamma):
+    xhat, rstd = cache
+    m = dy.shape[0] * dy.shape[1] * dy.shape[2]
+    dbeta = dy.sum(axis=(0, 1, 2))
+    dgamma = (dy * xhat).sum(axis=(0, 1, 2))
+    dx = (gamma * rstd) * (dy - dbeta / m - xhat * (dgamma / m))
+    return dx, dgamma, dbeta
+
+
+def relu(x):
+    return np.where(x > 0, x, 0.0)
+
+
+def relu_bwd(dy, x):
+    """ReLU'(0) = 0."""
+    return np.where(x > 0, dy, 0.0)
+
+
+def maxpool_fwd(x, k=3, stride=2, pad=1):
+    """Max over k x k windows; padding cells are -inf; first maximum in (h,w) scan order wins."""
+    n, h, w, c = x.shape
+    oh, ow = out_size(h, k, stride, pad), out_size(w, k, stride, pad)
+    xp = np.full((n, h + 2 * pad, w + 2 * pad, c), -np.inf, dtype=F)
+    xp[:, pad:pad + h, pad:pad + w, :] = x
+    best = np.full((n, oh, ow, c), -np.inf, dtype=F)
+    arg = np.zeros((n, oh, ow, c), dtype=np.int64)
+    for r in range(k):
+        for s in range(k):
+            v = xp[:, r:r + stride * (oh - 1) + 1:stride, s:s + stride * (ow - 1) + 1:stride, :]
+            better = v > best                      # strict: the first maximum is kept
+            best = np.where(better, v, best)
+            arg = np.where(better, r * k + s, arg)
+    return best, (arg, x.shape, k, stride, pad)
+
+
+def maxpool_bwd(dy, cache):
+    arg, x_shape, k, stride, pad = cache
+    n, h, w, c = x_shape
+    _, oh, ow, _ = dy.shape
+    dxp = np.zeros((n, h + 2 * pad, w + 2 * pad, c), dtype=F)
+    for r in range(k):
+        for s in range(k):
+            sel = np.where(arg == r * k + s, dy, 0.0)
+            dxp[:, r:r + stride * (oh - 1) + 1:stride, s:s + stride * (ow - 1) + 1:stride, :] += sel
+    return dxp[:, pad:pad + h, pad:pad + w, :].copy()
+
+
+def avgpool_fwd(x):
+    return x.mean(axis=(1, 2))
+
+
+def avgpool_bwd(dy, x_shape):
+    n, h, w, c = x_shape
+    return np.broadcast_to(dy[:, None, None, :] / (h * w), x_shape).astype(F)
+
+
+def linear_fwd(x, w, b):
+    return x @ w.T + b
+
+
+def softmax_ce(logits, labels):
+    """Mean over the batch of -log softmax(logits)[label]; gradient (softmax - onehot)/N."""
+    n = logits.shape[0]
+    z = logits - logits.max(axis=1, keepdims=True)
+    lse = np.log(np.exp(z).sum(axis=1, keepdims=True))
+    logp = z - lse
+    loss = -logp[np.arange(n), labels].mean()
+    g = np.exp(logp)
+    g[np.arange(n), labels] -= 1.0
+    return loss, g / n
+
+
+def local_loss(out, x_next, kappa, rho):
+    """Interior local loss (rho/2)||r||^2 + <kappa, r>, r = out - x_next, and its terminal adjoint."""
+    r = out - x_next
+    rn2 = float((r * r).sum())
+    loss = 0.5 * rho * rn2
+    seed = rho * r
+    if kappa is not None:
+        loss += float((kappa * r).sum())
+        seed = seed + kappa
+    return loss, rn2, r, seed
+
+
+# ----------------------------------------------------------------------------
+# network structure (derived from a workload dict)
+# ----------------------------------------------------------------------------
+AUX_BASE = 256
+
+
+def LP_AUX(k):
+    return AUX_BASE + k
+
+
+class Net:
+    """Static structure of one workload: blocks, module split, boundaries, parameter layouts."""
+
+    def __init__(self, cfg):
+        self.cfg = cfg
+        self.K = len(cfg["module_block_end"])
+        self.eps = float(cfg["bn_eps"])
+        self.kind = cfg["block_kind"]
+        assert self.kind in ("postbn", "preact")
+        # stem output geometry
+        h, w = cfg["H"], cfg["W"]
+        if cfg["stem_kind"] == "conv3x3":
+            self.stem = dict(R=3, stride=1, pad=1, pool=False)
+        else:
+            self.stem = dict(R=7, stride=2, pad=3, pool=True)
+            h, w = out_size(h, 7, 2, 3), out_size(w, 7, 2, 3)
+            h, w = out_size(h, 3, 2, 1), out_size(w, 3, 2, 1)
+        c = cfg["stem_channels"]
+        self.blocks = []
+        for ch, nb, st in zip(cfg["stage_channels"], cfg["stage_blocks"], cfg["stage_stride"]):
+            for b in range(nb):
+                s = st if b == 0 else 1
+                blk = dict(cin=c, cout=ch, stride=s, hin=h, win=w, proj=(s != 1 or c != ch))
+                h, w = out_size(h, 3, s, 1), out_size(w, 3, s, 1)
+                blk["hout"], blk["wout"] = h, w
+                self.blocks.append(blk)
+                c = ch
+        ends = list(cfg["module_block_end"])
+        assert ends[-1] == len(self.blocks)
+        self.module_blocks = [list(range(a, b)) for a, b in zip([0] + ends[:-1], ends)]
+        # boundary shapes: x_0 is the image batch, x_k the input of module k
+        self.boundary = [(cfg["N"], cfg["H"], cfg["W"], cfg["C_in"])]
+        for k in range(1, self.K):
+            b = self.blocks[self.module_blocks[k][0]]
+            self.boundary.append((cfg["N"], b["hin"], b["win"], b["cin"]))
+        # AuxNet_k : x_k -> x_{k+1}
+        self.aux = []
+        for k in range(self.K - 1):
+            _, hi, wi, ci = self.boundary[k]
+            _, ho, wo, co = self.boundary[k + 1]
+            total = hi // ho
+            assert total in (1, 2, 4) and hi == ho * total
+            if cfg["aux_convs"] == 1:
+                assert total in (1, 2)
+                convs = [dict(cin=ci, cout=co, stride=total)]
+            else:
+                hid = max(co // cfg["aux_width_div"], 1)
+                s1 = 2 if total >= 2 else 1
+                s2 = 2 if total == 4 else 1
+                convs = [dict(cin=ci, cout=hid, stride=s1), dict(cin=hid, cout=co, stride=s2)]
+            self.aux.append(convs)
+
+    # -- parameter layouts: list of (name, kind, shape) in blob order -----------
+    def param_layout(self, which):
+        L = []
+        if which >= AUX_BASE:
+            for i, cv in enumerate(self.aux[which - AUX_BASE]):
+                L.append(("conv%d.w" % (i + 1), "conv_w", (cv["cout"], 3, 3, cv["cin"])))
+                L.append(("bn%d.g" % (i + 1), "bn_gamma", (cv["cout"],)))
+                L.append(("bn%d.b" % (i + 1), "bn_beta", (cv["cout"],)))
+            return L
+        k = which
+        cfg = self.cfg
+        if k == 0:
+            R = self.stem["R"]
+            L.append(("stem.conv.w", "conv_w", (cfg["stem_channels"], R, R, cfg["C_in"])))
+            if self.kind == "postbn":
+                L.append(("stem.bn.g", "bn_gamma", (cfg["stem_channels"],)))
+                L.append(("stem.bn.b", "bn_beta", (cfg["stem_channels"],)))
+        for bi in self.module_blocks[k]:
+            b = self.blocks[bi]
+            p = "block%d." % bi
+            ci, co = b["cin"], b["cout"]
+            if self.kind == "postbn":
+                L += [(p + "conv1.w", "conv_w", (co, 3, 3, ci)), (p + "bn1.g", "bn_gamma", (co,)),
+                      (p + "bn1.b", "bn_beta", (co,)),
+                      (p + "conv2.w", "conv_w", (co, 3, 3, co)), (p + "bn2.g", "bn_gamma", (co,)),
+                      (p + "bn2.b", "bn_beta", (co,))]
+                if b["proj"]:
+                    L += [(p + "sc.w", "conv_w", (co, 1, 1, ci)), (p + "bns.g", "bn_gamma", (co,)),
+                          (p + "bns.b", "bn_beta", (co,))]
+            else:
+                L += [(p + "bn1.g", "bn_gamma", (ci,)), (p + "bn1.b", "bn_beta", (ci,)),
+                      (p + "conv1.w", "conv_w", (co, 3, 3, ci)),
+                      (p + "bn2.g", "bn_gamma", (co,)), (p + "bn2.b", "bn_beta", (co,)),
+                      (p + "conv2.w", "conv_w", (co, 3, 3, co))]
+                if b["proj"]:
+                    L.append((p + "sc.w", "conv_w", (co, 1, 1, ci)))
+        if k == self.K - 1:
+            c = self.blocks[-1]["cout"]
+            if self.kind == "preact":
+                L += [("head.bn.g", "bn_gamma", (c,)), ("head.bn.b", "bn_beta", (c,))]
+            L += [("head.fc.w", "fc_w", (cfg["num_classes"], c)), ("head.fc.b", "fc_b", (cfg["num_classes"],))]
+        return L
+
+    def param_count(self, which):
+        return int(sum(np.prod(s) for _, _, s in self.param_layout(which)))
+
+    def unpack(self, which, flat):
+        flat = np.asarray(flat, dtype=F)
+        out, off = {}, 0
+        for name, _, shape in self.param_layout(which):
+            n = int(np.prod(shape))
+            out[name] = flat[off:off + n].reshape(shape)
+            off += n
+        assert off == flat.size, (off, flat.size)
+        return out
+
+    def pack(self, which, named):
+        return np.concatenate([np.asarray(named[name], dtype=F).reshape(-1)
+                               for name, _, _ in self.param_layout(which)])
+
+
+# ----------------------------------------------------------------------------
+# AuxNet forward chain  (Eq. AV-Net-FP-lambda; Algorithm 1, first inner loop)
+# ----------------------------------------------------------------------------
+def auxnet_apply(net, k, p, x):
+    """x_{k+1} = AuxNet_k(x_k): conv3x3-BN[-ReLU-conv3x3-BN], batch statistics, no final ReLU."""
+    convs = net.aux[k]
+    h = conv_fwd(x, p["conv1.w"], convs[0]["stride"], 1)
+    h, _ = bn_fwd(h, p["bn1.g"], p["bn1.b"], net.eps)
+    if len(convs) == 2:
+        h = relu(h)
+        h = conv_fwd(h, p["conv2.w"], convs[1]["stride"], 1)
+        h, _ = bn_fwd(h, p["bn2.g"], p["bn2.b"], net.eps)
+    return h
+
+
+def auxnet_forward(net, aux_params, images, post=None):
+    """Serial chain x_0 = images, x_{k+1} = AuxNet_k(x_k).  ``post`` (optional) is applied to
+    each x_{k+1} before it feeds the next AuxNet (tests use it to model storage rounding)."""
+    xs, x = [], np.asarray(images, dtype=F)
+    for k in range(net.K - 1):
+        x = auxnet_apply(net, k, net.unpack(LP_AUX(k), aux_params[k]), x)
+        if post is not None:
+            x = np.asarray(post(x), dtype=F)
+        xs.append(x)
+    return xs
+
+
+# ----------------------------------------------------------------------------
+# module forward / backward
+# ----------------------------------------------------------------------------
+def _stem_fwd(net, p, x, cache):
+    st = net.stem
+    y = conv_fwd(x, p["stem.conv.w"], st["stride"], st["pad"])
+    cache["stem.x"] = x
+    if net.kind == "postbn":
+        z, cache["stem.bn"] = bn_fwd(y, p["stem.bn.g"], p["stem.bn.b"], net.eps)
+        cache["stem.z"] = z
+        y = relu(z)
+        if st["pool"]:
+            y, cache["stem.pool"] = maxpool_fwd(y)
+    return y
+
+
+def _stem_bwd(net, p, d, cache, g):
+    st = net.stem
+    if net.kind == "postbn":
+        if st["pool"]:
+            d = maxpool_bwd(d, cache["stem.pool"])
+        d = relu_bwd(d, cache["stem.z"])
+        d, g["stem.bn.g"], g["stem.bn.b"] = bn_bwd(d, cache["stem.bn"], p["stem.bn.g"])
+    g["stem.conv.w"] = conv_wgrad(cache["stem.x"], d, p["stem.conv.w"].shape, st["stride"], st["pad"])
+    return None        # the gradient with respect to the image is not used
+
+
+def _block_fwd(net, bi, p, x, cache):
+    """One residual block X + F(X, W) (Eq. ResNet-Training-Task), either block form."""
+    b = net.blocks[bi]
+    q = "block%d." % bi
+    c = cache.setdefault(bi, {})
+    c["x"] = x
+    if net.kind == "postbn":
+        y1 = conv_fwd(x, p[q + "conv1.w"], b["stride"], 1)
+        z1, c["bn1"] = bn_fwd(y1, p[q + "bn1.g"], p[q + "bn1.b"], net.eps)
+        a1 = relu(z1)
+        y2 = conv_fwd(a1, p[q + "conv2.w"], 1, 1)
+        z2, c["bn2"] = bn_fwd(y2, p[q + "bn2.g"], p[q + "bn2.b"], net.eps)
+        c["z1"], c["a1"] = z1, a1
+        if b["proj"]:
+            ys = conv_fwd(x, p[q + "sc.w"], b["stride"], 0)
+            sc, c["bns"] = bn_fwd(ys, p[q + "bns.g"], p[q + "bns.b"], net.eps)
+        else:
+            sc = x
+        return sc + z2
+    # pre-activation form
+    z0, c["bn1"] = bn_fwd(x, p[q + "bn1.g"], p[q + "bn1.b"], net.eps)
+    o = relu(z0)
+    y1 = conv_fwd(o, p[q + "conv1.w"], b["stride"], 1)
+    z1, c["bn2"] = bn_fwd(y1, p[q + "bn2.g"], p[q + "bn2.b"], net.eps)
+    a1 = relu(z1)
+    y2 = conv_fwd(a1, p[q + "conv2.w"], 1, 1)
+    c["z0"], c["o"], c["z1"], c["a1"] = z0, o, z1, a1
+    sc = conv_fwd(o, p[q + "sc.w"], b["stride"], 0) if b["proj"] else x
+    return sc + y2
+
+
+def _block_bwd(net, bi, p, d, cache, g):
+    """Adjoint step P_m = P_{m+1} dX_{m+1}/dX_m and the block's parameter gradients."""
+    b = net.blocks[bi]
+    q = "block%d." % bi
+    c = cache[bi]
+    x = c["x"]
+    if net.kind == "postbn":
+        dy2, g[q + "bn2.g"], g[q + "bn2.b"] = bn_bwd(d, c["bn2"], p[q + "bn2.g"])
+        g[q + "conv2.w"] = conv_wgrad(c["a1"], dy2, p[q + "conv2.w"].shape, 1, 1)
+        da1 = conv_dgrad(dy2, p[q + "conv2.w"], 1, 1, c["a1"].shape)
+        dz1 = relu_bwd(da1, c["z1"])
+        dy1, g[q + "bn1.g"], g[q + "bn1.b"] = bn_bwd(dz1, c["bn1"], p[q + "bn1.g"])
+        g[q + "conv1.w"] = conv_wgrad(x, dy1, p[q + "conv1.w"].shape, b["stride"], 1)
+        dx = conv_dgrad(dy1, p[q + "conv1.w"], b["stride"], 1, x.shape)
+        if b["proj"]:
+            dys, g[q + "bns.g"], g[q + "bns.b"] = bn_bwd(d, c["bns"], p[q + "bns.g"])
+            g[q + "sc.w"] = conv_wgrad(x, dys, p[q + "sc.w"].shape, b["stride"], 0)
+            dx = dx + conv_dgrad(dys, p[q + "sc.w"], b["stride"], 0, x.shape)
+        else:
+            dx = dx + d
+        return dx
+    # pre-activation form
+    g[q + "conv2.w"] = conv_wgrad(c["a1"], d, p[q + "conv2.w"].shape, 1, 1)
+    da1 = conv_dgrad(d, p[q + "conv2.w"], 1, 1, c["a1"].shape)
+    dz1 = relu_bwd(da1, c["z1"])
+    dy1, g[q + "bn2.g"], g[q + "bn2.b"] = bn_bwd(dz1, c["bn2"], p[q + "bn2.g"])
+    g[q + "conv1.w"] = conv_wgrad(c["o"], dy1, p[q + "conv1.w"].shape, b["stride"], 1)
+    do = conv_dgrad(dy1, p[q + "conv1.w"], b["stride"], 1, c["o"].shape)
+    dx_direct = 0.0
+    if b["proj"]:
+        g[q + "sc.w"] = conv_wgrad(c["o"], d, p[q + "sc.w"].shape, b["stride"], 0)
+        do = do + conv_dgrad(d, p[q + "sc.w"], b["stride"], 0, c["o"].shape)
+    else:
+        dx_direct = d
+    dz0 = relu_bwd(do, c["z0"])
+    dx, g[q + "bn1.g"], g[q + "bn1.b"] = bn_bwd(dz0, c["bn1"], p[q + "bn1.g"])
+    return dx + dx_direct
+
+
+def _head_fwd(net, p, x, cache):
+    cache["head.x"] = x
+    if net.kind == "preact":
+        z, cache["head.bn"] = bn_fwd(x, p["head.bn.g"], p["head.bn.b"], net.eps)
+        cache["head.z"] = z
+        x = relu(z)
+    pooled = avgpool_fwd(x)
+    cache["head.pooled"] = pooled
+    return linear_fwd(pooled, p["head.fc.w"], p["head.fc.b"])
+
+
+def _head_bwd(net, p, dlogits, cache, g):
+    g["head.fc.w"] = dlogits.T @ cache["head.pooled"]
+    g["head.fc.b"] = dlogits.sum(axis=0)
+    d = avgpool_bwd(dlogits @ p["head.fc.w"], cache["head.x"].shape)
+    if net.kind == "preact":
+        d = relu_bwd(d, cache["head.z"])
+        d, g["head.bn.g"], g["head.bn.b"] = bn_bwd(d, cache["head.bn"], p["head.bn.g"])
+    return d
+
+
+def module_forward(net, k, p, x_k, cache=None):
+    """F_k(x_k): stem (k = 0), the module's residual blocks, head (k = K-1: returns logits)."""
+    cache = {} if cache is None else cache
+    x = np.asarray(x_k, dtype=F)
+    if k == 0:
+        x = _stem_fwd(net, p, x, cache)
+    for bi in net.module_blocks[k]:
+        x = _block_fwd(net, bi, p, x, cache)
+    if k == net.K - 1:
+        x = _head_fwd(net, p, x, cache)
+    return x
+
+
+def module_fwd_bwd(net, k, params_flat, x_k, x_next_or_labels, kappa, rho):
+    """Forward of module k, its local loss, and the gradients of that loss with respect to the
+    module's parameters and its input x_k (x_{k+1} and kappa held constant).
+
+    Returns dict(loss, rnorm2, out, r, seed, grads (flat, blob order), dx (None for k = 0)).
+    """
+    p = net.unpack(k, params_flat)
+    cache = {}
+    out = module_forward(net, k, p, x_k, cache)
+    res = dict(out=out)
+    if k == net.K - 1:
+        loss, seed = softmax_ce(out, np.asarray(x_next_or_labels))
+        res.update(loss=loss, rnorm2=0.0, r=None, seed=seed)
+    else:
+        kap = None if kappa is None else np.asarray(kappa, dtype=F)
+        loss, rn2, r, seed = local_loss(out, np.asarray(x_next_or_labels, dtype=F), kap, rho)
+        res.update(loss=loss, rnorm2=rn2, r=r, seed=seed)
+    g = {}
+    d = seed
+    if k == net.K - 1:
+        d = _head_bwd(net, p, d, cache, g)
+    for bi in reversed(net.module_blocks[k]):
+        d = _block_bwd(net, bi, p, d, cache, g)
+    if k == 0:
+        d = _stem_bwd(net, p, d, cache, g)
+    res["grads"] = net.pack(k, g)
+    res["dx"] = d
+    return res
+
+
+# ----------------------------------------------------------------------------
+# update  (Eq. Parallel-ResNet-Backpropagation; Eq. Parallel-ResNet-Multiplier-Update)
+# ----------------------------------------------------------------------------
+def sgd_update(params_flat, grads_flat, lr, momentum=0.0, weight_decay=0.0, velocity=None):
+    """theta <- theta - lr * g   (plain SGD; optional weight decay and heavy-ball momentum)."""
+    g = np.asarray(grads_flat, dtype=F) + weight_decay * np.asarray(params_flat, dtype=F)
+    if momentum != 0.0:
+        velocity = g if velocity is None else momentum * velocity + g
+        g = velocity
+    return np.asarray(params_flat, dtype=F) - lr * g, velocity
+
+
+def kappa_update(kappa, r, kappa_step):
+    """kappa <- kappa + c * (F_k(x_k) - x_{k+1}).  The paper's step is c = eta/(2 beta) = lr/rho;
+    the method-of-multipliers step is c = rho (then the new kappa equals the terminal adjoint)."""
+    return np.asarray(kappa, dtype=F) + kappa_step * r
+
+
+# ----------------------------------------------------------------------------
+# layer-serial forward, written separately from the module code (consistency check)
+# ----------------------------------------------------------------------------
+def forward_serial(net, module_params, images):
+    """The undecomposed network X_0 = S(y), X_{l+1} = X_l + F(X_l, W_l), logits = T(X_L):
+    one pass over all blocks with the per-module parameter blobs, no module structure."""
+    named = {}
+    for k in range(net.K):
+        named.update(net.unpack(k, module_params[k]))
+    eps = net.eps
+    x = np.asarray(images, dtype=F)
+    st = net.stem
+    x = conv_fwd(x, named["stem.conv.w"], st["stride"], st["pad"])
+    if net.kind == "postbn":
+        x = relu(bn_fwd(x, named["stem.bn.g"], named["stem.bn.b"], eps)[0])
+        if st["pool"]:
+            x = maxpool_fwd(x)[0]
+    for bi, b in enumerate(net.blocks):
+        q = "block%d." % bi
+        if net.kind == "postbn":
+            t = conv_fwd(x, named[q + "conv1.w"], b["stride"], 1)
+            t = relu(bn_fwd(t, named[q + "bn1.g"], named[q + "bn1.b"], eps)[0])
+            t = conv_fwd(t, named[q + "conv2.w"], 1, 1)
+            t = bn_fwd(t, named[q + "bn2.g"], named[q + "bn2.b"], eps)[0]
+            if b["proj"]:
+                s = bn_fwd(conv_fwd(x, named[q + "sc.w"], b["stride"], 0),
+                           named[q + "bns.g"], named[q + "bns.b"], eps)[0]
+            else:
+                s = x
+            x = s + t
+        else:
+            o = relu(bn_fwd(x, named[q + "bn1.g"], named[q + "bn1.b"], eps)[0])
+            t = conv_fwd(o, named[q + "conv1.w"], b["stride"], 1)
+            t = relu(bn_fwd(t, named[q + "bn2.g"], named[q + "bn2.b"], eps)[0])
+            t = conv_fwd(t, named[q + "conv2.w"], 1, 1)
+            s = conv_fwd(o, named[q + "sc.w"], b["stride"], 0) if b["proj"] else x
+            x = s + t
+    if net.kind == "preact":
+        x = relu(bn_fwd(x, named["head.bn.g"], named["head.bn.b"], eps)[0])
+    return linear_fwd(avgpool_fwd(x), named["head.fc.w"], named["head.fc.b"])
+
+
+# ----------------------------------------------------------------------------
+# one whole layer-parallel step (Algorithm 1 without the AuxNet distillation)
+# ----------------------------------------------------------------------------
+def layer_parallel_step(net, module_params, aux_params, images, labels, kappas, rho, lr,
+                        kappa_step=None, post=None):
+    """AuxNet chain, K independent module forward+backward passes, SGD and multiplier updates.
+    ``kappas``: list of K-1 arrays or None (penalty method).  Returns the new parameters, new
+    multipliers and the per-module results."""
+    xs = [np.asarray(images, dtype=F)] + auxnet_forward(net, aux_params, images, post=post)
+    results, new_params, new_kappas = [], [], []
+    for k in range(net.K):
+        last = k == net.K - 1
+        tgt = labels if last else xs[k + 1]
+        kap = None if (kappas is None or last) else kappas[k]
+        res = module_fwd_bwd(net, k, module_params[k], xs[k], tgt, kap, rho)
+        results.append(res)
+        new_params.append(sgd_update(module_params[k], res["grads"], lr)[0])
+        if kap is not None:
+            c = rho if kappa_step is None else kappa_step
+            new_kappas.append(kappa_update(kap, res["r"], c))
+    return new_params, (new_kappas if kappas is not None else None), results, xs

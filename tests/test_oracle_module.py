@@ -1,0 +1,240 @@
+"""Pins for the oracle's module forward/backward, local losses, AuxNet chain and step.
+
+The paper prints no worked numeric example, so the pins are the facts it does fix:
+  (ii)  local back-propagation is the ordinary gradient of the local loss -> finite differences;
+  (iii) the penalty vanishes on the feasible set (psi(x, x) = 0): loss and all gradients are zero;
+  (iv)  kappa = 0 turns the augmented-Lagrangian method into the penalty method; the AL terms are
+        linear in kappa;
+  (v)   with consistent auxiliary variables the K modules reproduce the layer-serial network.
+A PyTorch-CPU autograd run on a tiny network is a secondary, library-based cross-check.
+"""
+import numpy as np
+import pytest
+
+from conftest import small_cfg
+from oracle import lp_oracle as O
+from workloads import gen, get_config
+
+
+def build(cfg, perturb=True):
+    net = O.Net(cfg)
+    mods = [gen.make_params(net.param_layout(k), cfg["seed"], "module%d" % k, perturb_bn=perturb)
+            for k in range(net.K)]
+    auxs = [gen.make_params(net.param_layout(O.LP_AUX(k)), cfg["seed"], "aux%d" % k, perturb_bn=perturb)
+            for k in range(net.K - 1)]
+    return net, mods, auxs
+
+
+ALL_CFGS = [
+    ("tiny", lambda: get_config("tiny")),
+    ("postbn-proj", lambda: small_cfg("postbn")),
+    ("preact-proj", lambda: small_cfg("preact")),
+    ("postbn-7x7", lambda: small_cfg("postbn", stem="conv7x7s2_maxpool", H=16, W=16, N=3,
+                                     stage_channels=(8, 8), stage_stride=(1, 1))),
+    ("preact-3mod", lambda: small_cfg("preact", stage_channels=(8, 16), stage_blocks=(2, 2),
+                                      module_block_end=(1, 3, 4), N=3)),
+]
+
+
+@pytest.mark.parametrize("name,mk", ALL_CFGS)
+def test_layouts_and_shapes(name, mk):
+    cfg = mk()
+    net, mods, auxs = build(cfg)
+    x = gen.make_images(cfg)
+    xs = O.auxnet_forward(net, auxs, x)
+    assert len(xs) == net.K - 1
+    for k in range(1, net.K):
+        assert xs[k - 1].shape == net.boundary[k]
+    for k in range(net.K - 1):
+        out = O.module_forward(net, k, net.unpack(k, mods[k]), x if k == 0 else xs[k - 1])
+        assert out.shape == net.boundary[k + 1]
+    for k in range(net.K):
+        assert mods[k].size == net.param_count(k)
+
+
+@pytest.mark.parametrize("name,mk", ALL_CFGS)
+def test_ii_finite_difference_gradients(name, mk):
+    cfg = mk()
+    net, mods, auxs = build(cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    xs = [x0] + O.auxnet_forward(net, auxs, x0)
+    labels = gen.make_labels(cfg)
+    rho = cfg["rho"]
+    for k in range(net.K):
+        last = k == net.K - 1
+        tgt = labels if last else xs[k + 1]
+        kap = None if last else gen.normal(5, "kap%d" % k, xs[k + 1].shape, std=0.3)
+        res = O.module_fwd_bwd(net, k, mods[k], xs[k], tgt, kap, rho)
+        p0 = mods[k].astype(np.float64)
+
+        def loss_of_params(p):
+            out = O.module_forward(net, k, net.unpack(k, p), xs[k])
+            return O.softmax_ce(out, labels)[0] if last else O.local_loss(out, tgt, kap, rho)[0]
+
+        def loss_of_x(xx):
+            out = O.module_forward(net, k, net.unpack(k, p0), xx)
+            return O.softmax_ce(out, labels)[0] if last else O.local_loss(out, tgt, kap, rho)[0]
+
+        # sample parameters from every tensor of the layout
+        off = 0
+        scale = max(1.0, abs(res["loss"]))
+        for pname, _, shape in net.param_layout(k):
+            n = int(np.prod(shape))
+            for j in sorted(set([off, off + n // 2, off + n - 1])):
+                h = 1e-5
+                pp, pm = p0.copy(), p0.copy()
+                pp[j] += h
+                pm[j] -= h
+                fd = (loss_of_params(pp) - loss_of_params(pm)) / (2 * h)
+                assert abs(fd - res["grads"][j]) < 2e-6 * scale + 1e-5 * abs(fd), (name, k, pname, j, fd, res["grads"][j])
+            off += n
+        if k > 0:
+            flat = xs[k].reshape(-1)
+            for j in [0, flat.size // 3, flat.size - 1]:
+                h = 1e-5
+                xp, xm = flat.copy(), flat.copy()
+                xp[j] += h
+                xm[j] -= h
+                fd = (loss_of_x(xp.reshape(xs[k].shape)) - loss_of_x(xm.reshape(xs[k].shape))) / (2 * h)
+                assert abs(fd - res["dx"].reshape(-1)[j]) < 2e-6 * scale + 1e-5 * abs(fd)
+        else:
+            assert res["dx"] is None
+
+
+@pytest.mark.parametrize("name,mk", ALL_CFGS)
+def test_iii_penalty_vanishes_on_feasible_set(name, mk):
+    cfg = mk()
+    net, mods, auxs = build(cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    xs = [x0] + O.auxnet_forward(net, auxs, x0)
+    for k in range(net.K - 1):
+        feasible = O.module_forward(net, k, net.unpack(k, mods[k]), xs[k])
+        res = O.module_fwd_bwd(net, k, mods[k], xs[k], feasible, None, 3.0)
+        assert res["loss"] == 0.0 and res["rnorm2"] == 0.0
+        assert np.all(res["grads"] == 0.0)
+        assert res["dx"] is None or np.all(res["dx"] == 0.0)
+
+
+@pytest.mark.parametrize("name,mk", ALL_CFGS[:3])
+def test_iv_al_reduces_to_penalty_and_is_linear_in_kappa(name, mk):
+    cfg = mk()
+    net, mods, auxs = build(cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    xs = [x0] + O.auxnet_forward(net, auxs, x0)
+    rho = 0.8
+    for k in range(net.K - 1):
+        tgt = xs[k + 1]
+        pen = O.module_fwd_bwd(net, k, mods[k], xs[k], tgt, None, rho)
+        al0 = O.module_fwd_bwd(net, k, mods[k], xs[k], tgt, np.zeros_like(tgt), rho)
+        assert al0["loss"] == pen["loss"]
+        np.testing.assert_array_equal(al0["grads"], pen["grads"])
+        np.testing.assert_array_equal(al0["seed"], pen["seed"])
+        kap = gen.normal(9, "k", tgt.shape, std=0.2)
+        al1 = O.module_fwd_bwd(net, k, mods[k], xs[k], tgt, kap, rho)
+        al2 = O.module_fwd_bwd(net, k, mods[k], xs[k], tgt, 2 * kap, rho)
+        assert abs((al1["loss"] - pen["loss"]) - float((kap * pen["r"]).sum())) < 1e-9 * max(1, abs(pen["loss"]))
+        d1 = al1["grads"] - pen["grads"]
+        d2 = al2["grads"] - pen["grads"]
+        np.testing.assert_allclose(d2, 2 * d1, rtol=1e-8, atol=1e-9 * np.abs(pen["grads"]).max())
+        # terminal adjoint: rho*r + kappa; with the multiplier step c = rho the new kappa equals it
+        np.testing.assert_allclose(al1["seed"], rho * al1["r"] + kap, rtol=1e-14)
+        np.testing.assert_allclose(O.kappa_update(kap, al1["r"], rho), al1["seed"], rtol=1e-14, atol=1e-15)
+
+
+@pytest.mark.parametrize("name,mk", ALL_CFGS)
+def test_v_consistent_chain_reproduces_layer_serial_network(name, mk):
+    cfg = mk()
+    net, mods, auxs = build(cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    x = x0
+    for k in range(net.K):
+        x = O.module_forward(net, k, net.unpack(k, mods[k]), x)      # x_{k+1} := F_k(x_k)
+    serial = O.forward_serial(net, mods, x0)
+    np.testing.assert_allclose(x, serial, rtol=1e-11, atol=1e-12)
+
+
+def test_identity_blocks_pass_features_through():
+    """Zero conv weights make F(X, W) = 0 in the pre-activation block, so X_{l+1} = X_l."""
+    cfg = small_cfg("preact", stage_channels=(8, 8), stage_stride=(1, 1), module_block_end=(1, 2))
+    net, mods, auxs = build(cfg)
+    named = net.unpack(1, mods[1])
+    named = {n: (np.zeros_like(v) if n.endswith("conv2.w") else v) for n, v in named.items()}
+    x1 = gen.normal(2, "x1", net.boundary[1])
+    c = {}
+    y = x1
+    for bi in net.module_blocks[1]:
+        y = O._block_fwd(net, bi, named, y, c)
+    np.testing.assert_array_equal(y, x1)
+
+
+def test_last_module_zero_head_gives_log_classes():
+    cfg = get_config("tiny")
+    net, mods, auxs = build(cfg)
+    named = net.unpack(1, mods[1])
+    named["head.fc.w"] = np.zeros_like(named["head.fc.w"])
+    named["head.fc.b"] = np.zeros_like(named["head.fc.b"])
+    x1 = gen.normal(2, "x1", net.boundary[1])
+    res = O.module_fwd_bwd(net, 1, net.pack(1, named), x1, gen.make_labels(cfg), None, 1.0)
+    assert abs(res["loss"] - np.log(10)) < 1e-12
+
+
+def test_step_two_updates_closed_form():
+    cfg = get_config("tiny")
+    net, mods, auxs = build(cfg)
+    x0 = gen.make_images(cfg)
+    labels = gen.make_labels(cfg)
+    kap = [gen.make_kappa(cfg, 0, net.boundary[1])]
+    newp, newk, results, xs = O.layer_parallel_step(net, mods, auxs, x0, labels, kap, 1.0, 0.1)
+    for k in range(net.K):
+        np.testing.assert_allclose(newp[k], mods[k] - 0.1 * results[k]["grads"], rtol=1e-15)
+    np.testing.assert_allclose(newk[0], results[0]["seed"], rtol=1e-13, atol=1e-15)
+    # a second step starts from the updated multiplier: the loss gains <kappa_new, r_new>
+    newp2, newk2, results2, _ = O.layer_parallel_step(net, newp, auxs, x0, labels, newk, 1.0, 0.1)
+    pen2 = O.module_fwd_bwd(net, 0, newp[0], x0, xs[1], None, 1.0)
+    assert abs(results2[0]["loss"] - pen2["loss"] - float((newk[0] * pen2["r"]).sum())) < 1e-9
+
+
+def test_torch_autograd_crosscheck():
+    """Secondary pin: PyTorch CPU autograd on a post-activation and a pre-activation module."""
+    torch = pytest.importorskip("torch")
+    import torch.nn.functional as Fn
+    for kind in ("postbn", "preact"):
+        cfg = small_cfg(kind)
+        net, mods, auxs = build(cfg)
+        k = 1
+        x = gen.normal(4, "x", net.boundary[1])
+        labels = gen.make_labels(cfg)
+        res = O.module_fwd_bwd(net, k, mods[k], x, labels, None, 1.0)
+        named = {n: torch.tensor(v, dtype=torch.float64, requires_grad=True)
+                 for n, v in net.unpack(k, mods[k]).items()}
+        xt = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+
+        def conv(t, w, stride, pad):
+            return Fn.conv2d(t.permute(0, 3, 1, 2), w.permute(0, 3, 1, 2), stride=stride, padding=pad).permute(0, 2, 3, 1)
+
+        def bn(t, g, b):
+            return Fn.batch_norm(t.permute(0, 3, 1, 2), None, None, g, b, True, 0.0, cfg["bn_eps"]).permute(0, 2, 3, 1)
+
+        h = xt
+        for bi in net.module_blocks[k]:
+            b = net.blocks[bi]
+            q = "block%d." % bi
+            if kind == "postbn":
+                t = torch.relu(bn(conv(h, named[q + "conv1.w"], b["stride"], 1), named[q + "bn1.g"], named[q + "bn1.b"]))
+                t = bn(conv(t, named[q + "conv2.w"], 1, 1), named[q + "bn2.g"], named[q + "bn2.b"])
+                s = bn(conv(h, named[q + "sc.w"], b["stride"], 0), named[q + "bns.g"], named[q + "bns.b"]) if b["proj"] else h
+            else:
+                o = torch.relu(bn(h, named[q + "bn1.g"], named[q + "bn1.b"]))
+                t = torch.relu(bn(conv(o, named[q + "conv1.w"], b["stride"], 1), named[q + "bn2.g"], named[q + "bn2.b"]))
+                t = conv(t, named[q + "conv2.w"], 1, 1)
+                s = conv(o, named[q + "sc.w"], b["stride"], 0) if b["proj"] else h
+            h = s + t
+        if kind == "preact":
+            h = torch.relu(bn(h, named["head.bn.g"], named["head.bn.b"]))
+        logits = h.mean(dim=(1, 2)) @ named["head.fc.w"].T + named["head.fc.b"]
+        loss = Fn.cross_entropy(logits, torch.tensor(labels, dtype=torch.long))
+        loss.backward()
+        assert abs(loss.item() - res["loss"]) < 1e-10
+        tg = net.pack(k, {n: v.grad.numpy() for n, v in named.items()})
+        np.testing.assert_allclose(res["grads"], tg, rtol=1e-7, atol=1e-10)
+        np.testing.assert_allclose(res["dx"], xt.grad.numpy(), rtol=1e-7, atol=1e-12)
