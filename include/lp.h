@@ -1,0 +1,192 @@
+/*
+ * lp.h - C ABI of the layer-parallel training step (single B200, sm_100a).
+ *
+ * One step of the method (paper Algorithm 1, penalty / augmented-Lagrangian form of
+ * Sections 3-4):
+ *   1. lp_auxnet_forward      x_{k+1} = AuxNet_k(x_k), k = 0..K-2          (Eq. AV-Net-FP-lambda)
+ *   2. lp_module_fwd_bwd(k)   out_k = F_k(x_k)                             (Eq. Parallel-ResNet-Feature-Flow)
+ *                             local loss + terminal adjoint                (Eq. Parallel-ResNet-Gradient-Propagation-Equation)
+ *                             parameter and input gradients                (Eq. Parallel-ResNet-Backpropagation)
+ *      lp_modules_fwd_bwd_all the same for all K modules concurrently      (Algorithm 1, "par for")
+ *   3. lp_step                theta <- theta - lr*g ; kappa <- kappa + c*r  (Eq. Parallel-ResNet-Multiplier-Update)
+ *
+ * Conventions
+ *   - Every function returns an lp_status (0 = LP_OK, negative = error).  Bad arguments are
+ *     reported on the host before anything is launched; nothing here aborts or throws.
+ *   - "device" pointers are CUDA device addresses, 16-byte aligned, owned by the caller and not
+ *     retained after the call returns unless stated.  "host" pointers are ordinary memory.
+ *   - Activations are NHWC in the descriptor's dtype (LP_F32: float, LP_BF16: bfloat16).
+ *     Convolution weights are [C_out][R][S][C_in] fp32 masters; labels are int32.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls are
+ *     asynchronous on it; lp_last_device_status synchronises and reports device-side errors.
+ *   - The library allocates no device memory for activations or parameters: the caller passes
+ *     one workspace of lp_workspace_bytes() bytes to lp_create, 256-byte aligned, and keeps it
+ *     alive until lp_destroy.
+ *   - Penalty coefficient: the paper's beta*||.||^2 is (rho/2)*||.||^2 here, rho = 2*beta.
+ *     `lambda_k` is the multiplier of the constraint F_k(x_k) = x_{k+1} (the paper's kappa_{k+1}).
+ */
+#ifndef LP_H_
+#define LP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lp_status {
+  LP_OK = 0,
+  LP_ERR_NULL = -1,           /* a required pointer is NULL */
+  LP_ERR_BAD_DESC = -2,       /* inconsistent or unsupported network descriptor */
+  LP_ERR_BAD_INDEX = -3,      /* module / AuxNet index out of range */
+  LP_ERR_ALIGN = -4,          /* a device pointer is not 16-byte aligned */
+  LP_ERR_WORKSPACE = -5,      /* workspace too small or misaligned */
+  LP_ERR_ORDER = -6,          /* call sequence violated (e.g. lp_step before any fwd_bwd) */
+  LP_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait ran out */
+  LP_ERR_CUDA = -8,           /* a CUDA runtime / driver call failed */
+  LP_ERR_SIZE = -9,           /* a size argument does not match the network */
+  LP_ERR_UNSUPPORTED = -10    /* valid request that this build does not implement */
+} lp_status;
+
+enum { LP_F32 = 0, LP_BF16 = 1 };
+enum { LP_STEM_CONV3X3 = 0, LP_STEM_CONV7X7S2_MAXPOOL = 1 };
+enum { LP_POSTBN = 0, LP_PREACT = 1 };
+/* `which` argument of the parameter calls: module k is k, AuxNet k is LP_AUX(k). */
+#define LP_AUX(k) (256 + (k))
+enum { LP_KIND_CONV_W = 0, LP_KIND_BN_GAMMA = 1, LP_KIND_BN_BETA = 2, LP_KIND_FC_W = 3, LP_KIND_FC_B = 4 };
+enum { LP_CONV_IMPL_AUTO = 0, LP_CONV_IMPL_SIMT = 1, LP_CONV_IMPL_TENSOR = 2 };
+enum { LP_CONV_FWD = 0, LP_CONV_DGRAD = 1, LP_CONV_WGRAD = 2 };
+
+#define LP_MAX_STAGES 8
+#define LP_MAX_MODULES 16
+
+/*
+ * Network and split.  A residual network: stem S, num_stages stages of residual blocks
+ * X + F(X, W) (Eq. ResNet-Training-Task), head T, cut into K modules of consecutive blocks
+ * (every n-th block, Section 4.1); the stem belongs to module 0 and the head to module K-1.
+ *   LP_POSTBN block: conv3x3-BN-ReLU-conv3x3-BN + shortcut (no ReLU after the sum)
+ *   LP_PREACT block: BN-ReLU-conv3x3-BN-ReLU-conv3x3 + shortcut
+ *   shortcut: identity, or a 1x1 convolution with the block's stride where shape changes
+ *             (followed by BN in LP_POSTBN; applied to the pre-activated tensor in LP_PREACT)
+ *   stem: LP_POSTBN conv-BN-ReLU (7x7/2 variant adds a 3x3/2 max-pool); LP_PREACT conv only
+ *   head: [BN-ReLU in LP_PREACT] global average pool, linear layer with bias, softmax CE
+ *   AuxNet_k: conv3x3(s1)-BN[-ReLU-conv3x3(s2)-BN] from x_k to the shape of x_{k+1}; hidden
+ *             width C_out/aux_width_div; strides chosen to reach the boundary's spatial size.
+ * Batch statistics everywhere (training mode), biased variance, eps = bn_eps.
+ */
+typedef struct lp_net_desc {
+  uint32_t struct_size;               /* sizeof(lp_net_desc) */
+  int32_t dtype;                      /* LP_F32 | LP_BF16 */
+  int32_t N, H, W, C_in, num_classes; /* input batch NHWC, classes */
+  int32_t stem_kind, stem_channels;
+  int32_t block_kind;
+  int32_t post_add_relu;              /* must be 0 */
+  int32_t num_stages;
+  int32_t stage_channels[LP_MAX_STAGES], stage_blocks[LP_MAX_STAGES], stage_stride[LP_MAX_STAGES];
+  int32_t K;                          /* number of modules, 1..LP_MAX_MODULES */
+  int32_t module_block_end[LP_MAX_MODULES]; /* cumulative block index ending each module */
+  int32_t aux_convs_per_boundary;     /* 1 or 2 */
+  int32_t aux_width_div;              /* >= 1 */
+  float bn_eps;
+  int32_t conv_impl;                  /* LP_CONV_IMPL_*: AUTO picks tensor cores where shapes allow */
+} lp_net_desc;
+
+typedef struct lp_param_entry {
+  char name[48];
+  int32_t kind;                       /* LP_KIND_* */
+  int32_t shape[4];                   /* unused trailing dims are 0 */
+  uint64_t offset;                    /* element offset in the flat fp32 blob */
+} lp_param_entry;
+
+typedef struct lp_handle lp_handle;
+
+const char* lp_status_string(int status);
+
+/* Host-only queries (no GPU needed). */
+size_t lp_workspace_bytes(const lp_net_desc* desc);     /* 0 on an invalid descriptor */
+int lp_validate_desc(const lp_net_desc* desc);
+/* Parameter layout of module `which` or AuxNet LP_AUX(k), in blob order.  `entries` may be NULL
+ * to query the count; at most `max_entries` are written; *n_entries receives the total. */
+int lp_param_layout(const lp_net_desc* desc, int which, lp_param_entry* entries, int max_entries,
+                    int* n_entries);
+/* Shape (NHWC) of x_k, k = 0..K-1 (x_0 is the image batch), from the descriptor alone. */
+int lp_boundary_shape_desc(const lp_net_desc* desc, int k, int shape_nhwc[4]);
+
+/* Create a handle over the caller's device workspace (zero-filled by this call on `stream`
+ * order of the default stream; parameters start at zero until lp_set_params).  The handle owns
+ * host memory, streams and events only. */
+int lp_create(const lp_net_desc* desc, void* dev_workspace, size_t bytes, lp_handle** out);
+int lp_destroy(lp_handle* h);
+
+int lp_param_count(lp_handle* h, int which, size_t* n);
+int lp_set_params(lp_handle* h, int which, const float* host, size_t n); /* synchronous */
+int lp_get_params(lp_handle* h, int which, float* host, size_t n);       /* synchronous */
+int lp_get_grads(lp_handle* h, int which, float* host, size_t n);        /* synchronous */
+int lp_boundary_shape(lp_handle* h, int k, int shape_nhwc[4]);
+
+/* Step 1.  images: device [N,H,W,C_in]; x_out: host array of K-1 device pointers, x_out[k-1]
+ * receives x_k (shape lp_boundary_shape(k)). */
+int lp_auxnet_forward(lp_handle* h, const void* images, void* const* x_out, void* stream);
+
+/* Step 2 for one module.  x_k: device input of module k (images for k = 0).
+ * x_next_or_labels: k < K-1: x_{k+1} (device, shape of boundary k+1); k == K-1: int32 labels[N].
+ * lambda_k: multiplier, same shape as x_{k+1}, or NULL for the penalty method (ignored for K-1).
+ * loss_out: device float[2] = { local loss, ||F_k(x_k) - x_{k+1}||^2 (0 for the last module) }.
+ * dx_k: device output, gradient of the local loss with respect to x_k (the paper's P^k_{kn});
+ *       may be NULL; ignored for k = 0.
+ * Parameter gradients stay in the workspace (lp_get_grads) until the next call for module k. */
+int lp_module_fwd_bwd(lp_handle* h, int k, const void* x_k, const void* x_next_or_labels,
+                      const void* lambda_k, float rho, float* loss_out, void* dx_k, void* stream);
+
+/* Step 2 for all modules at once: x[k] = x_k (K device pointers, x[0] = images), labels,
+ * lambdas[k] for k < K-1 (array or entries may be NULL), loss_out device float[K][2], dx[k]
+ * (array or entries may be NULL).  The K modules run on K internal streams forked from and
+ * joined back into `stream`. */
+int lp_modules_fwd_bwd_all(lp_handle* h, const void* const* x, const int32_t* labels,
+                           const void* const* lambdas, float rho, float* loss_out,
+                           void* const* dx, void* stream);
+
+/* Step 3.  SGD on every module whose gradients are fresh; kappa <- kappa + kappa_step * r for
+ * every interior module with a non-NULL lambdas_inout[k] (r = F_k(x_k) - x_{k+1} kept from the
+ * last fwd_bwd).  momentum = weight_decay = 0 is the paper's plain SGD. */
+int lp_step(lp_handle* h, float lr, float momentum, float weight_decay, float kappa_step,
+            void* const* lambdas_inout, void* stream);
+
+/* Layer-serial comparator (K = 1 in the paper's notation): forward through all modules with
+ * x_{k+1} := F_k(x_k); logits: device float[N][num_classes]. */
+int lp_forward_serial(lp_handle* h, const void* images, float* logits, void* stream);
+/* Layer-serial training pass with the same kernels: forward through all modules, cross-entropy,
+ * back-propagation through all modules in reverse; loss_out: device float[2]. */
+int lp_serial_fwd_bwd(lp_handle* h, const void* images, const int32_t* labels, float* loss_out,
+                      void* stream);
+
+/* Output of module k's last forward, F_k(x_k) - x_{k+1} residual and terminal adjoint, copied to
+ * host-visible device buffers for tests: dst device buffers of the boundary k+1 shape (NULL to
+ * skip).  Valid after lp_module_fwd_bwd(k) for k < K-1. */
+int lp_get_residual(lp_handle* h, int k, void* r_dst, void* seed_dst, void* stream);
+
+/* Synchronise `stream` and return LP_OK, LP_ERR_DEVICE_TIMEOUT or LP_ERR_CUDA. */
+int lp_last_device_status(lp_handle* h, void* stream);
+/* Number of kernels the library launched since the counter was last reset. */
+int64_t lp_launch_count(lp_handle* h, int reset);
+/* Time (ms, CUDA events on the launching stream) spent in tensor-core convolution kernels and
+ * their count since the last reset; only collected while profiling is enabled (serialises). */
+int lp_conv_profile(lp_handle* h, int enable, double* ms, double* flops, int64_t* launches);
+
+/* Stand-alone convolution on caller buffers (tests and kernel benchmarks).
+ * op = LP_CONV_FWD:   a = x [N,H,W,Cin],   b = w fp32 [Cout,R,R,Cin], out = y  [N,OH,OW,Cout]
+ * op = LP_CONV_DGRAD: a = dy [N,OH,OW,Cout], b = w fp32,               out = dx [N,H,W,Cin]
+ * op = LP_CONV_WGRAD: a = x,               b = dy (activation dtype),  out = dw fp32 [Cout,R,R,Cin]
+ * scratch: device buffer of lp_conv2d_scratch_bytes() (packed bf16 weights, statistics).
+ * stats (nullable, FWD only): device double[2*Cout] receives per-channel sum and sum of squares
+ * of y.  Returns LP_ERR_UNSUPPORTED if `impl` cannot run this shape. */
+size_t lp_conv2d_scratch_bytes(int Cin, int Cout, int R);
+int lp_conv2d(int op, int dtype, int impl, int N, int H, int W, int Cin, int Cout, int R,
+              int stride, int pad, const void* a, const void* b, void* out, double* stats,
+              void* scratch, size_t scratch_bytes, float* elapsed_ms, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LP_H_ */

@@ -1,0 +1,287 @@
+// Implicit-GEMM convolution on the 5th-generation tensor cores (forward and input gradient).
+//
+// GEMM view: M = output pixels (tiles of up to 128: a BW x BH x BNI box of the output grid),
+// N = output channels (tile of N_TILE <= 256), K = taps x input channels.  For every tap the
+// A operand is a 4-D TMA box of the NHWC activation tensor shifted by the tap offset (zero fill
+// outside the image supplies the padding; element strides supply the convolution stride); the B
+// operand is a 2-D TMA box of the bf16 weights [C_out][taps*C_in].  Both land in shared memory
+// in the K-major swizzled layout tcgen05.mma reads; accumulators live in tensor memory, double
+// buffered so the epilogue of one tile overlaps the MMAs of the next.
+//
+// Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = epilogue
+// (TMEM -> registers -> optional residual add -> bf16 store, per-channel sum / sum of squares
+// for the batch-norm that follows).  One persistent CTA per SM walks a contiguous tile range.
+#pragma once
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace lp {
+namespace tc {
+
+constexpr int kMaxStages = 12;
+constexpr int kTmemCols = 512;
+constexpr int kAccStride = 256;  // TMEM column offset between the two accumulator buffers
+
+struct ConvTcParams {
+  int Nimg, OHl, OWl;            // logical output grid
+  int BW, BH, BNI;               // tile box (logical pixels), BW*BH*BNI <= 128
+  int tiles_w, tiles_h, m_tiles, n_tiles, total_tiles;
+  int in_step;                   // input coordinate = logical * in_step + tap offset
+  int out_H, out_W, out_C;       // physical output tensor
+  int os, oo_h, oo_w;            // physical pixel = logical * os + oo
+  int n_tile_cols, Cout;
+  int ntaps;
+  int tap_dh[9], tap_dw[9], tap_w[9];
+  int Cin, KC, chunks;
+  int stages;
+  uint32_t stage_bytes, a_region_bytes, tx_bytes;
+  uint32_t idesc;
+  uint64_t desc_hi;
+  bf16* out;
+  const bf16* addend;            // nullable; same geometry as out
+  double* stats;                 // nullable; [2*Cout]
+  int* err;
+};
+
+struct TcSmemTail {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  int epi_ok;
+  float ssum[256];
+  float ssq[256];
+};
+
+// Sum 16 per-lane values over the 32 lanes of a warp; lane l ends with the total of column
+// ((l>>4)&1)*8 + ((l>>3)&1)*4 + ((l>>2)&1)*2 + ((l>>1)&1).
+__device__ __forceinline__ float transpose_reduce16(const float (&v)[16], int lane) {
+  float a[8], b[4], c[2];
+  const bool h4 = lane & 16, h3 = lane & 8, h2 = lane & 4, h1 = lane & 2;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float send = h4 ? v[j] : v[j + 8];
+    const float keep = h4 ? v[j + 8] : v[j];
+    a[j] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float send = h3 ? a[j] : a[j + 4];
+    const float keep = h3 ? a[j + 4] : a[j];
+    b[j] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+  }
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const float send = h2 ? b[j] : b[j + 2];
+    const float keep = h2 ? b[j + 2] : b[j];
+    c[j] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+  }
+  const float send = h1 ? c[0] : c[1];
+  const float keep = h1 ? c[1] : c[0];
+  float d = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+  d += __shfl_xor_sync(0xffffffffu, d, 1);
+  return d;
+}
+
+__global__ void __launch_bounds__(192, 1)
+conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ ConvTcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  TcSmemTail* tail = reinterpret_cast<TcSmemTail*>(smem + (size_t)p.stages * p.stage_bytes);
+  volatile int* abort_flag = &tail->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // contiguous tile range of this CTA
+  const int t_begin = (int)(((long long)p.total_tiles * blockIdx.x) / gridDim.x);
+  const int t_end = (int)(((long long)p.total_tiles * (blockIdx.x + 1)) / gridDim.x);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&tail->full[s], 1);
+      mbar_init(&tail->empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&tail->tmem_full[b], 1);
+      mbar_init(&tail->tmem_empty[b], 4);
+    }
+    tail->abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmB);
+  }
+  for (int i = threadIdx.x; i < 256; i += blockDim.x) {
+    tail->ssum[i] = 0.f;
+    tail->ssq[i] = 0.f;
+  }
+  if (warp == 2) {
+    tmem_alloc(&tail->tmem_base, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tail->tmem_base;
+  const int kiters = p.ntaps * p.chunks;
+  bool failed = false;
+
+  if (warp == 0) {
+    // ------------------------------- TMA producer -------------------------------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int t = t_begin; t < t_end && !failed; ++t) {
+        const int nt = t / p.m_tiles, m = t % p.m_tiles;
+        const int w0 = (m % p.tiles_w) * p.BW;
+        const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
+        const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
+        const int col0 = nt * p.n_tile_cols;
+        for (int tap = 0; tap < p.ntaps && !failed; ++tap) {
+          const int cw = w0 * p.in_step + p.tap_dw[tap];
+          const int ch = h0 * p.in_step + p.tap_dh[tap];
+          const int kb = p.tap_w[tap] * p.Cin;
+          for (int c = 0; c < p.chunks; ++c, ++it) {
+            const int s = it % p.stages;
+            const uint32_t ph = (it / p.stages) & 1;
+            if (!mbar_wait(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
+            uint8_t* sa = smem + (size_t)s * p.stage_bytes;
+            mbar_expect_tx(&tail->full[s], p.tx_bytes);
+            tma_load_4d(sa, &tmA, &tail->full[s], c * p.KC, cw, ch, n0);
+            tma_load_2d(sa + p.a_region_bytes, &tmB, &tail->full[s], kb + c * p.KC, col0);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer ---------------------------------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      int tl = 0;
+      for (int t = t_begin; t < t_end && !failed; ++t, ++tl) {
+        const int buf = tl & 1;
+        const uint32_t aph = (tl >> 1) & 1;
+        if (!mbar_wait(&tail->tmem_empty[buf], aph ^ 1, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * kAccStride;
+        for (int k = 0; k < kiters; ++k, ++it) {
+          const int s = it % p.stages;
+          const uint32_t ph = (it / p.stages) & 1;
+          if (!mbar_wait(&tail->full[s], ph, abort_flag)) { failed = true; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes);
+          const uint32_t b_addr = a_addr + p.a_region_bytes;
+          const uint64_t ad = smem_desc(p.desc_hi, a_addr), bd = smem_desc(p.desc_hi, b_addr);
+          const int nk = p.KC >> 4;
+          for (int j = 0; j < nk; ++j)  // +32 bytes (one K = 16 slice) per step, in 16-byte units
+            mma_bf16(d_tmem, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k | j) ? 1u : 0u);
+          mma_commit(&tail->empty[s]);
+        }
+        if (failed) break;
+        mma_commit(&tail->tmem_full[buf]);
+      }
+    }
+  } else {
+    // ------------------------------- epilogue -----------------------------------------
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    const int row = q * 32 + lane;
+    const int et = threadIdx.x - 64;  // 0..127
+    const int rows_used = p.BW * p.BH * p.BNI;
+    int tl = 0;
+    for (int t = t_begin; t < t_end && !failed; ++t, ++tl) {
+      const int buf = tl & 1;
+      const uint32_t aph = (tl >> 1) & 1;
+      const int nt = t / p.m_tiles, m = t % p.m_tiles;
+      const int w0 = (m % p.tiles_w) * p.BW;
+      const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
+      const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
+      const int col0 = nt * p.n_tile_cols;
+      const int ow = w0 + row % p.BW, oh = h0 + (row / p.BW) % p.BH, n = n0 + row / (p.BW * p.BH);
+      const bool valid = row < rows_used && ow < p.OWl && oh < p.OHl && n < p.Nimg;
+      const long long obase =
+          (((long long)n * p.out_H + (oh * p.os + p.oo_h)) * p.out_W + (ow * p.os + p.oo_w)) * p.out_C;
+      // one thread waits (bounded) and the 128 epilogue threads agree on the outcome, so that the
+      // named barriers below are reached by all of them or by none
+      if (et == 0) tail->epi_ok = mbar_wait(&tail->tmem_full[buf], aph, abort_flag) ? 1 : 0;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (!*(volatile int*)&tail->epi_ok) { failed = true; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + buf * kAccStride + ((uint32_t)(q * 32) << 16);
+      const int nchunk = p.n_tile_cols >> 4;
+      for (int cc = 0; cc < nchunk; ++cc) {
+        float v[16];
+        tmem_ld16(taddr + cc * 16, v);
+        const int col = col0 + cc * 16;
+        const bool lo_ok = valid && col < p.Cout, hi_ok = valid && col + 8 < p.Cout;
+        if (p.addend) {
+          float f[8];
+          if (lo_ok) {
+            ldv(p.addend + obase + col, f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] += f[j];
+          }
+          if (hi_ok) {
+            ldv(p.addend + obase + col + 8, f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[8 + j] += f[j];
+          }
+        }
+        if (lo_ok) stv(p.out + obase + col, *reinterpret_cast<float(*)[8]>(&v[0]));
+        if (hi_ok) stv(p.out + obase + col + 8, *reinterpret_cast<float(*)[8]>(&v[8]));
+        if (p.stats) {
+          float sq[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            if (!valid) v[j] = 0.f;
+            sq[j] = v[j] * v[j];
+          }
+          const float cs = transpose_reduce16(v, lane);
+          const float cq = transpose_reduce16(sq, lane);
+          if ((lane & 1) == 0) {
+            const int cidx = cc * 16 + ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 +
+                             ((lane >> 1) & 1);
+            atomicAdd(&tail->ssum[cidx], cs);
+            atomicAdd(&tail->ssq[cidx], cq);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tail->tmem_empty[buf]);
+      if (p.stats) {
+        // flush this tile's column sums (128 epilogue threads cooperate)
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        for (int c = et; c < p.n_tile_cols; c += 128) {
+          if (col0 + c < p.Cout) {
+            atomicAdd(&p.stats[col0 + c], (double)tail->ssum[c]);
+            atomicAdd(&p.stats[p.Cout + col0 + c], (double)tail->ssq[c]);
+          }
+          tail->ssum[c] = 0.f;
+          tail->ssq[c] = 0.f;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+      }
+    }
+  }
+
+  if (failed) {
+    *abort_flag = 1;
+    atomicExch(p.err, 1);
+    // let copies and MMAs already in flight land before shared / tensor memory is released
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && !failed) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace tc
+}  // namespace lp

@@ -1,0 +1,536 @@
+// Elementwise and reduction kernels of the step: batch-norm statistics / apply / backward, ReLU,
+// residual add, penalty / augmented-Lagrangian loss and terminal adjoint, pooling, head, updates.
+// All tensors are NHWC; every thread moves 16 bytes per access and keeps a fixed channel group,
+// so per-channel scale/shift live in registers (block size is a multiple of C / VEC).
+#pragma once
+#include "common.cuh"
+
+namespace lp {
+
+struct BnArgs {
+  const double* stats;  // [2*C]: per-channel sum, sum of squares
+  const float* gamma;
+  const float* beta;
+  double inv_count;     // 1 / (N*H*W)
+  float eps;
+};
+
+__device__ __forceinline__ void bn_mean_rstd(const BnArgs& a, int C, int c, float& mean, float& rstd) {
+  double m = a.stats[c] * a.inv_count;
+  double var = a.stats[C + c] * a.inv_count - m * m;
+  if (var < 0.0) var = 0.0;
+  mean = (float)m;
+  rstd = (float)(1.0 / sqrt(var + (double)a.eps));
+}
+
+// ---------------------------------------------------------------------------------------
+// per-channel sum / sum of squares  ->  stats[2C] (double atomics, one per block and channel)
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void bn_stats_kernel(const T* __restrict__ x, long long total_vecs, int C, double* __restrict__ stats) {
+  constexpr int V = VecT<T>::N;
+  extern __shared__ float sm[];  // [blockDim][2*V]
+  const int CV = C / V;
+  const int cg = threadIdx.x % CV;
+  float s[V], q[V];
+#pragma unroll
+  for (int j = 0; j < V; ++j) s[j] = q[j] = 0.f;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
+    float f[V];
+    ldv(x + i * V, f);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      s[j] += f[j];
+      q[j] += f[j] * f[j];
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < V; ++j) {
+    sm[threadIdx.x * 2 * V + j] = s[j];
+    sm[threadIdx.x * 2 * V + V + j] = q[j];
+  }
+  __syncthreads();
+  // thread t < 2*C sums one (channel, moment) column over the threads sharing its channel group
+  for (int t = threadIdx.x; t < 2 * C; t += blockDim.x) {
+    const int moment = t / C, c = t % C;
+    const int g = c / V, j = c % V;
+    float acc = 0.f;
+    for (int th = g; th < blockDim.x; th += CV) acc += sm[th * 2 * V + moment * V + j];
+    atomicAdd(&stats[moment * C + c], (double)acc);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// out = [relu]( bnA(x) [+ bnB(x2)] [+ addend] )
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void bn_apply_kernel(const T* __restrict__ x, BnArgs A, const T* __restrict__ x2, BnArgs B,
+                                const T* __restrict__ addend, T* __restrict__ out, long long total_vecs,
+                                int C, int relu) {
+  constexpr int V = VecT<T>::N;
+  const int CV = C / V;
+  const int c0 = (threadIdx.x % CV) * V;
+  float sa[V], ta[V], sb[V], tb[V];
+#pragma unroll
+  for (int j = 0; j < V; ++j) {
+    float mean, rstd;
+    bn_mean_rstd(A, C, c0 + j, mean, rstd);
+    sa[j] = A.gamma[c0 + j] * rstd;
+    ta[j] = A.beta[c0 + j] - mean * sa[j];
+    sb[j] = tb[j] = 0.f;
+    if (x2) {
+      bn_mean_rstd(B, C, c0 + j, mean, rstd);
+      sb[j] = B.gamma[c0 + j] * rstd;
+      tb[j] = B.beta[c0 + j] - mean * sb[j];
+    }
+  }
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
+    float f[V], y[V];
+    ldv(x + i * V, f);
+#pragma unroll
+    for (int j = 0; j < V; ++j) y[j] = f[j] * sa[j] + ta[j];
+    if (x2) {
+      ldv(x2 + i * V, f);
+#pragma unroll
+      for (int j = 0; j < V; ++j) y[j] += f[j] * sb[j] + tb[j];
+    }
+    if (addend) {
+      ldv(addend + i * V, f);
+#pragma unroll
+      for (int j = 0; j < V; ++j) y[j] += f[j];
+    }
+    if (relu) {
+#pragma unroll
+      for (int j = 0; j < V; ++j) y[j] = y[j] > 0.f ? y[j] : 0.f;
+    }
+    stv(out + i * V, y);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Interior local loss, fused into the kernel that produces the module output:
+//   out = bnA(x) [+ bnB(x2)] [+ addend];  r = out - x_next;  seed = rho*r + kappa
+// writes r and seed, accumulates sum r^2 and sum kappa*r (double atomics, one pair per block).
+// With x == nullptr the output is taken from `addend` alone (already final).
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void module_out_loss_kernel(const T* __restrict__ x, BnArgs A, const T* __restrict__ x2, BnArgs B,
+                                       const T* __restrict__ addend, const T* __restrict__ x_next,
+                                       const T* __restrict__ kappa, float rho, T* __restrict__ r_out,
+                                       T* __restrict__ seed_out, double* __restrict__ acc,
+                                       long long total_vecs, int C) {
+  constexpr int V = VecT<T>::N;
+  const int CV = C / V;
+  const int c0 = (threadIdx.x % CV) * V;
+  float sa[V], ta[V], sb[V], tb[V];
+#pragma unroll
+  for (int j = 0; j < V; ++j) {
+    sa[j] = ta[j] = sb[j] = tb[j] = 0.f;
+    float mean, rstd;
+    if (x) {
+      bn_mean_rstd(A, C, c0 + j, mean, rstd);
+      sa[j] = A.gamma[c0 + j] * rstd;
+      ta[j] = A.beta[c0 + j] - mean * sa[j];
+    }
+    if (x2) {
+      bn_mean_rstd(B, C, c0 + j, mean, rstd);
+      sb[j] = B.gamma[c0 + j] * rstd;
+      tb[j] = B.beta[c0 + j] - mean * sb[j];
+    }
+  }
+  float sum_rr = 0.f, sum_kr = 0.f;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
+    float f[V], y[V], k[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) y[j] = 0.f;
+    if (x) {
+      ldv(x + i * V, f);
+#pragma unroll
+      for (int j = 0; j < V; ++j) y[j] = f[j] * sa[j] + ta[j];
+    }
+    if (x2) {
+      ldv(x2 + i * V, f);
+#pragma unroll
+      for (int j = 0; j < V; ++j) y[j] += f[j] * sb[j] + tb[j];
+    }
+    if (addend) {
+      ldv(addend + i * V, f);
+#pragma unroll
+      for (int j = 0; j < V; ++j) y[j] += f[j];
+    }
+    ldv(x_next + i * V, f);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      y[j] -= f[j];  // r
+      sum_rr += y[j] * y[j];
+    }
+    stv(r_out + i * V, y);
+    if (kappa) {
+      ldv(kappa + i * V, k);
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        sum_kr += k[j] * y[j];
+        y[j] = rho * y[j] + k[j];
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < V; ++j) y[j] = rho * y[j];
+    }
+    stv(seed_out + i * V, y);
+  }
+  __shared__ float red[2][32];
+  sum_rr = warp_sum(sum_rr);
+  sum_kr = warp_sum(sum_kr);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  if (l == 0) {
+    red[0][w] = sum_rr;
+    red[1][w] = sum_kr;
+  }
+  __syncthreads();
+  if (w == 0) {
+    const int nw = (blockDim.x + 31) >> 5;
+    float a = l < nw ? red[0][l] : 0.f, b = l < nw ? red[1][l] : 0.f;
+    a = warp_sum(a);
+    b = warp_sum(b);
+    if (l == 0) {
+      atomicAdd(&acc[0], (double)a);
+      atomicAdd(&acc[1], (double)b);
+    }
+  }
+}
+
+__global__ void loss_finalize_kernel(const double* __restrict__ acc, float rho, float* __restrict__ loss_out) {
+  loss_out[0] = (float)(0.5 * (double)rho * acc[0] + acc[1]);
+  loss_out[1] = (float)acc[0];
+}
+
+// ---------------------------------------------------------------------------------------
+// BN backward.  dy_m = dy * [mask > 0] (mask optional: the stored post-ReLU activation).
+//   reduce: dbeta += sum dy_m ; dgamma += sum dy_m * xhat
+//   apply : dx = gamma*rstd*(dy_m - dbeta/M - xhat*dgamma/M) [+ addend]
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ x, const T* __restrict__ mask,
+                                     BnArgs A, float* __restrict__ dgamma, float* __restrict__ dbeta,
+                                     long long total_vecs, int C) {
+  constexpr int V = VecT<T>::N;
+  extern __shared__ float sm[];
+  const int CV = C / V;
+  const int c0 = (threadIdx.x % CV) * V;
+  float mean[V], rstd[V], sb[V], sg[V];
+#pragma unroll
+  for (int j = 0; j < V; ++j) {
+    bn_mean_rstd(A, C, c0 + j, mean[j], rstd[j]);
+    sb[j] = sg[j] = 0.f;
+  }
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
+    float d[V], f[V], m[V];
+    ldv(dy + i * V, d);
+    ldv(x + i * V, f);
+    if (mask) {
+      ldv(mask + i * V, m);
+#pragma unroll
+      for (int j = 0; j < V; ++j) d[j] = m[j] > 0.f ? d[j] : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      sb[j] += d[j];
+      sg[j] += d[j] * (f[j] - mean[j]) * rstd[j];
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < V; ++j) {
+    sm[threadIdx.x * 2 * V + j] = sb[j];
+    sm[threadIdx.x * 2 * V + V + j] = sg[j];
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < 2 * C; t += blockDim.x) {
+    const int which = t / C, c = t % C;
+    const int g = c / V, j = c % V;
+    float acc = 0.f;
+    for (int th = g; th < blockDim.x; th += CV) acc += sm[th * 2 * V + which * V + j];
+    atomicAdd(which ? &dgamma[c] : &dbeta[c], acc);
+  }
+}
+
+template <typename T>
+__global__ void bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ x, const T* __restrict__ mask,
+                                    BnArgs A, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
+                                    const T* __restrict__ addend, T* __restrict__ out, long long total_vecs, int C) {
+  constexpr int V = VecT<T>::N;
+  const int CV = C / V;
+  const int c0 = (threadIdx.x % CV) * V;
+  float mean[V], rstd[V], sc[V], mb[V], mg[V];
+  const float invM = (float)A.inv_count;
+#pragma unroll
+  for (int j = 0; j < V; ++j) {
+    bn_mean_rstd(A, C, c0 + j, mean[j], rstd[j]);
+    sc[j] = A.gamma[c0 + j] * rstd[j];
+    mb[j] = dbeta[c0 + j] * invM;
+    mg[j] = dgamma[c0 + j] * invM;
+  }
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
+    float d[V], f[V], m[V], o[V];
+    ldv(dy + i * V, d);
+    ldv(x + i * V, f);
+    if (mask) {
+      ldv(mask + i * V, m);
+#pragma unroll
+      for (int j = 0; j < V; ++j) d[j] = m[j] > 0.f ? d[j] : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < V; ++j) o[j] = sc[j] * (d[j] - mb[j] - (f[j] - mean[j]) * rstd[j] * mg[j]);
+    if (addend) {
+      ldv(addend + i * V, f);
+#pragma unroll
+      for (int j = 0; j < V; ++j) o[j] += f[j];
+    }
+    stv(out + i * V, o);
+  }
+}
+
+// out = a + b
+template <typename T>
+__global__ void add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, long long total_vecs) {
+  constexpr int V = VecT<T>::N;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
+    float f[V], g[V];
+    ldv(a + i * V, f);
+    ldv(b + i * V, g);
+#pragma unroll
+    for (int j = 0; j < V; ++j) f[j] += g[j];
+    stv(out + i * V, f);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// 3x3 / stride 2 / pad 1 max-pool; the first maximum in (r,s) scan order wins (stored as 0..8).
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void maxpool_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, uint8_t* __restrict__ arg, int N,
+                                   int H, int W, int C, int OH, int OW) {
+  const long long total = (long long)N * OH * OW * C;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int c = (int)(i % C);
+    long long p = i / C;
+    const int ow = (int)(p % OW);
+    p /= OW;
+    const int oh = (int)(p % OH);
+    const int n = (int)(p / OH);
+    float best = -INFINITY;
+    int ba = 0;
+    for (int r = 0; r < 3; ++r) {
+      const int ih = oh * 2 + r - 1;
+      if (ih < 0 || ih >= H) continue;
+      for (int s = 0; s < 3; ++s) {
+        const int iw = ow * 2 + s - 1;
+        if (iw < 0 || iw >= W) continue;
+        const float v = to_f(x[(((long long)n * H + ih) * W + iw) * C + c]);
+        if (v > best) {
+          best = v;
+          ba = r * 3 + s;
+        }
+      }
+    }
+    from_f(y[i], best);
+    arg[i] = (uint8_t)ba;
+  }
+}
+
+template <typename T>
+__global__ void maxpool_bwd_kernel(const T* __restrict__ dy, const uint8_t* __restrict__ arg, T* __restrict__ dx,
+                                   int N, int H, int W, int C, int OH, int OW) {
+  const long long total = (long long)N * H * W * C;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int c = (int)(i % C);
+    long long p = i / C;
+    const int iw = (int)(p % W);
+    p /= W;
+    const int ih = (int)(p % H);
+    const int n = (int)(p / H);
+    float acc = 0.f;
+    for (int r = 0; r < 3; ++r) {
+      const int t = ih + 1 - r;
+      if (t < 0 || (t & 1)) continue;
+      const int oh = t >> 1;
+      if (oh >= OH) continue;
+      for (int s = 0; s < 3; ++s) {
+        const int u = iw + 1 - s;
+        if (u < 0 || (u & 1)) continue;
+        const int ow = u >> 1;
+        if (ow >= OW) continue;
+        const long long o = (((long long)n * OH + oh) * OW + ow) * C + c;
+        if (arg[o] == r * 3 + s) acc += to_f(dy[o]);
+      }
+    }
+    from_f(dx[i], acc);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// head: global average pool, linear + softmax cross-entropy (mean over the batch), backward
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void avgpool_kernel(const T* __restrict__ x, float* __restrict__ pooled, int HW, int C) {
+  // grid: N blocks; thread c-strided
+  const int n = blockIdx.x;
+  for (int c = threadIdx.x; c < C; c += blockDim.x) {
+    float acc = 0.f;
+    const T* p = x + (long long)n * HW * C + c;
+    for (int i = 0; i < HW; ++i) acc += to_f(p[(long long)i * C]);
+    pooled[(long long)n * C + c] = acc / (float)HW;
+  }
+}
+
+// one block per sample; logits, softmax, loss (atomic mean), dlogits = (softmax - onehot)/N
+__global__ void head_fwd_kernel(const float* __restrict__ pooled, const float* __restrict__ Wt,
+                                const float* __restrict__ bias, const int32_t* __restrict__ labels,
+                                float* __restrict__ logits, float* __restrict__ dlogits, double* __restrict__ loss_acc,
+                                int N, int C, int classes) {
+  extern __shared__ float sh[];  // [classes] logits, then reduction scratch [32]
+  float* lg = sh;
+  float* red = sh + classes;
+  const int n = blockIdx.x;
+  const float* pv = pooled + (long long)n * C;
+  for (int j = threadIdx.x; j < classes; j += blockDim.x) {
+    float acc = bias[j];
+    const float* w = Wt + (long long)j * C;
+    for (int c = 0; c < C; ++c) acc += w[c] * pv[c];
+    lg[j] = acc;
+    logits[(long long)n * classes + j] = acc;
+  }
+  __syncthreads();
+  float mx = -INFINITY;
+  for (int j = threadIdx.x; j < classes; j += blockDim.x) mx = fmaxf(mx, lg[j]);
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  mx = -INFINITY;
+  for (int i = 0; i < (blockDim.x + 31) / 32; ++i) mx = fmaxf(mx, red[i]);
+  __syncthreads();
+  float se = 0.f;
+  for (int j = threadIdx.x; j < classes; j += blockDim.x) se += __expf(lg[j] - mx);
+  se = warp_sum(se);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = se;
+  __syncthreads();
+  se = 0.f;
+  for (int i = 0; i < (blockDim.x + 31) / 32; ++i) se += red[i];
+  const float lse = logf(se) + mx;
+  const int lab = labels[n];
+  for (int j = threadIdx.x; j < classes; j += blockDim.x) {
+    const float p = __expf(lg[j] - lse);
+    dlogits[(long long)n * classes + j] = (p - (j == lab ? 1.f : 0.f)) / (float)N;
+  }
+  if (threadIdx.x == 0) atomicAdd(loss_acc, (double)(lse - lg[lab]) / (double)N);
+}
+
+__global__ void ce_finalize_kernel(const double* __restrict__ acc, float* __restrict__ loss_out) {
+  loss_out[0] = (float)acc[0];
+  loss_out[1] = 0.f;
+}
+
+// dW[j][c] = sum_n dlogits[n][j]*pooled[n][c]; db[j] = sum_n dlogits[n][j]
+__global__ void head_bwd_w_kernel(const float* __restrict__ dlogits, const float* __restrict__ pooled,
+                                  float* __restrict__ dW, float* __restrict__ db, int N, int C, int classes) {
+  const long long total = (long long)classes * C;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int j = (int)(i / C), c = (int)(i % C);
+    float acc = 0.f;
+    for (int n = 0; n < N; ++n) acc += dlogits[(long long)n * classes + j] * pooled[(long long)n * C + c];
+    dW[i] = acc;
+    if (c == 0) {
+      float b = 0.f;
+      for (int n = 0; n < N; ++n) b += dlogits[(long long)n * classes + j];
+      db[j] = b;
+    }
+  }
+}
+
+// d[n,h,w,c] = (sum_j dlogits[n][j] W[j][c]) / HW, broadcast over the pixels
+template <typename T>
+__global__ void head_bwd_x_kernel(const float* __restrict__ dlogits, const float* __restrict__ Wt, T* __restrict__ d,
+                                  int HW, int C, int classes) {
+  const int n = blockIdx.x;
+  for (int c = threadIdx.x; c < C; c += blockDim.x) {
+    float acc = 0.f;
+    for (int j = 0; j < classes; ++j) acc += dlogits[(long long)n * classes + j] * Wt[(long long)j * C + c];
+    acc /= (float)HW;
+    T v;
+    from_f(v, acc);
+    T* p = d + (long long)n * HW * C + c;
+    for (int i = 0; i < HW; ++i) p[(long long)i * C] = v;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// updates
+// ---------------------------------------------------------------------------------------
+__global__ void sgd_kernel(float* __restrict__ p, const float* __restrict__ g, float* __restrict__ mom, long long n,
+                           float lr, float momentum, float wd) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    float gi = g[i] + wd * p[i];
+    if (momentum != 0.f) {
+      gi = momentum * mom[i] + gi;
+      mom[i] = gi;
+    }
+    p[i] -= lr * gi;
+  }
+}
+
+template <typename T>
+__global__ void kappa_update_kernel(T* __restrict__ kappa, const T* __restrict__ r, float c, long long total_vecs) {
+  constexpr int V = VecT<T>::N;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs;
+       i += (long long)gridDim.x * blockDim.x) {
+    float k[V], f[V];
+    ldv(kappa + i * V, k);
+    ldv(r + i * V, f);
+#pragma unroll
+    for (int j = 0; j < V; ++j) k[j] += c * f[j];
+    stv(kappa + i * V, k);
+  }
+}
+
+// bf16 operand copies of one convolution's fp32 master weights w[co][t][ci]:
+//   wf[co][t*Cin + ci]  (forward B operand, K-major)      wt[ci][t*Cout + co]  (dgrad B operand)
+struct PackEntry {
+  const float* w;
+  bf16* wf;
+  bf16* wt;  // may be null
+  int cout, taps, cin;
+  long long begin;  // first flat element index handled for this entry
+};
+
+__global__ void pack_weights_kernel(const PackEntry* __restrict__ tab, int n_entries, long long total) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    int lo = 0, hi = n_entries - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (tab[mid].begin <= i) lo = mid; else hi = mid - 1;
+    }
+    const PackEntry e = tab[lo];
+    const long long j = i - e.begin;
+    const float v = e.w[j];
+    const bf16 b = __float2bfloat16_rn(v);
+    e.wf[j] = b;
+    if (e.wt) {
+      const int ci = (int)(j % e.cin);
+      const long long q = j / e.cin;
+      const int t = (int)(q % e.taps);
+      const int co = (int)(q / e.taps);
+      e.wt[((long long)ci * e.taps + t) * e.cout + co] = b;
+    }
+  }
+}
+
+}  // namespace lp

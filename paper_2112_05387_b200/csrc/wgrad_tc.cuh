@@ -1,0 +1,292 @@
+// Weight gradient of a convolution on the tensor cores.
+//
+// dw[co][r][s][ci] = sum over output pixels of dy[pix][co] * x[pix shifted by (r,s)][ci].
+// GEMM view: M = rows (tap, ci) in tiles of 128, N = output channels (tile <= 256), K = pixels.
+// Both operands are stored pixel-major in memory (NHWC), i.e. MN-major for this product: a TMA
+// box [pixels][SC channels] lands in shared memory as rows of SC*2 bytes (swizzled), which is the
+// MN-major canonical layout with the 8-pixel group stride as SBO and the sub-box size as LBO.
+// An M tile is made of 128/SC_A sub-boxes, each with its own tap shift and channel offset, so
+// tiles stay full even when C_in is not a multiple of 128.  The pixel range is split over CTAs
+// (split-K); partial sums are added to dw with fp32 atomics (dw is zeroed by the caller).
+//
+// Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = epilogue.
+#pragma once
+#include <algorithm>
+
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace lp {
+namespace tc {
+
+constexpr int kWgMaxStages = 8;
+
+struct WgradParams {
+  int Nimg, OH, OW;
+  int BW, BH, BNI, tiles_w, tiles_h, pix_tiles;
+  int rows, rows_pad;            // pixels per K block, padded to a multiple of 16
+  int stride, pad, R;
+  int Cin, Cout, taps;
+  int sca, rpt, cin_chunks, total_chunks, m_tiles;   // A: sub-box channels, sub-boxes per tile
+  int scb, nb, n_tile, n_tiles;                      // B: sub-box channels, sub-boxes per tile
+  int splits;
+  int stages;
+  uint32_t a_sub_bytes, b_sub_bytes, a_region, stage_bytes, tx_bytes;
+  uint32_t idesc;
+  uint64_t adesc_hi, bdesc_hi;
+  uint32_t tmem_cols;
+  float* dw;
+  int* err;
+};
+
+struct WgSmemTail {
+  uint64_t full[kWgMaxStages];
+  uint64_t empty[kWgMaxStages];
+  uint64_t acc_full;
+  uint32_t tmem_base;
+  int abort_flag;
+  int epi_ok;
+};
+
+__global__ void __launch_bounds__(192, 1)
+wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmDY,
+                const __grid_constant__ WgradParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  WgSmemTail* tail = reinterpret_cast<WgSmemTail*>(smem + (size_t)p.stages * p.stage_bytes);
+  volatile int* abort_flag = &tail->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x;
+  const int m_tile = tile % p.m_tiles, n_tile = tile / p.m_tiles;
+  const int split = blockIdx.y;
+  const int pt_begin = (int)(((long long)p.pix_tiles * split) / p.splits);
+  const int pt_end = (int)(((long long)p.pix_tiles * (split + 1)) / p.splits);
+  const int n_iter = pt_end - pt_begin;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&tail->full[s], 1);
+      mbar_init(&tail->empty[s], 1);
+    }
+    mbar_init(&tail->acc_full, 1);
+    tail->abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmX);
+    prefetch_tmap(&tmDY);
+  }
+  // rows beyond the pixel box are never written by TMA: they must read as zero in the K dimension
+  if (p.rows_pad > p.rows) {
+    const int a_row_b = p.sca * 2, b_row_b = p.scb * 2;
+    for (int s = 0; s < p.stages; ++s) {
+      uint8_t* sa = smem + (size_t)s * p.stage_bytes;
+      for (int j = 0; j < p.rpt; ++j) {
+        uint8_t* base = sa + (size_t)j * p.a_sub_bytes + (size_t)p.rows * a_row_b;
+        const int nbytes = (p.rows_pad - p.rows) * a_row_b;
+        for (int i = threadIdx.x * 16; i < nbytes; i += blockDim.x * 16) *reinterpret_cast<uint4*>(base + i) = make_uint4(0, 0, 0, 0);
+      }
+      for (int j = 0; j < p.nb; ++j) {
+        uint8_t* base = sa + p.a_region + (size_t)j * p.b_sub_bytes + (size_t)p.rows * b_row_b;
+        const int nbytes = (p.rows_pad - p.rows) * b_row_b;
+        for (int i = threadIdx.x * 16; i < nbytes; i += blockDim.x * 16) *reinterpret_cast<uint4*>(base + i) = make_uint4(0, 0, 0, 0);
+      }
+    }
+    fence_proxy_async();
+  }
+  if (warp == 2) {
+    tmem_alloc(&tail->tmem_base, p.tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tail->tmem_base;
+  bool failed = false;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int it = 0; it < n_iter; ++it) {
+        const int pt = pt_begin + it;
+        const int w0 = (pt % p.tiles_w) * p.BW;
+        const int h0 = ((pt / p.tiles_w) % p.tiles_h) * p.BH;
+        const int n0 = (pt / (p.tiles_w * p.tiles_h)) * p.BNI;
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!mbar_wait(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
+        uint8_t* sa = smem + (size_t)s * p.stage_bytes;
+        mbar_expect_tx(&tail->full[s], p.tx_bytes);
+        for (int j = 0; j < p.rpt; ++j) {
+          int g = m_tile * p.rpt + j;
+          if (g >= p.total_chunks) g = p.total_chunks - 1;  // padding rows of the last tile: any finite data
+          const int tap = g / p.cin_chunks, c0 = (g % p.cin_chunks) * p.sca;
+          const int r = tap / p.R, q = tap % p.R;
+          tma_load_4d(sa + (size_t)j * p.a_sub_bytes, &tmX, &tail->full[s], c0, w0 * p.stride + q - p.pad,
+                      h0 * p.stride + r - p.pad, n0);
+        }
+        for (int j = 0; j < p.nb; ++j)
+          tma_load_4d(sa + p.a_region + (size_t)j * p.b_sub_bytes, &tmDY, &tail->full[s],
+                      n_tile * p.n_tile + j * p.scb, w0, h0, n0);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const int ksteps = p.rows_pad >> 4;
+      const uint32_t a_kstep = (uint32_t)(16 * p.sca * 2) >> 4, b_kstep = (uint32_t)(16 * p.scb * 2) >> 4;
+      for (int it = 0; it < n_iter; ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!mbar_wait(&tail->full[s], ph, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes);
+        const uint64_t ad = smem_desc(p.adesc_hi, a_addr), bd = smem_desc(p.bdesc_hi, a_addr + p.a_region);
+        for (int j = 0; j < ksteps; ++j)
+          mma_bf16(tmem_base, ad + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, (it | j) ? 1u : 0u);
+        mma_commit(&tail->empty[s]);
+      }
+      if (!failed) mma_commit(&tail->acc_full);
+    }
+  } else {
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const int et = threadIdx.x - 64;
+    if (et == 0) tail->epi_ok = (n_iter > 0 && mbar_wait(&tail->acc_full, 0, abort_flag)) ? 1 : 0;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (*(volatile int*)&tail->epi_ok) {
+      tc_fence_after();
+      const int g = m_tile * p.rpt + row / p.sca;
+      const bool valid = g < p.total_chunks;
+      const int tap = valid ? g / p.cin_chunks : 0;
+      const int ci = valid ? (g % p.cin_chunks) * p.sca + row % p.sca : 0;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+      const int co0 = n_tile * p.n_tile;
+      for (int cc = 0; cc < (p.n_tile >> 4); ++cc) {
+        float v[16];
+        tmem_ld16(taddr + cc * 16, v);
+        if (valid) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int co = co0 + cc * 16 + j;
+            if (co < p.Cout) atomicAdd(&p.dw[((long long)co * p.taps + tap) * p.Cin + ci], v[j]);
+          }
+        }
+      }
+      tc_fence_before();
+    } else if (n_iter > 0) {
+      failed = true;
+    }
+  }
+
+  if (failed) {
+    *abort_flag = 1;
+    atomicExch(p.err, 1);
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && !failed) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
+}  // namespace tc
+
+typedef CUresult (*WgEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static int wg_encode(WgEncodeFn enc, CUtensorMap* m, const void* base, int N, int H, int W, int C, int boxC, int BW,
+                     int BH, int BNI, int step) {
+  cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+  cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+  cuuint32_t box[4] = {(cuuint32_t)boxC, (cuuint32_t)((BW - 1) * step + 1), (cuuint32_t)((BH - 1) * step + 1),
+                       (cuuint32_t)BNI};
+  cuuint32_t es[4] = {1, (cuuint32_t)step, (cuuint32_t)step, 1};
+  const int row_bytes = boxC * 2;
+  const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : -8;
+}
+
+static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf16* dy, float* dw, int N, int H, int W,
+                           int Cin, int OH, int OW, int Cout, int R, int stride, int pad, int* dev_err,
+                           cudaStream_t st) {
+  tc::WgradParams p;
+  memset(&p, 0, sizeof(p));
+  p.Nimg = N; p.OH = OH; p.OW = OW;
+  // pixel box (K block): up to 128 output pixels
+  p.BW = std::min(OW, 128);
+  int bh = std::min(std::max(1, 128 / p.BW), OH);
+  const int th = (OH + bh - 1) / bh;
+  p.BH = (OH + th - 1) / th;
+  int bn = std::min(std::max(1, 128 / (p.BW * p.BH)), N);
+  const int tn = (N + bn - 1) / bn;
+  p.BNI = (N + tn - 1) / tn;
+  p.tiles_w = (OW + p.BW - 1) / p.BW;
+  p.tiles_h = (OH + p.BH - 1) / p.BH;
+  p.pix_tiles = p.tiles_w * p.tiles_h * ((N + p.BNI - 1) / p.BNI);
+  p.rows = p.BW * p.BH * p.BNI;
+  p.rows_pad = (p.rows + 15) / 16 * 16;
+  p.stride = stride; p.pad = pad; p.R = R;
+  p.Cin = Cin; p.Cout = Cout; p.taps = R * R;
+  p.sca = Cin % 64 == 0 ? 64 : (Cin % 32 == 0 ? 32 : 16);
+  p.rpt = 128 / p.sca;
+  p.cin_chunks = Cin / p.sca;
+  p.total_chunks = p.taps * p.cin_chunks;
+  p.m_tiles = (p.total_chunks + p.rpt - 1) / p.rpt;
+  int best_tile = 0;
+  for (int sc : {64, 32, 16}) {
+    if (Cout % sc) continue;
+    const int chunks = Cout / sc;
+    int nb = 1;
+    for (int d = 1; d <= chunks && d * sc <= 256; ++d)
+      if (chunks % d == 0) nb = d;
+    if (nb * sc > best_tile) { best_tile = nb * sc; p.scb = sc; p.nb = nb; }
+  }
+  if (!best_tile) return -10;
+  p.n_tile = best_tile;
+  p.n_tiles = Cout / p.n_tile;
+  const int tiles = p.m_tiles * p.n_tiles;
+  p.splits = std::max(1, std::min(p.pix_tiles, sm_count / std::max(1, tiles)));
+  p.a_sub_bytes = (uint32_t)(p.rows_pad * p.sca * 2);
+  p.b_sub_bytes = (uint32_t)(p.rows_pad * p.scb * 2);
+  p.a_sub_bytes = (p.a_sub_bytes + 1023) / 1024 * 1024;
+  p.b_sub_bytes = (p.b_sub_bytes + 1023) / 1024 * 1024;
+  p.a_region = p.a_sub_bytes * p.rpt;
+  p.stage_bytes = p.a_region + p.b_sub_bytes * p.nb;
+  p.tx_bytes = (uint32_t)(p.rows * (p.rpt * p.sca + p.nb * p.scb) * 2);
+  const size_t tail = sizeof(tc::WgSmemTail) + 1024;
+  int stages = (int)((220 * 1024 - tail) / p.stage_bytes);
+  stages = std::min(stages, tc::kWgMaxStages);
+  if (stages < 2) return -10;
+  p.stages = stages;
+  p.idesc = tc::instr_desc_bf16(128, p.n_tile, 1, 1);
+  p.adesc_hi = tc::smem_desc_hi(p.a_sub_bytes, 8 * p.sca * 2, tc::swizzle_code_for_row_bytes(p.sca * 2));
+  p.bdesc_hi = tc::smem_desc_hi(p.b_sub_bytes, 8 * p.scb * 2, tc::swizzle_code_for_row_bytes(p.scb * 2));
+  uint32_t cols = 32;
+  while ((int)cols < p.n_tile) cols *= 2;
+  p.tmem_cols = cols;
+  p.dw = dw; p.err = dev_err;
+  CUtensorMap tmX, tmDY;
+  if (wg_encode(enc, &tmX, x, N, H, W, Cin, p.sca, p.BW, p.BH, p.BNI, stride)) return -8;
+  if (wg_encode(enc, &tmDY, dy, N, OH, OW, Cout, p.scb, p.BW, p.BH, p.BNI, 1)) return -8;
+  size_t smem = std::max((size_t)stages * p.stage_bytes + tail, (size_t)120 * 1024);
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(tc::wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
+      return -8;
+    attr_set = true;
+  }
+  dim3 grid(tiles, p.splits);
+  tc::wgrad_tc_kernel<<<grid, 192, smem, st>>>(tmX, tmDY, p);
+  return cudaGetLastError() == cudaSuccess ? 0 : -8;
+}
+
+}  // namespace lp

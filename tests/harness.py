@@ -1,0 +1,118 @@
+"""Helpers shared by the GPU parity tests: run a workload through the C ABI and through the oracle."""
+import numpy as np
+
+from oracle import lp_oracle as O
+from workloads import gen
+
+
+def rel_err(a, b):
+    a = np.asarray(a, dtype=np.float64).reshape(-1)
+    b = np.asarray(b, dtype=np.float64).reshape(-1)
+    nb = np.linalg.norm(b)
+    return float(np.linalg.norm(a - b) / nb) if nb > 0 else float(np.linalg.norm(a))
+
+
+def torch_dtype(cfg):
+    import torch
+    return torch.float32 if cfg["dtype"] == "f32" else torch.bfloat16
+
+
+def to_dev(a, cfg, dev="cuda:0"):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dev).to(torch_dtype(cfg)).contiguous()
+
+
+def to_host(t):
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+def make_all_params(net, cfg, perturb=True):
+    mods = [gen.make_params(net.param_layout(k), cfg["seed"], "module%d" % k, perturb_bn=perturb, dtype=cfg["dtype"])
+            for k in range(net.K)]
+    auxs = [gen.make_params(net.param_layout(O.LP_AUX(k)), cfg["seed"], "aux%d" % k, perturb_bn=perturb,
+                            dtype=cfg["dtype"]) for k in range(net.K - 1)]
+    return mods, auxs
+
+
+def per_tensor_errors(net, which, got_flat, ref_flat):
+    out, off = {}, 0
+    for name, _, shape in net.param_layout(which):
+        n = int(np.prod(shape))
+        out[name] = rel_err(got_flat[off:off + n], ref_flat[off:off + n])
+        off += n
+    return out
+
+
+class GpuRun:
+    """One workload on the GPU: handle, parameters, device buffers."""
+
+    def __init__(self, cfg, conv_impl=0, perturb=True, kappa_std=None):
+        import torch
+        import paper_2112_05387_b200 as lp
+        self.lp, self.torch, self.cfg = lp, torch, cfg
+        self.net = O.Net(cfg)
+        self.desc = lp.desc_from_config(cfg, conv_impl)
+        self.h = lp.lp_create(self.desc)
+        self.mods, self.auxs = make_all_params(self.net, cfg, perturb)
+        for k in range(self.net.K):
+            lp.lp_set_params(self.h, k, self.mods[k])
+        for k in range(self.net.K - 1):
+            lp.lp_set_params(self.h, lp.LP_AUX(k), self.auxs[k])
+        self.images = gen.make_images(cfg)
+        self.labels = gen.make_labels(cfg)
+        self.d_images = to_dev(self.images, cfg)
+        self.d_labels = torch.from_numpy(self.labels).to("cuda:0")
+        K = self.net.K
+        self.d_x = [self.d_images] + [torch.zeros(self.net.boundary[k], dtype=torch_dtype(cfg), device="cuda:0")
+                                      for k in range(1, K)]
+        std = cfg["kappa_std"] if kappa_std is None else kappa_std
+        self.kappa = [gen.make_kappa(cfg, k, self.net.boundary[k + 1], std=std) for k in range(K - 1)]
+        self.use_kappa = cfg["loss"] == "al"
+        self.d_kappa = [to_dev(kp, cfg) for kp in self.kappa]
+        self.d_loss = torch.zeros(K, 2, dtype=torch.float32, device="cuda:0")
+        self.d_dx = [None] + [torch.zeros_like(self.d_x[k]) for k in range(1, K)]
+
+    def auxnet(self):
+        self.lp.lp_auxnet_forward(self.h, self.d_images, self.d_x[1:])
+        assert self.lp.lp_last_device_status(self.h) == 0
+        return [to_host(t) for t in self.d_x[1:]]
+
+    def set_boundaries(self, xs_host):
+        """Load x_1..x_{K-1} from host arrays (oracle AuxNet outputs rounded to the storage type)."""
+        for k in range(1, self.net.K):
+            self.d_x[k].copy_(to_dev(xs_host[k - 1], self.cfg))
+
+    def fwd_bwd_all(self, grouped=True):
+        lp, h = self.lp, self.h
+        lam = self.d_kappa if self.use_kappa else None
+        if grouped:
+            lp.lp_modules_fwd_bwd_all(h, self.d_x, self.d_labels, lam, self.cfg["rho"], self.d_loss, self.d_dx)
+        else:
+            for k in range(self.net.K):
+                last = k == self.net.K - 1
+                lp.lp_module_fwd_bwd(h, k, self.d_x[k], self.d_labels if last else self.d_x[k + 1],
+                                     None if (last or lam is None) else lam[k], self.cfg["rho"], self.d_loss[k],
+                                     self.d_dx[k])
+        st = lp.lp_last_device_status(h)
+        assert st == 0, lp.lp_status_string(st)
+        return [lp.lp_get_grads(h, k) for k in range(self.net.K)]
+
+    def step(self, kappa_step=None):
+        lam = self.d_kappa if self.use_kappa else None
+        c = self.cfg["rho"] if kappa_step is None else kappa_step
+        self.lp.lp_step(self.h, self.cfg["lr"], 0.0, 0.0, c, lam)
+        assert self.lp.lp_last_device_status(self.h) == 0
+
+
+def oracle_modules(run, xs_host, kappas=None, params=None):
+    """Oracle module_fwd_bwd for every module on the given boundary tensors (x_0 = images)."""
+    net, cfg = run.net, run.cfg
+    xs = [run.images.astype(np.float64)] + [np.asarray(x, dtype=np.float64) for x in xs_host]
+    params = run.mods if params is None else params
+    kappas = (run.kappa if run.use_kappa else None) if kappas is None else kappas
+    out = []
+    for k in range(net.K):
+        last = k == net.K - 1
+        out.append(O.module_fwd_bwd(net, k, params[k], xs[k], run.labels if last else xs[k + 1],
+                                    None if (last or kappas is None) else kappas[k], cfg["rho"]))
+    return out

@@ -1,0 +1,187 @@
+"""GPU parity of the whole layer-parallel step against the oracle, through the C ABI.
+
+Tolerances (relative L2 error per tensor): 1e-4 on the fp32 path, 2e-2 on the bf16 path, for
+losses, parameter gradients, input gradients, AuxNet outputs and updated parameters.
+"""
+import numpy as np
+import pytest
+
+from conftest import small_cfg
+from harness import GpuRun, oracle_modules, per_tensor_errors, rel_err, to_host
+from oracle import lp_oracle as O
+from workloads import gen, get_config, scaled
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+
+
+def check_modules(run, grads, ref, tol, dx_from=1):
+    net = run.net
+    loss = run.d_loss.cpu().numpy()
+    worst = 0.0
+    for k in range(net.K):
+        errs = per_tensor_errors(net, k, grads[k], ref[k]["grads"])
+        bad = {n: e for n, e in errs.items() if not e < tol}
+        assert not bad, (k, bad)
+        worst = max(worst, max(errs.values()))
+        lerr = abs(loss[k, 0] - ref[k]["loss"]) / max(abs(ref[k]["loss"]), 1e-30)
+        assert lerr < tol, (k, loss[k, 0], ref[k]["loss"])
+        if k < net.K - 1:
+            assert abs(loss[k, 1] - ref[k]["rnorm2"]) / ref[k]["rnorm2"] < tol
+        if k >= dx_from:
+            e = rel_err(to_host(run.d_dx[k]), ref[k]["dx"])
+            assert e < tol, (k, "dx", e)
+    return worst
+
+
+def full_step_parity(cfg, conv_impl=0, grouped=True, steps=1):
+    run = GpuRun(cfg, conv_impl=conv_impl)
+    net, tol = run.net, TOL[cfg["dtype"]]
+    # AuxNet chain: GPU against oracle (the oracle feeds each AuxNet the storage-rounded tensor)
+    post = (lambda a: gen.storage_round(a, cfg["dtype"]))
+    ox = O.auxnet_forward(net, run.auxs, run.images, post=post)
+    gx = run.auxnet()
+    for k in range(net.K - 1):
+        assert rel_err(gx[k], ox[k]) < tol, ("auxnet", k, rel_err(gx[k], ox[k]))
+    # module inputs come from the oracle, never from the CUDA path
+    run.set_boundaries(ox)
+    xs_host = [to_host(t) for t in run.d_x[1:]]
+    params = [m.astype(np.float64) for m in run.mods]
+    kappas = [k.astype(np.float64) for k in run.kappa] if run.use_kappa else None
+    lr = None
+    for step in range(steps):
+        grads = run.fwd_bwd_all(grouped=grouped)
+        ref = oracle_modules(run, xs_host, kappas=kappas, params=params)
+        check_modules(run, grads, ref, tol)
+        for k in range(net.K - 1):
+            r = run.torch.zeros_like(run.d_x[k + 1])
+            s = run.torch.zeros_like(run.d_x[k + 1])
+            run.lp.lp_get_residual(run.h, k, r, s)
+            assert rel_err(to_host(r), ref[k]["r"]) < tol
+            assert rel_err(to_host(s), ref[k]["seed"]) < tol
+        if lr is None:
+            # the penalty is a plain sum over the boundary tensor, so gradients are large: pick the
+            # learning rate (from the oracle's gradients) that moves the parameters by about 0.02
+            lr = 0.02 / max(float(np.abs(ref[k]["grads"]).max()) for k in range(net.K))
+        run.cfg["lr"] = lr
+        before = [run.lp.lp_get_params(run.h, k).astype(np.float64) for k in range(net.K)]
+        run.step()
+        new_params = [O.sgd_update(params[k], ref[k]["grads"], lr)[0] for k in range(net.K)]
+        for k in range(net.K):
+            got = run.lp.lp_get_params(run.h, k).astype(np.float64)
+            errs = per_tensor_errors(net, k, got, new_params[k])
+            assert max(errs.values()) < tol, (k, errs)
+            # the update itself, wherever it is large enough to be resolved in the fp32 master copy
+            off = 0
+            for name, _, shape in net.param_layout(k):
+                n = int(np.prod(shape))
+                sl = slice(off, off + n)
+                off += n
+                d_ref = new_params[k][sl] - params[k][sl]
+                if np.linalg.norm(d_ref) > 2e-3 * np.linalg.norm(params[k][sl]):
+                    assert rel_err(got[sl] - before[k][sl], d_ref) < tol, (k, name)
+        params = new_params
+        if kappas is not None:
+            kappas = [O.kappa_update(kappas[k], ref[k]["r"], cfg["rho"]) for k in range(net.K - 1)]
+            for k in range(net.K - 1):
+                assert rel_err(to_host(run.d_kappa[k]), kappas[k]) < tol
+        # the oracle continues from its own updated parameters and multipliers
+    return run
+
+
+def test_tiny_fp32_step_two_steps():
+    full_step_parity(get_config("tiny"), steps=2)
+
+
+def test_tiny_fp32_per_module_calls_and_penalty():
+    cfg = get_config("tiny")
+    cfg["loss"] = "penalty"
+    full_step_parity(cfg, grouped=False)
+
+
+@pytest.mark.parametrize("kind,stem", [("postbn", "conv3x3"), ("preact", "conv3x3"), ("postbn", "conv7x7s2_maxpool")])
+def test_small_fp32_block_kinds(kind, stem):
+    if stem == "conv3x3":
+        cfg = small_cfg(kind, N=4, H=8, W=8)
+    else:
+        cfg = small_cfg(kind, stem=stem, N=3, H=32, W=32, stage_channels=(8, 16), stage_stride=(1, 2))
+    full_step_parity(cfg, steps=1)
+
+
+@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("kind", ["postbn", "preact"])
+def test_small_bf16_block_kinds(kind, impl):
+    cfg = small_cfg(kind, N=8, H=16, W=16, dtype="bf16", stage_channels=(16, 32), stage_blocks=(2, 2),
+                    module_block_end=(1, 3, 4), stem_channels=16, classes=10)
+    full_step_parity(cfg, conv_impl=impl, steps=2)
+
+
+def test_resnet56_reduced_batch_bf16():
+    full_step_parity(scaled("resnet56", N=16), steps=1)
+
+
+def test_resnet110_reduced_batch_bf16_two_steps():
+    full_step_parity(scaled("resnet110", N=8), steps=2)
+
+
+def test_wrn28_10_reduced_batch_bf16():
+    full_step_parity(scaled("wrn28_10", N=6), steps=1)
+
+
+def test_resnet34_reduced_bf16():
+    full_step_parity(scaled("resnet34", N=2, H=64, W=64), steps=1)
+
+
+def test_serial_forward_matches_oracle_and_serial_backprop_is_bp():
+    """Layer-serial comparator: x_{k+1} := F_k(x_k) reproduces the undecomposed network, and
+    back-propagating the cross-entropy through all modules gives the ordinary BP gradients."""
+    cfg = small_cfg("preact", N=4, H=8, W=8, stage_channels=(8, 16), stage_blocks=(2, 2), module_block_end=(1, 3, 4))
+    run = GpuRun(cfg)
+    torch = run.torch
+    logits = torch.zeros(cfg["N"], cfg["num_classes"], dtype=torch.float32, device="cuda:0")
+    run.lp.lp_forward_serial(run.h, run.d_images, logits)
+    assert run.lp.lp_last_device_status(run.h) == 0
+    ref = O.forward_serial(run.net, run.mods, run.images)
+    assert rel_err(logits.cpu().numpy(), ref) < 1e-4
+    loss = torch.zeros(2, dtype=torch.float32, device="cuda:0")
+    run.lp.lp_serial_fwd_bwd(run.h, run.d_images, run.d_labels, loss)
+    assert run.lp.lp_last_device_status(run.h) == 0
+    # oracle BP: chain the modules, seed each with the next module's input gradient
+    net = run.net
+    xs = [run.images.astype(np.float64)]
+    for k in range(net.K - 1):
+        xs.append(O.module_forward(net, k, net.unpack(k, run.mods[k]), xs[k]))
+    res = O.module_fwd_bwd(net, net.K - 1, run.mods[-1], xs[-1], run.labels, None, 1.0)
+    assert abs(loss[0].item() - res["loss"]) < 1e-4 * abs(res["loss"])
+    errs = per_tensor_errors(net, net.K - 1, run.lp.lp_get_grads(run.h, net.K - 1), res["grads"])
+    assert max(errs.values()) < 1e-4, errs
+    # module K-2 receives dx of module K-1 as terminal adjoint: penalty with rho = 0 and kappa = dx
+    d = res["dx"]
+    for k in range(net.K - 2, -1, -1):
+        r2 = O.module_fwd_bwd(net, k, run.mods[k], xs[k], xs[k + 1], d, 0.0)
+        errs = per_tensor_errors(net, k, run.lp.lp_get_grads(run.h, k), r2["grads"])
+        assert max(errs.values()) < 2e-4, (k, errs)
+        d = r2["dx"]
+
+
+def test_argument_errors_are_reported_on_the_host():
+    cfg = get_config("tiny")
+    run = GpuRun(cfg)
+    lp = run.lp
+    with pytest.raises(lp.LpError) as e:
+        lp.lp_module_fwd_bwd(run.h, 5, run.d_x[0], run.d_x[1], None, 1.0, run.d_loss[0], None)
+    assert e.value.status == -3
+    with pytest.raises(lp.LpError) as e:
+        lp.lp_module_fwd_bwd(run.h, 0, None, run.d_x[1], None, 1.0, run.d_loss[0], None)
+    assert e.value.status == -1
+    with pytest.raises(lp.LpError) as e:
+        lp.lp_module_fwd_bwd(run.h, 0, run.d_x[0].data_ptr() + 4, run.d_x[1], None, 1.0, run.d_loss[0], None)
+    assert e.value.status == -4
+    with pytest.raises(lp.LpError) as e:
+        lp.lp_step(run.h, 0.1)
+    assert e.value.status == -6
+    with pytest.raises(lp.LpError) as e:
+        lp.lp_set_params(run.h, 0, np.zeros(3, dtype=np.float32))
+    assert e.value.status == -9
+    assert lp.lp_last_device_status(run.h) == 0
