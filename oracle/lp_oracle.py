@@ -186,6 +186,11 @@ class Net:
 
     def __init__(self, cfg):
         self.cfg = cfg
+        # Optional model of activation storage: a callable applied wherever the step keeps an
+        # activation or adjoint tensor between operators.  None (default) = exact arithmetic.
+        # Tests of reduced-precision storage pass a rounding function so that the decisions that
+        # floating point takes (ReLU masks, max-pool winners) are taken on the same values.
+        self.store = None
         self.K = len(cfg["module_block_end"])
         self.eps = float(cfg["bn_eps"])
         self.kind = cfg["block_kind"]
@@ -294,19 +299,23 @@ class Net:
                                for name, _, _ in self.param_layout(which)])
 
 
+def _st(net, a):
+    return a if net.store is None else np.asarray(net.store(a), dtype=F)
+
+
 # ----------------------------------------------------------------------------
 # AuxNet forward chain  (Eq. AV-Net-FP-lambda; Algorithm 1, first inner loop)
 # ----------------------------------------------------------------------------
 def auxnet_apply(net, k, p, x):
     """x_{k+1} = AuxNet_k(x_k): conv3x3-BN[-ReLU-conv3x3-BN], batch statistics, no final ReLU."""
     convs = net.aux[k]
-    h = conv_fwd(x, p["conv1.w"], convs[0]["stride"], 1)
+    h = _st(net, conv_fwd(x, p["conv1.w"], convs[0]["stride"], 1))
     h, _ = bn_fwd(h, p["bn1.g"], p["bn1.b"], net.eps)
     if len(convs) == 2:
-        h = relu(h)
-        h = conv_fwd(h, p["conv2.w"], convs[1]["stride"], 1)
+        h = _st(net, relu(h))
+        h = _st(net, conv_fwd(h, p["conv2.w"], convs[1]["stride"], 1))
         h, _ = bn_fwd(h, p["bn2.g"], p["bn2.b"], net.eps)
-    return h
+    return _st(net, h)
 
 
 def auxnet_forward(net, aux_params, images, post=None):
@@ -326,12 +335,12 @@ def auxnet_forward(net, aux_params, images, post=None):
 # ----------------------------------------------------------------------------
 def _stem_fwd(net, p, x, cache):
     st = net.stem
-    y = conv_fwd(x, p["stem.conv.w"], st["stride"], st["pad"])
+    y = _st(net, conv_fwd(x, p["stem.conv.w"], st["stride"], st["pad"]))
     cache["stem.x"] = x
     if net.kind == "postbn":
         z, cache["stem.bn"] = bn_fwd(y, p["stem.bn.g"], p["stem.bn.b"], net.eps)
         cache["stem.z"] = z
-        y = relu(z)
+        y = _st(net, relu(z))
         if st["pool"]:
             y, cache["stem.pool"] = maxpool_fwd(y)
     return y
@@ -341,9 +350,10 @@ def _stem_bwd(net, p, d, cache, g):
     st = net.stem
     if net.kind == "postbn":
         if st["pool"]:
-            d = maxpool_bwd(d, cache["stem.pool"])
+            d = _st(net, maxpool_bwd(d, cache["stem.pool"]))
         d = relu_bwd(d, cache["stem.z"])
         d, g["stem.bn.g"], g["stem.bn.b"] = bn_bwd(d, cache["stem.bn"], p["stem.bn.g"])
+        d = _st(net, d)
     g["stem.conv.w"] = conv_wgrad(cache["stem.x"], d, p["stem.conv.w"].shape, st["stride"], st["pad"])
     return None        # the gradient with respect to the image is not used
 
@@ -355,27 +365,27 @@ def _block_fwd(net, bi, p, x, cache):
     c = cache.setdefault(bi, {})
     c["x"] = x
     if net.kind == "postbn":
-        y1 = conv_fwd(x, p[q + "conv1.w"], b["stride"], 1)
+        y1 = _st(net, conv_fwd(x, p[q + "conv1.w"], b["stride"], 1))
         z1, c["bn1"] = bn_fwd(y1, p[q + "bn1.g"], p[q + "bn1.b"], net.eps)
-        a1 = relu(z1)
-        y2 = conv_fwd(a1, p[q + "conv2.w"], 1, 1)
+        a1 = _st(net, relu(z1))
+        y2 = _st(net, conv_fwd(a1, p[q + "conv2.w"], 1, 1))
         z2, c["bn2"] = bn_fwd(y2, p[q + "bn2.g"], p[q + "bn2.b"], net.eps)
         c["z1"], c["a1"] = z1, a1
         if b["proj"]:
-            ys = conv_fwd(x, p[q + "sc.w"], b["stride"], 0)
+            ys = _st(net, conv_fwd(x, p[q + "sc.w"], b["stride"], 0))
             sc, c["bns"] = bn_fwd(ys, p[q + "bns.g"], p[q + "bns.b"], net.eps)
         else:
             sc = x
         return sc + z2
     # pre-activation form
     z0, c["bn1"] = bn_fwd(x, p[q + "bn1.g"], p[q + "bn1.b"], net.eps)
-    o = relu(z0)
-    y1 = conv_fwd(o, p[q + "conv1.w"], b["stride"], 1)
+    o = _st(net, relu(z0))
+    y1 = _st(net, conv_fwd(o, p[q + "conv1.w"], b["stride"], 1))
     z1, c["bn2"] = bn_fwd(y1, p[q + "bn2.g"], p[q + "bn2.b"], net.eps)
-    a1 = relu(z1)
+    a1 = _st(net, relu(z1))
     y2 = conv_fwd(a1, p[q + "conv2.w"], 1, 1)
     c["z0"], c["o"], c["z1"], c["a1"] = z0, o, z1, a1
-    sc = conv_fwd(o, p[q + "sc.w"], b["stride"], 0) if b["proj"] else x
+    sc = _st(net, conv_fwd(o, p[q + "sc.w"], b["stride"], 0)) if b["proj"] else x
     return sc + y2
 
 
@@ -387,35 +397,39 @@ def _block_bwd(net, bi, p, d, cache, g):
     x = c["x"]
     if net.kind == "postbn":
         dy2, g[q + "bn2.g"], g[q + "bn2.b"] = bn_bwd(d, c["bn2"], p[q + "bn2.g"])
+        dy2 = _st(net, dy2)
         g[q + "conv2.w"] = conv_wgrad(c["a1"], dy2, p[q + "conv2.w"].shape, 1, 1)
-        da1 = conv_dgrad(dy2, p[q + "conv2.w"], 1, 1, c["a1"].shape)
+        da1 = _st(net, conv_dgrad(dy2, p[q + "conv2.w"], 1, 1, c["a1"].shape))
         dz1 = relu_bwd(da1, c["z1"])
         dy1, g[q + "bn1.g"], g[q + "bn1.b"] = bn_bwd(dz1, c["bn1"], p[q + "bn1.g"])
+        dy1 = _st(net, dy1)
         g[q + "conv1.w"] = conv_wgrad(x, dy1, p[q + "conv1.w"].shape, b["stride"], 1)
         dx = conv_dgrad(dy1, p[q + "conv1.w"], b["stride"], 1, x.shape)
         if b["proj"]:
             dys, g[q + "bns.g"], g[q + "bns.b"] = bn_bwd(d, c["bns"], p[q + "bns.g"])
+            dys = _st(net, dys)
             g[q + "sc.w"] = conv_wgrad(x, dys, p[q + "sc.w"].shape, b["stride"], 0)
-            dx = dx + conv_dgrad(dys, p[q + "sc.w"], b["stride"], 0, x.shape)
+            dx = _st(net, dx) + conv_dgrad(dys, p[q + "sc.w"], b["stride"], 0, x.shape)
         else:
             dx = dx + d
-        return dx
+        return _st(net, dx)
     # pre-activation form
     g[q + "conv2.w"] = conv_wgrad(c["a1"], d, p[q + "conv2.w"].shape, 1, 1)
-    da1 = conv_dgrad(d, p[q + "conv2.w"], 1, 1, c["a1"].shape)
+    da1 = _st(net, conv_dgrad(d, p[q + "conv2.w"], 1, 1, c["a1"].shape))
     dz1 = relu_bwd(da1, c["z1"])
     dy1, g[q + "bn2.g"], g[q + "bn2.b"] = bn_bwd(dz1, c["bn2"], p[q + "bn2.g"])
+    dy1 = _st(net, dy1)
     g[q + "conv1.w"] = conv_wgrad(c["o"], dy1, p[q + "conv1.w"].shape, b["stride"], 1)
-    do = conv_dgrad(dy1, p[q + "conv1.w"], b["stride"], 1, c["o"].shape)
+    do = _st(net, conv_dgrad(dy1, p[q + "conv1.w"], b["stride"], 1, c["o"].shape))
     dx_direct = 0.0
     if b["proj"]:
         g[q + "sc.w"] = conv_wgrad(c["o"], d, p[q + "sc.w"].shape, b["stride"], 0)
-        do = do + conv_dgrad(d, p[q + "sc.w"], b["stride"], 0, c["o"].shape)
+        do = _st(net, do + conv_dgrad(d, p[q + "sc.w"], b["stride"], 0, c["o"].shape))
     else:
         dx_direct = d
     dz0 = relu_bwd(do, c["z0"])
     dx, g[q + "bn1.g"], g[q + "bn1.b"] = bn_bwd(dz0, c["bn1"], p[q + "bn1.g"])
-    return dx + dx_direct
+    return _st(net, dx + dx_direct)
 
 
 def _head_fwd(net, p, x, cache):
@@ -423,7 +437,7 @@ def _head_fwd(net, p, x, cache):
     if net.kind == "preact":
         z, cache["head.bn"] = bn_fwd(x, p["head.bn.g"], p["head.bn.b"], net.eps)
         cache["head.z"] = z
-        x = relu(z)
+        x = _st(net, relu(z))
     pooled = avgpool_fwd(x)
     cache["head.pooled"] = pooled
     return linear_fwd(pooled, p["head.fc.w"], p["head.fc.b"])
@@ -432,10 +446,11 @@ def _head_fwd(net, p, x, cache):
 def _head_bwd(net, p, dlogits, cache, g):
     g["head.fc.w"] = dlogits.T @ cache["head.pooled"]
     g["head.fc.b"] = dlogits.sum(axis=0)
-    d = avgpool_bwd(dlogits @ p["head.fc.w"], cache["head.x"].shape)
+    d = _st(net, avgpool_bwd(dlogits @ p["head.fc.w"], cache["head.x"].shape))
     if net.kind == "preact":
         d = relu_bwd(d, cache["head.z"])
         d, g["head.bn.g"], g["head.bn.b"] = bn_bwd(d, cache["head.bn"], p["head.bn.g"])
+        d = _st(net, d)
     return d
 
 
@@ -445,8 +460,12 @@ def module_forward(net, k, p, x_k, cache=None):
     x = np.asarray(x_k, dtype=F)
     if k == 0:
         x = _stem_fwd(net, p, x, cache)
-    for bi in net.module_blocks[k]:
+    for i, bi in enumerate(net.module_blocks[k]):
         x = _block_fwd(net, bi, p, x, cache)
+        # an interior module's final output goes straight into the local loss; every other block
+        # output is kept as an activation tensor
+        if not (i == len(net.module_blocks[k]) - 1 and k < net.K - 1 and net.kind == "postbn"):
+            x = _st(net, x)
     if k == net.K - 1:
         x = _head_fwd(net, p, x, cache)
     return x
@@ -468,7 +487,8 @@ def module_fwd_bwd(net, k, params_flat, x_k, x_next_or_labels, kappa, rho):
     else:
         kap = None if kappa is None else np.asarray(kappa, dtype=F)
         loss, rn2, r, seed = local_loss(out, np.asarray(x_next_or_labels, dtype=F), kap, rho)
-        res.update(loss=loss, rnorm2=rn2, r=r, seed=seed)
+        res.update(loss=loss, rnorm2=rn2, r=_st(net, r), seed=seed)
+        seed = _st(net, seed)
     g = {}
     d = seed
     if k == net.K - 1:

@@ -104,9 +104,15 @@ class GpuRun:
         assert self.lp.lp_last_device_status(self.h) == 0
 
 
-def oracle_modules(run, xs_host, kappas=None, params=None):
-    """Oracle module_fwd_bwd for every module on the given boundary tensors (x_0 = images)."""
+def oracle_modules(run, xs_host, kappas=None, params=None, exact=False):
+    """Oracle module_fwd_bwd for every module on the given boundary tensors (x_0 = images).
+
+    For a bf16 workload the oracle rounds activations where the step stores them (unless
+    ``exact``): ReLU masks and max-pool winners are decisions taken by floating point, and both
+    sides must take them on the same values -- exact arithmetic alone moves gradient tensors of a
+    randomly initialised network by several percent through flipped masks."""
     net, cfg = run.net, run.cfg
+    net.store = None if (exact or cfg["dtype"] == "f32") else gen.round_bf16
     xs = [run.images.astype(np.float64)] + [np.asarray(x, dtype=np.float64) for x in xs_host]
     params = run.mods if params is None else params
     kappas = (run.kappa if run.use_kappa else None) if kappas is None else kappas
@@ -115,4 +121,5 @@ def oracle_modules(run, xs_host, kappas=None, params=None):
         last = k == net.K - 1
         out.append(O.module_fwd_bwd(net, k, params[k], xs[k], run.labels if last else xs[k + 1],
                                     None if (last or kappas is None) else kappas[k], cfg["rho"]))
+    net.store = None
     return out

@@ -54,6 +54,12 @@ def full_step_parity(cfg, conv_impl=0, grouped=True, steps=1):
         grads = run.fwd_bwd_all(grouped=grouped)
         ref = oracle_modules(run, xs_host, kappas=kappas, params=params)
         check_modules(run, grads, ref, tol)
+        if cfg["dtype"] == "bf16" and step == 0:
+            # against exact arithmetic: losses and residual norms within the same tolerance
+            exact = oracle_modules(run, xs_host, kappas=kappas, params=params, exact=True)
+            loss = run.d_loss.cpu().numpy()
+            for k in range(net.K):
+                assert abs(loss[k, 0] - exact[k]["loss"]) < tol * abs(exact[k]["loss"]), (k, "exact loss")
         for k in range(net.K - 1):
             r = run.torch.zeros_like(run.d_x[k + 1])
             s = run.torch.zeros_like(run.d_x[k + 1])
