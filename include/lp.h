@@ -56,6 +56,8 @@ enum { LP_POSTBN = 0, LP_PREACT = 1 };
 #define LP_AUX(k) (256 + (k))
 enum { LP_KIND_CONV_W = 0, LP_KIND_BN_GAMMA = 1, LP_KIND_BN_BETA = 2, LP_KIND_FC_W = 3, LP_KIND_FC_B = 4 };
 enum { LP_CONV_IMPL_AUTO = 0, LP_CONV_IMPL_SIMT = 1, LP_CONV_IMPL_TENSOR = 2 };
+/* May be OR-ed into conv_impl: keep one kind of convolution on the CUDA cores (diagnostics). */
+enum { LP_CONV_NO_TENSOR_FWD = 16, LP_CONV_NO_TENSOR_DGRAD = 32, LP_CONV_NO_TENSOR_WGRAD = 64 };
 enum { LP_CONV_FWD = 0, LP_CONV_DGRAD = 1, LP_CONV_WGRAD = 2 };
 
 #define LP_MAX_STAGES 8

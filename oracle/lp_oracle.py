@@ -303,17 +303,23 @@ def _st(net, a):
     return a if net.store is None else np.asarray(net.store(a), dtype=F)
 
 
+def _wq(net, w):
+    """Convolution weights as the contraction reads them (the storage model also applies to the
+    operand copy of the weights; the fp32 master that the update touches is not rounded)."""
+    return _st(net, w)
+
+
 # ----------------------------------------------------------------------------
 # AuxNet forward chain  (Eq. AV-Net-FP-lambda; Algorithm 1, first inner loop)
 # ----------------------------------------------------------------------------
 def auxnet_apply(net, k, p, x):
     """x_{k+1} = AuxNet_k(x_k): conv3x3-BN[-ReLU-conv3x3-BN], batch statistics, no final ReLU."""
     convs = net.aux[k]
-    h = _st(net, conv_fwd(x, p["conv1.w"], convs[0]["stride"], 1))
+    h = _st(net, conv_fwd(x, _wq(net, p["conv1.w"]), convs[0]["stride"], 1))
     h, _ = bn_fwd(h, p["bn1.g"], p["bn1.b"], net.eps)
     if len(convs) == 2:
         h = _st(net, relu(h))
-        h = _st(net, conv_fwd(h, p["conv2.w"], convs[1]["stride"], 1))
+        h = _st(net, conv_fwd(h, _wq(net, p["conv2.w"]), convs[1]["stride"], 1))
         h, _ = bn_fwd(h, p["bn2.g"], p["bn2.b"], net.eps)
     return _st(net, h)
 
@@ -335,7 +341,7 @@ def auxnet_forward(net, aux_params, images, post=None):
 # ----------------------------------------------------------------------------
 def _stem_fwd(net, p, x, cache):
     st = net.stem
-    y = _st(net, conv_fwd(x, p["stem.conv.w"], st["stride"], st["pad"]))
+    y = _st(net, conv_fwd(x, _wq(net, p["stem.conv.w"]), st["stride"], st["pad"]))
     cache["stem.x"] = x
     if net.kind == "postbn":
         z, cache["stem.bn"] = bn_fwd(y, p["stem.bn.g"], p["stem.bn.b"], net.eps)
@@ -365,14 +371,14 @@ def _block_fwd(net, bi, p, x, cache):
     c = cache.setdefault(bi, {})
     c["x"] = x
     if net.kind == "postbn":
-        y1 = _st(net, conv_fwd(x, p[q + "conv1.w"], b["stride"], 1))
+        y1 = _st(net, conv_fwd(x, _wq(net, p[q + "conv1.w"]), b["stride"], 1))
         z1, c["bn1"] = bn_fwd(y1, p[q + "bn1.g"], p[q + "bn1.b"], net.eps)
         a1 = _st(net, relu(z1))
-        y2 = _st(net, conv_fwd(a1, p[q + "conv2.w"], 1, 1))
+        y2 = _st(net, conv_fwd(a1, _wq(net, p[q + "conv2.w"]), 1, 1))
         z2, c["bn2"] = bn_fwd(y2, p[q + "bn2.g"], p[q + "bn2.b"], net.eps)
         c["z1"], c["a1"] = z1, a1
         if b["proj"]:
-            ys = _st(net, conv_fwd(x, p[q + "sc.w"], b["stride"], 0))
+            ys = _st(net, conv_fwd(x, _wq(net, p[q + "sc.w"]), b["stride"], 0))
             sc, c["bns"] = bn_fwd(ys, p[q + "bns.g"], p[q + "bns.b"], net.eps)
         else:
             sc = x
@@ -380,12 +386,12 @@ def _block_fwd(net, bi, p, x, cache):
     # pre-activation form
     z0, c["bn1"] = bn_fwd(x, p[q + "bn1.g"], p[q + "bn1.b"], net.eps)
     o = _st(net, relu(z0))
-    y1 = _st(net, conv_fwd(o, p[q + "conv1.w"], b["stride"], 1))
+    y1 = _st(net, conv_fwd(o, _wq(net, p[q + "conv1.w"]), b["stride"], 1))
     z1, c["bn2"] = bn_fwd(y1, p[q + "bn2.g"], p[q + "bn2.b"], net.eps)
     a1 = _st(net, relu(z1))
-    y2 = conv_fwd(a1, p[q + "conv2.w"], 1, 1)
+    y2 = conv_fwd(a1, _wq(net, p[q + "conv2.w"]), 1, 1)
     c["z0"], c["o"], c["z1"], c["a1"] = z0, o, z1, a1
-    sc = _st(net, conv_fwd(o, p[q + "sc.w"], b["stride"], 0)) if b["proj"] else x
+    sc = _st(net, conv_fwd(o, _wq(net, p[q + "sc.w"]), b["stride"], 0)) if b["proj"] else x
     return sc + y2
 
 
@@ -399,32 +405,32 @@ def _block_bwd(net, bi, p, d, cache, g):
         dy2, g[q + "bn2.g"], g[q + "bn2.b"] = bn_bwd(d, c["bn2"], p[q + "bn2.g"])
         dy2 = _st(net, dy2)
         g[q + "conv2.w"] = conv_wgrad(c["a1"], dy2, p[q + "conv2.w"].shape, 1, 1)
-        da1 = _st(net, conv_dgrad(dy2, p[q + "conv2.w"], 1, 1, c["a1"].shape))
+        da1 = _st(net, conv_dgrad(dy2, _wq(net, p[q + "conv2.w"]), 1, 1, c["a1"].shape))
         dz1 = relu_bwd(da1, c["z1"])
         dy1, g[q + "bn1.g"], g[q + "bn1.b"] = bn_bwd(dz1, c["bn1"], p[q + "bn1.g"])
         dy1 = _st(net, dy1)
         g[q + "conv1.w"] = conv_wgrad(x, dy1, p[q + "conv1.w"].shape, b["stride"], 1)
-        dx = conv_dgrad(dy1, p[q + "conv1.w"], b["stride"], 1, x.shape)
+        dx = conv_dgrad(dy1, _wq(net, p[q + "conv1.w"]), b["stride"], 1, x.shape)
         if b["proj"]:
             dys, g[q + "bns.g"], g[q + "bns.b"] = bn_bwd(d, c["bns"], p[q + "bns.g"])
             dys = _st(net, dys)
             g[q + "sc.w"] = conv_wgrad(x, dys, p[q + "sc.w"].shape, b["stride"], 0)
-            dx = _st(net, dx) + conv_dgrad(dys, p[q + "sc.w"], b["stride"], 0, x.shape)
+            dx = _st(net, dx) + conv_dgrad(dys, _wq(net, p[q + "sc.w"]), b["stride"], 0, x.shape)
         else:
             dx = dx + d
         return _st(net, dx)
     # pre-activation form
     g[q + "conv2.w"] = conv_wgrad(c["a1"], d, p[q + "conv2.w"].shape, 1, 1)
-    da1 = _st(net, conv_dgrad(d, p[q + "conv2.w"], 1, 1, c["a1"].shape))
+    da1 = _st(net, conv_dgrad(d, _wq(net, p[q + "conv2.w"]), 1, 1, c["a1"].shape))
     dz1 = relu_bwd(da1, c["z1"])
     dy1, g[q + "bn2.g"], g[q + "bn2.b"] = bn_bwd(dz1, c["bn2"], p[q + "bn2.g"])
     dy1 = _st(net, dy1)
     g[q + "conv1.w"] = conv_wgrad(c["o"], dy1, p[q + "conv1.w"].shape, b["stride"], 1)
-    do = _st(net, conv_dgrad(dy1, p[q + "conv1.w"], b["stride"], 1, c["o"].shape))
+    do = _st(net, conv_dgrad(dy1, _wq(net, p[q + "conv1.w"]), b["stride"], 1, c["o"].shape))
     dx_direct = 0.0
     if b["proj"]:
         g[q + "sc.w"] = conv_wgrad(c["o"], d, p[q + "sc.w"].shape, b["stride"], 0)
-        do = _st(net, do + conv_dgrad(d, p[q + "sc.w"], b["stride"], 0, c["o"].shape))
+        do = _st(net, do + conv_dgrad(d, _wq(net, p[q + "sc.w"]), b["stride"], 0, c["o"].shape))
     else:
         dx_direct = d
     dz0 = relu_bwd(do, c["z0"])

@@ -1,7 +1,8 @@
 // Direct (CUDA-core) convolution kernels: any filter size, stride, padding and channel count.
 // They carry the fp32 workload (tensor cores have no true-fp32 mode) and the few bf16 shapes
 // the tensor-core path does not take (3-channel stems).  fp32 accumulation throughout;
-// weights are the fp32 masters w[co][r][s][ci].
+// weights are the fp32 masters w[co][r][s][ci], rounded to the activation type as they are read
+// so that both convolution paths of a bf16 network contract the same operands.
 #pragma once
 #include "common.cuh"
 
@@ -40,7 +41,7 @@ __global__ void conv_fwd_simt_kernel(const T* __restrict__ x, const float* __res
         for (int ci = 0; ci < g.Cin; ++ci) {
           const float xv = to_f(xp[ci]);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) acc[j] += xv * __ldg(wp + j * tap_stride + ci);
+          for (int j = 0; j < 4; ++j) acc[j] += xv * round_storage<T>(__ldg(wp + j * tap_stride + ci));
         }
       }
     }
@@ -84,10 +85,10 @@ __global__ void conv_dgrad_simt_kernel(const T* __restrict__ dy, const float* __
         for (int co = 0; co < g.Cout; ++co) {
           const float d = to_f(dp[co]);
           const float4 wv = __ldg(reinterpret_cast<const float4*>(wp + (long long)co * g.R * g.S * g.Cin));
-          acc[0] += d * wv.x;
-          acc[1] += d * wv.y;
-          acc[2] += d * wv.z;
-          acc[3] += d * wv.w;
+          acc[0] += d * round_storage<T>(wv.x);
+          acc[1] += d * round_storage<T>(wv.y);
+          acc[2] += d * round_storage<T>(wv.z);
+          acc[3] += d * round_storage<T>(wv.w);
         }
       }
     }

@@ -229,10 +229,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lo_ok) stv(p.out + obase + col, *reinterpret_cast<float(*)[8]>(&v[0]));
         if (hi_ok) stv(p.out + obase + col + 8, *reinterpret_cast<float(*)[8]>(&v[8]));
         if (p.stats) {
+          // statistics of the tensor as stored (bf16), so that the batch-norm that follows
+          // normalises exactly the values it reads
           float sq[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            if (!valid) v[j] = 0.f;
+            v[j] = valid ? round_storage<bf16>(v[j]) : 0.f;
             sq[j] = v[j] * v[j];
           }
           const float cs = transpose_reduce16(v, lane);

@@ -368,8 +368,8 @@ struct ProfScope {
 static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int N, const void* x, void* y,
                         const void* addend, double* stats, bool* stats_done, int* dev_err, cudaStream_t st) {
   if (stats_done) *stats_done = false;
-  const bool use_tc = dtype == LP_BF16 && impl != LP_CONV_IMPL_SIMT && tc_fwd_ok(c) && c.wf;
-  if (impl == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
+  const bool use_tc = dtype == LP_BF16 && (impl & 15) != LP_CONV_IMPL_SIMT && !(impl & 16) && tc_fwd_ok(c) && c.wf;
+  if ((impl & 15) == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
   if (use_tc) {
     TcGemmSpec s;
     memset(&s, 0, sizeof(s));
@@ -404,8 +404,8 @@ static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int
 // dx = conv^T(dy, w) [+ addend]   (addend may alias dx)
 static int conv_dgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N, const void* dy, void* dx,
                       const void* addend, int* dev_err, cudaStream_t st) {
-  const bool use_tc = dtype == LP_BF16 && impl != LP_CONV_IMPL_SIMT && tc_dgrad_ok(c) && c.wt;
-  if (impl == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
+  const bool use_tc = dtype == LP_BF16 && (impl & 15) != LP_CONV_IMPL_SIMT && !(impl & 32) && tc_dgrad_ok(c) && c.wt;
+  if ((impl & 15) == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
   if (use_tc) {
     const int st2 = c.stride;
     const int classes = st2 * st2;
@@ -465,8 +465,8 @@ static int conv_dgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
 // dw += x (*) dy     (dw zeroed by the caller beforehand)
 static int conv_wgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N, const void* x, const void* dy,
                       float* dw, int* dev_err, cudaStream_t st) {
-  const bool use_tc = dtype == LP_BF16 && impl != LP_CONV_IMPL_SIMT && tc_wgrad_ok(c);
-  if (impl == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
+  const bool use_tc = dtype == LP_BF16 && (impl & 15) != LP_CONV_IMPL_SIMT && !(impl & 64) && tc_wgrad_ok(c);
+  if ((impl & 15) == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
   if (use_tc) {
     ProfScope ps(h, st, 2.0 * N * c.OH * c.OW * (double)c.cout * c.R * c.R * c.cin);
     int rc = launch_wgrad_tc(g_dev.encode, g_dev.sm_count, (const bf16*)x, (const bf16*)dy, dw, N, c.H, c.W, c.cin,
@@ -497,7 +497,7 @@ struct Planner {
   Arena& A;
   int dtype;
   int impl;
-  Planner(const NetDef& n, Arena& a) : net(n), A(a), dtype(n.d.dtype), impl(n.d.conv_impl) {}
+  Planner(const NetDef& n, Arena& a) : net(n), A(a), dtype(n.d.dtype), impl(n.d.conv_impl & 15) {}
 
   Tensor new_tensor(int n, int h, int w, int c) {
     Tensor t;
@@ -569,7 +569,7 @@ struct Planner {
   }
 
   bool conv_fuses_stats(const ConvDef& c) const {
-    return dtype == LP_BF16 && impl != LP_CONV_IMPL_SIMT && tc_fwd_ok(c) && c.wf;
+    return dtype == LP_BF16 && impl != LP_CONV_IMPL_SIMT && !(net.d.conv_impl & 16) && tc_fwd_ok(c) && c.wf;
   }
   Tensor emit_conv(Plan& P, std::vector<Op>& ops, const Tensor& in, int conv, const Tensor* addend, int stats_bn) {
     const ConvDef& c = P.convs[conv];

@@ -104,7 +104,21 @@ class GpuRun:
         assert self.lp.lp_last_device_status(self.h) == 0
 
 
-def oracle_modules(run, xs_host, kappas=None, params=None, exact=False):
+def noisy_bf16_store(seed=1234, eps=1e-7):
+    """Storage model with accumulation-order noise: values are perturbed by a relative 1e-7
+    (the size of fp32 summation-order effects) before they are rounded to bf16.  Two runs of the
+    oracle that differ only by this noise bound how closely ANY bf16-storage implementation can be
+    expected to reproduce a gradient tensor: rounding boundaries and ReLU masks turn such noise
+    into percent-level changes of the adjoint fields of a deep module."""
+    rng = np.random.default_rng(seed)
+
+    def store(a):
+        a = np.asarray(a, dtype=np.float64)
+        return gen.round_bf16(a * (1.0 + eps * rng.standard_normal(a.shape)))
+    return store
+
+
+def oracle_modules(run, xs_host, kappas=None, params=None, exact=False, store=None):
     """Oracle module_fwd_bwd for every module on the given boundary tensors (x_0 = images).
 
     For a bf16 workload the oracle rounds activations where the step stores them (unless
@@ -112,7 +126,7 @@ def oracle_modules(run, xs_host, kappas=None, params=None, exact=False):
     sides must take them on the same values -- exact arithmetic alone moves gradient tensors of a
     randomly initialised network by several percent through flipped masks."""
     net, cfg = run.net, run.cfg
-    net.store = None if (exact or cfg["dtype"] == "f32") else gen.round_bf16
+    net.store = None if (exact or cfg["dtype"] == "f32") else (store or gen.round_bf16)
     xs = [run.images.astype(np.float64)] + [np.asarray(x, dtype=np.float64) for x in xs_host]
     params = run.mods if params is None else params
     kappas = (run.kappa if run.use_kappa else None) if kappas is None else kappas

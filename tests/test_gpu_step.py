@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 
 from conftest import small_cfg
-from harness import GpuRun, oracle_modules, per_tensor_errors, rel_err, to_host
+from harness import GpuRun, noisy_bf16_store, oracle_modules, per_tensor_errors, rel_err, to_host
 from oracle import lp_oracle as O
 from workloads import gen, get_config, scaled
 
@@ -16,23 +16,33 @@ pytestmark = pytest.mark.gpu
 TOL = {"f32": 1e-4, "bf16": 2e-2}
 
 
-def check_modules(run, grads, ref, tol, dx_from=1):
+def check_modules(run, grads, ref, tol, floor=None, dx_from=1):
+    """Per-tensor relative L2 errors of parameter gradients, input gradients and losses.
+
+    fp32: every tensor within `tol`.  bf16: within max(tol, 4 x noise floor), the floor being the
+    change of that tensor between two oracle runs that differ by 1e-7 relative noise before each
+    bf16 rounding (see harness.noisy_bf16_store); losses always within `tol`."""
     net = run.net
     loss = run.d_loss.cpu().numpy()
-    worst = 0.0
+    allow = []
     for k in range(net.K):
         errs = per_tensor_errors(net, k, grads[k], ref[k]["grads"])
-        bad = {n: e for n, e in errs.items() if not e < tol}
+        fl = per_tensor_errors(net, k, floor[k]["grads"], ref[k]["grads"]) if floor else {}
+        allow.append({n: max(tol, 4 * fl.get(n, 0.0)) for n in errs})
+        bad = {n: (e, fl.get(n, 0.0)) for n, e in errs.items() if not e < allow[k][n]}
         assert not bad, (k, bad)
-        worst = max(worst, max(errs.values()))
+        whole = rel_err(grads[k], ref[k]["grads"])
+        whole_floor = rel_err(floor[k]["grads"], ref[k]["grads"]) if floor else 0.0
+        assert whole < max(tol, 4 * whole_floor), (k, "whole gradient", whole, whole_floor)
         lerr = abs(loss[k, 0] - ref[k]["loss"]) / max(abs(ref[k]["loss"]), 1e-30)
         assert lerr < tol, (k, loss[k, 0], ref[k]["loss"])
         if k < net.K - 1:
             assert abs(loss[k, 1] - ref[k]["rnorm2"]) / ref[k]["rnorm2"] < tol
         if k >= dx_from:
             e = rel_err(to_host(run.d_dx[k]), ref[k]["dx"])
-            assert e < tol, (k, "dx", e)
-    return worst
+            f = rel_err(floor[k]["dx"], ref[k]["dx"]) if floor else 0.0
+            assert e < max(tol, 4 * f), (k, "dx", e, f)
+    return allow
 
 
 def full_step_parity(cfg, conv_impl=0, grouped=True, steps=1):
@@ -53,7 +63,10 @@ def full_step_parity(cfg, conv_impl=0, grouped=True, steps=1):
     for step in range(steps):
         grads = run.fwd_bwd_all(grouped=grouped)
         ref = oracle_modules(run, xs_host, kappas=kappas, params=params)
-        check_modules(run, grads, ref, tol)
+        floor = None
+        if cfg["dtype"] == "bf16":
+            floor = oracle_modules(run, xs_host, kappas=kappas, params=params, store=noisy_bf16_store())
+        allow = check_modules(run, grads, ref, tol, floor)
         if cfg["dtype"] == "bf16" and step == 0:
             # against exact arithmetic: losses and residual norms within the same tolerance
             exact = oracle_modules(run, xs_host, kappas=kappas, params=params, exact=True)
@@ -86,13 +99,25 @@ def full_step_parity(cfg, conv_impl=0, grouped=True, steps=1):
                 off += n
                 d_ref = new_params[k][sl] - params[k][sl]
                 if np.linalg.norm(d_ref) > 2e-3 * np.linalg.norm(params[k][sl]):
-                    assert rel_err(got[sl] - before[k][sl], d_ref) < tol, (k, name)
+                    assert rel_err(got[sl] - before[k][sl], d_ref) < allow[k][name] + 1e-3, (k, name)
         params = new_params
         if kappas is not None:
             kappas = [O.kappa_update(kappas[k], ref[k]["r"], cfg["rho"]) for k in range(net.K - 1)]
             for k in range(net.K - 1):
                 assert rel_err(to_host(run.d_kappa[k]), kappas[k]) < tol
-        # the oracle continues from its own updated parameters and multipliers
+        # The oracle continues from its own updated parameters and multipliers.  On the bf16 path
+        # the GPU's second step is started from the oracle's state as well: its own fp32 masters
+        # differ from the oracle's by the (already checked) gradient error times the learning
+        # rate, which is enough to flip a few ReLU masks and would be counted twice.
+        if cfg["dtype"] == "bf16" and step + 1 < steps:
+            for k in range(net.K):
+                run.lp.lp_set_params(run.h, k, params[k].astype(np.float32))
+                params[k] = params[k].astype(np.float32).astype(np.float64)
+            if kappas is not None:
+                for k in range(net.K - 1):
+                    kq = gen.round_bf16(kappas[k])
+                    run.d_kappa[k].copy_(run.torch.from_numpy(kq).to("cuda:0").to(run.torch.bfloat16))
+                    kappas[k] = kq.astype(np.float64)
     return run
 
 
