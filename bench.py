@@ -1,0 +1,435 @@
+#!/usr/bin/env python
+"""Benchmark of the layer-parallel training step on B200 (one process per GPU).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload wrn28_10] [--impl ours|reference]
+
+A step is one pass of the whole hot path over one synthetic batch: AuxNet forward chain, all K
+modules' forward + local loss + backward (concurrently, on K streams), parameter / multiplier
+update.  The step is recorded once into a CUDA graph and replayed.  `value` is images/s with the
+inputs resident in HBM; `e2e` is the same step driven from pinned host buffers (images and labels
+copied in, the K losses copied out, every step).  With N > 1 the ranks are independent replicas
+(the path does not shard: no collective), and `value` is the sum over ranks.
+
+`--impl reference` times the CPU oracle (oracle/lp_oracle.py, as it stands) on a bounded sample of
+the same workload on the host cores.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "images/sec per layer-parallel step"
+UNIT = "images/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="wrn28_10")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (0 = the workload's own)")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-serial", action="store_true")
+    ap.add_argument("--conv-impl", type=int, default=0)
+    return ap.parse_args()
+
+
+# ---------------------------------------------------------------------------------------------
+# workload FLOP accounting (true sizes, multiply-add = 2 FLOPs, backward = 2 x forward)
+# ---------------------------------------------------------------------------------------------
+def conv_flops_forward(cfg):
+    """Forward conv FLOPs per step: main network (stem + blocks) and AuxNet, from the oracle-free
+    shape walk below (this is bookkeeping for the report, not part of the path)."""
+    def out(h, r, s, p):
+        return (h + 2 * p - r) // s + 1
+    n = cfg["N"]
+    h, w = cfg["H"], cfg["W"]
+    fl = 0.0
+    if cfg["stem_kind"] == "conv3x3":
+        fl += 2.0 * n * h * w * cfg["stem_channels"] * 9 * cfg["C_in"]
+    else:
+        h, w = out(h, 7, 2, 3), out(w, 7, 2, 3)
+        fl += 2.0 * n * h * w * cfg["stem_channels"] * 49 * cfg["C_in"]
+        h, w = out(h, 3, 2, 1), out(w, 3, 2, 1)
+    c = cfg["stem_channels"]
+    shapes = []
+    for ch, nb, st in zip(cfg["stage_channels"], cfg["stage_blocks"], cfg["stage_stride"]):
+        for b in range(nb):
+            s = st if b == 0 else 1
+            shapes.append((h, w, c))
+            ho, wo = out(h, 3, s, 1), out(w, 3, s, 1)
+            fl += 2.0 * n * ho * wo * ch * 9 * c + 2.0 * n * ho * wo * ch * 9 * ch
+            if s != 1 or c != ch:
+                fl += 2.0 * n * ho * wo * ch * c
+            h, w, c = ho, wo, ch
+    # AuxNet
+    aux = 0.0
+    ends = cfg["module_block_end"]
+    bshape = [(cfg["H"], cfg["W"], cfg["C_in"])] + [shapes[e] for e in ends[:-1]]
+    for k in range(len(ends) - 1):
+        (hi, wi, ci), (ho, wo, co) = bshape[k], bshape[k + 1]
+        total = hi // ho
+        if cfg["aux_convs"] == 1:
+            aux += 2.0 * n * ho * wo * co * 9 * ci
+        else:
+            hid = co // cfg["aux_width_div"]
+            s1 = 2 if total >= 2 else 1
+            hm, wm = out(hi, 3, s1, 1), out(wi, 3, s1, 1)
+            aux += 2.0 * n * hm * wm * hid * 9 * ci + 2.0 * n * ho * wo * co * 9 * hid
+    return fl, aux
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks sampling during the timed region
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.rows = []
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            parts = [p.strip() for p in r.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle timing (bounded sample)
+# ---------------------------------------------------------------------------------------------
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle_step(cfg_name, sample_batch, repeats=1):
+    """One layer-parallel step of the oracle (AuxNet chain, K module forward+backward, updates) on
+    `sample_batch` images of the workload; returns (images/s, seconds per step)."""
+    from oracle import lp_oracle as O
+    from workloads import gen, scaled
+    cfg = scaled(cfg_name, N=sample_batch)
+    net = O.Net(cfg)
+    mods = [gen.make_params(net.param_layout(k), 0, "module%d" % k) for k in range(net.K)]
+    auxs = [gen.make_params(net.param_layout(O.LP_AUX(k)), 0, "aux%d" % k) for k in range(net.K - 1)]
+    images, labels = gen.make_images(cfg), gen.make_labels(cfg)
+    kappas = None
+    if cfg["loss"] == "al":
+        kappas = [np.zeros(net.boundary[k + 1]) for k in range(net.K - 1)]
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        O.layer_parallel_step(net, mods, auxs, images, labels, kappas, cfg["rho"], 1e-4)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return sample_batch / best, best
+
+
+def oracle_sample_batch(cfg):
+    # about 10-30 s of CPU work: the oracle sustains roughly 50-100 GFLOP/s of fp64 matmul
+    fwd, aux = conv_flops_forward(cfg)
+    per_image = (3 * fwd + aux) / cfg["N"]
+    target = 1.2e12
+    return int(max(1, min(cfg["N"], target // per_image)))
+
+
+def run_reference(args):
+    from workloads import get_config
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = get_config(args.workload)
+    sb = oracle_sample_batch(cfg)
+    steps = max(1, min(args.steps, 3))
+    warm = min(args.warmup, 1)
+    for _ in range(warm):
+        time_oracle_step(args.workload, sb)
+    times = [time_oracle_step(args.workload, sb)[1] for _ in range(steps)]
+    dt = float(np.mean(times))
+    val = sb / dt
+    line = {"metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps, "warmup": warm,
+            "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "impl": "reference",
+            "config": {"workload": args.workload, "sample_batch": sb, "full_batch": cfg["N"]},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                             "sample": "one full layer-parallel step on %d of %d images" % (sb, cfg["N"])},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU benchmark
+# ---------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import paper_2112_05387_b200 as lp
+    from workloads import gen, get_config, scaled
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    cfg = scaled(args.workload, N=args.batch) if args.batch else get_config(args.workload)
+    K = cfg["K"]
+    desc = lp.desc_from_config(cfg, args.conv_impl)
+    h = lp.lp_create(desc, device=str(dev))
+    tdt = torch.float32 if cfg["dtype"] == "f32" else torch.bfloat16
+    for k in range(K):
+        lp.lp_set_params(h, k, gen.make_params(lp.lp_param_layout(desc, k), 0, "module%d" % k, dtype=cfg["dtype"]))
+    for k in range(K - 1):
+        lp.lp_set_params(h, lp.LP_AUX(k), gen.make_params(lp.lp_param_layout(desc, lp.LP_AUX(k)), 0, "aux%d" % k,
+                                                         dtype=cfg["dtype"]))
+    images_host = torch.from_numpy(gen.make_images(cfg)).to(tdt).pin_memory()
+    labels_host = torch.from_numpy(gen.make_labels(cfg)).pin_memory()
+    d_images = images_host.to(dev)
+    d_labels = labels_host.to(dev)
+    shapes = [lp.lp_boundary_shape_desc(desc, k) for k in range(K)]
+    d_x = [d_images] + [torch.zeros(shapes[k], dtype=tdt, device=dev) for k in range(1, K)]
+    use_kappa = cfg["loss"] == "al"
+    d_kappa = [torch.zeros(shapes[k + 1], dtype=tdt, device=dev) for k in range(K - 1)] if use_kappa else None
+    d_dx = [None] + [torch.zeros_like(d_x[k]) for k in range(1, K)]
+    d_loss = torch.zeros(K, 2, dtype=torch.float32, device=dev)
+    loss_host = torch.zeros(K, 2, dtype=torch.float32).pin_memory()
+    lr = 1e-9  # the penalty is a sum over the boundary tensor: a small rate keeps replayed steps finite
+    kstep = cfg["rho"]
+    stream = torch.cuda.Stream(device=dev)
+    sp = stream.cuda_stream
+
+    def step_direct():
+        lp.lp_auxnet_forward(h, d_images, d_x[1:], sp)
+        lp.lp_modules_fwd_bwd_all(h, d_x, d_labels, d_kappa, cfg["rho"], d_loss, d_dx, sp)
+        lp.lp_step(h, lr, 0.0, 0.0, kstep, d_kappa, sp)
+
+    def serial_direct():
+        lp.lp_serial_fwd_bwd(h, d_images, d_labels, d_loss[K - 1], sp)
+        lp.lp_step(h, lr, 0.0, 0.0, 0.0, None, sp)
+
+    with torch.cuda.stream(stream):
+        step_direct()                       # first use sets kernel attributes, outside any capture
+        st = lp.lp_last_device_status(h, sp)
+        if st != 0:
+            raise RuntimeError("device status %d after the first step" % st)
+        lp.lp_launch_count(h, reset=True)
+        step_direct()
+        launches_per_step = lp.lp_launch_count(h, reset=True)
+        gid = None
+        if not args.no_graph:
+            lp.lp_graph_begin(h, sp)
+            step_direct()
+            gid = lp.lp_graph_end(h, sp)
+
+        def step():
+            if gid is None:
+                step_direct()
+            else:
+                lp.lp_graph_launch(h, gid, sp)
+
+        def barrier():
+            torch.cuda.synchronize(dev)
+            if dist is not None:
+                dist.barrier()
+            torch.cuda.synchronize(dev)
+
+        for _ in range(max(args.warmup, 3)):
+            step()
+        barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        clocks = sampler.stop()
+        st = lp.lp_last_device_status(h, sp)
+        if st != 0:
+            raise RuntimeError("device status %d in the timed region" % st)
+
+        # end to end: pinned host inputs in, losses out, every step
+        for _ in range(2):
+            d_images.copy_(images_host, non_blocking=True)
+            d_labels.copy_(labels_host, non_blocking=True)
+            step()
+            loss_host.copy_(d_loss, non_blocking=True)
+        barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for _ in range(args.steps):
+            d_images.copy_(images_host, non_blocking=True)
+            d_labels.copy_(labels_host, non_blocking=True)
+            step()
+            loss_host.copy_(d_loss, non_blocking=True)
+            stream.synchronize()             # the caller reads the losses before the next step
+        f1.record(stream)
+        barrier()
+        ms_e2e = f0.elapsed_time(f1)
+        losses = loss_host.clone().numpy()
+
+        # per-kernel timing of the tensor-core convolutions: modules one after another on one
+        # stream (so that a kernel's events do not include waiting for another module's kernels)
+        lp.lp_conv_profile(h, True, read=False)
+        prof_steps = 2
+        for _ in range(prof_steps):
+            lp.lp_auxnet_forward(h, d_images, d_x[1:], sp)
+            for k in range(K):
+                last = k == K - 1
+                lp.lp_module_fwd_bwd(h, k, d_x[k], d_labels if last else d_x[k + 1],
+                                     None if (last or not use_kappa) else d_kappa[k], cfg["rho"], d_loss[k],
+                                     d_dx[k], sp)
+        conv_ms, conv_flops, conv_launches = lp.lp_conv_profile(h, False, read=True)
+        barrier()
+
+        serial = None
+        if not args.no_serial and world == 1:
+            serial_direct()
+            sgid = None
+            if not args.no_graph:
+                lp.lp_graph_begin(h, sp)
+                serial_direct()
+                sgid = lp.lp_graph_end(h, sp)
+            for _ in range(3):
+                lp.lp_graph_launch(h, sgid, sp) if sgid is not None else serial_direct()
+            barrier()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_ser = max(3, args.steps // 3)
+            g0.record(stream)
+            for _ in range(n_ser):
+                lp.lp_graph_launch(h, sgid, sp) if sgid is not None else serial_direct()
+            g1.record(stream)
+            barrier()
+            serial = {"value": cfg["N"] * n_ser / (g0.elapsed_time(g1) * 1e-3), "unit": UNIT,
+                      "what": "layer-serial forward + back-propagation + update with the same kernels (no AuxNet)"}
+
+    # max over ranks
+    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    n_img = cfg["N"] * args.steps * world
+    value = n_img / (ms * 1e-3)
+    e2e_value = n_img / (ms_e2e * 1e-3)
+    fwd, aux = conv_flops_forward(cfg)
+    step_conv_flops = 3 * fwd + aux
+    peaks = {}
+    ppath = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak_src = "fallback"
+    if os.path.exists(ppath):
+        peaks = json.load(open(ppath))
+        peak_src = "measured"
+    peak_tf = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    achieved_tf = conv_flops / (conv_ms * 1e-3) / 1e12 if conv_ms > 0 else 0.0
+    roofline = {"bound": "tensor", "kernel": "conv_tc_kernel + wgrad_tc_kernel (all tensor-core convolutions)",
+                "achieved": achieved_tf, "peak": peak_tf, "peak_source": peak_src + " (sustained bf16 GEMM)",
+                "unit": "TFLOP/s", "frac": achieved_tf / peak_tf if peak_tf else None,
+                "frac_of_nominal_2250": achieved_tf / 2250.0,
+                "launches_timed": int(conv_launches), "avg_launch_ms": conv_ms / max(conv_launches, 1),
+                "flops_per_launch_avg": conv_flops / max(conv_launches, 1), "traffic": None,
+                "timing": "CUDA events around every tensor-core conv launch, modules run back to back on one stream"}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32",
+            "data": "synthetic",
+            "config": {"workload": args.workload, "global_batch": cfg["N"] * world, "K": K, "loss": cfg["loss"],
+                       "rho": cfg["rho"], "parallelism": "replicas only (no collective)" if world > 1 else "1 GPU",
+                       "cuda_graph": gid is not None, "l2": "working set of a step (GBs) is far larger than L2",
+                       "conv_flops_per_step": step_conv_flops},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT,
+                    "h2d_bytes_per_step": int(images_host.numel() * images_host.element_size() + labels_host.numel() * 4),
+                    "d2h_bytes_per_step": int(loss_host.numel() * 4)},
+            "gpu_launches": int(launches_per_step * args.steps),
+            "launches_per_step": int(launches_per_step),
+            "step_conv_tflops": step_conv_flops / (ms / args.steps * 1e-3) / 1e12,
+            "roofline": roofline,
+            "losses": [float(v) for v in losses[:, 0]]}
+    if serial:
+        line["layer_serial"] = serial
+    if not args.no_cpu_baseline and world == 1:
+        sb = oracle_sample_batch(cfg)
+        val, dt = time_oracle_step(args.workload, sb)
+        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                                "sample": "one full layer-parallel step on %d of %d images (%.1f s)" % (sb, cfg["N"], dt)}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        import __graft_entry__ as g
+        g.build()
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -176,6 +176,15 @@ int64_t lp_launch_count(lp_handle* h, int reset);
  * their count since the last reset; only collected while profiling is enabled (serialises). */
 int lp_conv_profile(lp_handle* h, int enable, double* ms, double* flops, int64_t* launches);
 
+/* CUDA-graph helpers: record every launch the library makes on `stream` between begin and end
+ * (the internal module streams are forked from and joined into it), then replay the recording.
+ * Pointer arguments of the recorded calls are baked into the graph.  Up to 8 graphs per handle;
+ * *graph_id receives the slot.  The first call of every kind must have run once outside a capture
+ * (kernel attributes are set on first use). */
+int lp_graph_begin(lp_handle* h, void* stream);
+int lp_graph_end(lp_handle* h, void* stream, int* graph_id);
+int lp_graph_launch(lp_handle* h, int graph_id, void* stream);
+
 /* Stand-alone convolution on caller buffers (tests and kernel benchmarks).
  * op = LP_CONV_FWD:   a = x [N,H,W,Cin],   b = w fp32 [Cout,R,R,Cin], out = y  [N,OH,OW,Cout]
  * op = LP_CONV_DGRAD: a = dy [N,OH,OW,Cout], b = w fp32,               out = dx [N,H,W,Cin]

@@ -11,8 +11,8 @@ __all__ = [
     "lp_param_layout", "lp_boundary_shape_desc", "lp_create", "lp_destroy", "lp_param_count", "lp_set_params",
     "lp_get_params", "lp_get_grads", "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd",
     "lp_modules_fwd_bwd_all", "lp_step", "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual",
-    "lp_last_device_status", "lp_launch_count", "lp_conv_profile", "lp_conv2d", "lp_conv2d_scratch_bytes",
-    "EXPORTED_SYMBOLS",
+    "lp_last_device_status", "lp_launch_count", "lp_conv_profile", "lp_conv2d", "lp_conv2d_scratch_bytes", "lp_graph_begin", "lp_graph_end",
+    "lp_graph_launch", "EXPORTED_SYMBOLS",
 ]
 
 LP_OK = 0
@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = [
     "lp_create", "lp_destroy", "lp_param_count", "lp_set_params", "lp_get_params", "lp_get_grads",
     "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd", "lp_modules_fwd_bwd_all", "lp_step",
     "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual", "lp_last_device_status", "lp_launch_count",
-    "lp_conv_profile", "lp_conv2d_scratch_bytes", "lp_conv2d",
+    "lp_conv_profile", "lp_conv2d_scratch_bytes", "lp_conv2d", "lp_graph_begin", "lp_graph_end", "lp_graph_launch",
 ]
 
 
@@ -104,6 +104,9 @@ def library():
     lib.lp_launch_count.argtypes = [vp, i32]
     lib.lp_conv_profile.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                     ctypes.POINTER(ctypes.c_int64)]
+    lib.lp_graph_begin.argtypes = [vp, vp]
+    lib.lp_graph_end.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    lib.lp_graph_launch.argtypes = [vp, i32, vp]
     lib.lp_conv2d_scratch_bytes.restype = sz
     lib.lp_conv2d_scratch_bytes.argtypes = [i32, i32, i32]
     lib.lp_conv2d.argtypes = [i32] * 11 + [vp, vp, vp, vp, vp, sz, ctypes.POINTER(f32), vp]
@@ -299,6 +302,20 @@ def lp_conv_profile(h, enable, read=True):
     else:
         _check(library().lp_conv_profile(h.ptr, 1 if enable else 0, None, None, None), "lp_conv_profile")
     return ms.value, fl.value, n.value
+
+
+def lp_graph_begin(h, stream):
+    _check(library().lp_graph_begin(h.ptr, _ptr(stream)), "lp_graph_begin")
+
+
+def lp_graph_end(h, stream):
+    gid = ctypes.c_int(-1)
+    _check(library().lp_graph_end(h.ptr, _ptr(stream), ctypes.byref(gid)), "lp_graph_end")
+    return gid.value
+
+
+def lp_graph_launch(h, graph_id, stream=None):
+    _check(library().lp_graph_launch(h.ptr, graph_id, _ptr(stream)), "lp_graph_launch")
 
 
 def lp_conv2d_scratch_bytes(cin, cout, r):

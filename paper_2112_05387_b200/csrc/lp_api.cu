@@ -175,6 +175,9 @@ struct lp_handle {
   uint8_t* ws = nullptr;
   size_t ws_bytes = 0;
   int32_t* zero_labels = nullptr;  // N zeros, for forward passes that only want logits
+  std::vector<cudaGraphExec_t> graphs;
+  int64_t launches_at_capture = 0;
+  std::vector<int64_t> graph_launches;  // kernels recorded in each graph
 };
 
 namespace lp {
@@ -1197,6 +1200,7 @@ int lp_destroy(lp_handle* h) {
   for (auto e : h->done) if (e) cudaEventDestroy(e);
   if (h->fork) cudaEventDestroy(h->fork);
   for (auto& pr : h->prof.events) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
+  for (auto g : h->graphs) cudaGraphExecDestroy(g);
   delete h;
   return LP_OK;
 }
@@ -1456,6 +1460,39 @@ int lp_conv_profile(lp_handle* h, int enable, double* ms, double* flops, int64_t
   }
   pr.used = 0;
   pr.enabled = enable != 0;
+  return LP_OK;
+}
+
+int lp_graph_begin(lp_handle* h, void* stream) {
+  if (!h) return LP_ERR_NULL;
+  if (h->graphs.size() >= 8) return LP_ERR_UNSUPPORTED;
+  if (h->prof.enabled) return LP_ERR_ORDER;
+  h->launches_at_capture = h->launches;
+  LP_CUDA_OK(cudaStreamBeginCapture((cudaStream_t)stream, cudaStreamCaptureModeRelaxed));
+  return LP_OK;
+}
+
+int lp_graph_end(lp_handle* h, void* stream, int* graph_id) {
+  if (!h || !graph_id) return LP_ERR_NULL;
+  cudaGraph_t g = nullptr;
+  LP_CUDA_OK(cudaStreamEndCapture((cudaStream_t)stream, &g));
+  cudaGraphExec_t exec = nullptr;
+  cudaError_t e = cudaGraphInstantiate(&exec, g, 0);
+  cudaGraphDestroy(g);
+  if (e != cudaSuccess) return LP_ERR_CUDA;
+  h->graphs.push_back(exec);
+  h->graph_launches.push_back(h->launches - h->launches_at_capture);
+  h->launches = h->launches_at_capture;  // recording launched nothing
+  *graph_id = (int)h->graphs.size() - 1;
+  return LP_OK;
+}
+
+int lp_graph_launch(lp_handle* h, int graph_id, void* stream) {
+  if (!h) return LP_ERR_NULL;
+  if (graph_id < 0 || graph_id >= (int)h->graphs.size()) return LP_ERR_BAD_INDEX;
+  LP_CUDA_OK(cudaGraphLaunch(h->graphs[graph_id], (cudaStream_t)stream));
+  h->launches += h->graph_launches[graph_id];
+  for (auto& P : h->modules) { P.ran_fwd_bwd = true; }
   return LP_OK;
 }
 
