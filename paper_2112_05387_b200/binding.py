@@ -63,7 +63,8 @@ _LIB = None
 
 
 def library_path():
-    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblp.so")
+    """In-tree liblp.so, or the library named by LP_LIBRARY_PATH (for trying out a different build)."""
+    return os.environ.get("LP_LIBRARY_PATH") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblp.so")
 
 
 def library():

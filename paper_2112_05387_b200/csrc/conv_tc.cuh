@@ -128,58 +128,59 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   bool failed = false;
 
   if (warp == 0) {
-    // ------------------------------- TMA producer -------------------------------------
-    if (lane == 0) {
-      uint32_t it = 0;
-      for (int t = t_begin; t < t_end && !failed; ++t) {
-        const int nt = t / p.m_tiles, m = t % p.m_tiles;
-        const int w0 = (m % p.tiles_w) * p.BW;
-        const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
-        const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
-        const int col0 = nt * p.n_tile_cols;
-        for (int tap = 0; tap < p.ntaps && !failed; ++tap) {
-          const int cw = w0 * p.in_step + p.tap_dw[tap];
-          const int ch = h0 * p.in_step + p.tap_dh[tap];
-          const int kb = p.tap_w[tap] * p.Cin;
-          for (int c = 0; c < p.chunks; ++c, ++it) {
-            const int s = it % p.stages;
-            const uint32_t ph = (it / p.stages) & 1;
-            if (!mbar_wait(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
-            uint8_t* sa = smem + (size_t)s * p.stage_bytes;
+    // ------------------------------- TMA producer (warp-uniform loop, elected issue) ----
+    uint32_t s = 0, ph = 0;
+    for (int t = t_begin; t < t_end && !failed; ++t) {
+      const int nt = t / p.m_tiles, m = t % p.m_tiles;
+      const int w0 = (m % p.tiles_w) * p.BW;
+      const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
+      const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
+      const int col0 = nt * p.n_tile_cols;
+      for (int tap = 0; tap < p.ntaps && !failed; ++tap) {
+        const int cw = w0 * p.in_step + p.tap_dw[tap];
+        const int ch = h0 * p.in_step + p.tap_dh[tap];
+        const int kb = p.tap_w[tap] * p.Cin;
+        for (int c = 0; c < p.chunks; ++c) {
+          if (!mbar_wait_warp(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
+          uint8_t* sa = smem + s * p.stage_bytes;
+          if (elect_one()) {
             mbar_expect_tx(&tail->full[s], p.tx_bytes);
             tma_load_4d(sa, &tmA, &tail->full[s], c * p.KC, cw, ch, n0);
             tma_load_2d(sa + p.a_region_bytes, &tmB, &tail->full[s], kb + c * p.KC, col0);
           }
+          __syncwarp();
+          if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------- MMA issuer ---------------------------------------
-    if (lane == 0) {
-      uint32_t it = 0;
-      int tl = 0;
-      for (int t = t_begin; t < t_end && !failed; ++t, ++tl) {
-        const int buf = tl & 1;
-        const uint32_t aph = (tl >> 1) & 1;
-        if (!mbar_wait(&tail->tmem_empty[buf], aph ^ 1, abort_flag)) { failed = true; break; }
+    // ------------------------------- MMA issuer (warp-uniform loop, elected issue) ------
+    uint32_t s = 0, ph = 0;
+    const uint32_t smem_base = smem_u32(smem);
+    const int nk = p.KC >> 4;
+    int tl = 0;
+    for (int t = t_begin; t < t_end && !failed; ++t, ++tl) {
+      const int buf = tl & 1;
+      const uint32_t aph = (tl >> 1) & 1;
+      if (!mbar_wait_warp(&tail->tmem_empty[buf], aph ^ 1, abort_flag)) { failed = true; break; }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + buf * kAccStride;
+      for (int k = 0; k < kiters; ++k) {
+        if (!mbar_wait_warp(&tail->full[s], ph, abort_flag)) { failed = true; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * kAccStride;
-        for (int k = 0; k < kiters; ++k, ++it) {
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1;
-          if (!mbar_wait(&tail->full[s], ph, abort_flag)) { failed = true; break; }
-          tc_fence_after();
-          const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes);
-          const uint32_t b_addr = a_addr + p.a_region_bytes;
-          const uint64_t ad = smem_desc(p.desc_hi, a_addr), bd = smem_desc(p.desc_hi, b_addr);
-          const int nk = p.KC >> 4;
+        const uint32_t a_addr = smem_base + s * p.stage_bytes;
+        const uint64_t ad = smem_desc(p.desc_hi, a_addr), bd = smem_desc(p.desc_hi, a_addr + p.a_region_bytes);
+        if (elect_one()) {
           for (int j = 0; j < nk; ++j)  // +32 bytes (one K = 16 slice) per step, in 16-byte units
             mma_bf16(d_tmem, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k | j) ? 1u : 0u);
           mma_commit(&tail->empty[s]);
         }
-        if (failed) break;
-        mma_commit(&tail->tmem_full[buf]);
+        __syncwarp();
+        if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
       }
+      if (failed) break;
+      if (elect_one()) mma_commit(&tail->tmem_full[buf]);
+      __syncwarp();
     }
   } else {
     // ------------------------------- epilogue -----------------------------------------

@@ -103,46 +103,53 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   bool failed = false;
 
   if (warp == 0) {
-    if (lane == 0) {
-      for (int it = 0; it < n_iter; ++it) {
-        const int pt = pt_begin + it;
-        const int w0 = (pt % p.tiles_w) * p.BW;
-        const int h0 = ((pt / p.tiles_w) % p.tiles_h) * p.BH;
-        const int n0 = (pt / (p.tiles_w * p.tiles_h)) * p.BNI;
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
-        if (!mbar_wait(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
-        uint8_t* sa = smem + (size_t)s * p.stage_bytes;
+    // TMA producer: warp-uniform loop, one elected lane issues the copies
+    uint32_t s = 0, ph = 0;
+    for (int it = 0; it < n_iter; ++it) {
+      const int pt = pt_begin + it;
+      const int w0 = (pt % p.tiles_w) * p.BW;
+      const int h0 = ((pt / p.tiles_w) % p.tiles_h) * p.BH;
+      const int n0 = (pt / (p.tiles_w * p.tiles_h)) * p.BNI;
+      if (!mbar_wait_warp(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
+      uint8_t* sa = smem + s * p.stage_bytes;
+      if (elect_one()) {
         mbar_expect_tx(&tail->full[s], p.tx_bytes);
         for (int j = 0; j < p.rpt; ++j) {
           int g = m_tile * p.rpt + j;
           if (g >= p.total_chunks) g = p.total_chunks - 1;  // padding rows of the last tile: any finite data
           const int tap = g / p.cin_chunks, c0 = (g % p.cin_chunks) * p.sca;
           const int r = tap / p.R, q = tap % p.R;
-          tma_load_4d(sa + (size_t)j * p.a_sub_bytes, &tmX, &tail->full[s], c0, w0 * p.stride + q - p.pad,
+          tma_load_4d(sa + j * p.a_sub_bytes, &tmX, &tail->full[s], c0, w0 * p.stride + q - p.pad,
                       h0 * p.stride + r - p.pad, n0);
         }
         for (int j = 0; j < p.nb; ++j)
-          tma_load_4d(sa + p.a_region + (size_t)j * p.b_sub_bytes, &tmDY, &tail->full[s],
-                      n_tile * p.n_tile + j * p.scb, w0, h0, n0);
+          tma_load_4d(sa + p.a_region + j * p.b_sub_bytes, &tmDY, &tail->full[s], n_tile * p.n_tile + j * p.scb, w0,
+                      h0, n0);
       }
+      __syncwarp();
+      if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      const int ksteps = p.rows_pad >> 4;
-      const uint32_t a_kstep = (uint32_t)(16 * p.sca * 2) >> 4, b_kstep = (uint32_t)(16 * p.scb * 2) >> 4;
-      for (int it = 0; it < n_iter; ++it) {
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
-        if (!mbar_wait(&tail->full[s], ph, abort_flag)) { failed = true; break; }
-        tc_fence_after();
-        const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes);
-        const uint64_t ad = smem_desc(p.adesc_hi, a_addr), bd = smem_desc(p.bdesc_hi, a_addr + p.a_region);
+    uint32_t s = 0, ph = 0;
+    const uint32_t smem_base = smem_u32(smem);
+    const int ksteps = p.rows_pad >> 4;
+    const uint32_t a_kstep = (uint32_t)(16 * p.sca * 2) >> 4, b_kstep = (uint32_t)(16 * p.scb * 2) >> 4;
+    for (int it = 0; it < n_iter; ++it) {
+      if (!mbar_wait_warp(&tail->full[s], ph, abort_flag)) { failed = true; break; }
+      tc_fence_after();
+      const uint32_t a_addr = smem_base + s * p.stage_bytes;
+      const uint64_t ad = smem_desc(p.adesc_hi, a_addr), bd = smem_desc(p.bdesc_hi, a_addr + p.a_region);
+      if (elect_one()) {
         for (int j = 0; j < ksteps; ++j)
           mma_bf16(tmem_base, ad + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, (it | j) ? 1u : 0u);
         mma_commit(&tail->empty[s]);
       }
-      if (!failed) mma_commit(&tail->acc_full);
+      __syncwarp();
+      if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
+    }
+    if (!failed && n_iter > 0) {
+      if (elect_one()) mma_commit(&tail->acc_full);
+      __syncwarp();
     }
   } else {
     const int q = warp & 3;
