@@ -212,6 +212,23 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------------------
+# aggregation over replicas (the only cross-rank step: no data-path collective)
+# ---------------------------------------------------------------------------------------------
+def max_over_ranks(values, dist=None, device=None):
+    """Element-wise maximum of a list of per-rank scalars over all ranks (identity without dist)."""
+    import torch
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_images_per_s(batch_per_rank, steps, world, ms_max_over_ranks):
+    """Every rank processes `batch_per_rank` images per step; the job is as slow as its slowest rank."""
+    return batch_per_rank * steps * world / (ms_max_over_ranks * 1e-3)
+
+
+# ---------------------------------------------------------------------------------------------
 # GPU benchmark
 # ---------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -363,18 +380,14 @@ def run_ours(args):
                       "what": "layer-serial forward + back-propagation + update with the same kernels (no AuxNet)"}
 
     # max over ranks
-    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], dist, dev)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    n_img = cfg["N"] * args.steps * world
-    value = n_img / (ms * 1e-3)
-    e2e_value = n_img / (ms_e2e * 1e-3)
+    value = whole_job_images_per_s(cfg["N"], args.steps, world, ms)
+    e2e_value = whole_job_images_per_s(cfg["N"], args.steps, world, ms_e2e)
     fwd, aux = conv_flops_forward(cfg)
     step_conv_flops = 3 * fwd + aux
     peaks = {}

@@ -1,0 +1,105 @@
+"""Full-size parity in the launch configuration the benchmark times (WRN-28-10, N = 128, grouped call).
+
+The oracle cannot run the whole step at this size in seconds, so the test checks properties that hold
+at any size, and compares ONE module against the oracle element by element."""
+import numpy as np
+import pytest
+
+from harness import GpuRun, noisy_bf16_store, oracle_modules, per_tensor_errors, rel_err, to_host
+from oracle import lp_oracle as O
+from workloads import gen, get_config
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def wrn():
+    cfg = get_config("wrn28_10")
+    cfg["loss"] = "al"                      # exercise the multiplier path; kappa = 0 must equal the penalty
+    run = GpuRun(cfg, kappa_std=0.0)
+    run.auxnet()                            # boundaries from the GPU AuxNet: only properties are checked on them
+    return run
+
+
+def test_kappa_zero_equals_penalty_and_loss_is_linear_in_kappa(wrn):
+    run, torch = wrn, wrn.torch
+    K = run.net.K
+    for t in run.d_kappa:
+        t.zero_()
+    g_al0 = run.fwd_bwd_all()
+    loss_al0 = run.d_loss.cpu().numpy().copy()
+    run.use_kappa = False
+    g_pen = run.fwd_bwd_all()
+    loss_pen = run.d_loss.cpu().numpy().copy()
+    run.use_kappa = True
+    np.testing.assert_allclose(loss_al0, loss_pen, rtol=1e-6)
+    for k in range(K):
+        assert rel_err(g_al0[k], g_pen[k]) < 1e-4      # split-K atomics reorder fp32 sums, nothing else differs
+    # L_AL - L_P = <kappa, r>
+    r = [torch.zeros_like(run.d_x[k + 1]) for k in range(K - 1)]
+    for k in range(K - 1):
+        run.lp.lp_get_residual(run.h, k, r[k], None)
+        run.d_kappa[k].copy_((0.05 * torch.randn(run.d_kappa[k].shape, device="cuda:0",
+                                                 generator=torch.Generator(device="cuda:0").manual_seed(k))).to(torch.bfloat16))
+    run.fwd_bwd_all()
+    loss_al = run.d_loss.cpu().numpy().copy()
+    for k in range(K - 1):
+        inner = float((run.d_kappa[k].double() * r[k].double()).sum())
+        assert abs((loss_al[k, 0] - loss_pen[k, 0]) - inner) < 2e-2 * abs(inner) + 1e-6 * abs(loss_pen[k, 0])
+        np.testing.assert_allclose(loss_al[k, 1], loss_pen[k, 1], rtol=1e-6)
+
+
+def test_multiplier_step_rho_gives_terminal_adjoint(wrn):
+    run, torch = wrn, wrn.torch
+    K = run.net.K
+    run.fwd_bwd_all()
+    seeds = [torch.zeros_like(run.d_x[k + 1]) for k in range(K - 1)]
+    for k in range(K - 1):
+        run.lp.lp_get_residual(run.h, k, None, seeds[k])
+    run.cfg["lr"] = 0.0
+    run.step(kappa_step=run.cfg["rho"])
+    for k in range(K - 1):
+        assert rel_err(to_host(run.d_kappa[k]), to_host(seeds[k])) < 1e-2
+
+
+def test_scale_invariance_of_convs_feeding_a_batch_norm(wrn):
+    """<w, dL/dw> = 0 for a convolution whose output goes straight into a batch norm (eps -> 0)."""
+    run = wrn
+    run.fwd_bwd_all()
+    desc = run.desc
+    for k in range(run.net.K):
+        p = run.lp.lp_get_params(run.h, k).astype(np.float64)
+        g = run.lp.lp_get_grads(run.h, k).astype(np.float64)
+        off = 0
+        for name, kind, shape in run.lp.lp_param_layout(desc, k):
+            n = int(np.prod(shape))
+            if name.endswith("conv1.w"):
+                w, d = p[off:off + n], g[off:off + n]
+                assert abs(w @ d) < 2e-2 * np.linalg.norm(w) * np.linalg.norm(d), (k, name)
+            off += n
+
+
+def test_one_module_against_the_oracle_at_full_size(wrn):
+    run = wrn
+    net, cfg = run.net, run.cfg
+    k = 3                                          # last module: 3 blocks at 640 channels + head + cross-entropy
+    x3 = gen.round_bf16(gen.normal(7, "x3", net.boundary[3]))
+    run.d_x[3].copy_(run.torch.from_numpy(x3).to("cuda:0").to(run.torch.bfloat16))
+    run.fwd_bwd_all()
+    grads = run.lp.lp_get_grads(run.h, k)
+    loss = run.d_loss.cpu().numpy()
+
+    def oracle(store):
+        net.store = store
+        res = O.module_fwd_bwd(net, k, run.mods[k], x3.astype(np.float64), run.labels, None, cfg["rho"])
+        net.store = None
+        return res
+    ref = oracle(gen.round_bf16)
+    floor = oracle(noisy_bf16_store())
+    assert abs(loss[k, 0] - ref["loss"]) < 2e-2 * abs(ref["loss"])
+    errs = per_tensor_errors(net, k, grads, ref["grads"])
+    fl = per_tensor_errors(net, k, floor["grads"], ref["grads"])
+    bad = {n: (e, fl[n]) for n, e in errs.items() if not e < max(2e-2, 4 * fl[n])}
+    assert not bad, bad
+    e = rel_err(to_host(run.d_dx[k]), ref["dx"])
+    assert e < max(2e-2, 4 * rel_err(floor["dx"], ref["dx"])), e
