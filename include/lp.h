@@ -197,6 +197,33 @@ int lp_conv2d(int op, int dtype, int impl, int N, int H, int W, int Cin, int Cou
               int stride, int pad, const void* a, const void* b, void* out, double* stats,
               void* scratch, size_t scratch_bytes, float* elapsed_ms, void* stream);
 
+/*
+ * Forward convolution for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of lp_conv2d(LP_CONV_FWD, LP_BF16, tensor cores).)
+ *
+ * Some callers may not call cudaMalloc at all: code that runs inside a memory pool it does not
+ * own, plug-ins whose host forbids driver allocations after start-up, or a latency-critical loop
+ * in which an allocation would synchronise the device.  lp_conv2d needs a scratch buffer from
+ * its caller (bf16 operand copy of the weights, an error word, a small table); this entry point
+ * keeps that scratch in a fixed array inside the library instead, LP_NOALLOC_SCRATCH_BYTES long,
+ * which every GPU that loads the library holds until the process exits.  It calls no cudaMalloc,
+ * cudaFree or allocating library routine; the caller passes only inputs and outputs.
+ *
+ *   x: device bf16 [N,H,W,Cin]; w: device fp32 [Cout,R,R,Cin]; y: device bf16 [N,OH,OW,Cout].
+ *   Same shape rules as the tensor-core path of lp_conv2d (Cin, Cout multiples of 8, R in {1,3},
+ *   stride in {1,2}); LP_ERR_UNSUPPORTED otherwise.  The call is synchronous on `stream`.
+ *   LP_ERR_SIZE ("size mismatch") if 2*Cout*R*R*Cin + 1024 bytes exceed the array.
+ *
+ * The first call on a device looks up the array's device address (once per device, with that
+ * device current) and sets kernel attributes: make it before any stream capture.  All calls share
+ * the one array, which keeps the previous call's contents; the words that must start at zero are
+ * cleared by each call.  Two calls that overlap on the GPU (different streams or threads) race on
+ * the array: serialise them.
+ */
+#define LP_NOALLOC_SCRATCH_BYTES (8u << 20)
+int lp_conv2d_fwd_noalloc(int N, int H, int W, int Cin, int Cout, int R, int stride, int pad, const void* x,
+                          const float* w, void* y, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

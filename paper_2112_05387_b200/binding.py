@@ -12,7 +12,7 @@ __all__ = [
     "lp_get_params", "lp_get_grads", "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd",
     "lp_modules_fwd_bwd_all", "lp_step", "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual",
     "lp_last_device_status", "lp_launch_count", "lp_conv_profile", "lp_conv2d", "lp_conv2d_scratch_bytes", "lp_graph_begin", "lp_graph_end",
-    "lp_graph_launch", "EXPORTED_SYMBOLS",
+    "lp_graph_launch", "lp_conv2d_fwd_noalloc", "LP_NOALLOC_SCRATCH_BYTES", "EXPORTED_SYMBOLS",
 ]
 
 LP_OK = 0
@@ -20,6 +20,7 @@ LP_F32, LP_BF16 = 0, 1
 LP_CONV_IMPL_AUTO, LP_CONV_IMPL_SIMT, LP_CONV_IMPL_TENSOR = 0, 1, 2
 LP_CONV_FWD, LP_CONV_DGRAD, LP_CONV_WGRAD = 0, 1, 2
 LP_MAX_STAGES, LP_MAX_MODULES = 8, 16
+LP_NOALLOC_SCRATCH_BYTES = 8 << 20
 _KINDS = ["conv_w", "bn_gamma", "bn_beta", "fc_w", "fc_b"]
 
 EXPORTED_SYMBOLS = [
@@ -28,6 +29,7 @@ EXPORTED_SYMBOLS = [
     "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd", "lp_modules_fwd_bwd_all", "lp_step",
     "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual", "lp_last_device_status", "lp_launch_count",
     "lp_conv_profile", "lp_conv2d_scratch_bytes", "lp_conv2d", "lp_graph_begin", "lp_graph_end", "lp_graph_launch",
+    "lp_conv2d_fwd_noalloc",
 ]
 
 
@@ -108,6 +110,7 @@ def library():
     lib.lp_graph_begin.argtypes = [vp, vp]
     lib.lp_graph_end.argtypes = [vp, vp, ctypes.POINTER(i32)]
     lib.lp_graph_launch.argtypes = [vp, i32, vp]
+    lib.lp_conv2d_fwd_noalloc.argtypes = [i32] * 8 + [vp, vp, vp, vp]
     lib.lp_conv2d_scratch_bytes.restype = sz
     lib.lp_conv2d_scratch_bytes.argtypes = [i32, i32, i32]
     lib.lp_conv2d.argtypes = [i32] * 11 + [vp, vp, vp, vp, vp, sz, ctypes.POINTER(f32), vp]
@@ -331,3 +334,9 @@ def lp_conv2d(op, dtype, impl, N, H, W, Cin, Cout, R, stride, pad, a, b, out, st
                              _ptr(stats), _ptr(scratch), scratch_bytes, ctypes.byref(ms) if timed else None,
                              _ptr(stream))
     return st, (ms.value if timed else None)
+
+
+def lp_conv2d_fwd_noalloc(N, H, W, Cin, Cout, R, stride, pad, x, w, y, stream=None):
+    """Forward convolution whose scratch is a fixed array inside the library: for callers that may
+    not allocate device memory.  Returns the status (0 = ok); see include/lp.h for the limits."""
+    return library().lp_conv2d_fwd_noalloc(N, H, W, Cin, Cout, R, stride, pad, _ptr(x), _ptr(w), _ptr(y), _ptr(stream))

@@ -1582,4 +1582,58 @@ int lp_conv2d(int op, int dtype, int impl, int N, int H, int W, int Cin, int Cou
   return e ? LP_ERR_DEVICE_TIMEOUT : LP_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Forward convolution without any caller- or library-side allocation: the scratch that lp_conv2d
+// takes from its caller lives in this fixed device array instead.  In host code the array's name
+// is only a handle: its device address is looked up once per device with cudaGetSymbolAddress.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[LP_NOALLOC_SCRATCH_BYTES];
+static void* g_noalloc_ptr[64] = {nullptr};
+
+int lp_conv2d_fwd_noalloc(int N, int H, int W, int Cin, int Cout, int R, int stride, int pad, const void* x,
+                          const float* w, void* y, void* stream) {
+  if (!x || !w || !y) return LP_ERR_NULL;
+  if (N < 1 || H < 1 || W < 1 || Cin < 1 || Cout < 1 || R < 1 || stride < 1 || pad < 0) return LP_ERR_SIZE;
+  if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return LP_ERR_ALIGN;
+  const size_t n = (size_t)Cin * Cout * R * R;
+  const size_t need = 256 + align_up(n * 2, 256) + 256;  // error word | bf16 weights | one-entry table
+  if (need > (size_t)LP_NOALLOC_SCRATCH_BYTES) return LP_ERR_SIZE;
+  int rc = g_dev.init();
+  if (rc != LP_OK) return rc;
+  int dev = 0;
+  LP_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return LP_ERR_UNSUPPORTED;
+  if (!g_noalloc_ptr[dev]) {  // set-up, once per device, with that device current
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return LP_ERR_CUDA;
+    g_noalloc_ptr[dev] = ptr;
+  }
+  uint8_t* sp = (uint8_t*)g_noalloc_ptr[dev];
+  cudaStream_t st = (cudaStream_t)stream;
+  ConvDef c;
+  c.cin = Cin; c.cout = Cout; c.R = R; c.stride = stride; c.pad = pad; c.H = H; c.W = W;
+  c.OH = conv_out(H, R, stride, pad); c.OW = conv_out(W, R, stride, pad);
+  if (c.OH < 1 || c.OW < 1) return LP_ERR_SIZE;
+  if (!tc_fwd_ok(c)) return LP_ERR_UNSUPPORTED;
+  int* dev_err = (int*)sp;
+  c.w = const_cast<float*>(w);
+  c.wf = (bf16*)(sp + 256);
+  c.wt = nullptr;
+  PackEntry pe;
+  pe.w = c.w; pe.wf = c.wf; pe.wt = nullptr; pe.cout = Cout; pe.taps = R * R; pe.cin = Cin; pe.begin = 0;
+  PackEntry* dpe = (PackEntry*)(sp + 256 + align_up(n * 2, 256));
+  LP_CUDA_OK(cudaMemsetAsync(dev_err, 0, 4, st));  // the only word that must start at zero
+  LP_CUDA_OK(cudaMemcpyAsync(dpe, &pe, sizeof(pe), cudaMemcpyHostToDevice, st));
+  LP_CUDA_OK(cudaStreamSynchronize(st));
+  pack_weights_kernel<<<grid_for((long long)n, 256, g_dev.sm_count, 8), 256, 0, st>>>(dpe, 1, (long long)n);
+  LP_CUDA_OK(cudaGetLastError());
+  bool done = false;
+  rc = conv_forward(nullptr, LP_BF16, LP_CONV_IMPL_TENSOR, c, N, x, y, nullptr, nullptr, &done, dev_err, st);
+  if (rc != LP_OK) return rc;
+  LP_CUDA_OK(cudaStreamSynchronize(st));
+  int e = 0;
+  LP_CUDA_OK(cudaMemcpy(&e, dev_err, 4, cudaMemcpyDeviceToHost));
+  return e ? LP_ERR_DEVICE_TIMEOUT : LP_OK;
+}
+
 }  // extern "C"
