@@ -229,11 +229,14 @@ static void pick_pixel_box(int OWl, int OHl, int Nimg, int& BW, int& BH, int& BN
   BNI = (Nimg + tn - 1) / tn;
 }
 
+// K chunk (channels per pipeline stage).  Every stage costs a fixed amount (barrier round trip,
+// TMA and MMA issue) worth roughly 48 channels of tensor work, so fewer, larger chunks win even
+// when the last chunk of a tap is partly zero fill (160 channels: 3 chunks of 64, not 5 of 32).
 static int pick_kc(int Cin) {
-  int best = 16, best_pad = 1 << 30;
+  int best = 16, best_cost = 1 << 30;
   for (int kc : {64, 32, 16}) {
-    const int padded = (Cin + kc - 1) / kc * kc;
-    if (padded < best_pad) { best_pad = padded; best = kc; }
+    const int cost = (Cin + kc - 1) / kc * (kc + 48);
+    if (cost < best_cost) { best_cost = cost; best = kc; }
   }
   return best;
 }

@@ -261,7 +261,19 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf
   p.n_tile = best_tile;
   p.n_tiles = Cout / p.n_tile;
   const int tiles = p.m_tiles * p.n_tiles;
-  p.splits = std::max(1, std::min(p.pix_tiles, sm_count / std::max(1, tiles)));
+  // split the pixel range so that the CTAs fill whole waves of SMs: time ~ waves x (K blocks per
+  // CTA + fixed prologue/epilogue worth about 4 K blocks)
+  {
+    int best_s = 1;
+    double best_t = 1e30;
+    const int max_s = std::min(p.pix_tiles, 64);
+    for (int sp = 1; sp <= max_s; ++sp) {
+      const int waves = (tiles * sp + sm_count - 1) / sm_count;
+      const double t = waves * ((double)((p.pix_tiles + sp - 1) / sp) + 4.0);
+      if (t < best_t - 1e-9) { best_t = t; best_s = sp; }
+    }
+    p.splits = best_s;
+  }
   p.a_sub_bytes = (uint32_t)(p.rows_pad * p.sca * 2);
   p.b_sub_bytes = (uint32_t)(p.rows_pad * p.scb * 2);
   p.a_sub_bytes = (p.a_sub_bytes + 1023) / 1024 * 1024;
