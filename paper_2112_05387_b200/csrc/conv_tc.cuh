@@ -5,8 +5,13 @@
 // A operand is a 4-D TMA box of the NHWC activation tensor shifted by the tap offset (zero fill
 // outside the image supplies the padding; element strides supply the convolution stride); the B
 // operand is a 2-D TMA box of the bf16 weights [C_out][taps*C_in].  Both land in shared memory
-// in the K-major swizzled layout tcgen05.mma reads; accumulators live in tensor memory, double
-// buffered so the epilogue of one tile overlaps the MMAs of the next.
+// in the K-major swizzled layout tcgen05.mma reads; accumulators live in tensor memory.
+//
+// Operand reuse: a CTA works on up to two consecutive pixel tiles at once ("pair"): both A tiles
+// are multiplied with the same B stage, which halves the weight traffic per FLOP (the kernel is
+// otherwise bound by L2 -> SM bandwidth).  The accumulators form a ring of 512 / N_TILE slots in
+// tensor memory (3 for N_TILE = 160), so the epilogue of one unit overlaps the MMAs of the next
+// as far as slots are free.
 //
 // Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = epilogue
 // (TMEM -> registers -> optional residual add -> bf16 store, per-channel sum / sum of squares
@@ -20,7 +25,7 @@ namespace tc {
 
 constexpr int kMaxStages = 12;
 constexpr int kTmemCols = 512;
-constexpr int kAccStride = 256;  // TMEM column offset between the two accumulator buffers
+constexpr int kMaxSlots = 4;     // accumulator slots in tensor memory
 
 struct ConvTcParams {
   int Nimg, OHl, OWl;            // logical output grid
@@ -34,7 +39,9 @@ struct ConvTcParams {
   int tap_dh[9], tap_dw[9], tap_w[9];
   int Cin, KC, chunks;
   int stages;
-  uint32_t stage_bytes, a_region_bytes, tx_bytes;
+  int mpair;                     // pixel tiles per unit: 1 or 2
+  int nslots, acc_stride;        // accumulator ring: slots and their TMEM column stride
+  uint32_t stage_bytes, a_region_bytes, b_offset, tx_a, tx_b;
   uint32_t idesc;
   uint64_t desc_hi;
   bf16* out;
@@ -46,8 +53,8 @@ struct ConvTcParams {
 struct TcSmemTail {
   uint64_t full[kMaxStages];
   uint64_t empty[kMaxStages];
-  uint64_t tmem_full[2];
-  uint64_t tmem_empty[2];
+  uint64_t tmem_full[kMaxSlots];
+  uint64_t tmem_empty[kMaxSlots];
   uint32_t tmem_base;
   int abort_flag;
   int epi_ok;
@@ -103,7 +110,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(&tail->full[s], 1);
       mbar_init(&tail->empty[s], 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < kMaxSlots; ++b) {
       mbar_init(&tail->tmem_full[b], 1);
       mbar_init(&tail->tmem_empty[b], 4);
     }
@@ -127,60 +134,85 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int kiters = p.ntaps * p.chunks;
   bool failed = false;
 
+  // All three roles walk the same sequence of units: a unit is one pixel tile, or two consecutive
+  // ones of the same channel tile, and takes the next one or two accumulator slots of the ring.
   if (warp == 0) {
     // ------------------------------- TMA producer (warp-uniform loop, elected issue) ----
     uint32_t s = 0, ph = 0;
-    for (int t = t_begin; t < t_end && !failed; ++t) {
+    for (int t = t_begin; t < t_end && !failed;) {
       const int nt = t / p.m_tiles, m = t % p.m_tiles;
-      const int w0 = (m % p.tiles_w) * p.BW;
-      const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
-      const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
+      const int cnt = (p.mpair == 2 && t + 1 < t_end && m + 1 < p.m_tiles) ? 2 : 1;
+      int w0[2], h0[2], n0[2];
+      for (int a = 0; a < 2; ++a) {
+        const int mm = m + a;
+        w0[a] = (mm % p.tiles_w) * p.BW;
+        h0[a] = ((mm / p.tiles_w) % p.tiles_h) * p.BH;
+        n0[a] = (mm / (p.tiles_w * p.tiles_h)) * p.BNI;
+      }
       const int col0 = nt * p.n_tile_cols;
+      const uint32_t tx = p.tx_b + cnt * p.tx_a;
       for (int tap = 0; tap < p.ntaps && !failed; ++tap) {
-        const int cw = w0 * p.in_step + p.tap_dw[tap];
-        const int ch = h0 * p.in_step + p.tap_dh[tap];
         const int kb = p.tap_w[tap] * p.Cin;
         for (int c = 0; c < p.chunks; ++c) {
           if (!mbar_wait_warp(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
           uint8_t* sa = smem + s * p.stage_bytes;
           if (elect_one()) {
-            mbar_expect_tx(&tail->full[s], p.tx_bytes);
-            tma_load_4d(sa, &tmA, &tail->full[s], c * p.KC, cw, ch, n0);
-            tma_load_2d(sa + p.a_region_bytes, &tmB, &tail->full[s], kb + c * p.KC, col0);
+            mbar_expect_tx(&tail->full[s], tx);
+            tma_load_4d(sa, &tmA, &tail->full[s], c * p.KC, w0[0] * p.in_step + p.tap_dw[tap],
+                        h0[0] * p.in_step + p.tap_dh[tap], n0[0]);
+            if (cnt == 2)
+              tma_load_4d(sa + p.a_region_bytes, &tmA, &tail->full[s], c * p.KC, w0[1] * p.in_step + p.tap_dw[tap],
+                          h0[1] * p.in_step + p.tap_dh[tap], n0[1]);
+            tma_load_2d(sa + p.b_offset, &tmB, &tail->full[s], kb + c * p.KC, col0);
           }
           __syncwarp();
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
         }
       }
+      t += cnt;
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer (warp-uniform loop, elected issue) ------
     uint32_t s = 0, ph = 0;
     const uint32_t smem_base = smem_u32(smem);
     const int nk = p.KC >> 4;
-    int tl = 0;
-    for (int t = t_begin; t < t_end && !failed; ++t, ++tl) {
-      const int buf = tl & 1;
-      const uint32_t aph = (tl >> 1) & 1;
-      if (!mbar_wait_warp(&tail->tmem_empty[buf], aph ^ 1, abort_flag)) { failed = true; break; }
+    uint32_t slot = 0, slot_phase = 0;  // bit b of slot_phase: parity of the number of uses of slot b
+    for (int t = t_begin; t < t_end && !failed;) {
+      const int m = t % p.m_tiles;
+      const int cnt = (p.mpair == 2 && t + 1 < t_end && m + 1 < p.m_tiles) ? 2 : 1;
+      uint32_t sl[2];
+      sl[0] = slot;
+      sl[1] = slot + 1 == (uint32_t)p.nslots ? 0 : slot + 1;
+      for (int a = 0; a < cnt && !failed; ++a)
+        if (!mbar_wait_warp(&tail->tmem_empty[sl[a]], ((slot_phase >> sl[a]) & 1) ^ 1, abort_flag)) failed = true;
+      if (failed) break;
       tc_fence_after();
-      const uint32_t d_tmem = tmem_base + buf * kAccStride;
+      const uint32_t d0 = tmem_base + sl[0] * p.acc_stride, d1 = tmem_base + sl[1] * p.acc_stride;
       for (int k = 0; k < kiters; ++k) {
         if (!mbar_wait_warp(&tail->full[s], ph, abort_flag)) { failed = true; break; }
         tc_fence_after();
         const uint32_t a_addr = smem_base + s * p.stage_bytes;
-        const uint64_t ad = smem_desc(p.desc_hi, a_addr), bd = smem_desc(p.desc_hi, a_addr + p.a_region_bytes);
+        const uint64_t ad0 = smem_desc(p.desc_hi, a_addr), ad1 = smem_desc(p.desc_hi, a_addr + p.a_region_bytes);
+        const uint64_t bd = smem_desc(p.desc_hi, a_addr + p.b_offset);
         if (elect_one()) {
-          for (int j = 0; j < nk; ++j)  // +32 bytes (one K = 16 slice) per step, in 16-byte units
-            mma_bf16(d_tmem, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k | j) ? 1u : 0u);
+          for (int j = 0; j < nk; ++j) {  // +32 bytes (one K = 16 slice) per step, in 16-byte units
+            mma_bf16(d0, ad0 + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k | j) ? 1u : 0u);
+            if (cnt == 2) mma_bf16(d1, ad1 + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k | j) ? 1u : 0u);
+          }
           mma_commit(&tail->empty[s]);
         }
         __syncwarp();
         if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
       }
       if (failed) break;
-      if (elect_one()) mma_commit(&tail->tmem_full[buf]);
+      if (elect_one()) {
+        mma_commit(&tail->tmem_full[sl[0]]);
+        if (cnt == 2) mma_commit(&tail->tmem_full[sl[1]]);
+      }
       __syncwarp();
+      for (int a = 0; a < cnt; ++a) slot_phase ^= 1u << sl[a];
+      slot = cnt == 2 ? (sl[1] + 1 == (uint32_t)p.nslots ? 0 : sl[1] + 1) : sl[1];
+      t += cnt;
     }
   } else {
     // ------------------------------- epilogue -----------------------------------------
@@ -188,82 +220,90 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int row = q * 32 + lane;
     const int et = threadIdx.x - 64;  // 0..127
     const int rows_used = p.BW * p.BH * p.BNI;
-    int tl = 0;
-    for (int t = t_begin; t < t_end && !failed; ++t, ++tl) {
-      const int buf = tl & 1;
-      const uint32_t aph = (tl >> 1) & 1;
-      const int nt = t / p.m_tiles, m = t % p.m_tiles;
-      const int w0 = (m % p.tiles_w) * p.BW;
-      const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
-      const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
+    uint32_t slot = 0, slot_phase = 0;
+    for (int t = t_begin; t < t_end && !failed;) {
+      const int nt = t / p.m_tiles, m0 = t % p.m_tiles;
+      const int cnt = (p.mpair == 2 && t + 1 < t_end && m0 + 1 < p.m_tiles) ? 2 : 1;
       const int col0 = nt * p.n_tile_cols;
-      const int ow = w0 + row % p.BW, oh = h0 + (row / p.BW) % p.BH, n = n0 + row / (p.BW * p.BH);
-      const bool valid = row < rows_used && ow < p.OWl && oh < p.OHl && n < p.Nimg;
-      const long long obase =
-          (((long long)n * p.out_H + (oh * p.os + p.oo_h)) * p.out_W + (ow * p.os + p.oo_w)) * p.out_C;
-      // one thread waits (bounded) and the 128 epilogue threads agree on the outcome, so that the
-      // named barriers below are reached by all of them or by none
-      if (et == 0) tail->epi_ok = mbar_wait(&tail->tmem_full[buf], aph, abort_flag) ? 1 : 0;
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (!*(volatile int*)&tail->epi_ok) { failed = true; break; }
-      tc_fence_after();
-      const uint32_t taddr = tmem_base + buf * kAccStride + ((uint32_t)(q * 32) << 16);
-      const int nchunk = p.n_tile_cols >> 4;
-      for (int cc = 0; cc < nchunk; ++cc) {
-        float v[16];
-        tmem_ld16(taddr + cc * 16, v);
-        const int col = col0 + cc * 16;
-        const bool lo_ok = valid && col < p.Cout, hi_ok = valid && col + 8 < p.Cout;
-        if (p.addend) {
-          float f[8];
-          if (lo_ok) {
-            ldv(p.addend + obase + col, f);
+      for (int a = 0; a < cnt && !failed; ++a) {
+        const int m = m0 + a;
+        const uint32_t buf = slot;
+        const int w0 = (m % p.tiles_w) * p.BW;
+        const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
+        const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
+        const int ow = w0 + row % p.BW, oh = h0 + (row / p.BW) % p.BH, n = n0 + row / (p.BW * p.BH);
+        const bool valid = row < rows_used && ow < p.OWl && oh < p.OHl && n < p.Nimg;
+        const long long obase =
+            (((long long)n * p.out_H + (oh * p.os + p.oo_h)) * p.out_W + (ow * p.os + p.oo_w)) * p.out_C;
+        // one thread waits (bounded) and the 128 epilogue threads agree on the outcome, so that the
+        // named barriers below are reached by all of them or by none
+        if (et == 0) tail->epi_ok = mbar_wait(&tail->tmem_full[buf], (slot_phase >> buf) & 1, abort_flag) ? 1 : 0;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (!*(volatile int*)&tail->epi_ok) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + buf * p.acc_stride + ((uint32_t)(q * 32) << 16);
+        const int nchunk = p.n_tile_cols >> 4;
+        for (int cc = 0; cc < nchunk; ++cc) {
+          float v[16];
+          tmem_ld16(taddr + cc * 16, v);
+          const int col = col0 + cc * 16;
+          const bool lo_ok = valid && col < p.Cout, hi_ok = valid && col + 8 < p.Cout;
+          if (p.addend) {
+            float f[8];
+            if (lo_ok) {
+              ldv(p.addend + obase + col, f);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] += f[j];
+              for (int j = 0; j < 8; ++j) v[j] += f[j];
+            }
+            if (hi_ok) {
+              ldv(p.addend + obase + col + 8, f);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) v[8 + j] += f[j];
+            }
           }
-          if (hi_ok) {
-            ldv(p.addend + obase + col + 8, f);
+          if (lo_ok) stv(p.out + obase + col, *reinterpret_cast<float(*)[8]>(&v[0]));
+          if (hi_ok) stv(p.out + obase + col + 8, *reinterpret_cast<float(*)[8]>(&v[8]));
+          if (p.stats) {
+            // statistics of the tensor as stored (bf16), so that the batch-norm that follows
+            // normalises exactly the values it reads
+            float sq[16];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) v[8 + j] += f[j];
+            for (int j = 0; j < 16; ++j) {
+              v[j] = valid ? round_storage<bf16>(v[j]) : 0.f;
+              sq[j] = v[j] * v[j];
+            }
+            const float cs = transpose_reduce16(v, lane);
+            const float cq = transpose_reduce16(sq, lane);
+            if ((lane & 1) == 0) {
+              const int cidx = cc * 16 + ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 +
+                               ((lane >> 1) & 1);
+              atomicAdd(&tail->ssum[cidx], cs);
+              atomicAdd(&tail->ssq[cidx], cq);
+            }
           }
         }
-        if (lo_ok) stv(p.out + obase + col, *reinterpret_cast<float(*)[8]>(&v[0]));
-        if (hi_ok) stv(p.out + obase + col + 8, *reinterpret_cast<float(*)[8]>(&v[8]));
-        if (p.stats) {
-          // statistics of the tensor as stored (bf16), so that the batch-norm that follows
-          // normalises exactly the values it reads
-          float sq[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            v[j] = valid ? round_storage<bf16>(v[j]) : 0.f;
-            sq[j] = v[j] * v[j];
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tail->tmem_empty[buf]);
+        slot_phase ^= 1u << buf;
+        slot = slot + 1 == (uint32_t)p.nslots ? 0 : slot + 1;
+        // flush the column sums when the channel tile is about to change (or at the very end)
+        const bool last_of_unit = a + 1 == cnt;
+        const bool flush = p.stats && last_of_unit && (t + cnt >= t_end || (t + cnt) / p.m_tiles != nt);
+        if (flush) {
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          for (int c = et; c < p.n_tile_cols; c += 128) {
+            if (col0 + c < p.Cout) {
+              atomicAdd(&p.stats[col0 + c], (double)tail->ssum[c]);
+              atomicAdd(&p.stats[p.Cout + col0 + c], (double)tail->ssq[c]);
+            }
+            tail->ssum[c] = 0.f;
+            tail->ssq[c] = 0.f;
           }
-          const float cs = transpose_reduce16(v, lane);
-          const float cq = transpose_reduce16(sq, lane);
-          if ((lane & 1) == 0) {
-            const int cidx = cc * 16 + ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 +
-                             ((lane >> 1) & 1);
-            atomicAdd(&tail->ssum[cidx], cs);
-            atomicAdd(&tail->ssq[cidx], cq);
-          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&tail->tmem_empty[buf]);
-      if (p.stats) {
-        // flush this tile's column sums (128 epilogue threads cooperate)
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        for (int c = et; c < p.n_tile_cols; c += 128) {
-          if (col0 + c < p.Cout) {
-            atomicAdd(&p.stats[col0 + c], (double)tail->ssum[c]);
-            atomicAdd(&p.stats[p.Cout + col0 + c], (double)tail->ssq[c]);
-          }
-          tail->ssum[c] = 0.f;
-          tail->ssq[c] = 0.f;
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-      }
+      t += cnt;
     }
   }
 

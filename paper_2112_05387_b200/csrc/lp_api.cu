@@ -310,9 +310,18 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   const int row_bytes = p.KC * 2;
   p.a_region_bytes = (uint32_t)align_up((size_t)128 * row_bytes, 1024);
   const uint32_t b_region = (uint32_t)align_up((size_t)p.n_tile_cols * row_bytes, 1024);
-  p.stage_bytes = p.a_region_bytes + b_region;
-  p.tx_bytes = (uint32_t)((p.BW * p.BH * p.BNI + p.n_tile_cols) * row_bytes);
   const size_t tail = sizeof(tc::TcSmemTail) + 1024;
+  // two pixel tiles per weight tile wherever a CTA has at least two tiles and three stages still fit
+  p.mpair = 1;
+  if (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, g_dev.sm_count) &&
+      (kTcMaxSmem - tail) / (2 * p.a_region_bytes + b_region) >= 3)
+    p.mpair = 2;
+  p.b_offset = p.mpair * p.a_region_bytes;
+  p.stage_bytes = p.b_offset + b_region;
+  p.tx_a = (uint32_t)(p.BW * p.BH * p.BNI * row_bytes);
+  p.tx_b = (uint32_t)(p.n_tile_cols * row_bytes);
+  p.acc_stride = (p.n_tile_cols + 31) / 32 * 32;
+  p.nslots = std::min(tc::kMaxSlots, tc::kTmemCols / p.acc_stride);
   int stages = (int)((kTcMaxSmem - tail) / p.stage_bytes);
   stages = std::min(stages, tc::kMaxStages);
   if (stages < 2) return LP_ERR_UNSUPPORTED;

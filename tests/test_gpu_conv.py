@@ -85,6 +85,10 @@ TC_CASES = [
     (3, 7, 7, 128, 128, 3, 1, 1),     # 7x7 pairs of images, odd batch
     (2, 32, 32, 40, 160, 3, 1, 1),    # AuxNet hidden width (C_in = 40)
     (2, 32, 32, 160, 80, 3, 2, 1),    # AuxNet strided
+    (32, 32, 32, 64, 64, 3, 1, 1),    # 256 pixel tiles: CTAs work on pairs of tiles sharing the weight stage
+    (29, 32, 32, 32, 48, 3, 1, 1),    # 232 tiles: CTAs with one tile and CTAs with a pair
+    (64, 16, 16, 32, 320, 3, 1, 1),   # pairs with two channel tiles (ranges cross the channel-tile boundary)
+    (37, 16, 16, 160, 160, 3, 2, 1),  # pairs, stride 2, odd tile count (input gradient: parity classes)
 ]
 
 
