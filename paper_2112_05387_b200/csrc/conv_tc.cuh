@@ -13,7 +13,8 @@
 // tensor memory (3 for N_TILE = 160), so the epilogue of one unit overlaps the MMAs of the next
 // as far as slots are free.
 //
-// Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = epilogue
+// Roles (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = epilogue, two
+// warps per TMEM lane quarter taking alternate 32-column groups
 // (TMEM -> registers -> optional residual add -> bf16 store, per-channel sum / sum of squares
 // for the batch-norm that follows).  One persistent CTA per SM walks a contiguous tile range.
 #pragma once
@@ -92,7 +93,14 @@ __device__ __forceinline__ float transpose_reduce16(const float (&v)[16], int la
   return d;
 }
 
-__global__ void __launch_bounds__(192, 1)
+#ifndef LP_EPI_WARPS
+#define LP_EPI_WARPS 4
+#endif
+constexpr int kEpiThreads = 32 * LP_EPI_WARPS;
+constexpr int kConvThreads = 64 + kEpiThreads;
+constexpr int kEpiGroups = LP_EPI_WARPS / 4;
+
+__global__ void __launch_bounds__(kConvThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ ConvTcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -112,7 +120,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int b = 0; b < kMaxSlots; ++b) {
       mbar_init(&tail->tmem_full[b], 1);
-      mbar_init(&tail->tmem_empty[b], 4);
+      mbar_init(&tail->tmem_empty[b], kEpiThreads / 32);
     }
     tail->abort_flag = 0;
     fence_barrier_init();
@@ -216,10 +224,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else {
     // ------------------------------- epilogue -----------------------------------------
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    const int q = warp & 3;              // TMEM lane quarter this warp may read
+    const int grp = (warp - 2) >> 2;     // which of the two warps of the quarter
     const int row = q * 32 + lane;
-    const int et = threadIdx.x - 64;  // 0..127
+    const int et = threadIdx.x - 64;     // 0..255
     const int rows_used = p.BW * p.BH * p.BNI;
+    const int ngroups = (p.n_tile_cols + 31) >> 5;
     uint32_t slot = 0, slot_phase = 0;
     for (int t = t_begin; t < t_end && !failed;) {
       const int nt = t / p.m_tiles, m0 = t % p.m_tiles;
@@ -235,50 +245,61 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool valid = row < rows_used && ow < p.OWl && oh < p.OHl && n < p.Nimg;
         const long long obase =
             (((long long)n * p.out_H + (oh * p.os + p.oo_h)) * p.out_W + (ow * p.os + p.oo_w)) * p.out_C;
-        // one thread waits (bounded) and the 128 epilogue threads agree on the outcome, so that the
+        // one thread waits (bounded) and all epilogue threads agree on the outcome, so that the
         // named barriers below are reached by all of them or by none
         if (et == 0) tail->epi_ok = mbar_wait(&tail->tmem_full[buf], (slot_phase >> buf) & 1, abort_flag) ? 1 : 0;
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
         if (!*(volatile int*)&tail->epi_ok) { failed = true; break; }
         tc_fence_after();
         const uint32_t taddr = tmem_base + buf * p.acc_stride + ((uint32_t)(q * 32) << 16);
-        const int nchunk = p.n_tile_cols >> 4;
-        for (int cc = 0; cc < nchunk; ++cc) {
-          float v[16];
-          tmem_ld16(taddr + cc * 16, v);
-          const int col = col0 + cc * 16;
-          const bool lo_ok = valid && col < p.Cout, hi_ok = valid && col + 8 < p.Cout;
+        for (int g = grp; g < ngroups; g += kEpiGroups) {
+          const int c_in_tile = g * 32;
+          const int col = col0 + c_in_tile;
+          const bool wide = c_in_tile + 32 <= p.n_tile_cols;   // a 16-column tail otherwise
+          const int nv = wide ? 4 : 2;                         // 8-channel vectors in this group
+          // residual operand first: its latency overlaps the TMEM read
+          float add[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) add[j] = 0.f;
           if (p.addend) {
-            float f[8];
-            if (lo_ok) {
-              ldv(p.addend + obase + col, f);
 #pragma unroll
-              for (int j = 0; j < 8; ++j) v[j] += f[j];
-            }
-            if (hi_ok) {
-              ldv(p.addend + obase + col + 8, f);
-#pragma unroll
-              for (int j = 0; j < 8; ++j) v[8 + j] += f[j];
-            }
+            for (int u = 0; u < 4; ++u)
+              if (u < nv && valid && col + 8 * u < p.Cout)
+                ldv(p.addend + obase + col + 8 * u, *reinterpret_cast<float(*)[8]>(&add[8 * u]));
           }
-          if (lo_ok) stv(p.out + obase + col, *reinterpret_cast<float(*)[8]>(&v[0]));
-          if (hi_ok) stv(p.out + obase + col + 8, *reinterpret_cast<float(*)[8]>(&v[8]));
+          float v[32];
+          if (wide) {
+            tmem_ld32(taddr + c_in_tile, v);
+          } else {
+            tmem_ld16(taddr + c_in_tile, *reinterpret_cast<float(*)[16]>(&v[0]));
+#pragma unroll
+            for (int j = 16; j < 32; ++j) v[j] = 0.f;
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] += add[j];
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            if (u < nv && valid && col + 8 * u < p.Cout)
+              stv(p.out + obase + col + 8 * u, *reinterpret_cast<float(*)[8]>(&v[8 * u]));
           if (p.stats) {
             // statistics of the tensor as stored (bf16), so that the batch-norm that follows
             // normalises exactly the values it reads
-            float sq[16];
+            float sq[32];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
+            for (int j = 0; j < 32; ++j) {
               v[j] = valid ? round_storage<bf16>(v[j]) : 0.f;
               sq[j] = v[j] * v[j];
             }
-            const float cs = transpose_reduce16(v, lane);
-            const float cq = transpose_reduce16(sq, lane);
-            if ((lane & 1) == 0) {
-              const int cidx = cc * 16 + ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 +
-                               ((lane >> 1) & 1);
-              atomicAdd(&tail->ssum[cidx], cs);
-              atomicAdd(&tail->ssq[cidx], cq);
+            const int cl = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              if (hf == 1 && !wide) break;
+              const float cs = transpose_reduce16(*reinterpret_cast<float(*)[16]>(&v[16 * hf]), lane);
+              const float cq = transpose_reduce16(*reinterpret_cast<float(*)[16]>(&sq[16 * hf]), lane);
+              if ((lane & 1) == 0) {
+                atomicAdd(&tail->ssum[c_in_tile + 16 * hf + cl], cs);
+                atomicAdd(&tail->ssq[c_in_tile + 16 * hf + cl], cq);
+              }
             }
           }
         }
@@ -291,8 +312,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool last_of_unit = a + 1 == cnt;
         const bool flush = p.stats && last_of_unit && (t + cnt >= t_end || (t + cnt) / p.m_tiles != nt);
         if (flush) {
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          for (int c = et; c < p.n_tile_cols; c += 128) {
+          asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+          for (int c = et; c < p.n_tile_cols; c += kEpiThreads) {
             if (col0 + c < p.Cout) {
               atomicAdd(&p.stats[col0 + c], (double)tail->ssum[c]);
               atomicAdd(&p.stats[p.Cout + col0 + c], (double)tail->ssq[c]);
@@ -300,7 +321,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tail->ssum[c] = 0.f;
             tail->ssq[c] = 0.f;
           }
-          asm volatile("bar.sync 1, 128;" ::: "memory");
+          asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
         }
       }
       t += cnt;

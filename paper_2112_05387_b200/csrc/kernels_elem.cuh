@@ -507,7 +507,8 @@ struct PackEntry {
   bf16* wf;
   bf16* wt;  // may be null
   int cout, taps, cin;
-  long long begin;  // first flat element index handled for this entry
+  long long begin;       // first flat element index handled for this entry
+  long long tile_begin;  // first 32x32 tile index of this entry (tiled kernel)
 };
 
 __global__ void pack_weights_kernel(const PackEntry* __restrict__ tab, int n_entries, long long total) {
@@ -530,6 +531,42 @@ __global__ void pack_weights_kernel(const PackEntry* __restrict__ tab, int n_ent
       const int co = (int)(q / e.taps);
       e.wt[((long long)ci * e.taps + t) * e.cout + co] = b;
     }
+  }
+}
+
+// Same copies, one 32 (c_out) x 32 (c_in) tile of one tap per block: reads and both writes are
+// coalesced (the transposed copy goes through shared memory).  blockDim = (32, 8).
+__global__ void pack_weights_tiled_kernel(const PackEntry* __restrict__ tab, int n_entries) {
+  __shared__ float tile[32][33];
+  const long long b = blockIdx.x;
+  int lo = 0, hi = n_entries - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (tab[mid].tile_begin <= b) lo = mid; else hi = mid - 1;
+  }
+  const PackEntry e = tab[lo];
+  const int tiles_ci = (e.cin + 31) >> 5, tiles_co = (e.cout + 31) >> 5;
+  int r = (int)(b - e.tile_begin);
+  const int ci0 = (r % tiles_ci) << 5;
+  r /= tiles_ci;
+  const int co0 = (r % tiles_co) << 5;
+  const int t = r / tiles_co;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  for (int i = ty; i < 32; i += 8) {
+    const int co = co0 + i, ci = ci0 + tx;
+    float v = 0.f;
+    if (co < e.cout && ci < e.cin) {
+      const long long j = ((long long)co * e.taps + t) * e.cin + ci;
+      v = e.w[j];
+      e.wf[j] = __float2bfloat16_rn(v);
+    }
+    tile[i][tx] = v;
+  }
+  if (!e.wt) return;
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int ci = ci0 + i, co = co0 + tx;
+    if (co < e.cout && ci < e.cin) e.wt[((long long)ci * e.taps + t) * e.cout + co] = __float2bfloat16_rn(tile[tx][i]);
   }
 }
 

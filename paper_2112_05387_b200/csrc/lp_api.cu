@@ -71,6 +71,7 @@ struct ParamSet {
   PackEntry* dev_pack = nullptr;
   std::vector<PackEntry> host_pack;
   long long pack_total = 0;
+  long long pack_tiles = 0;
   bool grads_fresh = false;
   bool momentum_used = false;
 };
@@ -342,7 +343,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     attr_set = true;
   }
   const int grid = std::min(p.total_tiles, g_dev.sm_count);
-  tc::conv_tc_kernel<<<grid, 192, smem, st>>>(tmA, tmB, p);
+  tc::conv_tc_kernel<<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
   if (h) h->launches++;
   LP_CUDA_OK(cudaGetLastError());
   return LP_OK;
@@ -555,7 +556,9 @@ struct Planner {
       PackEntry pe;
       pe.w = c.w; pe.wf = c.wf; pe.wt = c.wt; pe.cout = cout; pe.taps = R * R; pe.cin = cin;
       pe.begin = P.ps.pack_total;
+      pe.tile_begin = P.ps.pack_tiles;
       P.ps.pack_total += (long long)n;
+      P.ps.pack_tiles += (long long)R * R * ((cin + 31) / 32) * ((cout + 31) / 32);
       P.ps.host_pack.push_back(pe);
     }
     P.convs.push_back(c);
@@ -1058,8 +1061,8 @@ static int zero_forward_state(Plan& P, cudaStream_t st) {
 
 static int pack_weights(lp_handle* h, Plan& P, cudaStream_t st) {
   if (P.ps.host_pack.empty()) return LP_OK;
-  pack_weights_kernel<<<grid_for(P.ps.pack_total, 256, g_dev.sm_count, 8), 256, 0, st>>>(
-      P.ps.dev_pack, (int)P.ps.host_pack.size(), P.ps.pack_total);
+  pack_weights_tiled_kernel<<<(unsigned)P.ps.pack_tiles, dim3(32, 8), 0, st>>>(P.ps.dev_pack,
+                                                                              (int)P.ps.host_pack.size());
   h->launches++;
   LP_CUDA_OK(cudaGetLastError());
   return LP_OK;
@@ -1539,7 +1542,7 @@ int lp_conv2d(int op, int dtype, int impl, int N, int H, int W, int Cin, int Cou
       // pack on the fly: one-entry table placed after the two weight copies is not available on the
       // device, so build it in pinned-free fashion: the table lives in the scratch tail
       PackEntry pe;
-      pe.w = c.w; pe.wf = c.wf; pe.wt = c.wt; pe.cout = Cout; pe.taps = R * R; pe.cin = Cin; pe.begin = 0;
+      pe.w = c.w; pe.wf = c.wf; pe.wt = c.wt; pe.cout = Cout; pe.taps = R * R; pe.cin = Cin; pe.begin = 0; pe.tile_begin = 0;
       PackEntry* dpe = (PackEntry*)(sp + 256 + 2 * align_up(n * 2, 256));
       LP_CUDA_OK(cudaMemcpyAsync(dpe, &pe, sizeof(pe), cudaMemcpyHostToDevice, st));
       LP_CUDA_OK(cudaStreamSynchronize(st));
@@ -1632,7 +1635,7 @@ int lp_conv2d_fwd_noalloc(int N, int H, int W, int Cin, int Cout, int R, int str
   c.wf = (bf16*)(sp + 256);
   c.wt = nullptr;
   PackEntry pe;
-  pe.w = c.w; pe.wf = c.wf; pe.wt = nullptr; pe.cout = Cout; pe.taps = R * R; pe.cin = Cin; pe.begin = 0;
+  pe.w = c.w; pe.wf = c.wf; pe.wt = nullptr; pe.cout = Cout; pe.taps = R * R; pe.cin = Cin; pe.begin = 0; pe.tile_begin = 0;
   PackEntry* dpe = (PackEntry*)(sp + 256 + align_up(n * 2, 256));
   LP_CUDA_OK(cudaMemsetAsync(dev_err, 0, 4, st));  // the only word that must start at zero
   LP_CUDA_OK(cudaMemcpyAsync(dpe, &pe, sizeof(pe), cudaMemcpyHostToDevice, st));
