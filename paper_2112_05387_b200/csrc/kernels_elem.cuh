@@ -90,7 +90,7 @@ __global__ void bn_apply_kernel(const T* __restrict__ x, BnArgs A, const T* __re
     float f[V], y[V];
     ldv(x + i * V, f);
 #pragma unroll
-    for (int j = 0; j < V; ++j) y[j] = f[j] * sa[j] + ta[j];
+    for (int j = 0; j < V; ++j) y[j] = fmaf(f[j], sa[j], ta[j]);
     if (x2) {
       ldv(x2 + i * V, f);
 #pragma unroll
@@ -208,33 +208,35 @@ __global__ void loss_finalize_kernel(const double* __restrict__ acc, float rho, 
 }
 
 // ---------------------------------------------------------------------------------------
-// BN backward.  dy_m = dy * [mask > 0] (mask optional: the stored post-ReLU activation).
+// BN backward.  dy_m = dy * [bn(x) > 0] when a ReLU followed the normalisation (relu_mask): the
+// mask is recomputed from x with the forward kernel's own expression instead of being read back.
 //   reduce: dbeta += sum dy_m ; dgamma += sum dy_m * xhat
 //   apply : dx = gamma*rstd*(dy_m - dbeta/M - xhat*dgamma/M) [+ addend]
 // ---------------------------------------------------------------------------------------
 template <typename T>
-__global__ void bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ x, const T* __restrict__ mask,
+__global__ void bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_mask,
                                      BnArgs A, float* __restrict__ dgamma, float* __restrict__ dbeta,
                                      long long total_vecs, int C) {
   constexpr int V = VecT<T>::N;
   extern __shared__ float sm[];
   const int CV = C / V;
   const int c0 = (threadIdx.x % CV) * V;
-  float mean[V], rstd[V], sb[V], sg[V];
+  float mean[V], rstd[V], sb[V], sg[V], sa[V], ta[V];
 #pragma unroll
   for (int j = 0; j < V; ++j) {
     bn_mean_rstd(A, C, c0 + j, mean[j], rstd[j]);
+    sa[j] = A.gamma[c0 + j] * rstd[j];
+    ta[j] = A.beta[c0 + j] - mean[j] * sa[j];
     sb[j] = sg[j] = 0.f;
   }
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
-    float d[V], f[V], m[V];
+    float d[V], f[V];
     ldv(dy + i * V, d);
     ldv(x + i * V, f);
-    if (mask) {
-      ldv(mask + i * V, m);
+    if (relu_mask) {
 #pragma unroll
-      for (int j = 0; j < V; ++j) d[j] = m[j] > 0.f ? d[j] : 0.f;
+      for (int j = 0; j < V; ++j) d[j] = fmaf(f[j], sa[j], ta[j]) > 0.f ? d[j] : 0.f;
     }
 #pragma unroll
     for (int j = 0; j < V; ++j) {
@@ -258,30 +260,30 @@ __global__ void bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restri
 }
 
 template <typename T>
-__global__ void bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ x, const T* __restrict__ mask,
+__global__ void bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_mask,
                                     BnArgs A, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
                                     const T* __restrict__ addend, T* __restrict__ out, long long total_vecs, int C) {
   constexpr int V = VecT<T>::N;
   const int CV = C / V;
   const int c0 = (threadIdx.x % CV) * V;
-  float mean[V], rstd[V], sc[V], mb[V], mg[V];
+  float mean[V], rstd[V], sc[V], mb[V], mg[V], ta[V];
   const float invM = (float)A.inv_count;
 #pragma unroll
   for (int j = 0; j < V; ++j) {
     bn_mean_rstd(A, C, c0 + j, mean[j], rstd[j]);
     sc[j] = A.gamma[c0 + j] * rstd[j];
+    ta[j] = A.beta[c0 + j] - mean[j] * sc[j];
     mb[j] = dbeta[c0 + j] * invM;
     mg[j] = dgamma[c0 + j] * invM;
   }
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
-    float d[V], f[V], m[V], o[V];
+    float d[V], f[V], o[V];
     ldv(dy + i * V, d);
     ldv(x + i * V, f);
-    if (mask) {
-      ldv(mask + i * V, m);
+    if (relu_mask) {
 #pragma unroll
-      for (int j = 0; j < V; ++j) d[j] = m[j] > 0.f ? d[j] : 0.f;
+      for (int j = 0; j < V; ++j) d[j] = fmaf(f[j], sc[j], ta[j]) > 0.f ? d[j] : 0.f;
     }
 #pragma unroll
     for (int j = 0; j < V; ++j) o[j] = sc[j] * (d[j] - mb[j] - (f[j] - mean[j]) * rstd[j] * mg[j]);

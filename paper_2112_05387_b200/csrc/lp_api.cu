@@ -988,7 +988,7 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       if (!threads) return LP_ERR_UNSUPPORTED;
       const long long vecs = op.in2.elems() / V;
       BnArgs A = bn_args(b, eps);
-      const T* mask = op.mask.defined() ? (const T*)resolve(op.mask, c) : nullptr;
+      const int mask = op.mask.defined() ? 1 : 0;  // a ReLU followed this BN in the forward pass
       const T* addend = op.addend.defined() ? (const T*)resolve(op.addend, c) : nullptr;
       const int grid_r = grid_for(vecs, threads * 8, g_dev.sm_count, 4);
       bn_bwd_reduce_kernel<T><<<grid_r, threads, (size_t)threads * 2 * V * 4, st>>>(
