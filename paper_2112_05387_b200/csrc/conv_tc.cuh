@@ -59,8 +59,8 @@ struct TcSmemTail {
   uint32_t tmem_base;
   int abort_flag;
   int epi_ok;
-  float ssum[256];
-  float ssq[256];
+  float ssum[8][256];   // per epilogue warp: plain read-modify-write, no shared-memory atomics
+  float ssq[8][256];
 };
 
 // Sum 16 per-lane values over the 32 lanes of a warp; lane l ends with the total of column
@@ -127,9 +127,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
   }
-  for (int i = threadIdx.x; i < 256; i += blockDim.x) {
-    tail->ssum[i] = 0.f;
-    tail->ssq[i] = 0.f;
+  for (int i = threadIdx.x; i < 8 * 256; i += blockDim.x) {
+    (&tail->ssum[0][0])[i] = 0.f;
+    (&tail->ssq[0][0])[i] = 0.f;
   }
   if (warp == 2) {
     tmem_alloc(&tail->tmem_base, kTmemCols);
@@ -252,60 +252,75 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!*(volatile int*)&tail->epi_ok) { failed = true; break; }
         tc_fence_after();
         const uint32_t taddr = tmem_base + buf * p.acc_stride + ((uint32_t)(q * 32) << 16);
-        for (int g = grp; g < ngroups; g += kEpiGroups) {
-          const int c_in_tile = g * 32;
-          const int col = col0 + c_in_tile;
-          const bool wide = c_in_tile + 32 <= p.n_tile_cols;   // a 16-column tail otherwise
-          const int nv = wide ? 4 : 2;                         // 8-channel vectors in this group
-          // residual operand first: its latency overlaps the TMEM read
-          float add[32];
+        // Drain the accumulator into registers first (up to kBatch x 32 columns per pass) and hand
+        // the TMEM slot back to the MMA warp; stores and statistics then work from registers.
+        constexpr int kBatch = 5;
+        for (int g0 = grp; g0 < ngroups; g0 += kBatch * kEpiGroups) {
+          uint32_t raw[kBatch][32];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) add[j] = 0.f;
-          if (p.addend) {
+          for (int i = 0; i < kBatch; ++i) {
+            const int g = g0 + i * kEpiGroups;
+            if (g < ngroups) {
+              if (g * 32 + 32 <= p.n_tile_cols) tmem_ld32_issue(taddr + g * 32, raw[i]);
+              else tmem_ld16_issue(taddr + g * 32, raw[i]);
+            }
+          }
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < kBatch; ++i) tmem_ld_fence(raw[i]);
+          if (g0 + kBatch * kEpiGroups >= ngroups) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tail->tmem_empty[buf]);
+          }
+#pragma unroll
+          for (int i = 0; i < kBatch; ++i) {
+            const int g = g0 + i * kEpiGroups;
+            if (g >= ngroups) continue;
+            const int c_in_tile = g * 32;
+            const int col = col0 + c_in_tile;
+            const bool wide = c_in_tile + 32 <= p.n_tile_cols;   // a 16-column tail otherwise
+            const int nv = wide ? 4 : 2;                         // 8-channel vectors in this group
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = (wide || j < 16) ? __uint_as_float(raw[i][j]) : 0.f;
+            if (p.addend) {
+#pragma unroll
+              for (int u = 0; u < 4; ++u)
+                if (u < nv && valid && col + 8 * u < p.Cout) {
+                  float f[8];
+                  ldv(p.addend + obase + col + 8 * u, f);
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) v[8 * u + j] += f[j];
+                }
+            }
 #pragma unroll
             for (int u = 0; u < 4; ++u)
               if (u < nv && valid && col + 8 * u < p.Cout)
-                ldv(p.addend + obase + col + 8 * u, *reinterpret_cast<float(*)[8]>(&add[8 * u]));
-          }
-          float v[32];
-          if (wide) {
-            tmem_ld32(taddr + c_in_tile, v);
-          } else {
-            tmem_ld16(taddr + c_in_tile, *reinterpret_cast<float(*)[16]>(&v[0]));
+                stv(p.out + obase + col + 8 * u, *reinterpret_cast<float(*)[8]>(&v[8 * u]));
+            if (p.stats) {
+              // statistics of the tensor as stored (bf16), so that the batch-norm that follows
+              // normalises exactly the values it reads
+              float sq[32];
 #pragma unroll
-            for (int j = 16; j < 32; ++j) v[j] = 0.f;
-          }
+              for (int j = 0; j < 32; ++j) {
+                v[j] = valid ? round_storage<bf16>(v[j]) : 0.f;
+                sq[j] = v[j] * v[j];
+              }
+              const int cl = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] += add[j];
-#pragma unroll
-          for (int u = 0; u < 4; ++u)
-            if (u < nv && valid && col + 8 * u < p.Cout)
-              stv(p.out + obase + col + 8 * u, *reinterpret_cast<float(*)[8]>(&v[8 * u]));
-          if (p.stats) {
-            // statistics of the tensor as stored (bf16), so that the batch-norm that follows
-            // normalises exactly the values it reads
-            float sq[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              v[j] = valid ? round_storage<bf16>(v[j]) : 0.f;
-              sq[j] = v[j] * v[j];
-            }
-            const int cl = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-              if (hf == 1 && !wide) break;
-              const float cs = transpose_reduce16(*reinterpret_cast<float(*)[16]>(&v[16 * hf]), lane);
-              const float cq = transpose_reduce16(*reinterpret_cast<float(*)[16]>(&sq[16 * hf]), lane);
-              if ((lane & 1) == 0) {
-                atomicAdd(&tail->ssum[c_in_tile + 16 * hf + cl], cs);
-                atomicAdd(&tail->ssq[c_in_tile + 16 * hf + cl], cq);
+              for (int hf = 0; hf < 2; ++hf) {
+                if (hf == 1 && !wide) break;
+                const float cs = transpose_reduce16(*reinterpret_cast<float(*)[16]>(&v[16 * hf]), lane);
+                const float cq = transpose_reduce16(*reinterpret_cast<float(*)[16]>(&sq[16 * hf]), lane);
+                if ((lane & 1) == 0) {
+                  tail->ssum[warp - 2][c_in_tile + 16 * hf + cl] += cs;
+                  tail->ssq[warp - 2][c_in_tile + 16 * hf + cl] += cq;
+                }
               }
             }
           }
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&tail->tmem_empty[buf]);
         slot_phase ^= 1u << buf;
         slot = slot + 1 == (uint32_t)p.nslots ? 0 : slot + 1;
         // flush the column sums when the channel tile is about to change (or at the very end)
@@ -314,12 +329,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (flush) {
           asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
           for (int c = et; c < p.n_tile_cols; c += kEpiThreads) {
-            if (col0 + c < p.Cout) {
-              atomicAdd(&p.stats[col0 + c], (double)tail->ssum[c]);
-              atomicAdd(&p.stats[p.Cout + col0 + c], (double)tail->ssq[c]);
+            float a_s = 0.f, a_q = 0.f;
+            for (int wi = 0; wi < kEpiThreads / 32; ++wi) {
+              a_s += tail->ssum[wi][c];
+              a_q += tail->ssq[wi][c];
+              tail->ssum[wi][c] = 0.f;
+              tail->ssq[wi][c] = 0.f;
             }
-            tail->ssum[c] = 0.f;
-            tail->ssq[c] = 0.f;
+            if (col0 + c < p.Cout) {
+              atomicAdd(&p.stats[col0 + c], (double)a_s);
+              atomicAdd(&p.stats[p.Cout + col0 + c], (double)a_q);
+            }
           }
           asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
         }
