@@ -13,8 +13,9 @@
 // tensor memory (3 for N_TILE = 160), so the epilogue of one unit overlaps the MMAs of the next
 // as far as slots are free.
 //
-// Roles (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = epilogue, two
-// warps per TMEM lane quarter taking alternate 32-column groups
+// Roles: warp 0 = TMA producer; warps 1 and 2 = MMA issuers, one per accumulator of a pair (a
+// tcgen05.mma costs its issuing thread about 65 cycles, close to the 80 cycles of tensor work of
+// an N = 160 instruction, so one issuer cannot keep the pipe full); warps 3.. = epilogue
 // (TMEM -> registers -> optional residual add -> bf16 store, per-channel sum / sum of squares
 // for the batch-norm that follows).  One persistent CTA per SM walks a contiguous tile range.
 #pragma once
@@ -97,7 +98,8 @@ __device__ __forceinline__ float transpose_reduce16(const float (&v)[16], int la
 #define LP_EPI_WARPS 4
 #endif
 constexpr int kEpiThreads = 32 * LP_EPI_WARPS;
-constexpr int kConvThreads = 64 + kEpiThreads;
+constexpr int kConvThreads = 96 + kEpiThreads;
+constexpr int kFirstEpiWarp = 3;
 constexpr int kEpiGroups = LP_EPI_WARPS / 4;
 
 __global__ void __launch_bounds__(kConvThreads, 1)
@@ -116,7 +118,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(&tail->full[s], 1);
-      mbar_init(&tail->empty[s], 1);
+      mbar_init(&tail->empty[s], 2);   // one arrival per MMA warp
     }
     for (int b = 0; b < kMaxSlots; ++b) {
       mbar_init(&tail->tmem_full[b], 1);
@@ -131,7 +133,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     (&tail->ssum[0][0])[i] = 0.f;
     (&tail->ssq[0][0])[i] = 0.f;
   }
-  if (warp == 2) {
+  if (warp == kFirstEpiWarp) {
     tmem_alloc(&tail->tmem_base, kTmemCols);
     tmem_relinquish();
   }
@@ -179,8 +181,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
       t += cnt;
     }
-  } else if (warp == 1) {
-    // ------------------------------- MMA issuer (warp-uniform loop, elected issue) ------
+  } else if (warp == 1 || warp == 2) {
+    // ------------------------------- MMA issuers (warp-uniform loops, elected issue) ----
+    // Warp 1 owns the first accumulator of every unit, warp 2 the second one of a pair.  Both
+    // wait for every stage and both arrive on its "empty" barrier: with a commit after their
+    // MMAs, or (warp 2 in a single-tile unit) with a plain arrive.
+    const int me = warp - 1;
     uint32_t s = 0, ph = 0;
     const uint32_t smem_base = smem_u32(smem);
     const int nk = p.KC >> 4;
@@ -191,32 +197,32 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t sl[2];
       sl[0] = slot;
       sl[1] = slot + 1 == (uint32_t)p.nslots ? 0 : slot + 1;
-      for (int a = 0; a < cnt && !failed; ++a)
-        if (!mbar_wait_warp(&tail->tmem_empty[sl[a]], ((slot_phase >> sl[a]) & 1) ^ 1, abort_flag)) failed = true;
-      if (failed) break;
-      tc_fence_after();
-      const uint32_t d0 = tmem_base + sl[0] * p.acc_stride, d1 = tmem_base + sl[1] * p.acc_stride;
+      const bool active = me < cnt;
+      if (active) {
+        if (!mbar_wait_warp(&tail->tmem_empty[sl[me]], ((slot_phase >> sl[me]) & 1) ^ 1, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+      }
+      const uint32_t d = tmem_base + sl[me] * p.acc_stride;
       for (int k = 0; k < kiters; ++k) {
         if (!mbar_wait_warp(&tail->full[s], ph, abort_flag)) { failed = true; break; }
         tc_fence_after();
         const uint32_t a_addr = smem_base + s * p.stage_bytes;
-        const uint64_t ad0 = smem_desc(p.desc_hi, a_addr), ad1 = smem_desc(p.desc_hi, a_addr + p.a_region_bytes);
+        const uint64_t ad = smem_desc(p.desc_hi, a_addr + me * p.a_region_bytes);
         const uint64_t bd = smem_desc(p.desc_hi, a_addr + p.b_offset);
         if (elect_one()) {
-          for (int j = 0; j < nk; ++j) {  // +32 bytes (one K = 16 slice) per step, in 16-byte units
-            mma_bf16(d0, ad0 + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k | j) ? 1u : 0u);
-            if (cnt == 2) mma_bf16(d1, ad1 + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k | j) ? 1u : 0u);
+          if (active) {
+            for (int j = 0; j < nk; ++j)  // +32 bytes (one K = 16 slice) per step, in 16-byte units
+              mma_bf16(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k | j) ? 1u : 0u);
+            mma_commit(&tail->empty[s]);
+          } else {
+            mbar_arrive(&tail->empty[s]);
           }
-          mma_commit(&tail->empty[s]);
         }
         __syncwarp();
         if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
       }
       if (failed) break;
-      if (elect_one()) {
-        mma_commit(&tail->tmem_full[sl[0]]);
-        if (cnt == 2) mma_commit(&tail->tmem_full[sl[1]]);
-      }
+      if (active && elect_one()) mma_commit(&tail->tmem_full[sl[me]]);
       __syncwarp();
       for (int a = 0; a < cnt; ++a) slot_phase ^= 1u << sl[a];
       slot = cnt == 2 ? (sl[1] + 1 == (uint32_t)p.nslots ? 0 : sl[1] + 1) : sl[1];
@@ -225,9 +231,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else {
     // ------------------------------- epilogue -----------------------------------------
     const int q = warp & 3;              // TMEM lane quarter this warp may read
-    const int grp = (warp - 2) >> 2;     // which of the two warps of the quarter
+    const int grp = (warp - kFirstEpiWarp) >> 2;  // which warp of the quarter (more than four epilogue warps)
     const int row = q * 32 + lane;
-    const int et = threadIdx.x - 64;     // 0..255
+    const int et = threadIdx.x - 32 * kFirstEpiWarp;
     const int rows_used = p.BW * p.BH * p.BNI;
     const int ngroups = (p.n_tile_cols + 31) >> 5;
     uint32_t slot = 0, slot_phase = 0;
@@ -314,8 +320,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const float cs = transpose_reduce16(*reinterpret_cast<float(*)[16]>(&v[16 * hf]), lane);
                 const float cq = transpose_reduce16(*reinterpret_cast<float(*)[16]>(&sq[16 * hf]), lane);
                 if ((lane & 1) == 0) {
-                  tail->ssum[warp - 2][c_in_tile + 16 * hf + cl] += cs;
-                  tail->ssq[warp - 2][c_in_tile + 16 * hf + cl] += cq;
+                  tail->ssum[warp - kFirstEpiWarp][c_in_tile + 16 * hf + cl] += cs;
+                  tail->ssq[warp - kFirstEpiWarp][c_in_tile + 16 * hf + cl] += cq;
                 }
               }
             }
@@ -361,7 +367,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);
   }
   __syncthreads();
-  if (warp == 2) {
+  if (warp == kFirstEpiWarp) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
