@@ -27,6 +27,8 @@ def main():
     ap.add_argument("--impl", type=int, default=2)
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--stats", action="store_true")
+    ap.add_argument("--sustain", type=float, default=0.0, help="also run back to back for this many seconds "
+                    "and report the sustained rate with the clocks and power seen (the part is power-capped)")
     a = ap.parse_args()
     pad = 1 if a.R == 3 else (0 if a.R == 1 else a.R // 2)
     OH = (a.H + 2 * pad - a.R) // a.stride + 1
@@ -57,9 +59,28 @@ def main():
             times.append(ms)
     flops = 2.0 * a.N * OH * OW * a.Cout * a.R * a.R * a.Cin
     med = float(np.median(times))
-    print(json.dumps({"op": a.op, "shape": [a.N, a.H, a.W, a.Cin, a.Cout, a.R, a.stride], "ms_median": med,
-                      "ms_min": float(min(times)), "tflops_median": flops / med / 1e9,
-                      "tflops_best": flops / min(times) / 1e9}))
+    out_line = {"op": a.op, "shape": [a.N, a.H, a.W, a.Cin, a.Cout, a.R, a.stride], "ms_median": med,
+                "ms_min": float(min(times)), "tflops_median": flops / med / 1e9,
+                "tflops_best": flops / min(times) / 1e9}
+    if a.sustain > 0:
+        import subprocess
+        import time
+        q = subprocess.Popen(["nvidia-smi", "-i", "0", "--query-gpu=clocks.sm,power.draw", "--format=csv,noheader,nounits",
+                              "-lms", "100"], stdout=subprocess.PIPE, text=True)
+        t0 = time.time()
+        sus = []
+        while time.time() - t0 < a.sustain:
+            for _ in range(50):
+                st, ms = lp.lp_conv2d(op, lp.LP_BF16, a.impl, a.N, a.H, a.W, a.Cin, a.Cout, a.R, a.stride, pad, ta, tb,
+                                      out, stats, base, nbytes, timed=True)
+                sus.append(ms)
+        q.terminate()
+        rows = [r.split(",") for r in q.stdout.read().strip().splitlines() if "," in r]
+        tail_ms = float(np.median(sus[len(sus) // 2:]))
+        out_line.update({"sustained_tflops": flops / tail_ms / 1e9,
+                         "sm_mhz_median": float(np.median([float(r[0]) for r in rows[len(rows) // 2:]])) if rows else None,
+                         "power_w_median": float(np.median([float(r[1]) for r in rows[len(rows) // 2:]])) if rows else None})
+    print(json.dumps(out_line))
 
 
 if __name__ == "__main__":
