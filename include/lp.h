@@ -155,6 +155,17 @@ int lp_modules_fwd_bwd_all(lp_handle* h, const void* const* x, const int32_t* la
 int lp_step(lp_handle* h, float lr, float momentum, float weight_decay, float kappa_step,
             void* const* lambdas_inout, void* stream);
 
+/* Steps 1-3 in one call with every dependency of Algorithm 1 and no more: the AuxNet chain runs
+ * on its own stream; module k starts as soon as x_k exists, takes its local loss as soon as
+ * x_{k+1} exists, and updates its own parameters (and multiplier) right after its own backward
+ * pass ("update unlocking", Section 4.1) without waiting for the other modules.  Arguments as in
+ * lp_auxnet_forward (x_out[k-1] receives x_k), lp_modules_fwd_bwd_all (loss_out float[K][2];
+ * dx[k] for k >= 1, array or entries may be NULL) and lp_step.  Everything is joined back into
+ * `stream` before the call's work is complete in stream order. */
+int lp_layer_parallel_step(lp_handle* h, const void* images, void* const* x_out, const int32_t* labels,
+                           void* const* lambdas_inout, float rho, float* loss_out, void* const* dx, float lr,
+                           float momentum, float weight_decay, float kappa_step, void* stream);
+
 /* Layer-serial comparator (K = 1 in the paper's notation): forward through all modules with
  * x_{k+1} := F_k(x_k); logits: device float[N][num_classes]. */
 int lp_forward_serial(lp_handle* h, const void* images, float* logits, void* stream);

@@ -12,7 +12,7 @@ __all__ = [
     "lp_get_params", "lp_get_grads", "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd",
     "lp_modules_fwd_bwd_all", "lp_step", "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual",
     "lp_last_device_status", "lp_launch_count", "lp_conv_profile", "lp_conv2d", "lp_conv2d_scratch_bytes", "lp_graph_begin", "lp_graph_end",
-    "lp_graph_launch", "lp_conv2d_fwd_noalloc", "LP_NOALLOC_SCRATCH_BYTES", "EXPORTED_SYMBOLS",
+    "lp_graph_launch", "lp_conv2d_fwd_noalloc", "LP_NOALLOC_SCRATCH_BYTES", "lp_layer_parallel_step", "EXPORTED_SYMBOLS",
 ]
 
 LP_OK = 0
@@ -29,7 +29,7 @@ EXPORTED_SYMBOLS = [
     "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd", "lp_modules_fwd_bwd_all", "lp_step",
     "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual", "lp_last_device_status", "lp_launch_count",
     "lp_conv_profile", "lp_conv2d_scratch_bytes", "lp_conv2d", "lp_graph_begin", "lp_graph_end", "lp_graph_launch",
-    "lp_conv2d_fwd_noalloc",
+    "lp_conv2d_fwd_noalloc", "lp_layer_parallel_step",
 ]
 
 
@@ -99,6 +99,8 @@ def library():
     lib.lp_modules_fwd_bwd_all.argtypes = [vp, ctypes.POINTER(vp), vp, ctypes.POINTER(vp), f32, vp,
                                            ctypes.POINTER(vp), vp]
     lib.lp_step.argtypes = [vp, f32, f32, f32, f32, ctypes.POINTER(vp), vp]
+    lib.lp_layer_parallel_step.argtypes = [vp, vp, ctypes.POINTER(vp), vp, ctypes.POINTER(vp), f32, vp,
+                                           ctypes.POINTER(vp), f32, f32, f32, f32, vp]
     lib.lp_forward_serial.argtypes = [vp, vp, vp, vp]
     lib.lp_serial_fwd_bwd.argtypes = [vp, vp, vp, vp, vp]
     lib.lp_get_residual.argtypes = [vp, i32, vp, vp, vp]
@@ -275,6 +277,16 @@ def lp_modules_fwd_bwd_all(h, x, labels, lambdas, rho, loss_out, dx, stream=None
 def lp_step(h, lr, momentum=0.0, weight_decay=0.0, kappa_step=0.0, lambdas_inout=None, stream=None):
     la = _ptr_array(lambdas_inout, h.K) if lambdas_inout is not None else None
     _check(library().lp_step(h.ptr, lr, momentum, weight_decay, kappa_step, la, _ptr(stream)), "lp_step")
+
+
+def lp_layer_parallel_step(h, images, x_out, labels, lambdas_inout, rho, loss_out, dx, lr, momentum=0.0,
+                           weight_decay=0.0, kappa_step=0.0, stream=None):
+    xa = _ptr_array(x_out, h.K - 1)
+    la = _ptr_array(lambdas_inout, h.K) if lambdas_inout is not None else None
+    da = _ptr_array(dx, h.K) if dx is not None else None
+    _check(library().lp_layer_parallel_step(h.ptr, _ptr(images), xa, _ptr(labels), la, rho, _ptr(loss_out), da, lr,
+                                            momentum, weight_decay, kappa_step, _ptr(stream)),
+           "lp_layer_parallel_step")
 
 
 def lp_forward_serial(h, images, logits, stream=None):

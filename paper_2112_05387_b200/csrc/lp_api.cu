@@ -122,6 +122,7 @@ struct RunCtx {
   float rho = 0.f;
   float* loss_out = nullptr;
   bool serial = false;       // layer-serial mode: interior modules produce `out`, no local loss
+  cudaEvent_t loss_wait = nullptr;  // recorded when x_{k+1} is ready: awaited just before the local loss
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -170,6 +171,9 @@ struct lp_handle {
   std::vector<cudaStream_t> streams;
   std::vector<cudaEvent_t> done;
   cudaEvent_t fork = nullptr;
+  cudaStream_t aux_stream = nullptr;
+  std::vector<cudaEvent_t> aux_done;  // aux_done[k]: x_{k+1} has been produced
+  cudaEvent_t aux_end = nullptr;
   int64_t launches = 0;
   ConvProfile prof;
   int conv_impl = LP_CONV_IMPL_AUTO;
@@ -958,6 +962,7 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       break;
     }
     case OP_OUT_LOSS: {
+      if (c.loss_wait && !c.serial) LP_CUDA_OK(cudaStreamWaitEvent(st, c.loss_wait, 0));
       const int C = op.out.c;
       const int threads = threads_for_channels(C, dtype);
       if (!threads) return LP_ERR_UNSUPPORTED;
@@ -1071,11 +1076,11 @@ static int pack_weights(lp_handle* h, Plan& P, cudaStream_t st) {
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 static int module_fwd_bwd(lp_handle* h, int k, const void* x_k, const void* x_next_or_labels, const void* lambda_k,
-                          float rho, float* loss_out, void* dx_k, cudaStream_t st) {
+                          float rho, float* loss_out, void* dx_k, cudaStream_t st, cudaEvent_t loss_wait = nullptr) {
   Plan& P = h->modules[k];
   const bool last = k == h->net.K - 1;
   RunCtx c;
-  c.st = st; c.x = x_k; c.rho = rho; c.loss_out = loss_out; c.dx = dx_k;
+  c.st = st; c.x = x_k; c.rho = rho; c.loss_out = loss_out; c.dx = dx_k; c.loss_wait = loss_wait;
   if (last) c.labels = (const int32_t*)x_next_or_labels;
   else { c.xnext = x_next_or_labels; c.kappa = lambda_k; }
   int rc = zero_forward_state(P, st);
@@ -1204,6 +1209,11 @@ int lp_create(const lp_net_desc* desc, void* dev_workspace, size_t bytes, lp_han
     }
   }
   if (cudaEventCreateWithFlags(&h->fork, cudaEventDisableTiming) != cudaSuccess) { delete h; return LP_ERR_CUDA; }
+  if (cudaStreamCreateWithFlags(&h->aux_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->aux_end, cudaEventDisableTiming) != cudaSuccess) { delete h; return LP_ERR_CUDA; }
+  h->aux_done.resize(net.K > 1 ? net.K - 1 : 0);
+  for (auto& e : h->aux_done)
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { delete h; return LP_ERR_CUDA; }
   *out = h;
   return LP_OK;
 }
@@ -1214,6 +1224,9 @@ int lp_destroy(lp_handle* h) {
   for (auto s : h->streams) if (s) cudaStreamDestroy(s);
   for (auto e : h->done) if (e) cudaEventDestroy(e);
   if (h->fork) cudaEventDestroy(h->fork);
+  if (h->aux_stream) cudaStreamDestroy(h->aux_stream);
+  if (h->aux_end) cudaEventDestroy(h->aux_end);
+  for (auto e : h->aux_done) if (e) cudaEventDestroy(e);
   for (auto& pr : h->prof.events) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
   for (auto g : h->graphs) cudaGraphExecDestroy(g);
   delete h;
@@ -1340,6 +1353,31 @@ int lp_modules_fwd_bwd_all(lp_handle* h, const void* const* x, const int32_t* la
   return LP_OK;
 }
 
+static int update_module(lp_handle* h, int k, float lr, float momentum, float weight_decay, float kappa_step,
+                         void* lambda_inout, cudaStream_t st) {
+  Plan& P = h->modules[k];
+  sgd_kernel<<<grid_for((long long)P.ps.n, 256, g_dev.sm_count, 8), 256, 0, st>>>(P.ps.p, P.ps.g, P.ps.m,
+                                                                                  (long long)P.ps.n, lr, momentum,
+                                                                                  weight_decay);
+  h->launches++;
+  LP_CUDA_OK(cudaGetLastError());
+  int rc = pack_weights(h, P, st);
+  if (rc != LP_OK) return rc;
+  P.ps.grads_fresh = false;
+  if (lambda_inout && k + 1 < h->net.K) {
+    const long long n = P.r.elems();
+    if (h->dtype == LP_F32)
+      kappa_update_kernel<float><<<grid_for(n / 4, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+          (float*)lambda_inout, (const float*)P.r.p, kappa_step, n / 4);
+    else
+      kappa_update_kernel<bf16><<<grid_for(n / 8, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+          (bf16*)lambda_inout, (const bf16*)P.r.p, kappa_step, n / 8);
+    h->launches++;
+    LP_CUDA_OK(cudaGetLastError());
+  }
+  return LP_OK;
+}
+
 int lp_step(lp_handle* h, float lr, float momentum, float weight_decay, float kappa_step, void* const* lambdas_inout,
             void* stream) {
   if (!h) return LP_ERR_NULL;
@@ -1352,28 +1390,62 @@ int lp_step(lp_handle* h, float lr, float momentum, float weight_decay, float ka
     for (int k = 0; k + 1 < K; ++k)
       if (lambdas_inout[k] && !aligned16(lambdas_inout[k])) return LP_ERR_ALIGN;
   for (int k = 0; k < K; ++k) {
-    Plan& P = h->modules[k];
-    if (!P.ps.grads_fresh) continue;
-    sgd_kernel<<<grid_for((long long)P.ps.n, 256, g_dev.sm_count, 8), 256, 0, st>>>(P.ps.p, P.ps.g, P.ps.m,
-                                                                                    (long long)P.ps.n, lr, momentum,
-                                                                                    weight_decay);
-    h->launches++;
-    LP_CUDA_OK(cudaGetLastError());
-    int rc = pack_weights(h, P, st);
+    if (!h->modules[k].ps.grads_fresh) continue;
+    int rc = update_module(h, k, lr, momentum, weight_decay, kappa_step,
+                           (lambdas_inout && k + 1 < K) ? lambdas_inout[k] : nullptr, st);
     if (rc != LP_OK) return rc;
-    P.ps.grads_fresh = false;
-    if (lambdas_inout && k + 1 < K && lambdas_inout[k]) {
-      const long long n = P.r.elems();
-      if (h->dtype == LP_F32)
-        kappa_update_kernel<float><<<grid_for(n / 4, 256, g_dev.sm_count, 8), 256, 0, st>>>(
-            (float*)lambdas_inout[k], (const float*)P.r.p, kappa_step, n / 4);
-      else
-        kappa_update_kernel<bf16><<<grid_for(n / 8, 256, g_dev.sm_count, 8), 256, 0, st>>>(
-            (bf16*)lambdas_inout[k], (const bf16*)P.r.p, kappa_step, n / 8);
-      h->launches++;
-      LP_CUDA_OK(cudaGetLastError());
-    }
   }
+  return LP_OK;
+}
+
+int lp_layer_parallel_step(lp_handle* h, const void* images, void* const* x_out, const int32_t* labels,
+                           void* const* lambdas_inout, float rho, float* loss_out, void* const* dx, float lr,
+                           float momentum, float weight_decay, float kappa_step, void* stream) {
+  if (!h || !images || !labels || !loss_out) return LP_ERR_NULL;
+  const int K = h->net.K;
+  if (K > 1 && !x_out) return LP_ERR_NULL;
+  if (!aligned16(images)) return LP_ERR_ALIGN;
+  for (int k = 0; k + 1 < K; ++k) {
+    if (!x_out[k]) return LP_ERR_NULL;
+    if (!aligned16(x_out[k]) || (lambdas_inout && lambdas_inout[k] && !aligned16(lambdas_inout[k])) ||
+        (dx && dx[k + 1] && !aligned16(dx[k + 1])))
+      return LP_ERR_ALIGN;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  LP_CUDA_OK(cudaEventRecord(h->fork, st));
+  // AuxNet chain on its own stream; aux_done[k] marks x_{k+1}
+  LP_CUDA_OK(cudaStreamWaitEvent(h->aux_stream, h->fork, 0));
+  {
+    RunCtx c;
+    c.st = h->aux_stream; c.images = images; c.xout = x_out;
+    for (int k = 0; k + 1 < K; ++k) {
+      int rc = zero_forward_state(h->auxs[k], c.st);
+      if (rc != LP_OK) return rc;
+      rc = run_ops(h, h->auxs[k], h->auxs[k].fwd, c);
+      if (rc != LP_OK) return rc;
+      LP_CUDA_OK(cudaEventRecord(h->aux_done[k], h->aux_stream));
+    }
+    LP_CUDA_OK(cudaEventRecord(h->aux_end, h->aux_stream));
+  }
+  // module k starts as soon as x_k exists, takes its local loss as soon as x_{k+1} exists, and
+  // updates its own parameters right after its own backward pass
+  for (int k = 0; k < K; ++k) {
+    cudaStream_t sk = h->streams[k];
+    LP_CUDA_OK(cudaStreamWaitEvent(sk, h->fork, 0));
+    if (k > 0) LP_CUDA_OK(cudaStreamWaitEvent(sk, h->aux_done[k - 1], 0));
+    const bool last = k == K - 1;
+    const void* xk = k == 0 ? images : x_out[k - 1];
+    const void* tgt = last ? (const void*)labels : (const void*)x_out[k];
+    void* lam = (lambdas_inout && !last) ? lambdas_inout[k] : nullptr;
+    int rc = module_fwd_bwd(h, k, xk, tgt, lam, rho, loss_out + 2 * k, dx ? dx[k] : nullptr, sk,
+                            last ? nullptr : h->aux_done[k]);
+    if (rc != LP_OK) return rc;
+    rc = update_module(h, k, lr, momentum, weight_decay, kappa_step, lam, sk);
+    if (rc != LP_OK) return rc;
+    LP_CUDA_OK(cudaEventRecord(h->done[k], sk));
+  }
+  LP_CUDA_OK(cudaStreamWaitEvent(st, h->aux_end, 0));
+  for (int k = 0; k < K; ++k) LP_CUDA_OK(cudaStreamWaitEvent(st, h->done[k], 0));
   return LP_OK;
 }
 

@@ -196,6 +196,39 @@ def test_serial_forward_matches_oracle_and_serial_backprop_is_bp():
         d = r2["dx"]
 
 
+@pytest.mark.parametrize("which", ["tiny", "bf16-preact", "bf16-postbn"])
+def test_fused_step_equals_the_three_separate_calls(which):
+    """lp_layer_parallel_step (AuxNet stream, per-module start / loss / update events) computes what
+    lp_auxnet_forward + lp_modules_fwd_bwd_all + lp_step compute: same boundaries, losses, gradients,
+    updated parameters and multipliers (only the order of fp32 atomic sums differs)."""
+    if which == "tiny":
+        cfg, tol = get_config("tiny"), 1e-5
+    else:
+        cfg = small_cfg(which.split("-")[1], N=8, H=16, W=16, dtype="bf16", stage_channels=(16, 32), stage_blocks=(2, 2),
+                        module_block_end=(1, 3, 4), stem_channels=16, classes=10)
+        tol = 2e-2
+    a, b = GpuRun(cfg), GpuRun(cfg)
+    K, lp = a.net.K, a.lp
+    lr, c = 1e-4, cfg["rho"]
+    a.cfg["lr"] = lr
+    a.auxnet()
+    ga = a.fwd_bwd_all()
+    a.step(kappa_step=c)
+    lp.lp_layer_parallel_step(b.h, b.d_images, b.d_x[1:], b.d_labels, b.d_kappa if b.use_kappa else None, cfg["rho"],
+                              b.d_loss, b.d_dx, lr, 0.0, 0.0, c)
+    assert lp.lp_last_device_status(b.h) == 0
+    for k in range(1, K):
+        assert rel_err(to_host(b.d_x[k]), to_host(a.d_x[k])) < tol
+        assert rel_err(to_host(b.d_dx[k]), to_host(a.d_dx[k])) < tol
+    np.testing.assert_allclose(b.d_loss.cpu().numpy(), a.d_loss.cpu().numpy(), rtol=max(tol, 1e-5))
+    for k in range(K):
+        assert rel_err(lp.lp_get_grads(b.h, k), ga[k]) < tol
+        assert rel_err(lp.lp_get_params(b.h, k), lp.lp_get_params(a.h, k)) < tol
+    if a.use_kappa:
+        for k in range(K - 1):
+            assert rel_err(to_host(b.d_kappa[k]), to_host(a.d_kappa[k])) < tol
+
+
 def test_argument_errors_are_reported_on_the_host():
     cfg = get_config("tiny")
     run = GpuRun(cfg)
