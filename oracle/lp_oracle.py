@@ -324,6 +324,63 @@ def auxnet_apply(net, k, p, x):
     return _st(net, h)
 
 
+def auxnet_fwd_bwd(net, k, params_flat, x_in, target):
+    """Distillation loss D = ||target - AuxNet_k(x_in)||^2 (Eq. AV-Net-lambda: `target` is the
+    corrected auxiliary variable, held constant) and its gradient with respect to AuxNet_k's
+    parameters.  Returns dict(out, loss, grads (flat, blob order))."""
+    p = net.unpack(LP_AUX(k), params_flat)
+    convs = net.aux[k]
+    x_in = np.asarray(x_in, dtype=F)
+    y1 = _st(net, conv_fwd(x_in, _wq(net, p["conv1.w"]), convs[0]["stride"], 1))
+    z1, c1 = bn_fwd(y1, p["bn1.g"], p["bn1.b"], net.eps)
+    g = {}
+    if len(convs) == 2:
+        h = _st(net, relu(z1))
+        y2 = _st(net, conv_fwd(h, _wq(net, p["conv2.w"]), convs[1]["stride"], 1))
+        z2, c2 = bn_fwd(y2, p["bn2.g"], p["bn2.b"], net.eps)
+        out = _st(net, z2)
+    else:
+        out = _st(net, z1)
+    diff = out - np.asarray(target, dtype=F)
+    loss = float((diff * diff).sum())
+    d = _st(net, 2.0 * diff)
+    if len(convs) == 2:
+        dy2, g["bn2.g"], g["bn2.b"] = bn_bwd(d, c2, p["bn2.g"])
+        dy2 = _st(net, dy2)
+        g["conv2.w"] = conv_wgrad(h, dy2, p["conv2.w"].shape, convs[1]["stride"], 1)
+        dh = _st(net, conv_dgrad(dy2, _wq(net, p["conv2.w"]), convs[1]["stride"], 1, h.shape))
+        d = relu_bwd(dh, z1)
+    dy1, g["bn1.g"], g["bn1.b"] = bn_bwd(d, c1, p["bn1.g"])
+    dy1 = _st(net, dy1)
+    g["conv1.w"] = conv_wgrad(x_in, dy1, p["conv1.w"].shape, convs[0]["stride"], 1)
+    return dict(out=out, loss=loss, grads=net.pack(LP_AUX(k), g))
+
+
+def aux_correction(x_k, dx_k, seed_prev, lr_lambda):
+    """Correction of the auxiliary variable x_k (Eq. Parallel-ResNet-Slack-Variables-Update):
+    x_k <- x_k - lr * (P^k_{kn} + beta dpsi(x_k, out_{k-1})/dx_k - kappa_k).  With psi the squared
+    l2 norm and beta = rho/2 the last two terms are -(rho r_{k-1} + kappa_k), minus the terminal
+    adjoint of module k-1, so the direction is g_k = dx_k - seed_{k-1}."""
+    g = np.asarray(dx_k, dtype=F) - np.asarray(seed_prev, dtype=F)
+    return np.asarray(x_k, dtype=F) - lr_lambda * g, g
+
+
+def auxnet_distill_step(net, aux_params, images, xs, dxs, seeds, lr_lambda, lr_aux):
+    """Second parallel loop of Algorithm 1 for every boundary k = 1..K-1: correct x_k, then one SGD
+    step of AuxNet_{k-1} on ||x_k_new - AuxNet_{k-1}(x_{k-1})||^2 (x_{k-1} and x_k_new constant).
+    xs[k-1] = x_k, dxs[k-1] = dx_k, seeds[k-1] = terminal adjoint of module k-1."""
+    new_params, new_x, losses, grads = [], [], [], []
+    for k in range(1, net.K):
+        x_new, _ = aux_correction(xs[k - 1], dxs[k - 1], seeds[k - 1], lr_lambda)
+        x_in = images if k == 1 else xs[k - 2]
+        res = auxnet_fwd_bwd(net, k - 1, aux_params[k - 1], x_in, x_new)
+        new_params.append(sgd_update(aux_params[k - 1], res["grads"], lr_aux)[0])
+        new_x.append(x_new)
+        losses.append(res["loss"])
+        grads.append(res["grads"])
+    return new_params, new_x, losses, grads
+
+
 def auxnet_forward(net, aux_params, images, post=None):
     """Serial chain x_0 = images, x_{k+1} = AuxNet_k(x_k).  ``post`` (optional) is applied to
     each x_{k+1} before it feeds the next AuxNet (tests use it to model storage rounding)."""

@@ -238,3 +238,60 @@ def test_torch_autograd_crosscheck():
         tg = net.pack(k, {n: v.grad.numpy() for n, v in named.items()})
         np.testing.assert_allclose(res["grads"], tg, rtol=1e-7, atol=1e-10)
         np.testing.assert_allclose(res["dx"], xt.grad.numpy(), rtol=1e-7, atol=1e-12)
+
+
+# -- AuxNet correction and distillation (second loop of Algorithm 1) ---------------------------
+@pytest.mark.parametrize("name,mk", ALL_CFGS[:3] + ALL_CFGS[4:])
+def test_auxnet_distillation_gradients(name, mk):
+    cfg = mk()
+    net, mods, auxs = build(cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    xs = [x0] + O.auxnet_forward(net, auxs, x0)
+    for k in range(net.K - 1):
+        target = xs[k + 1] + 0.3 * gen.normal(8, "t%d" % k, xs[k + 1].shape)
+        res = O.auxnet_fwd_bwd(net, k, auxs[k], xs[k], target)
+        np.testing.assert_allclose(res["out"], xs[k + 1], rtol=1e-12, atol=1e-12)     # same forward as the chain
+        assert abs(res["loss"] - float(((xs[k + 1] - target) ** 2).sum())) < 1e-9 * res["loss"]
+        p0 = auxs[k].astype(np.float64)
+
+        def loss_of(p):
+            out = O.auxnet_apply(net, k, net.unpack(O.LP_AUX(k), p), xs[k])
+            return float(((out - target) ** 2).sum())
+        off = 0
+        for pname, _, shape in net.param_layout(O.LP_AUX(k)):
+            n = int(np.prod(shape))
+            for j in sorted(set([off, off + n // 2, off + n - 1])):
+                h = 1e-5
+                pp, pm = p0.copy(), p0.copy()
+                pp[j] += h
+                pm[j] -= h
+                fd = (loss_of(pp) - loss_of(pm)) / (2 * h)
+                assert abs(fd - res["grads"][j]) < 2e-6 * max(1.0, res["loss"]) + 1e-5 * abs(fd), (name, k, pname, j)
+            off += n
+        # the target reproduced exactly: zero loss, zero gradients
+        zero = O.auxnet_fwd_bwd(net, k, auxs[k], xs[k], xs[k + 1])
+        assert zero["loss"] == 0.0 and np.all(zero["grads"] == 0.0)
+
+
+def test_aux_correction_direction_and_distillation_is_linear_in_the_step():
+    """g_k = P^k_{kn} + rho (x_k - out_{k-1}) - kappa_k = dx_k - seed_{k-1}; the distillation gradient
+    for the target x_k - lr*g_k is 2*lr*J^T g_k, linear in lr."""
+    cfg = get_config("tiny")
+    net, mods, auxs = build(cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    xs = [x0] + O.auxnet_forward(net, auxs, x0)
+    labels = gen.make_labels(cfg)
+    rho = 0.7
+    kap = gen.normal(3, "kap", xs[1].shape, std=0.2)
+    r0 = O.module_fwd_bwd(net, 0, mods[0], xs[0], xs[1], kap, rho)
+    r1 = O.module_fwd_bwd(net, 1, mods[1], xs[1], labels, None, rho)
+    x_new, g = O.aux_correction(xs[1], r1["dx"], r0["seed"], 0.05)
+    np.testing.assert_allclose(g, r1["dx"] + rho * (xs[1] - r0["out"]) - kap, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(x_new, xs[1] - 0.05 * g, rtol=1e-14)
+    g1 = O.auxnet_fwd_bwd(net, 0, auxs[0], x0, xs[1] - 0.05 * g)["grads"]
+    g2 = O.auxnet_fwd_bwd(net, 0, auxs[0], x0, xs[1] - 0.10 * g)["grads"]
+    np.testing.assert_allclose(g2, 2 * g1, rtol=1e-9, atol=1e-12)
+    newp, newx, losses, grads = O.auxnet_distill_step(net, auxs, x0, xs[1:], [r1["dx"]], [r0["seed"]], 0.05, 0.01)
+    np.testing.assert_allclose(grads[0], g1, rtol=1e-12)
+    np.testing.assert_allclose(newp[0], auxs[0] - 0.01 * g1, rtol=1e-12, atol=1e-15)
+    assert abs(losses[0] - 0.05 ** 2 * float((g * g).sum())) < 1e-12 * max(1.0, losses[0])
