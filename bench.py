@@ -364,6 +364,33 @@ def run_ours(args):
         conv_ms, conv_flops, conv_launches = lp.lp_conv_profile(h, False, read=True)
         barrier()
 
+        distill = None
+        if not args.no_serial and world == 1 and K > 1:
+            d_dloss = torch.zeros(K - 1, dtype=torch.float32, device=dev)
+
+            def step_with_distill():
+                step_direct()
+                lp.lp_auxnet_distill(h, d_images, d_x[1:], d_dx, 1e-9, 1e-9, None, d_dloss, sp)
+            step_with_distill()
+            dgid = None
+            if not args.no_graph:
+                lp.lp_graph_begin(h, sp)
+                step_with_distill()
+                dgid = lp.lp_graph_end(h, sp)
+            for _ in range(3):
+                lp.lp_graph_launch(h, dgid, sp) if dgid is not None else step_with_distill()
+            barrier()
+            d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_d = max(3, args.steps // 3)
+            d0.record(stream)
+            for _ in range(n_d):
+                lp.lp_graph_launch(h, dgid, sp) if dgid is not None else step_with_distill()
+            d1.record(stream)
+            barrier()
+            distill = {"value": cfg["N"] * n_d / (d0.elapsed_time(d1) * 1e-3), "unit": UNIT,
+                       "what": "the step followed by lp_auxnet_distill (auxiliary-variable correction + one AuxNet "
+                               "distillation step per boundary): all of Algorithm 1"}
+
         three = None
         if not args.no_serial and world == 1:
             step_three_calls()
@@ -453,6 +480,8 @@ def run_ours(args):
         line["layer_serial"] = serial
     if three:
         line["three_calls"] = three
+    if distill:
+        line["with_distillation"] = distill
     if not args.no_cpu_baseline and world == 1:
         sb = oracle_sample_batch(cfg)
         val, dt = time_oracle_step(args.workload, sb)

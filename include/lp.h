@@ -166,6 +166,20 @@ int lp_layer_parallel_step(lp_handle* h, const void* images, void* const* x_out,
                            void* const* lambdas_inout, float rho, float* loss_out, void* const* dx, float lr,
                            float momentum, float weight_decay, float kappa_step, void* stream);
 
+/* Second parallel loop of Algorithm 1, for every boundary k = 1..K-1: the correction direction of
+ * the auxiliary variable, g_k = dx_k - seed_{k-1} (Eq. Parallel-ResNet-Slack-Variables-Update: the
+ * input gradient of module k plus the gradient of module k-1's penalty/AL term with respect to
+ * x_k, which is minus its terminal adjoint), the corrected variable x_k_new = x_k - lr_lambda*g_k,
+ * and ONE SGD step (rate lr_aux) of AuxNet_{k-1} on ||x_k_new - AuxNet_{k-1}(x_{k-1})||^2 with
+ * x_{k-1} and x_k_new held constant (Eq. AV-Net-lambda, local knowledge distillation).
+ * Call after lp_auxnet_forward and the module passes of the same batch (the AuxNet activations and
+ * the terminal adjoints are taken from the workspace).
+ *   x[k-1] = x_k as produced by lp_auxnet_forward (K-1 device pointers); dx[k] = dx_k (K entries,
+ *   entry 0 unused); x_new[k-1] (array or entries may be NULL) receives x_k_new;
+ *   loss_out: device float[K-1], the distillation losses before the update (= lr_lambda^2 ||g_k||^2). */
+int lp_auxnet_distill(lp_handle* h, const void* images, void* const* x, const void* const* dx, float lr_lambda,
+                      float lr_aux, void* const* x_new, float* loss_out, void* stream);
+
 /* Layer-serial comparator (K = 1 in the paper's notation): forward through all modules with
  * x_{k+1} := F_k(x_k); logits: device float[N][num_classes]. */
 int lp_forward_serial(lp_handle* h, const void* images, float* logits, void* stream);

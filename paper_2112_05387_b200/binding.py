@@ -12,7 +12,7 @@ __all__ = [
     "lp_get_params", "lp_get_grads", "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd",
     "lp_modules_fwd_bwd_all", "lp_step", "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual",
     "lp_last_device_status", "lp_launch_count", "lp_conv_profile", "lp_conv2d", "lp_conv2d_scratch_bytes", "lp_graph_begin", "lp_graph_end",
-    "lp_graph_launch", "lp_conv2d_fwd_noalloc", "LP_NOALLOC_SCRATCH_BYTES", "lp_layer_parallel_step", "EXPORTED_SYMBOLS",
+    "lp_graph_launch", "lp_conv2d_fwd_noalloc", "LP_NOALLOC_SCRATCH_BYTES", "lp_layer_parallel_step", "lp_auxnet_distill", "EXPORTED_SYMBOLS",
 ]
 
 LP_OK = 0
@@ -29,7 +29,7 @@ EXPORTED_SYMBOLS = [
     "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd", "lp_modules_fwd_bwd_all", "lp_step",
     "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual", "lp_last_device_status", "lp_launch_count",
     "lp_conv_profile", "lp_conv2d_scratch_bytes", "lp_conv2d", "lp_graph_begin", "lp_graph_end", "lp_graph_launch",
-    "lp_conv2d_fwd_noalloc", "lp_layer_parallel_step",
+    "lp_conv2d_fwd_noalloc", "lp_layer_parallel_step", "lp_auxnet_distill",
 ]
 
 
@@ -101,6 +101,7 @@ def library():
     lib.lp_step.argtypes = [vp, f32, f32, f32, f32, ctypes.POINTER(vp), vp]
     lib.lp_layer_parallel_step.argtypes = [vp, vp, ctypes.POINTER(vp), vp, ctypes.POINTER(vp), f32, vp,
                                            ctypes.POINTER(vp), f32, f32, f32, f32, vp]
+    lib.lp_auxnet_distill.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), f32, f32, ctypes.POINTER(vp), vp, vp]
     lib.lp_forward_serial.argtypes = [vp, vp, vp, vp]
     lib.lp_serial_fwd_bwd.argtypes = [vp, vp, vp, vp, vp]
     lib.lp_get_residual.argtypes = [vp, i32, vp, vp, vp]
@@ -287,6 +288,14 @@ def lp_layer_parallel_step(h, images, x_out, labels, lambdas_inout, rho, loss_ou
     _check(library().lp_layer_parallel_step(h.ptr, _ptr(images), xa, _ptr(labels), la, rho, _ptr(loss_out), da, lr,
                                             momentum, weight_decay, kappa_step, _ptr(stream)),
            "lp_layer_parallel_step")
+
+
+def lp_auxnet_distill(h, images, x, dx, lr_lambda, lr_aux, x_new, loss_out, stream=None):
+    xa = _ptr_array(x, h.K - 1)
+    da = _ptr_array(dx, h.K)
+    na = _ptr_array(x_new, h.K - 1) if x_new is not None else None
+    _check(library().lp_auxnet_distill(h.ptr, _ptr(images), xa, da, lr_lambda, lr_aux, na, _ptr(loss_out), _ptr(stream)),
+           "lp_auxnet_distill")
 
 
 def lp_forward_serial(h, images, logits, stream=None):

@@ -502,6 +502,50 @@ __global__ void kappa_update_kernel(T* __restrict__ kappa, const T* __restrict__
   }
 }
 
+// Correction of an auxiliary variable and seed of the AuxNet distillation:
+//   g = dx_k - seed_{k-1};  x_new = x_k - lr*g (optional output);  d = 2*(x_k - x_new) = 2*lr*g;
+//   acc[0] += sum (lr*g)^2   (the distillation loss ||x_new - AuxNet(x_{k-1})||^2 before the update)
+template <typename T>
+__global__ void distill_seed_kernel(const T* __restrict__ xk, const T* __restrict__ dxk, const T* __restrict__ seed_prev,
+                                    float lr, T* __restrict__ x_new, T* __restrict__ d_out, double* __restrict__ acc,
+                                    long long total_vecs) {
+  constexpr int V = VecT<T>::N;
+  float sum = 0.f;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs;
+       i += (long long)gridDim.x * blockDim.x) {
+    float a[V], b[V], x[V];
+    ldv(dxk + i * V, a);
+    ldv(seed_prev + i * V, b);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      a[j] = lr * (a[j] - b[j]);
+      sum += a[j] * a[j];
+    }
+    if (x_new) {
+      ldv(xk + i * V, x);
+#pragma unroll
+      for (int j = 0; j < V; ++j) x[j] -= a[j];
+      stv(x_new + i * V, x);
+    }
+#pragma unroll
+    for (int j = 0; j < V; ++j) a[j] *= 2.f;
+    stv(d_out + i * V, a);
+  }
+  __shared__ float red[32];
+  sum = warp_sum(sum);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float v = threadIdx.x < (blockDim.x + 31) / 32 ? red[threadIdx.x] : 0.f;
+    v = warp_sum(v);
+    if (threadIdx.x == 0) atomicAdd(&acc[0], (double)v);
+  }
+}
+
+__global__ void distill_loss_kernel(const double* __restrict__ acc, float* __restrict__ loss_out) {
+  loss_out[0] = (float)acc[0];
+}
+
 // bf16 operand copies of one convolution's fp32 master weights w[co][t][ci]:
 //   wf[co][t*Cin + ci]  (forward B operand, K-major)      wt[ci][t*Cout + co]  (dgrad B operand)
 struct PackEntry {

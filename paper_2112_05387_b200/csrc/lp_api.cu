@@ -360,7 +360,7 @@ static bool tc_dgrad_ok(const ConvDef& c) {
   return tc_fwd_ok(c) && (c.stride == 1 || (c.H % 2 == 0 && c.W % 2 == 0));
 }
 static bool tc_wgrad_ok(const ConvDef& c) {
-  return c.cin % 16 == 0 && c.cout % 16 == 0 && (c.R == 1 || c.R == 3) && (c.stride == 1 || c.stride == 2);
+  return c.cin % 8 == 0 && c.cout % 16 == 0 && (c.R == 1 || c.R == 3) && (c.stride == 1 || c.stride == 2);
 }
 
 struct ProfScope {
@@ -863,13 +863,17 @@ struct Planner {
     std::vector<int> ci, bi;
     for (size_t i = 0; i < cv.size(); ++i) {
       const std::string id = std::to_string(i + 1);
-      ci.push_back(add_conv(P, "conv" + id + ".w", cv[i].cin, cv[i].cout, 3, cv[i].stride, 1, cv[i].hin, cv[i].win, false));
+      // the distillation step back-propagates through the second convolution into the first
+      ci.push_back(add_conv(P, "conv" + id + ".w", cv[i].cin, cv[i].cout, 3, cv[i].stride, 1, cv[i].hin, cv[i].win, i > 0));
       bi.push_back(add_bn(P, "bn" + id, cv[i].cout, (long long)s.n * cv[i].hout * cv[i].wout));
     }
     finish_stats(P);
     Tensor cur = x;
+    std::vector<Tensor> ins, ys, acts;
     for (size_t i = 0; i < cv.size(); ++i) {
+      ins.push_back(cur);
       Tensor y = emit_conv(P, P.fwd, cur, ci[i], nullptr, bi[i]);
+      ys.push_back(y);
       const bool final_conv = i + 1 == cv.size();
       Tensor out;
       Op op;
@@ -882,9 +886,20 @@ struct Planner {
       }
       op.out = out;
       P.fwd.push_back(op);
+      acts.push_back(out);
       cur = out;
     }
     P.out = cur;
+    // backward of the distillation loss ||x_{k+1}^{new} - AuxNet_k(x_k)||^2, seeded in P.seed
+    const Shape4 o = net.boundary[k + 1];
+    P.seed = new_tensor(o.n, o.h, o.w, o.c);
+    Tensor d = P.seed;
+    for (int i = (int)cv.size() - 1; i >= 0; --i) {
+      const bool relu_after = i + 1 < (int)cv.size();
+      Tensor dy = emit_bn_bwd(P.bwd, d, ys[i], relu_after ? &acts[i] : nullptr, bi[i], nullptr);
+      emit_wgrad(P.bwd, ins[i], dy, ci[i]);
+      if (i > 0) d = emit_dgrad(P, P.bwd, dy, ci[i], nullptr, nullptr);
+    }
   }
 };
 
@@ -1446,6 +1461,48 @@ int lp_layer_parallel_step(lp_handle* h, const void* images, void* const* x_out,
   }
   LP_CUDA_OK(cudaStreamWaitEvent(st, h->aux_end, 0));
   for (int k = 0; k < K; ++k) LP_CUDA_OK(cudaStreamWaitEvent(st, h->done[k], 0));
+  return LP_OK;
+}
+
+int lp_auxnet_distill(lp_handle* h, const void* images, void* const* x, const void* const* dx, float lr_lambda,
+                      float lr_aux, void* const* x_new, float* loss_out, void* stream) {
+  if (!h || !images || !x || !dx || !loss_out) return LP_ERR_NULL;
+  const int K = h->net.K;
+  if (!aligned16(images)) return LP_ERR_ALIGN;
+  for (int k = 1; k < K; ++k) {
+    if (!x[k - 1] || !dx[k]) return LP_ERR_NULL;
+    if (!aligned16(x[k - 1]) || !aligned16(dx[k]) || (x_new && x_new[k - 1] && !aligned16(x_new[k - 1]))) return LP_ERR_ALIGN;
+    if (!h->modules[k - 1].ran_fwd_bwd) return LP_ERR_ORDER;  // its terminal adjoint is the other half of g_k
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  RunCtx c;
+  c.st = st; c.images = images; c.xout = x;
+  for (int k = 1; k < K; ++k) {
+    Plan& A = h->auxs[k - 1];
+    const long long n = A.seed.elems();
+    LP_CUDA_OK(cudaMemsetAsync(A.loss_acc, 0, 2 * sizeof(double), st));
+    LP_CUDA_OK(cudaMemsetAsync(A.ps.g, 0, A.ps.n * 4, st));
+    void* xn = x_new ? x_new[k - 1] : nullptr;
+    if (h->dtype == LP_F32)
+      distill_seed_kernel<float><<<grid_for(n / 4, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+          (const float*)x[k - 1], (const float*)dx[k], (const float*)h->modules[k - 1].seed.p, lr_lambda,
+          (float*)xn, (float*)A.seed.p, A.loss_acc, n / 4);
+    else
+      distill_seed_kernel<bf16><<<grid_for(n / 8, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+          (const bf16*)x[k - 1], (const bf16*)dx[k], (const bf16*)h->modules[k - 1].seed.p, lr_lambda, (bf16*)xn,
+          (bf16*)A.seed.p, A.loss_acc, n / 8);
+    distill_loss_kernel<<<1, 1, 0, st>>>(A.loss_acc, loss_out + (k - 1));
+    h->launches += 2;
+    LP_CUDA_OK(cudaGetLastError());
+    int rc = run_ops(h, A, A.bwd, c);
+    if (rc != LP_OK) return rc;
+    sgd_kernel<<<grid_for((long long)A.ps.n, 256, g_dev.sm_count, 8), 256, 0, st>>>(A.ps.p, A.ps.g, A.ps.m,
+                                                                                    (long long)A.ps.n, lr_aux, 0.f, 0.f);
+    h->launches++;
+    LP_CUDA_OK(cudaGetLastError());
+    rc = pack_weights(h, A, st);
+    if (rc != LP_OK) return rc;
+  }
   return LP_OK;
 }
 

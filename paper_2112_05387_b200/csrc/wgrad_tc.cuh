@@ -170,9 +170,10 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       tc_fence_after();
       for (int a = 0; a < cnt; ++a) {
         const int g = (m_tile + a) * p.rpt + row / p.sca;
-        const bool valid = g < p.total_chunks;
+        const int ci_raw = (g % p.cin_chunks) * p.sca + row % p.sca;
+        const bool valid = g < p.total_chunks && ci_raw < p.Cin;
         const int tap = valid ? g / p.cin_chunks : 0;
-        const int ci = valid ? (g % p.cin_chunks) * p.sca + row % p.sca : 0;
+        const int ci = valid ? ci_raw : 0;
         const uint32_t taddr = tmem_base + a * 256 + ((uint32_t)(q * 32) << 16);
         const int co0 = n_tile * p.n_tile;
         for (int cc = 0; cc < (p.n_tile >> 4); ++cc) {
@@ -241,9 +242,11 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf
   p.Nimg = N; p.OH = OH; p.OW = OW;
   p.stride = stride; p.pad = pad; p.R = R;
   p.Cin = Cin; p.Cout = Cout; p.taps = R * R;
+  // sub-box width of x: the widest that divides C_in; otherwise 16 with zero fill past the last
+  // channel (C_in = 40: chunks 0-15, 16-31, 32-47)
   p.sca = Cin % 64 == 0 ? 64 : (Cin % 32 == 0 ? 32 : 16);
   p.rpt = 128 / p.sca;
-  p.cin_chunks = Cin / p.sca;
+  p.cin_chunks = (Cin + p.sca - 1) / p.sca;
   p.total_chunks = p.taps * p.cin_chunks;
   p.m_tiles = (p.total_chunks + p.rpt - 1) / p.rpt;
   int best_tile = 0;

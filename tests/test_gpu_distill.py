@@ -1,0 +1,76 @@
+"""GPU parity of the auxiliary-variable correction and AuxNet distillation (lp_auxnet_distill)
+against the oracle: corrected variables, distillation losses, AuxNet parameter updates."""
+import numpy as np
+import pytest
+
+from conftest import small_cfg
+from harness import GpuRun, oracle_modules, per_tensor_errors, rel_err, to_host
+from oracle import lp_oracle as O
+from workloads import gen, get_config
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(cfg, tol, lr_lambda=0.05, lr_aux=0.01):
+    run = GpuRun(cfg)
+    net, lp, torch = run.net, run.lp, run.torch
+    K = net.K
+    post = (lambda a: gen.storage_round(a, cfg["dtype"]))
+    ox = O.auxnet_forward(net, run.auxs, run.images, post=post)
+    run.auxnet()                      # fills the AuxNet activations in the workspace
+    run.set_boundaries(ox)            # module inputs and distillation inputs are the oracle's
+    xs_host = [to_host(t) for t in run.d_x[1:]]
+    run.fwd_bwd_all()
+    ref = oracle_modules(run, xs_host)
+    d_new = [torch.zeros_like(run.d_x[k]) for k in range(1, K)]
+    d_loss = torch.zeros(K - 1, dtype=torch.float32, device="cuda:0")
+    before = [lp.lp_get_params(run.h, lp.LP_AUX(k)).astype(np.float64) for k in range(K - 1)]
+    lp.lp_auxnet_distill(run.h, run.d_images, run.d_x[1:], run.d_dx, lr_lambda, lr_aux, d_new, d_loss)
+    assert lp.lp_last_device_status(run.h) == 0
+    # oracle: same storage model as the module comparison
+    net.store = None if cfg["dtype"] == "f32" else gen.round_bf16
+    newp, newx, losses, grads = O.auxnet_distill_step(net, run.auxs, run.images.astype(np.float64), xs_host,
+                                                     [r["dx"] for r in ref[1:]], [r["seed"] for r in ref[:-1]],
+                                                     lr_lambda, lr_aux)
+    net.store = None
+    got_loss = d_loss.cpu().numpy()
+    for k in range(K - 1):
+        assert rel_err(to_host(d_new[k]), newx[k]) < tol, ("x_new", k)
+        assert abs(got_loss[k] - losses[k]) < 2 * tol * losses[k], ("loss", k, got_loss[k], losses[k])
+        g_gpu = lp.lp_get_grads(run.h, lp.LP_AUX(k))
+        errs = per_tensor_errors(net, O.LP_AUX(k), g_gpu, grads[k])
+        assert max(errs.values()) < tol, (k, errs)
+        after = lp.lp_get_params(run.h, lp.LP_AUX(k)).astype(np.float64)
+        assert rel_err(after, newp[k]) < tol
+        upd = per_tensor_errors(net, O.LP_AUX(k), after - before[k], newp[k] - run.auxs[k])
+        big = {n: e for n, e in upd.items() if e >= tol + 1e-3}
+        assert not big or cfg["dtype"] == "bf16", (k, big)
+
+
+def test_distill_tiny_fp32():
+    run_case(get_config("tiny"), 1e-4)
+
+
+@pytest.mark.parametrize("kind", ["postbn", "preact"])
+def test_distill_small_fp32_two_conv_auxnets(kind):
+    cfg = small_cfg(kind, N=4, H=8, W=8, stage_channels=(8, 16), stage_blocks=(2, 2), module_block_end=(1, 3, 4))
+    run_case(cfg, 1e-4)
+
+
+def test_distill_small_bf16():
+    # K = 2: the only AuxNet reads the image, so its stored activations on the GPU and in the oracle
+    # come from identical inputs (with K > 2 the GPU chain feeds AuxNet_1 its own bf16 x_1, which
+    # differs from the oracle's by rounding noise and flips ReLU masks of so small a tensor)
+    cfg = small_cfg("preact", N=16, H=16, W=16, dtype="bf16", stage_channels=(16, 32), stage_blocks=(2, 2),
+                    module_block_end=(2, 4), stem_channels=16, classes=10)
+    run_case(cfg, 3e-2)
+
+
+def test_distill_needs_module_passes_first():
+    cfg = get_config("tiny")
+    run = GpuRun(cfg)
+    run.auxnet()
+    with pytest.raises(run.lp.LpError) as e:
+        run.lp.lp_auxnet_distill(run.h, run.d_images, run.d_x[1:], run.d_dx, 0.1, 0.1, None,
+                                 run.torch.zeros(1, device="cuda:0"))
+    assert e.value.status == -6
