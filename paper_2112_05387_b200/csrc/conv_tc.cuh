@@ -13,6 +13,20 @@
 // tensor memory (3 for N_TILE = 160), so the epilogue of one unit overlaps the MMAs of the next
 // as far as slots are free.
 //
+// Tap reuse ("halo" mode, 3x3 stride-1 convolutions with 64-channel K chunks): all nine taps of
+// a K chunk read the same activations, shifted by whole pixels.  The tile is 8 pixels wide and its
+// rows are ordered (w, image, h); ONE box with a one-pixel halo all round, (8+2) x BNI x (BH+2)
+// rows of 128 bytes, is fetched per K chunk and tile.  An 8-row group of the A operand (one image
+// row segment) is then 8 consecutive box rows, consecutive groups are 10 rows (1280 bytes)
+// apart, and tap (dy, dx) starts dy*10*BNI + dx rows into the box.  The shared-memory descriptor
+// takes exactly that: its start address moves by whole 128-byte rows and its stride byte offset is
+// 1280.  Neither is a multiple of the 1024-byte swizzle atom; that works because the 128-byte
+// swizzle is a function of the shared-memory address bits (16-byte chunk index ^= address bits
+// 7..9), for the TMA write and for the MMA read alike, so any row of the box can be the first row
+// of an operand (checked against the CPU oracle by the parity tests).  Activations and weights
+// travel in separate rings: an activation stage per K chunk (nine taps), a weight stage per tap.
+// This cuts the bytes fetched per MMA from 52 KB to 25 KB per eight instructions.
+//
 // Roles: warp 0 = TMA producer; warps 1 and 2 = MMA issuers, one per accumulator of a pair (a
 // tcgen05.mma costs its issuing thread about 65 cycles, close to the 80 cycles of tensor work of
 // an N = 160 instruction, so one issuer cannot keep the pipe full); warps 3.. = epilogue
@@ -28,6 +42,10 @@ namespace tc {
 constexpr int kMaxStages = 12;
 constexpr int kTmemCols = 512;
 constexpr int kMaxSlots = 4;     // accumulator slots in tensor memory
+
+#ifndef LP_EPI_WARPS
+#define LP_EPI_WARPS 4
+#endif
 
 struct ConvTcParams {
   int Nimg, OHl, OWl;            // logical output grid
@@ -50,18 +68,30 @@ struct ConvTcParams {
   const bf16* addend;            // nullable; same geometry as out
   double* stats;                 // nullable; [2*Cout]
   int* err;
+  // halo mode
+  int halo;                      // 1: one activation box with a halo per K chunk serves all nine taps
+  int nA, nB;                    // ring depths
+  uint32_t a_halo_bytes;         // one activation box (1024-aligned)
+  uint32_t a_stage_bytes;        // mpair boxes
+  uint32_t b_stage_bytes, b_ring_offset;
+  uint32_t tail_offset;          // barriers and scratch after the rings
+  int tap_widx9[9];              // weight tap index of the nine taps in (dy, dx) order
+  uint32_t tap_off9[9];          // byte offset of the tap's first row inside the box
+  uint64_t desc_hi_a;            // descriptor of the activation operand (row-group stride of the box)
 };
 
 struct TcSmemTail {
   uint64_t full[kMaxStages];
   uint64_t empty[kMaxStages];
+  uint64_t full_b[kMaxStages];
+  uint64_t empty_b[kMaxStages];
   uint64_t tmem_full[kMaxSlots];
   uint64_t tmem_empty[kMaxSlots];
   uint32_t tmem_base;
   int abort_flag;
   int epi_ok;
-  float ssum[8][256];   // per epilogue warp: plain read-modify-write, no shared-memory atomics
-  float ssq[8][256];
+  float ssum[LP_EPI_WARPS][256];   // per epilogue warp: plain read-modify-write, no shared-memory atomics
+  float ssq[LP_EPI_WARPS][256];
 };
 
 // Sum 16 per-lane values over the 32 lanes of a warp; lane l ends with the total of column
@@ -94,9 +124,6 @@ __device__ __forceinline__ float transpose_reduce16(const float (&v)[16], int la
   return d;
 }
 
-#ifndef LP_EPI_WARPS
-#define LP_EPI_WARPS 4
-#endif
 constexpr int kEpiThreads = 32 * LP_EPI_WARPS;
 constexpr int kConvThreads = 96 + kEpiThreads;
 constexpr int kFirstEpiWarp = 3;
@@ -107,7 +134,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const __grid_constant__ ConvTcParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  TcSmemTail* tail = reinterpret_cast<TcSmemTail*>(smem + (size_t)p.stages * p.stage_bytes);
+  TcSmemTail* tail = reinterpret_cast<TcSmemTail*>(smem + p.tail_offset);
   volatile int* abort_flag = &tail->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -116,9 +143,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int t_end = (int)(((long long)p.total_tiles * (blockIdx.x + 1)) / gridDim.x);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) {
+    for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(&tail->full[s], 1);
       mbar_init(&tail->empty[s], 2);   // one arrival per MMA warp
+      mbar_init(&tail->full_b[s], 1);
+      mbar_init(&tail->empty_b[s], 2);
     }
     for (int b = 0; b < kMaxSlots; ++b) {
       mbar_init(&tail->tmem_full[b], 1);
@@ -129,7 +158,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
   }
-  for (int i = threadIdx.x; i < 8 * 256; i += blockDim.x) {
+  for (int i = threadIdx.x; i < LP_EPI_WARPS * 256; i += blockDim.x) {
     (&tail->ssum[0][0])[i] = 0.f;
     (&tail->ssq[0][0])[i] = 0.f;
   }
@@ -146,7 +175,101 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   // All three roles walk the same sequence of units: a unit is one pixel tile, or two consecutive
   // ones of the same channel tile, and takes the next one or two accumulator slots of the ring.
-  if (warp == 0) {
+  if (warp == 0 && p.halo) {
+    // ------------------------------- TMA producer, halo mode ----------------------------
+    uint32_t sa = 0, pha = 0, sb = 0, phb = 0;
+    uint8_t* b_ring = smem + p.b_ring_offset;
+    for (int t = t_begin; t < t_end && !failed;) {
+      const int nt = t / p.m_tiles, m = t % p.m_tiles;
+      const int cnt = (p.mpair == 2 && t + 1 < t_end && m + 1 < p.m_tiles) ? 2 : 1;
+      int w0[2], h0[2], n0[2];
+      for (int a = 0; a < 2; ++a) {
+        const int mm = m + a;
+        w0[a] = (mm % p.tiles_w) * p.BW;
+        h0[a] = ((mm / p.tiles_w) % p.tiles_h) * p.BH;
+        n0[a] = (mm / (p.tiles_w * p.tiles_h)) * p.BNI;
+      }
+      const int col0 = nt * p.n_tile_cols;
+      for (int c = 0; c < p.chunks && !failed; ++c) {
+        if (!mbar_wait_warp(&tail->empty[sa], pha ^ 1, abort_flag)) { failed = true; break; }
+        uint8_t* pa = smem + sa * p.a_stage_bytes;
+        if (elect_one()) {
+          mbar_expect_tx(&tail->full[sa], cnt * p.tx_a);
+          tma_load_4d(pa, &tmA, &tail->full[sa], c * p.KC, w0[0] - 1, n0[0], h0[0] - 1);
+          if (cnt == 2) tma_load_4d(pa + p.a_halo_bytes, &tmA, &tail->full[sa], c * p.KC, w0[1] - 1, n0[1], h0[1] - 1);
+        }
+        __syncwarp();
+        if (++sa == (uint32_t)p.nA) { sa = 0; pha ^= 1; }
+        for (int ti = 0; ti < 9; ++ti) {
+          if (!mbar_wait_warp(&tail->empty_b[sb], phb ^ 1, abort_flag)) { failed = true; break; }
+          if (elect_one()) {
+            mbar_expect_tx(&tail->full_b[sb], p.tx_b);
+            tma_load_2d(b_ring + sb * p.b_stage_bytes, &tmB, &tail->full_b[sb], p.tap_widx9[ti] * p.Cin + c * p.KC, col0);
+          }
+          __syncwarp();
+          if (++sb == (uint32_t)p.nB) { sb = 0; phb ^= 1; }
+        }
+      }
+      t += cnt;
+    }
+  } else if ((warp == 1 || warp == 2) && p.halo) {
+    // ------------------------------- MMA issuers, halo mode -----------------------------
+    const int me = warp - 1;
+    uint32_t sa = 0, pha = 0, sb = 0, phb = 0;
+    const uint32_t smem_base = smem_u32(smem);
+    const int nk = p.KC >> 4;
+    uint32_t slot = 0, slot_phase = 0;
+    for (int t = t_begin; t < t_end && !failed;) {
+      const int m = t % p.m_tiles;
+      const int cnt = (p.mpair == 2 && t + 1 < t_end && m + 1 < p.m_tiles) ? 2 : 1;
+      uint32_t sl[2];
+      sl[0] = slot;
+      sl[1] = slot + 1 == (uint32_t)p.nslots ? 0 : slot + 1;
+      const bool active = me < cnt;
+      if (active) {
+        if (!mbar_wait_warp(&tail->tmem_empty[sl[me]], ((slot_phase >> sl[me]) & 1) ^ 1, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+      }
+      const uint32_t d = tmem_base + sl[me] * p.acc_stride;
+      uint32_t accum = 0;
+      for (int c = 0; c < p.chunks && !failed; ++c) {
+        const uint32_t a_addr = smem_base + sa * p.a_stage_bytes + me * p.a_halo_bytes;
+        for (int ti = 0; ti < 9; ++ti) {
+          // The box barrier is polled together with the first weight stage and released together
+          // with the last one: a separate trip (poll, election, commit) at every chunk boundary
+          // costs about 500 cycles in which the tensor pipe runs dry.
+          bool ok = ti ? true : mbar_wait(&tail->full[sa], pha, abort_flag);
+          ok = mbar_wait(&tail->full_b[sb], phb, abort_flag) && ok;
+          if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+          tc_fence_after();
+          const uint64_t ad = smem_desc(p.desc_hi_a, a_addr + p.tap_off9[ti]);
+          const uint64_t bd = smem_desc(p.desc_hi, smem_base + p.b_ring_offset + sb * p.b_stage_bytes);
+          if (elect_one()) {
+            if (active) {
+              for (int j = 0; j < nk; ++j)
+                mma_bf16(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (accum | j) ? 1u : 0u);
+              mma_commit(&tail->empty_b[sb]);
+              if (ti == 8) mma_commit(&tail->empty[sa]);
+            } else {
+              mbar_arrive(&tail->empty_b[sb]);
+              if (ti == 8) mbar_arrive(&tail->empty[sa]);
+            }
+          }
+          __syncwarp();
+          accum = 1;
+          if (++sb == (uint32_t)p.nB) { sb = 0; phb ^= 1; }
+        }
+        if (failed) break;
+        if (++sa == (uint32_t)p.nA) { sa = 0; pha ^= 1; }
+      }
+      if (failed) break;
+      if (active && elect_one()) mma_commit(&tail->tmem_full[sl[me]]);
+      __syncwarp();
+      for (int a = 0; a < cnt; ++a) slot_phase ^= 1u << sl[a];
+      slot = cnt == 2 ? (sl[1] + 1 == (uint32_t)p.nslots ? 0 : sl[1] + 1) : sl[1];
+      t += cnt;
+    }
+  } else if (warp == 0) {
     // ------------------------------- TMA producer (warp-uniform loop, elected issue) ----
     uint32_t s = 0, ph = 0;
     for (int t = t_begin; t < t_end && !failed;) {
@@ -247,7 +370,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int w0 = (m % p.tiles_w) * p.BW;
         const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
         const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
-        const int ow = w0 + row % p.BW, oh = h0 + (row / p.BW) % p.BH, n = n0 + row / (p.BW * p.BH);
+        // rows of a tile: (w, h, image), or (w, image, h) in halo mode
+        const int ow = w0 + row % p.BW;
+        const int oh = h0 + (p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH);
+        const int n = n0 + (p.halo ? (row / p.BW) % p.BNI : row / (p.BW * p.BH));
         const bool valid = row < rows_used && ow < p.OWl && oh < p.OHl && n < p.Nimg;
         const long long obase =
             (((long long)n * p.out_H + (oh * p.os + p.oo_h)) * p.out_W + (ow * p.os + p.oo_w)) * p.out_C;

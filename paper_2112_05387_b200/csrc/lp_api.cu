@@ -292,11 +292,54 @@ static int encode_mat_map(CUtensorMap* m, const void* base, long long K, int row
 static const size_t kTcMinSmem = 120 * 1024;   // more than half an SM: one CTA (and one TMEM owner) per SM
 static const size_t kTcMaxSmem = 220 * 1024;
 
+// Halo mode (one activation box per K chunk serves all nine taps, see conv_tc.cuh): a 3x3 stride-1
+// tap set, 64-channel K chunks and an output width that is a multiple of 8.
+static const int kHaloBoxW = 10;   // 8-pixel tile width plus one halo pixel on each side
+
+static bool pick_halo_box(const TcGemmSpec& s, int& BW, int& BH, int& BNI, int tapw3[3][3]) {
+  if (s.ntaps != 9 || s.in_step != 1 || s.os != 1 || s.OWl % 8) return false;
+  bool seen[3][3] = {};
+  for (int i = 0; i < 9; ++i) {
+    const int dx = s.dw[i] + 1, dy = s.dh[i] + 1;
+    if (dx < 0 || dx > 2 || dy < 0 || dy > 2 || seen[dx][dy]) return false;
+    seen[dx][dy] = true;
+    tapw3[dx][dy] = s.widx[i];
+  }
+  BW = 8;
+  if (8 * s.OHl <= 64) {
+    BH = s.OHl;
+    BNI = std::min(s.aN, 128 / (8 * BH));
+  } else {
+    BNI = 1;
+    BH = std::min(s.OHl, 16);
+    const int th = (s.OHl + BH - 1) / BH;
+    BH = (s.OHl + th - 1) / th;
+  }
+  return BH >= 2 && 8 * BH * BNI >= 96;
+}
+
+static int encode_act_map_halo(CUtensorMap* m, const void* base, int N, int H, int W, int C, int boxC, int boxW, int BH,
+                               int BNI, int row_bytes) {
+  // dimension order (C, W, image, H): the image row is the slowest coordinate of the box
+  cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)N, (cuuint64_t)H};
+  cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)H * W * C * 2, (cuuint64_t)W * C * 2};
+  cuuint32_t box[4] = {(cuuint32_t)boxC, (cuuint32_t)boxW, (cuuint32_t)BNI, (cuuint32_t)(BH + 2)};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+  CUresult r = g_dev.encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LP_OK : LP_ERR_CUDA;
+}
+
 static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaStream_t st) {
   tc::ConvTcParams p;
   memset(&p, 0, sizeof(p));
   p.Nimg = s.aN; p.OHl = s.OHl; p.OWl = s.OWl;
-  pick_pixel_box(s.OWl, s.OHl, s.aN, p.BW, p.BH, p.BNI);
+  int tapw3[3][3];
+  p.halo = (pick_kc(s.aC) == 64 && pick_halo_box(s, p.BW, p.BH, p.BNI, tapw3)) ? 1 : 0;
+  if (!p.halo) pick_pixel_box(s.OWl, s.OHl, s.aN, p.BW, p.BH, p.BNI);
   p.tiles_w = (s.OWl + p.BW - 1) / p.BW;
   p.tiles_h = (s.OHl + p.BH - 1) / p.BH;
   const int tiles_n = (s.aN + p.BNI - 1) / p.BNI;
@@ -316,30 +359,71 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   p.a_region_bytes = (uint32_t)align_up((size_t)128 * row_bytes, 1024);
   const uint32_t b_region = (uint32_t)align_up((size_t)p.n_tile_cols * row_bytes, 1024);
   const size_t tail = sizeof(tc::TcSmemTail) + 1024;
-  // two pixel tiles per weight tile wherever a CTA has at least two tiles and three stages still fit
-  p.mpair = 1;
-  if (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, g_dev.sm_count) &&
-      (kTcMaxSmem - tail) / (2 * p.a_region_bytes + b_region) >= 3)
-    p.mpair = 2;
-  p.b_offset = p.mpair * p.a_region_bytes;
-  p.stage_bytes = p.b_offset + b_region;
-  p.tx_a = (uint32_t)(p.BW * p.BH * p.BNI * row_bytes);
   p.tx_b = (uint32_t)(p.n_tile_cols * row_bytes);
   p.acc_stride = (p.n_tile_cols + 31) / 32 * 32;
   p.nslots = std::min(tc::kMaxSlots, tc::kTmemCols / p.acc_stride);
-  int stages = (int)((kTcMaxSmem - tail) / p.stage_bytes);
-  stages = std::min(stages, tc::kMaxStages);
-  if (stages < 2) return LP_ERR_UNSUPPORTED;
-  p.stages = stages;
+  if (p.halo) {
+    // activation ring: three boxes deep if at least three weight stages still fit, else two
+    const int halo_rows = kHaloBoxW * p.BNI * (p.BH + 2);
+    p.a_halo_bytes = (uint32_t)align_up((size_t)halo_rows * row_bytes, 1024);
+    for (int dy = 0; dy < 3; ++dy)
+      for (int dx = 0; dx < 3; ++dx) {
+        p.tap_widx9[dy * 3 + dx] = tapw3[dx][dy];
+        p.tap_off9[dy * 3 + dx] = (uint32_t)((dy * kHaloBoxW * p.BNI + dx) * row_bytes);
+      }
+    // 8-row groups of the operand are one box row (kHaloBoxW pixels) apart
+    p.desc_hi_a = tc::smem_desc_hi(16, kHaloBoxW * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
+    p.b_stage_bytes = b_region;
+    p.tx_a = (uint32_t)(halo_rows * row_bytes);
+    const size_t avail = kTcMaxSmem - tail;
+    // two activation stages (each lasts nine weight stages), the rest of shared memory for weights
+    bool fits = false;
+    p.nA = 2;
+    for (int pair = (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, g_dev.sm_count)) ? 2 : 1;
+         pair >= 1 && !fits; --pair) {
+      const size_t a_bytes = (size_t)p.nA * pair * p.a_halo_bytes;
+      if (a_bytes >= avail) continue;
+      const int nb = (int)std::min<size_t>((avail - a_bytes) / b_region, 8);
+      if (nb >= 3) { p.mpair = pair; p.nB = nb; fits = true; }
+    }
+    if (fits) {
+      p.a_stage_bytes = p.mpair * p.a_halo_bytes;
+      p.b_ring_offset = p.nA * p.a_stage_bytes;
+      p.tail_offset = p.b_ring_offset + p.nB * p.b_stage_bytes;
+    } else {
+      p.halo = 0;
+      pick_pixel_box(s.OWl, s.OHl, s.aN, p.BW, p.BH, p.BNI);
+      p.tiles_w = (s.OWl + p.BW - 1) / p.BW;
+      p.tiles_h = (s.OHl + p.BH - 1) / p.BH;
+      p.m_tiles = p.tiles_w * p.tiles_h * ((s.aN + p.BNI - 1) / p.BNI);
+      p.total_tiles = p.m_tiles * p.n_tiles;
+    }
+  }
+  if (!p.halo) {
+    // two pixel tiles per weight tile wherever a CTA has at least two tiles and three stages still fit
+    p.mpair = 1;
+    if (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, g_dev.sm_count) &&
+        (kTcMaxSmem - tail) / (2 * p.a_region_bytes + b_region) >= 3)
+      p.mpair = 2;
+    p.b_offset = p.mpair * p.a_region_bytes;
+    p.stage_bytes = p.b_offset + b_region;
+    p.tx_a = (uint32_t)(p.BW * p.BH * p.BNI * row_bytes);
+    int stages = (int)((kTcMaxSmem - tail) / p.stage_bytes);
+    stages = std::min(stages, tc::kMaxStages);
+    if (stages < 2) return LP_ERR_UNSUPPORTED;
+    p.stages = stages;
+    p.tail_offset = (uint32_t)(stages * p.stage_bytes);
+  }
   p.idesc = tc::instr_desc_bf16(128, p.n_tile_cols, 0, 0);
   p.desc_hi = tc::smem_desc_hi(16, 8 * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
   p.out = s.out; p.addend = s.addend; p.stats = s.stats; p.err = dev_err;
   CUtensorMap tmA, tmB;
-  int rc = encode_act_map(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, p.KC, p.BW, p.BH, p.BNI, s.in_step, row_bytes);
+  int rc = p.halo ? encode_act_map_halo(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, p.KC, kHaloBoxW, p.BH, p.BNI, row_bytes)
+                  : encode_act_map(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, p.KC, p.BW, p.BH, p.BNI, s.in_step, row_bytes);
   if (rc != LP_OK) return rc;
   rc = encode_mat_map(&tmB, s.wmat, s.w_K, s.w_rows, p.KC, p.n_tile_cols, row_bytes);
   if (rc != LP_OK) return rc;
-  size_t smem = (size_t)stages * p.stage_bytes + tail;
+  size_t smem = (size_t)p.tail_offset + tail;
   smem = std::max(smem, kTcMinSmem);
   static bool attr_set = false;
   if (!attr_set) {

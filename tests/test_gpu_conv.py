@@ -89,6 +89,10 @@ TC_CASES = [
     (29, 32, 32, 32, 48, 3, 1, 1),    # 232 tiles: CTAs with one tile and CTAs with a pair
     (64, 16, 16, 32, 320, 3, 1, 1),   # pairs with two channel tiles (ranges cross the channel-tile boundary)
     (37, 16, 16, 160, 160, 3, 2, 1),  # pairs, stride 2, odd tile count (input gradient: parity classes)
+    (3, 12, 24, 64, 64, 3, 1, 1),     # 24-wide boxes of 4 rows with a one-row halo, 96 of 128 tile rows used
+    (2, 56, 56, 64, 64, 3, 1, 1),     # 56-wide boxes of 2 rows
+    (9, 4, 4, 64, 32, 3, 1, 1),       # 4x4 images, eight per tile, ragged last tile
+    (40, 32, 32, 160, 160, 3, 1, 1),  # 320 halo tiles of 16x8 pixels: pairs, three K chunks with zero fill
 ]
 
 
