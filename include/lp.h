@@ -201,6 +201,44 @@ int64_t lp_launch_count(lp_handle* h, int reset);
  * their count since the last reset; only collected while profiling is enabled (serialises). */
 int lp_conv_profile(lp_handle* h, int enable, double* ms, double* flops, int64_t* launches);
 
+/* Per-operation time line of everything the library launches while it is enabled: one record per
+ * operation of a module or AuxNet plan (a convolution, a batch-norm pass, the local loss, the
+ * update, ...), timed with CUDA events on the stream the operation runs on, so that the phases of
+ * the paper's cost model (Section 4.3: T_f, T_b per module, t_psi, the AuxNet pass and the AuxNet
+ * distillation) can be measured per module while the modules overlap.  Events cannot be recorded
+ * into a graph: lp_graph_begin returns LP_ERR_ORDER while the time line is enabled.
+ *   enable       0/1: state after the call (records collected so far are dropped either way)
+ *   records      host array of max_records entries, or NULL; when given (or n_records is), the
+ *                device is synchronised and the records collected so far are written, times in ms
+ *                relative to the earliest recorded start
+ *   n_records    receives the number of records collected (may exceed max_records) */
+#define LP_PHASE_AUX_FORWARD 0
+#define LP_PHASE_FORWARD 1
+#define LP_PHASE_BACKWARD 2
+#define LP_PHASE_UPDATE 3
+#define LP_PHASE_DISTILL 4
+/* operation kinds in lp_timeline_record.op */
+#define LP_OP_CONV_FWD 0
+#define LP_OP_CONV_DGRAD 1
+#define LP_OP_CONV_WGRAD 2
+#define LP_OP_BN_STATS 3
+#define LP_OP_BN_APPLY 4
+#define LP_OP_OUT_LOSS 5
+#define LP_OP_BN_BWD 6
+#define LP_OP_MAXPOOL_FWD 7
+#define LP_OP_MAXPOOL_BWD 8
+#define LP_OP_HEAD_FWD 9
+#define LP_OP_HEAD_BWD 10
+#define LP_OP_COPY 11
+#define LP_OP_UPDATE 12
+typedef struct lp_timeline_record {
+  int32_t plan;   /* module k, or LP_AUX(k) */
+  int32_t op;     /* LP_OP_* */
+  int32_t phase;  /* LP_PHASE_* */
+  float start_ms, end_ms;
+} lp_timeline_record;
+int lp_timeline(lp_handle* h, int enable, int max_records, lp_timeline_record* records, int* n_records);
+
 /* CUDA-graph helpers: record every launch the library makes on `stream` between begin and end
  * (the internal module streams are forked from and joined into it), then replay the recording.
  * Pointer arguments of the recorded calls are baked into the graph.  Up to 8 graphs per handle;

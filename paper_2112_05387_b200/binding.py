@@ -12,7 +12,8 @@ __all__ = [
     "lp_get_params", "lp_get_grads", "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd",
     "lp_modules_fwd_bwd_all", "lp_step", "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual",
     "lp_last_device_status", "lp_launch_count", "lp_conv_profile", "lp_conv2d", "lp_conv2d_scratch_bytes", "lp_graph_begin", "lp_graph_end",
-    "lp_graph_launch", "lp_conv2d_fwd_noalloc", "LP_NOALLOC_SCRATCH_BYTES", "lp_layer_parallel_step", "lp_auxnet_distill", "EXPORTED_SYMBOLS",
+    "lp_graph_launch", "lp_conv2d_fwd_noalloc", "LP_NOALLOC_SCRATCH_BYTES", "lp_layer_parallel_step", "lp_auxnet_distill", "lp_timeline", "lp_timeline_record",
+    "LP_PHASE_NAMES", "LP_OP_NAMES", "EXPORTED_SYMBOLS",
 ]
 
 LP_OK = 0
@@ -22,6 +23,9 @@ LP_CONV_FWD, LP_CONV_DGRAD, LP_CONV_WGRAD = 0, 1, 2
 LP_MAX_STAGES, LP_MAX_MODULES = 8, 16
 LP_NOALLOC_SCRATCH_BYTES = 8 << 20
 _KINDS = ["conv_w", "bn_gamma", "bn_beta", "fc_w", "fc_b"]
+LP_PHASE_NAMES = ["aux_forward", "forward", "backward", "update", "distill"]
+LP_OP_NAMES = ["conv_fwd", "conv_dgrad", "conv_wgrad", "bn_stats", "bn_apply", "out_loss", "bn_bwd", "maxpool_fwd",
+               "maxpool_bwd", "head_fwd", "head_bwd", "copy", "update"]
 
 EXPORTED_SYMBOLS = [
     "lp_status_string", "lp_workspace_bytes", "lp_validate_desc", "lp_param_layout", "lp_boundary_shape_desc",
@@ -29,7 +33,7 @@ EXPORTED_SYMBOLS = [
     "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd", "lp_modules_fwd_bwd_all", "lp_step",
     "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual", "lp_last_device_status", "lp_launch_count",
     "lp_conv_profile", "lp_conv2d_scratch_bytes", "lp_conv2d", "lp_graph_begin", "lp_graph_end", "lp_graph_launch",
-    "lp_conv2d_fwd_noalloc", "lp_layer_parallel_step", "lp_auxnet_distill",
+    "lp_conv2d_fwd_noalloc", "lp_layer_parallel_step", "lp_auxnet_distill", "lp_timeline",
 ]
 
 
@@ -59,6 +63,11 @@ class lp_net_desc(ctypes.Structure):
 class lp_param_entry(ctypes.Structure):
     _fields_ = [("name", ctypes.c_char * 48), ("kind", ctypes.c_int32), ("shape", ctypes.c_int32 * 4),
                 ("offset", ctypes.c_uint64)]
+
+
+class lp_timeline_record(ctypes.Structure):
+    _fields_ = [("plan", ctypes.c_int32), ("op", ctypes.c_int32), ("phase", ctypes.c_int32),
+                ("start_ms", ctypes.c_float), ("end_ms", ctypes.c_float)]
 
 
 _LIB = None
@@ -108,6 +117,8 @@ def library():
     lib.lp_last_device_status.argtypes = [vp, vp]
     lib.lp_launch_count.restype = ctypes.c_int64
     lib.lp_launch_count.argtypes = [vp, i32]
+    lib.lp_timeline.argtypes = [vp, i32, i32, ctypes.POINTER(lp_timeline_record), ctypes.POINTER(ctypes.c_int)]
+    lib.lp_timeline.restype = i32
     lib.lp_conv_profile.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                     ctypes.POINTER(ctypes.c_int64)]
     lib.lp_graph_begin.argtypes = [vp, vp]
@@ -327,6 +338,19 @@ def lp_conv_profile(h, enable, read=True):
     else:
         _check(library().lp_conv_profile(h.ptr, 1 if enable else 0, None, None, None), "lp_conv_profile")
     return ms.value, fl.value, n.value
+
+
+def lp_timeline(h, enable, read=True, max_records=4096):
+    """Enable/disable the per-operation time line; with ``read`` returns the records collected so far
+    as a list of dicts (plan, op, phase, start_ms, end_ms)."""
+    if not read:
+        _check(library().lp_timeline(h.ptr, 1 if enable else 0, 0, None, None), "lp_timeline")
+        return []
+    recs = (lp_timeline_record * max_records)()
+    n = ctypes.c_int(0)
+    _check(library().lp_timeline(h.ptr, 1 if enable else 0, max_records, recs, ctypes.byref(n)), "lp_timeline")
+    return [dict(plan=r.plan, op=LP_OP_NAMES[r.op], phase=LP_PHASE_NAMES[r.phase], start_ms=r.start_ms, end_ms=r.end_ms)
+            for r in recs[:min(n.value, max_records)]]
 
 
 def lp_graph_begin(h, stream):

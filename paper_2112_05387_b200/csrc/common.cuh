@@ -33,6 +33,21 @@ __device__ __forceinline__ void ldv(const bf16* p, float (&f)[8]) {
     f[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
   }
 }
+// The same in two steps: a raw 16-byte load now, the conversion when the values are needed, so
+// that several loads can be in flight per thread without holding their unpacked values.
+template <typename T>
+__device__ __forceinline__ uint4 ld_raw(const T* p) { return *reinterpret_cast<const uint4*>(p); }
+__device__ __forceinline__ void cvt_raw(const uint4& v, float (&f)[4]) {
+  f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+}
+__device__ __forceinline__ void cvt_raw(const uint4& v, float (&f)[8]) {
+  const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(u[i] << 16);
+    f[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+  }
+}
 __device__ __forceinline__ void stv(float* p, const float (&f)[4]) {
   *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
 }

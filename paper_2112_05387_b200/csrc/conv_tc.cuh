@@ -46,6 +46,12 @@ constexpr int kMaxSlots = 4;     // accumulator slots in tensor memory
 #ifndef LP_EPI_WARPS
 #define LP_EPI_WARPS 4
 #endif
+#ifndef LP_CONV_MIN_BLOCKS
+#define LP_CONV_MIN_BLOCKS 1
+#endif
+#ifndef LP_EPI_BATCH
+#define LP_EPI_BATCH 5
+#endif
 
 struct ConvTcParams {
   int Nimg, OHl, OWl;            // logical output grid
@@ -129,7 +135,7 @@ constexpr int kConvThreads = 96 + kEpiThreads;
 constexpr int kFirstEpiWarp = 3;
 constexpr int kEpiGroups = LP_EPI_WARPS / 4;
 
-__global__ void __launch_bounds__(kConvThreads, 1)
+__global__ void __launch_bounds__(kConvThreads, LP_CONV_MIN_BLOCKS)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ ConvTcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -386,7 +392,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t taddr = tmem_base + buf * p.acc_stride + ((uint32_t)(q * 32) << 16);
         // Drain the accumulator into registers first (up to kBatch x 32 columns per pass) and hand
         // the TMEM slot back to the MMA warp; stores and statistics then work from registers.
-        constexpr int kBatch = 5;
+        constexpr int kBatch = LP_EPI_BATCH;
         for (int g0 = grp; g0 < ngroups; g0 += kBatch * kEpiGroups) {
           uint32_t raw[kBatch][32];
 #pragma unroll

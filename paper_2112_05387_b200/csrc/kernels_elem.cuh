@@ -15,12 +15,47 @@ struct BnArgs {
   float eps;
 };
 
-__device__ __forceinline__ void bn_mean_rstd(const BnArgs& a, int C, int c, float& mean, float& rstd) {
-  double m = a.stats[c] * a.inv_count;
-  double var = a.stats[C + c] * a.inv_count - m * m;
-  if (var < 0.0) var = 0.0;
-  mean = (float)m;
-  rstd = (float)(1.0 / sqrt(var + (double)a.eps));
+// The constants of V consecutive channels c0..c0+V-1 (V = 4 or 8, c0 a multiple of V): mean,
+// 1/sqrt(var+eps), gamma, beta.  16-byte loads wherever the pointers allow: every thread of every
+// block runs this prologue, and scalar loads at a stride of V channels between neighbouring
+// threads (32 sectors per warp instruction, 4*V instructions) took longer than the pass itself.
+template <int V>
+__device__ __forceinline__ void bn_load_consts(const BnArgs& a, int C, int c0, float (&mean)[V], float (&rstd)[V],
+                                               float (&gamma)[V], float (&beta)[V]) {
+  double s1[V], s2[V];
+  if ((reinterpret_cast<uintptr_t>(a.stats) & 15) == 0 && (C & 1) == 0) {
+#pragma unroll
+    for (int j = 0; j < V; j += 2) {
+      const double2 u = *reinterpret_cast<const double2*>(a.stats + c0 + j);
+      const double2 w = *reinterpret_cast<const double2*>(a.stats + C + c0 + j);
+      s1[j] = u.x; s1[j + 1] = u.y; s2[j] = w.x; s2[j + 1] = w.y;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < V; ++j) { s1[j] = a.stats[c0 + j]; s2[j] = a.stats[C + c0 + j]; }
+  }
+  if (((reinterpret_cast<uintptr_t>(a.gamma + c0) | reinterpret_cast<uintptr_t>(a.beta + c0)) & 15) == 0) {
+#pragma unroll
+    for (int j = 0; j < V; j += 4) {
+      const float4 g = *reinterpret_cast<const float4*>(a.gamma + c0 + j);
+      const float4 b = *reinterpret_cast<const float4*>(a.beta + c0 + j);
+      gamma[j] = g.x; gamma[j + 1] = g.y; gamma[j + 2] = g.z; gamma[j + 3] = g.w;
+      beta[j] = b.x; beta[j + 1] = b.y; beta[j + 2] = b.z; beta[j + 3] = b.w;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < V; ++j) { gamma[j] = a.gamma[c0 + j]; beta[j] = a.beta[c0 + j]; }
+  }
+#pragma unroll
+  for (int j = 0; j < V; ++j) {
+    const double m = s1[j] * a.inv_count;
+    const double var = fma(-m, m, s2[j] * a.inv_count);
+    mean[j] = (float)m;
+    const float v = fmaxf((float)var, 0.f) + a.eps;
+    float r = rsqrtf(v);
+    r = r * fmaf(-0.5f * v * r, r, 1.5f);
+    rstd[j] = r;
+  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -64,49 +99,83 @@ __global__ void bn_stats_kernel(const T* __restrict__ x, long long total_vecs, i
 // ---------------------------------------------------------------------------------------
 // out = [relu]( bnA(x) [+ bnB(x2)] [+ addend] )
 // ---------------------------------------------------------------------------------------
-template <typename T>
-__global__ void bn_apply_kernel(const T* __restrict__ x, BnArgs A, const T* __restrict__ x2, BnArgs B,
-                                const T* __restrict__ addend, T* __restrict__ out, long long total_vecs,
-                                int C, int relu) {
+// X2 / ADD select at compile time whether a second normalised input and a plain addend exist, so
+// that the common one-input form keeps few enough registers for four 256-thread blocks per SM.
+template <typename T, bool X2, bool ADD>
+__global__ void __launch_bounds__(256, X2 ? 2 : (ADD ? 3 : 4))
+bn_apply_kernel(const T* __restrict__ x, BnArgs A, const T* __restrict__ x2, BnArgs B,
+                const T* __restrict__ addend, T* __restrict__ out, long long total_vecs, int C, int relu) {
   constexpr int V = VecT<T>::N;
   const int CV = C / V;
   const int c0 = (threadIdx.x % CV) * V;
-  float sa[V], ta[V], sb[V], tb[V];
+  float sa[V], ta[V], sb[X2 ? V : 1], tb[X2 ? V : 1];
+  {
+    float mean[V], rstd[V], gamma[V], beta[V];
+    bn_load_consts<V>(A, C, c0, mean, rstd, gamma, beta);
 #pragma unroll
-  for (int j = 0; j < V; ++j) {
-    float mean, rstd;
-    bn_mean_rstd(A, C, c0 + j, mean, rstd);
-    sa[j] = A.gamma[c0 + j] * rstd;
-    ta[j] = A.beta[c0 + j] - mean * sa[j];
-    sb[j] = tb[j] = 0.f;
-    if (x2) {
-      bn_mean_rstd(B, C, c0 + j, mean, rstd);
-      sb[j] = B.gamma[c0 + j] * rstd;
-      tb[j] = B.beta[c0 + j] - mean * sb[j];
+    for (int j = 0; j < V; ++j) {
+      sa[j] = gamma[j] * rstd[j];
+      ta[j] = beta[j] - mean[j] * sa[j];
+    }
+    if (X2) {
+      bn_load_consts<V>(B, C, c0, mean, rstd, gamma, beta);
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        sb[X2 ? j : 0] = gamma[j] * rstd[j];
+        tb[X2 ? j : 0] = beta[j] - mean[j] * sb[X2 ? j : 0];
+      }
     }
   }
   const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
-    float f[V], y[V];
-    ldv(x + i * V, f);
+  // U vectors per thread and trip, all loads issued before the first use: with one 16-byte load
+  // per thread a grid that fills the machine keeps only a few MB in flight, less than the
+  // bandwidth-latency product of the memory system
+  constexpr int U = 4;
+  for (long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i0 < total_vecs; i0 += U * stride) {
+    uint4 rf[U], rg[X2 ? U : 1], ra[ADD ? U : 1];
 #pragma unroll
-    for (int j = 0; j < V; ++j) y[j] = fmaf(f[j], sa[j], ta[j]);
-    if (x2) {
-      ldv(x2 + i * V, f);
-#pragma unroll
-      for (int j = 0; j < V; ++j) y[j] += f[j] * sb[j] + tb[j];
+    for (int u = 0; u < U; ++u) {
+      const long long i = i0 + u * stride;
+      if (i < total_vecs) {
+        rf[u] = ld_raw(x + i * V);
+        if (X2) rg[X2 ? u : 0] = ld_raw(x2 + i * V);
+        if (ADD) ra[ADD ? u : 0] = ld_raw(addend + i * V);
+      }
     }
-    if (addend) {
-      ldv(addend + i * V, f);
 #pragma unroll
-      for (int j = 0; j < V; ++j) y[j] += f[j];
-    }
-    if (relu) {
+    for (int u = 0; u < U; ++u) {
+      const long long i = i0 + u * stride;
+      if (i >= total_vecs) break;
+      float f[V], y[V];
+      cvt_raw(rf[u], f);
 #pragma unroll
-      for (int j = 0; j < V; ++j) y[j] = y[j] > 0.f ? y[j] : 0.f;
+      for (int j = 0; j < V; ++j) y[j] = fmaf(f[j], sa[j], ta[j]);
+      if (X2) {
+        cvt_raw(rg[X2 ? u : 0], f);
+#pragma unroll
+        for (int j = 0; j < V; ++j) y[j] += f[j] * sb[X2 ? j : 0] + tb[X2 ? j : 0];
+      }
+      if (ADD) {
+        cvt_raw(ra[ADD ? u : 0], f);
+#pragma unroll
+        for (int j = 0; j < V; ++j) y[j] += f[j];
+      }
+      if (relu) {
+#pragma unroll
+        for (int j = 0; j < V; ++j) y[j] = y[j] > 0.f ? y[j] : 0.f;
+      }
+      stv(out + i * V, y);
     }
-    stv(out + i * V, y);
   }
+}
+
+template <typename T>
+void launch_bn_apply(int grid, int threads, cudaStream_t st, const T* x, const BnArgs& A, const T* x2, const BnArgs& B,
+                     const T* addend, T* out, long long total_vecs, int C, int relu) {
+  if (x2 && addend) bn_apply_kernel<T, true, true><<<grid, threads, 0, st>>>(x, A, x2, B, addend, out, total_vecs, C, relu);
+  else if (x2) bn_apply_kernel<T, true, false><<<grid, threads, 0, st>>>(x, A, x2, B, addend, out, total_vecs, C, relu);
+  else if (addend) bn_apply_kernel<T, false, true><<<grid, threads, 0, st>>>(x, A, x2, B, addend, out, total_vecs, C, relu);
+  else bn_apply_kernel<T, false, false><<<grid, threads, 0, st>>>(x, A, x2, B, addend, out, total_vecs, C, relu);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -126,18 +195,24 @@ __global__ void module_out_loss_kernel(const T* __restrict__ x, BnArgs A, const 
   const int c0 = (threadIdx.x % CV) * V;
   float sa[V], ta[V], sb[V], tb[V];
 #pragma unroll
-  for (int j = 0; j < V; ++j) {
-    sa[j] = ta[j] = sb[j] = tb[j] = 0.f;
-    float mean, rstd;
+  for (int j = 0; j < V; ++j) sa[j] = ta[j] = sb[j] = tb[j] = 0.f;
+  {
+    float mean[V], rstd[V], gamma[V], beta[V];
     if (x) {
-      bn_mean_rstd(A, C, c0 + j, mean, rstd);
-      sa[j] = A.gamma[c0 + j] * rstd;
-      ta[j] = A.beta[c0 + j] - mean * sa[j];
+      bn_load_consts<V>(A, C, c0, mean, rstd, gamma, beta);
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        sa[j] = gamma[j] * rstd[j];
+        ta[j] = beta[j] - mean[j] * sa[j];
+      }
     }
     if (x2) {
-      bn_mean_rstd(B, C, c0 + j, mean, rstd);
-      sb[j] = B.gamma[c0 + j] * rstd;
-      tb[j] = B.beta[c0 + j] - mean * sb[j];
+      bn_load_consts<V>(B, C, c0, mean, rstd, gamma, beta);
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        sb[j] = gamma[j] * rstd[j];
+        tb[j] = beta[j] - mean[j] * sb[j];
+      }
     }
   }
   float sum_rr = 0.f, sum_kr = 0.f;
@@ -214,7 +289,8 @@ __global__ void loss_finalize_kernel(const double* __restrict__ acc, float rho, 
 //   apply : dx = gamma*rstd*(dy_m - dbeta/M - xhat*dgamma/M) [+ addend]
 // ---------------------------------------------------------------------------------------
 template <typename T>
-__global__ void bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_mask,
+__global__ void __launch_bounds__(256, 3)
+bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_mask,
                                      BnArgs A, float* __restrict__ dgamma, float* __restrict__ dbeta,
                                      long long total_vecs, int C) {
   constexpr int V = VecT<T>::N;
@@ -222,26 +298,43 @@ __global__ void bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restri
   const int CV = C / V;
   const int c0 = (threadIdx.x % CV) * V;
   float mean[V], rstd[V], sb[V], sg[V], sa[V], ta[V];
-#pragma unroll
-  for (int j = 0; j < V; ++j) {
-    bn_mean_rstd(A, C, c0 + j, mean[j], rstd[j]);
-    sa[j] = A.gamma[c0 + j] * rstd[j];
-    ta[j] = A.beta[c0 + j] - mean[j] * sa[j];
-    sb[j] = sg[j] = 0.f;
-  }
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
-    float d[V], f[V];
-    ldv(dy + i * V, d);
-    ldv(x + i * V, f);
-    if (relu_mask) {
-#pragma unroll
-      for (int j = 0; j < V; ++j) d[j] = fmaf(f[j], sa[j], ta[j]) > 0.f ? d[j] : 0.f;
-    }
+  {
+    float gamma[V], beta[V];
+    bn_load_consts<V>(A, C, c0, mean, rstd, gamma, beta);
 #pragma unroll
     for (int j = 0; j < V; ++j) {
-      sb[j] += d[j];
-      sg[j] += d[j] * (f[j] - mean[j]) * rstd[j];
+      sa[j] = gamma[j] * rstd[j];
+      ta[j] = beta[j] - mean[j] * sa[j];
+      sb[j] = sg[j] = 0.f;
+    }
+  }
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  constexpr int U = 2;
+  for (long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i0 < total_vecs; i0 += U * stride) {
+    uint4 rd[U], rx[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const long long i = i0 + u * stride;
+      if (i < total_vecs) {
+        rd[u] = ld_raw(dy + i * V);
+        rx[u] = ld_raw(x + i * V);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (i0 + u * stride >= total_vecs) break;
+      float d[V], f[V];
+      cvt_raw(rd[u], d);
+      cvt_raw(rx[u], f);
+      if (relu_mask) {
+#pragma unroll
+        for (int j = 0; j < V; ++j) d[j] = fmaf(f[j], sa[j], ta[j]) > 0.f ? d[j] : 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        sb[j] += d[j];
+        sg[j] += d[j] * (f[j] - mean[j]) * rstd[j];
+      }
     }
   }
 #pragma unroll
@@ -260,39 +353,74 @@ __global__ void bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restri
 }
 
 template <typename T>
-__global__ void bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_mask,
-                                    BnArgs A, const float* __restrict__ dgamma, const float* __restrict__ dbeta,
-                                    const T* __restrict__ addend, T* __restrict__ out, long long total_vecs, int C) {
+__global__ void __launch_bounds__(256, 3)
+bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_mask, BnArgs A,
+                    const float* __restrict__ dgamma, const float* __restrict__ dbeta,
+                    const T* __restrict__ addend, T* __restrict__ out, long long total_vecs, int C) {
   constexpr int V = VecT<T>::N;
   const int CV = C / V;
   const int c0 = (threadIdx.x % CV) * V;
-  float mean[V], rstd[V], sc[V], mb[V], mg[V], ta[V];
+  // dx = sc*(dy_m - mb - xhat*mg) = sc*dy_m + a2*x + a3   with xhat = (x - mean)*rstd
+  float sc[V], ta[V], a2[V], a3[V];
   const float invM = (float)A.inv_count;
+  {
+    float mean[V], rstd[V], gamma[V], beta[V];
+    bn_load_consts<V>(A, C, c0, mean, rstd, gamma, beta);
+    const bool vec = ((reinterpret_cast<uintptr_t>(dbeta + c0) | reinterpret_cast<uintptr_t>(dgamma + c0)) & 15) == 0;
 #pragma unroll
-  for (int j = 0; j < V; ++j) {
-    bn_mean_rstd(A, C, c0 + j, mean[j], rstd[j]);
-    sc[j] = A.gamma[c0 + j] * rstd[j];
-    ta[j] = A.beta[c0 + j] - mean[j] * sc[j];
-    mb[j] = dbeta[c0 + j] * invM;
-    mg[j] = dgamma[c0 + j] * invM;
+    for (int j = 0; j < V; j += 4) {
+      float4 b, g;
+      if (vec) {
+        b = *reinterpret_cast<const float4*>(dbeta + c0 + j);
+        g = *reinterpret_cast<const float4*>(dgamma + c0 + j);
+      } else {
+        b = make_float4(dbeta[c0 + j], dbeta[c0 + j + 1], dbeta[c0 + j + 2], dbeta[c0 + j + 3]);
+        g = make_float4(dgamma[c0 + j], dgamma[c0 + j + 1], dgamma[c0 + j + 2], dgamma[c0 + j + 3]);
+      }
+      const float mb[4] = {b.x * invM, b.y * invM, b.z * invM, b.w * invM};
+      const float mg[4] = {g.x * invM, g.y * invM, g.z * invM, g.w * invM};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        sc[j + q] = gamma[j + q] * rstd[j + q];
+        ta[j + q] = beta[j + q] - mean[j + q] * sc[j + q];
+        a2[j + q] = -sc[j + q] * rstd[j + q] * mg[q];
+        a3[j + q] = -sc[j + q] * mb[q] - a2[j + q] * mean[j + q];
+      }
+    }
   }
   const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
-    float d[V], f[V], o[V];
-    ldv(dy + i * V, d);
-    ldv(x + i * V, f);
-    if (relu_mask) {
+  constexpr int U = 2;
+  for (long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i0 < total_vecs; i0 += U * stride) {
+    uint4 rd[U], rx[U], ra[U];
 #pragma unroll
-      for (int j = 0; j < V; ++j) d[j] = fmaf(f[j], sc[j], ta[j]) > 0.f ? d[j] : 0.f;
+    for (int u = 0; u < U; ++u) {
+      const long long i = i0 + u * stride;
+      if (i < total_vecs) {
+        rd[u] = ld_raw(dy + i * V);
+        rx[u] = ld_raw(x + i * V);
+        if (addend) ra[u] = ld_raw(addend + i * V);
+      }
     }
 #pragma unroll
-    for (int j = 0; j < V; ++j) o[j] = sc[j] * (d[j] - mb[j] - (f[j] - mean[j]) * rstd[j] * mg[j]);
-    if (addend) {
-      ldv(addend + i * V, f);
+    for (int u = 0; u < U; ++u) {
+      const long long i = i0 + u * stride;
+      if (i >= total_vecs) break;
+      float d[V], f[V], o[V];
+      cvt_raw(rd[u], d);
+      cvt_raw(rx[u], f);
+      if (relu_mask) {
 #pragma unroll
-      for (int j = 0; j < V; ++j) o[j] += f[j];
+        for (int j = 0; j < V; ++j) d[j] = fmaf(f[j], sc[j], ta[j]) > 0.f ? d[j] : 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < V; ++j) o[j] = fmaf(sc[j], d[j], fmaf(a2[j], f[j], a3[j]));
+      if (addend) {
+        cvt_raw(ra[u], f);
+#pragma unroll
+        for (int j = 0; j < V; ++j) o[j] += f[j];
+      }
+      stv(out + i * V, o);
     }
-    stv(out + i * V, o);
   }
 }
 

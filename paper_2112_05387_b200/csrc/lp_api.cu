@@ -56,6 +56,9 @@ enum OpType {
   OP_MAXPOOL_BWD, OP_HEAD_FWD, OP_HEAD_BWD, OP_COPY
 };
 
+static_assert(OP_CONV_FWD == LP_OP_CONV_FWD && OP_BN_BWD == LP_OP_BN_BWD && OP_COPY == LP_OP_COPY && LP_OP_UPDATE == OP_COPY + 1,
+              "operation codes of the time line follow OpType");
+
 struct Op {
   OpType type;
   Tensor in, in2, addend, mask, out;
@@ -123,6 +126,8 @@ struct RunCtx {
   float* loss_out = nullptr;
   bool serial = false;       // layer-serial mode: interior modules produce `out`, no local loss
   cudaEvent_t loss_wait = nullptr;  // recorded when x_{k+1} is ready: awaited just before the local loss
+  int plan_id = 0;           // time line: module k, or LP_AUX(k)
+  int phase = 0;             // time line: LP_PHASE_*
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -152,6 +157,20 @@ struct Device {
 };
 static Device g_dev;
 
+// Per-operation time line: a pair of events around every operation of every plan, on the stream
+// the operation runs on.  Events do not serialise the streams; they cannot be recorded into a graph.
+struct TimelineRec {
+  cudaEvent_t a = nullptr, b = nullptr;
+  int plan = 0, op_type = 0, phase = 0;
+};
+struct Timeline {
+  bool enabled = false;
+  cudaEvent_t base = nullptr;
+  bool base_recorded = false;
+  std::vector<TimelineRec> recs;
+  size_t used = 0;
+};
+
 struct ConvProfile {
   bool enabled = false;
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> events;
@@ -176,6 +195,7 @@ struct lp_handle {
   cudaEvent_t aux_end = nullptr;
   int64_t launches = 0;
   ConvProfile prof;
+  Timeline tl;
   int conv_impl = LP_CONV_IMPL_AUTO;
   uint8_t* ws = nullptr;
   size_t ws_bytes = 0;
@@ -1055,8 +1075,8 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       const T* x2 = nullptr;
       if (op.in2.defined()) { x2 = (const T*)resolve(op.in2, c); B2 = bn_args(P.bns[op.bn2], eps); }
       const T* addend = op.addend.defined() ? (const T*)resolve(op.addend, c) : nullptr;
-      bn_apply_kernel<T><<<grid, threads, 0, st>>>((const T*)resolve(op.in, c), A, x2, B2, addend,
-                                                   (T*)resolve(op.out, c), vecs, b.C, op.relu);
+      launch_bn_apply<T>(grid, threads, st, (const T*)resolve(op.in, c), A, x2, B2, addend, (T*)resolve(op.out, c), vecs,
+                         b.C, op.relu);
       h->launches++;
       break;
     }
@@ -1076,7 +1096,7 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       const T* addend = op.addend.defined() ? (const T*)resolve(op.addend, c) : nullptr;
       if (c.serial) {
         if (!x) break;  // the producing convolution already wrote the module output
-        bn_apply_kernel<T><<<grid, threads, 0, st>>>(x, A, x2, B2, addend, (T*)P.out.p, vecs, C, 0);
+        launch_bn_apply<T>(grid, threads, st, x, A, x2, B2, addend, (T*)P.out.p, vecs, C, 0);
         h->launches++;
         break;
       }
@@ -1149,8 +1169,28 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
   return LP_OK;
 }
 
+struct TimelineScope {
+  lp_handle* h; cudaStream_t st; TimelineRec* r = nullptr;
+  TimelineScope(lp_handle* h_, cudaStream_t st_, int plan, int op_type, int phase) : h(h_), st(st_) {
+    if (!h || !h->tl.enabled) return;
+    Timeline& tl = h->tl;
+    if (tl.used == tl.recs.size()) {
+      TimelineRec n;
+      if (cudaEventCreate(&n.a) != cudaSuccess || cudaEventCreate(&n.b) != cudaSuccess) return;
+      tl.recs.push_back(n);
+    }
+    r = &tl.recs[tl.used++];
+    r->plan = plan; r->op_type = op_type; r->phase = phase;
+    cudaEventRecord(r->a, st);
+  }
+  ~TimelineScope() {
+    if (r) cudaEventRecord(r->b, st);
+  }
+};
+
 static int run_ops(lp_handle* h, Plan& P, const std::vector<Op>& ops, const RunCtx& c) {
   for (const Op& op : ops) {
+    TimelineScope ts(h, c.st, c.plan_id, (int)op.type, c.phase);
     int rc = h->dtype == LP_F32 ? run_op_t<float>(h, P, op, c) : run_op_t<bf16>(h, P, op, c);
     if (rc != LP_OK) return rc;
   }
@@ -1185,8 +1225,11 @@ static int module_fwd_bwd(lp_handle* h, int k, const void* x_k, const void* x_ne
   int rc = zero_forward_state(P, st);
   if (rc != LP_OK) return rc;
   LP_CUDA_OK(cudaMemsetAsync(P.ps.g, 0, P.ps.n * 4, st));
+  c.plan_id = k;
+  c.phase = LP_PHASE_FORWARD;
   rc = run_ops(h, P, P.fwd, c);
   if (rc != LP_OK) return rc;
+  c.phase = LP_PHASE_BACKWARD;
   rc = run_ops(h, P, P.bwd, c);
   if (rc != LP_OK) return rc;
   P.ps.grads_fresh = true;
@@ -1404,7 +1447,8 @@ int lp_auxnet_forward(lp_handle* h, const void* images, void* const* x_out, void
   for (int k = 0; k + 1 < K; ++k) {
     int rc = zero_forward_state(h->auxs[k], c.st);
     if (rc != LP_OK) return rc;
-    rc = run_ops(h, h->auxs[k], h->auxs[k].fwd, c);
+    c.plan_id = LP_AUX(k); c.phase = LP_PHASE_AUX_FORWARD;
+      rc = run_ops(h, h->auxs[k], h->auxs[k].fwd, c);
     if (rc != LP_OK) return rc;
   }
   return LP_OK;
@@ -1455,6 +1499,7 @@ int lp_modules_fwd_bwd_all(lp_handle* h, const void* const* x, const int32_t* la
 static int update_module(lp_handle* h, int k, float lr, float momentum, float weight_decay, float kappa_step,
                          void* lambda_inout, cudaStream_t st) {
   Plan& P = h->modules[k];
+  TimelineScope ts(h, st, k, LP_OP_UPDATE, LP_PHASE_UPDATE);
   sgd_kernel<<<grid_for((long long)P.ps.n, 256, g_dev.sm_count, 8), 256, 0, st>>>(P.ps.p, P.ps.g, P.ps.m,
                                                                                   (long long)P.ps.n, lr, momentum,
                                                                                   weight_decay);
@@ -1520,6 +1565,7 @@ int lp_layer_parallel_step(lp_handle* h, const void* images, void* const* x_out,
     for (int k = 0; k + 1 < K; ++k) {
       int rc = zero_forward_state(h->auxs[k], c.st);
       if (rc != LP_OK) return rc;
+      c.plan_id = LP_AUX(k); c.phase = LP_PHASE_AUX_FORWARD;
       rc = run_ops(h, h->auxs[k], h->auxs[k].fwd, c);
       if (rc != LP_OK) return rc;
       LP_CUDA_OK(cudaEventRecord(h->aux_done[k], h->aux_stream));
@@ -1578,8 +1624,10 @@ int lp_auxnet_distill(lp_handle* h, const void* images, void* const* x, const vo
     distill_loss_kernel<<<1, 1, 0, st>>>(A.loss_acc, loss_out + (k - 1));
     h->launches += 2;
     LP_CUDA_OK(cudaGetLastError());
+    c.plan_id = LP_AUX(k - 1); c.phase = LP_PHASE_DISTILL;
     int rc = run_ops(h, A, A.bwd, c);
     if (rc != LP_OK) return rc;
+    TimelineScope ts(h, st, LP_AUX(k - 1), LP_OP_UPDATE, LP_PHASE_DISTILL);
     sgd_kernel<<<grid_for((long long)A.ps.n, 256, g_dev.sm_count, 8), 256, 0, st>>>(A.ps.p, A.ps.g, A.ps.m,
                                                                                     (long long)A.ps.n, lr_aux, 0.f, 0.f);
     h->launches++;
@@ -1599,6 +1647,7 @@ static int serial_forward(lp_handle* h, const void* images, const int32_t* label
     c.st = st; c.x = x; c.serial = true; c.labels = labels; c.loss_out = loss_out;
     int rc = zero_forward_state(P, st);
     if (rc != LP_OK) return rc;
+    c.plan_id = k; c.phase = LP_PHASE_FORWARD;
     rc = run_ops(h, P, P.fwd, c);
     if (rc != LP_OK) return rc;
     x = P.out.p;
@@ -1632,6 +1681,7 @@ int lp_serial_fwd_bwd(lp_handle* h, const void* images, const int32_t* labels, f
     c.st = st; c.serial = true; c.labels = labels;
     c.x = k == 0 ? images : h->modules[k - 1].out.p;
     c.dx = k > 0 ? h->modules[k - 1].seed.p : nullptr;  // adjoint handed to the previous module
+    c.plan_id = k; c.phase = LP_PHASE_BACKWARD;
     rc = run_ops(h, P, P.bwd, c);
     if (rc != LP_OK) return rc;
     P.ps.grads_fresh = true;
@@ -1691,10 +1741,39 @@ int lp_conv_profile(lp_handle* h, int enable, double* ms, double* flops, int64_t
   return LP_OK;
 }
 
+int lp_timeline(lp_handle* h, int enable, int max_records, lp_timeline_record* records, int* n_records) {
+  if (!h) return LP_ERR_NULL;
+  Timeline& tl = h->tl;
+  if (records || n_records) {
+    LP_CUDA_OK(cudaDeviceSynchronize());
+    int n = 0;
+    // times are relative to the earliest start among the records
+    std::vector<float> t0(tl.used, 0.f), t1(tl.used, 0.f);
+    size_t first = 0;
+    for (size_t i = 1; i < tl.used; ++i) {
+      float d = 0.f;
+      if (cudaEventElapsedTime(&d, tl.recs[first].a, tl.recs[i].a) == cudaSuccess && d < 0.f) first = i;
+    }
+    for (size_t i = 0; i < tl.used; ++i) {
+      if (cudaEventElapsedTime(&t0[i], tl.recs[first].a, tl.recs[i].a) != cudaSuccess) return LP_ERR_CUDA;
+      if (cudaEventElapsedTime(&t1[i], tl.recs[first].a, tl.recs[i].b) != cudaSuccess) return LP_ERR_CUDA;
+      if (records && n < max_records) {
+        records[n].plan = tl.recs[i].plan; records[n].op = tl.recs[i].op_type; records[n].phase = tl.recs[i].phase;
+        records[n].start_ms = t0[i]; records[n].end_ms = t1[i];
+      }
+      ++n;
+    }
+    if (n_records) *n_records = n;
+  }
+  tl.used = 0;
+  tl.enabled = enable != 0;
+  return LP_OK;
+}
+
 int lp_graph_begin(lp_handle* h, void* stream) {
   if (!h) return LP_ERR_NULL;
   if (h->graphs.size() >= 8) return LP_ERR_UNSUPPORTED;
-  if (h->prof.enabled) return LP_ERR_ORDER;
+  if (h->prof.enabled || h->tl.enabled) return LP_ERR_ORDER;
   h->launches_at_capture = h->launches;
   LP_CUDA_OK(cudaStreamBeginCapture((cudaStream_t)stream, cudaStreamCaptureModeRelaxed));
   return LP_OK;

@@ -229,6 +229,49 @@ def test_fused_step_equals_the_three_separate_calls(which):
             assert rel_err(to_host(b.d_kappa[k]), to_host(a.d_kappa[k])) < tol
 
 
+def test_timeline_records_every_operation_of_a_step():
+    """lp_timeline: one record per operation and phase, ordered in time within a module, and a
+    step run with the time line enabled gives the same losses as one without."""
+    cfg = get_config("tiny")
+    run = GpuRun(cfg)
+    lp, h, K = run.lp, run.h, run.net.K
+    lam = run.d_kappa if run.use_kappa else None
+
+    def step():
+        lp.lp_layer_parallel_step(h, run.d_images, run.d_x[1:], run.d_labels, lam, cfg["rho"], run.d_loss, run.d_dx,
+                                  0.0, 0.0, 0.0, 0.0)
+        assert lp.lp_last_device_status(h) == 0
+        return to_host(run.d_loss).copy()
+
+    ref = step()
+    assert lp.lp_timeline(h, True, read=False) == []
+    got = step()
+    recs = lp.lp_timeline(h, False)
+    np.testing.assert_array_equal(got, ref)
+    assert lp.lp_timeline(h, False) == []          # reading drops the records
+    phases = {r["phase"] for r in recs}
+    assert {"aux_forward", "forward", "backward", "update"} <= phases
+    for k in range(K):
+        mine = [r for r in recs if r["plan"] == k]
+        assert sum(r["op"] == "update" for r in mine) == 1
+        assert sum(r["op"] == "out_loss" for r in mine) == (1 if k < K - 1 else 0)
+        assert sum(r["op"] == "head_fwd" for r in mine) == (1 if k == K - 1 else 0)
+        n_fwd = sum(r["op"] == "conv_fwd" for r in mine)
+        assert n_fwd == sum(r["op"] == "conv_wgrad" for r in mine) and n_fwd >= 2
+        # operations of one module run on one stream, in the order they were issued
+        for a, b in zip(mine, mine[1:]):
+            assert a["start_ms"] <= a["end_ms"] <= b["start_ms"] + 1e-3
+        order = [r["phase"] for r in mine]
+        assert order == sorted(order, key=["forward", "backward", "update"].index)
+    assert all(r["plan"] >= 256 for r in recs if r["phase"] == "aux_forward")
+    assert min(r["start_ms"] for r in recs) == 0.0
+    # a graph cannot hold events that are read back: recording is refused while the time line is on
+    lp.lp_timeline(h, True, read=False)
+    with pytest.raises(lp.LpError):
+        lp.lp_graph_begin(h, None)
+    lp.lp_timeline(h, False, read=False)
+
+
 def test_argument_errors_are_reported_on_the_host():
     cfg = get_config("tiny")
     run = GpuRun(cfg)
