@@ -464,7 +464,7 @@ static bool tc_dgrad_ok(const ConvDef& c) {
   return tc_fwd_ok(c) && (c.stride == 1 || (c.H % 2 == 0 && c.W % 2 == 0));
 }
 static bool tc_wgrad_ok(const ConvDef& c) {
-  return c.cin % 8 == 0 && c.cout % 16 == 0 && (c.R == 1 || c.R == 3) && (c.stride == 1 || c.stride == 2);
+  return c.cin % 8 == 0 && c.cout % 8 == 0 && (c.R == 1 || c.R == 3) && (c.stride == 1 || c.stride == 2);
 }
 
 struct ProfScope {

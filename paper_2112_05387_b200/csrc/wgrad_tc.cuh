@@ -251,8 +251,10 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf
   p.m_tiles = (p.total_chunks + p.rpt - 1) / p.rpt;
   int best_tile = 0;
   for (int sc : {64, 32, 16}) {
-    if (Cout % sc) continue;
-    const int chunks = Cout / sc;
+    // 16-channel sub-boxes also serve a C_out that is only a multiple of 8: the last sub-box is
+    // half zero fill (C_out = 40: 32 + 16) and the epilogue skips the channels past C_out
+    if (Cout % sc && sc != 16) continue;
+    const int chunks = (Cout + sc - 1) / sc;
     int nb = 1;
     for (int d = 1; d <= chunks && d * sc <= 256; ++d)
       if (chunks % d == 0) nb = d;
@@ -260,7 +262,7 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf
   }
   if (!best_tile) return -10;
   p.n_tile = best_tile;
-  p.n_tiles = Cout / p.n_tile;
+  p.n_tiles = (Cout + p.n_tile - 1) / p.n_tile;
   // two row tiles per CTA pay off with 64-channel sub-boxes (few, large copies per stage); with
   // narrower sub-boxes the two pipeline stages that still fit do not hide the copy latency
   p.mpair = (p.m_tiles >= 2 && p.sca == 64) ? 2 : 1;

@@ -272,6 +272,22 @@ def test_timeline_records_every_operation_of_a_step():
     lp.lp_timeline(h, False, read=False)
 
 
+def test_speedup_accounting_on_the_tiny_workload():
+    """The speed-up accounting (Section 4.3) runs end to end: K = 1 has no auxiliary phases and the
+    model ratio 1; K = 2 has all five phases and a model ratio between 1 and K."""
+    from paper_2112_05387_b200 import speedup_accounting as sa
+    one = sa.measure("tiny", 1, reps=3)
+    two = sa.measure("tiny", 2, reps=3)
+    assert one["module_block_end"] == [2] and two["module_block_end"] == [1, 2]
+    p1, p2 = one["phases_ms"], two["phases_ms"]
+    assert p1["t_psi"] == p1["t_f_lambda"] == p1["t_b_lambda"] == 0.0 and one["rho_model_K_devices"] == 1.0
+    assert all(v > 0 for v in p2.values())
+    assert 1.0 < two["rho_model_K_devices"] < 2.0
+    for r in (one, two):
+        assert all(v > 0 for v in r["step_ms"].values())
+        assert r["rho_measured_one_gpu"] == pytest.approx(r["step_ms"]["layer_serial"] / r["step_ms"]["layer_parallel"])
+
+
 def test_argument_errors_are_reported_on_the_host():
     cfg = get_config("tiny")
     run = GpuRun(cfg)

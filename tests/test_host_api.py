@@ -5,6 +5,7 @@ import ctypes
 import os
 import re
 
+import numpy as np
 import pytest
 
 import paper_2112_05387_b200 as lp
@@ -80,3 +81,23 @@ def test_bad_descriptors_are_rejected():
     assert "null" in lp.lp_status_string(-1)
     with pytest.raises(lp.LpError):
         lp.lp_param_layout(good, 9)
+
+
+def test_with_modules_splits_the_blocks_evenly_and_validates():
+    """Re-splitting a workload into K modules (the K sweep of the speed-up accounting) keeps the
+    network and yields descriptors the library accepts; K = 1 is the layer-serial network."""
+    import paper_2112_05387_b200 as lp
+    from workloads import with_modules
+    for name, total in (("wrn28_10", 12), ("resnet110", 54), ("tiny", 2)):
+        for K in (1, 2, 3, 4, 6):
+            if K > total:
+                with pytest.raises(ValueError):
+                    with_modules(name, K)
+                continue
+            cfg = with_modules(name, K)
+            ends = cfg["module_block_end"]
+            assert len(ends) == K == cfg["K"] and ends[-1] == total and ends == sorted(set(ends))
+            sizes = np.diff([0] + ends)
+            assert sizes.max() - sizes.min() <= 1
+            assert lp.lp_validate_desc(lp.desc_from_config(cfg)) == 0
+            assert O.Net(cfg).K == K

@@ -6,6 +6,6 @@ settings) and draws every random tensor from one counter-based generator.  It
 contains none of the method's arithmetic: no convolution, no normalisation,
 no loss.
 """
-from .configs import CONFIGS, get_config, scaled  # noqa: F401
+from .configs import CONFIGS, get_config, scaled, with_modules  # noqa: F401
 from .gen import (normal, uniform_int, make_images, make_labels, make_params,  # noqa: F401
                   make_kappa, round_bf16, augment_crop_flip)

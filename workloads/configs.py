@@ -83,3 +83,15 @@ def scaled(name, N=None, H=None, W=None, dtype=None):
     if dtype is not None:
         cfg["dtype"] = dtype
     return cfg
+
+
+def with_modules(name, K, **kw):
+    """The workload `name` re-split into K modules of (nearly) equal block count; K = 1 is the
+    layer-serial network (no auxiliary variables).  Extra keywords go to `scaled`."""
+    cfg = scaled(name, **kw)
+    total = sum(cfg["stage_blocks"])
+    if not 1 <= K <= total:
+        raise ValueError("K must be in 1..%d" % total)
+    cfg["module_block_end"] = [(total * (k + 1)) // K for k in range(K)]
+    cfg["K"] = K
+    return cfg
