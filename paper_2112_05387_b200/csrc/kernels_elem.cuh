@@ -744,4 +744,73 @@ __global__ void pack_weights_tiled_kernel(const PackEntry* __restrict__ tab, int
   }
 }
 
+// The update and the weight copies in one pass over the packed convolution weights:
+//   w <- w - lr*(g + wd*w [momentum])   then the two bf16 copies of the new w, as above.
+// `p_base` / `g_base` / `m_base` are the parameter, gradient and momentum blobs the entries point
+// into (m_base may be null when momentum is 0).
+__global__ void sgd_pack_tiled_kernel(const PackEntry* __restrict__ tab, int n_entries, float* __restrict__ p_base,
+                                      const float* __restrict__ g_base, float* __restrict__ m_base, float lr,
+                                      float momentum, float wd) {
+  __shared__ float tile[32][33];
+  const long long b = blockIdx.x;
+  int lo = 0, hi = n_entries - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (tab[mid].tile_begin <= b) lo = mid; else hi = mid - 1;
+  }
+  const PackEntry e = tab[lo];
+  const long long base = e.w - p_base;
+  const int tiles_ci = (e.cin + 31) >> 5, tiles_co = (e.cout + 31) >> 5;
+  int r = (int)(b - e.tile_begin);
+  const int ci0 = (r % tiles_ci) << 5;
+  r /= tiles_ci;
+  const int co0 = (r % tiles_co) << 5;
+  const int t = r / tiles_co;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  for (int i = ty; i < 32; i += 8) {
+    const int co = co0 + i, ci = ci0 + tx;
+    float v = 0.f;
+    if (co < e.cout && ci < e.cin) {
+      const long long j = ((long long)co * e.taps + t) * e.cin + ci;
+      v = p_base[base + j];
+      float gi = g_base[base + j] + wd * v;
+      if (momentum != 0.f) {
+        gi = momentum * m_base[base + j] + gi;
+        m_base[base + j] = gi;
+      }
+      v -= lr * gi;
+      p_base[base + j] = v;
+      e.wf[j] = __float2bfloat16_rn(v);
+    }
+    tile[i][tx] = v;
+  }
+  if (!e.wt) return;
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int ci = ci0 + i, co = co0 + tx;
+    if (co < e.cout && ci < e.cin) e.wt[((long long)ci * e.taps + t) * e.cout + co] = __float2bfloat16_rn(tile[tx][i]);
+  }
+}
+
+// Plain update of the parameters that have no packed copy (normalisation, head, convolutions on
+// the CUDA-core path): one block per range of the blob.
+struct SgdRange {
+  long long begin;
+  int count;
+};
+__global__ void sgd_ranges_kernel(const SgdRange* __restrict__ ranges, float* __restrict__ p,
+                                  const float* __restrict__ g, float* __restrict__ mom, float lr, float momentum,
+                                  float wd) {
+  const SgdRange r = ranges[blockIdx.x];
+  for (int i = threadIdx.x; i < r.count; i += blockDim.x) {
+    const long long j = r.begin + i;
+    float gi = g[j] + wd * p[j];
+    if (momentum != 0.f) {
+      gi = momentum * mom[j] + gi;
+      mom[j] = gi;
+    }
+    p[j] -= lr * gi;
+  }
+}
+
 }  // namespace lp

@@ -73,6 +73,8 @@ struct ParamSet {
   float *p = nullptr, *g = nullptr, *m = nullptr;
   PackEntry* dev_pack = nullptr;
   std::vector<PackEntry> host_pack;
+  std::vector<SgdRange> host_ranges;   // the parts of the blob that have no packed copy
+  SgdRange* dev_ranges = nullptr;
   long long pack_total = 0;
   long long pack_tiles = 0;
   bool grads_fresh = false;
@@ -691,7 +693,21 @@ struct Planner {
     size_t off = 0;
     for (auto& b : P.bns) { b.stats = base + off; off += (size_t)2 * b.C; }
     P.loss_acc = (double*)A.alloc(2 * sizeof(double));
-    if (!P.ps.host_pack.empty()) P.ps.dev_pack = (PackEntry*)A.alloc(P.ps.host_pack.size() * sizeof(PackEntry));
+    if (!P.ps.host_pack.empty()) {
+      P.ps.dev_pack = (PackEntry*)A.alloc(P.ps.host_pack.size() * sizeof(PackEntry));
+      // complement of the packed entries in [0, n), cut into ranges of at most 16384 elements
+      std::vector<std::pair<long long, long long>> packed;
+      for (const PackEntry& e : P.ps.host_pack)
+        packed.push_back({(long long)(e.w - P.ps.p), (long long)(e.w - P.ps.p) + (long long)e.cout * e.taps * e.cin});
+      std::sort(packed.begin(), packed.end());
+      long long pos = 0;
+      auto add = [&](long long a, long long b) {
+        for (long long q = a; q < b; q += 16384) P.ps.host_ranges.push_back({q, (int)std::min<long long>(16384, b - q)});
+      };
+      for (const auto& pr : packed) { add(pos, pr.first); pos = pr.second; }
+      add(pos, (long long)P.ps.n);
+      if (!P.ps.host_ranges.empty()) P.ps.dev_ranges = (SgdRange*)A.alloc(P.ps.host_ranges.size() * sizeof(SgdRange));
+    }
   }
 
   bool conv_fuses_stats(const ConvDef& c) const {
@@ -1212,6 +1228,31 @@ static int pack_weights(lp_handle* h, Plan& P, cudaStream_t st) {
   return LP_OK;
 }
 
+// theta <- theta - lr*(g + wd*theta [momentum]) and, for the tensor-core path, fresh bf16 copies of
+// the convolution weights: one fused pass over the packed weights plus a small one over the rest.
+static int sgd_update(lp_handle* h, Plan& P, float lr, float momentum, float weight_decay, cudaStream_t st) {
+  float* mom = momentum != 0.f ? P.ps.m : nullptr;
+  if (P.ps.host_pack.empty()) {
+    sgd_kernel<<<grid_for((long long)P.ps.n, 256, g_dev.sm_count, 8), 256, 0, st>>>(P.ps.p, P.ps.g, P.ps.m,
+                                                                                    (long long)P.ps.n, lr, momentum,
+                                                                                    weight_decay);
+    h->launches++;
+    LP_CUDA_OK(cudaGetLastError());
+    return LP_OK;
+  }
+  if (!P.ps.host_ranges.empty()) {
+    sgd_ranges_kernel<<<(unsigned)P.ps.host_ranges.size(), 256, 0, st>>>(P.ps.dev_ranges, P.ps.p, P.ps.g, mom, lr,
+                                                                         momentum, weight_decay);
+    h->launches++;
+  }
+  sgd_pack_tiled_kernel<<<(unsigned)P.ps.pack_tiles, dim3(32, 8), 0, st>>>(P.ps.dev_pack, (int)P.ps.host_pack.size(),
+                                                                           P.ps.p, P.ps.g, mom, lr, momentum,
+                                                                           weight_decay);
+  h->launches++;
+  LP_CUDA_OK(cudaGetLastError());
+  return LP_OK;
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 static int module_fwd_bwd(lp_handle* h, int k, const void* x_k, const void* x_next_or_labels, const void* lambda_k,
@@ -1337,6 +1378,9 @@ int lp_create(const lp_net_desc* desc, void* dev_workspace, size_t bytes, lp_han
     if (P.ps.host_pack.empty()) return LP_OK;
     LP_CUDA_OK(cudaMemcpy(P.ps.dev_pack, P.ps.host_pack.data(), P.ps.host_pack.size() * sizeof(PackEntry),
                           cudaMemcpyHostToDevice));
+    if (!P.ps.host_ranges.empty())
+      LP_CUDA_OK(cudaMemcpy(P.ps.dev_ranges, P.ps.host_ranges.data(), P.ps.host_ranges.size() * sizeof(SgdRange),
+                            cudaMemcpyHostToDevice));
     return LP_OK;
   };
   for (auto& P : h->modules) if ((rc = upload(P)) != LP_OK) { delete h; return rc; }
@@ -1500,12 +1544,7 @@ static int update_module(lp_handle* h, int k, float lr, float momentum, float we
                          void* lambda_inout, cudaStream_t st) {
   Plan& P = h->modules[k];
   TimelineScope ts(h, st, k, LP_OP_UPDATE, LP_PHASE_UPDATE);
-  sgd_kernel<<<grid_for((long long)P.ps.n, 256, g_dev.sm_count, 8), 256, 0, st>>>(P.ps.p, P.ps.g, P.ps.m,
-                                                                                  (long long)P.ps.n, lr, momentum,
-                                                                                  weight_decay);
-  h->launches++;
-  LP_CUDA_OK(cudaGetLastError());
-  int rc = pack_weights(h, P, st);
+  int rc = sgd_update(h, P, lr, momentum, weight_decay, st);
   if (rc != LP_OK) return rc;
   P.ps.grads_fresh = false;
   if (lambda_inout && k + 1 < h->net.K) {
@@ -1628,11 +1667,7 @@ int lp_auxnet_distill(lp_handle* h, const void* images, void* const* x, const vo
     int rc = run_ops(h, A, A.bwd, c);
     if (rc != LP_OK) return rc;
     TimelineScope ts(h, st, LP_AUX(k - 1), LP_OP_UPDATE, LP_PHASE_DISTILL);
-    sgd_kernel<<<grid_for((long long)A.ps.n, 256, g_dev.sm_count, 8), 256, 0, st>>>(A.ps.p, A.ps.g, A.ps.m,
-                                                                                    (long long)A.ps.n, lr_aux, 0.f, 0.f);
-    h->launches++;
-    LP_CUDA_OK(cudaGetLastError());
-    rc = pack_weights(h, A, st);
+    rc = sgd_update(h, A, lr_aux, 0.f, 0.f, st);
     if (rc != LP_OK) return rc;
   }
   return LP_OK;

@@ -272,6 +272,40 @@ def test_timeline_records_every_operation_of_a_step():
     lp.lp_timeline(h, False, read=False)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_update_with_momentum_and_weight_decay(dtype):
+    """lp_step with heavy-ball momentum and weight decay, two steps from the same gradients, against
+    the oracle's update (the velocity starts at zero).  fp32 nets take the plain update kernel; bf16
+    nets the pass that also refreshes the packed bf16 weights, so the second forward must see them."""
+    if dtype == "f32":
+        cfg = get_config("tiny")
+    else:
+        cfg = small_cfg("preact", N=8, H=16, W=16, dtype="bf16", stage_channels=(16, 32), stage_blocks=(1, 1),
+                        module_block_end=(1, 2), stem_channels=16, classes=10)
+    run = GpuRun(cfg)
+    lp, h, K = run.lp, run.h, run.net.K
+    run.auxnet()
+    grads = run.fwd_bwd_all()
+    scale = max(np.abs(g).max() for g in grads)
+    lr, mom, wd = 0.05 / scale, 0.9, 0.01
+    p0 = [lp.lp_get_params(h, k) for k in range(K)]
+    lp.lp_step(h, lr, mom, wd, 0.0, None)
+    p1 = [lp.lp_get_params(h, k) for k in range(K)]
+    vel = []
+    for k in range(K):
+        want, v = O.sgd_update(p0[k], grads[k], lr, momentum=mom, weight_decay=wd)
+        vel.append(v)
+        np.testing.assert_allclose(p1[k], want, rtol=2e-6, atol=1e-7)
+    # second step: same inputs, new parameters; the oracle update uses the GPU's own new gradients
+    loss_before = to_host(run.d_loss).copy()
+    grads2 = run.fwd_bwd_all()
+    assert not np.array_equal(to_host(run.d_loss), loss_before)   # the forward used the updated weights
+    lp.lp_step(h, lr, mom, wd, 0.0, None)
+    for k in range(K):
+        want, _ = O.sgd_update(p1[k], grads2[k], lr, momentum=mom, weight_decay=wd, velocity=vel[k])
+        np.testing.assert_allclose(lp.lp_get_params(h, k), want, rtol=2e-6, atol=1e-7)
+
+
 def test_speedup_accounting_on_the_tiny_workload():
     """The speed-up accounting (Section 4.3) runs end to end: K = 1 has no auxiliary phases and the
     model ratio 1; K = 2 has all five phases and a model ratio between 1 and K."""
