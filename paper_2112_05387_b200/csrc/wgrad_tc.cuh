@@ -11,7 +11,12 @@
 // A CTA computes two row tiles at once where there are at least two: both multiply the same dy
 // stage, which cuts the L2 -> SM traffic per FLOP by about 30 %.
 //
-// Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = epilogue.
+// 3x3 stride-1 convolutions with C_out tiles of at most 160 take wgrad_halo_kernel instead: the
+// three taps of one kernel row read the same x pixels shifted by one pixel each, so ONE x box with
+// a one-pixel halo in w serves all three (see that kernel), which halves the bytes per MMA.
+//
+// Roles (224 threads): warps 0 and 6 = TMA producers (x and dy), warp 1 = MMA issuer, warps 2..5 =
+// epilogue.
 #pragma once
 #include <algorithm>
 
@@ -40,6 +45,12 @@ struct WgradParams {
   uint32_t tmem_cols;
   float* dw;
   int* err;
+  // halo kernel (3x3, stride 1)
+  int groups, acc_stride;        // (ci chunk, kernel row) groups; TMEM column stride of an accumulator
+  uint32_t a_box_bytes;          // one x box: (8+2) x BNI x BH pixels x 64 channels
+  uint32_t a_start3[3];          // first row of the three accumulators' A operands (bytes into the A region)
+  uint64_t adesc_hi3[3];         // their descriptors (the leading byte offset differs)
+  uint32_t a_kstep_bytes;        // 16 pixels further along K
 };
 
 struct WgSmemTail {
@@ -51,7 +62,7 @@ struct WgSmemTail {
   int epi_ok;
 };
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(224, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmDY,
                 const __grid_constant__ WgradParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -69,7 +80,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
-      mbar_init(&tail->full[s], 1);
+      mbar_init(&tail->full[s], 2);    // one expect_tx arrival per producer warp
       mbar_init(&tail->empty[s], 1);
     }
     mbar_init(&tail->acc_full, 1);
@@ -106,8 +117,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const uint32_t tmem_base = tail->tmem_base;
   bool failed = false;
 
-  if (warp == 0) {
-    // TMA producer: warp-uniform loop, one elected lane issues the copies
+  if (warp == 0 || warp == 6) {
+    // TMA producers: warp 0 copies the x sub-boxes, warp 6 the dy sub-boxes (a copy costs its
+    // issuing thread about 100 cycles, and a stage has up to 11 of them for 16 MMAs); warp-uniform
+    // loops, one elected lane issues
+    const bool do_a = warp == 0;
     uint32_t s = 0, ph = 0;
     for (int it = 0; it < n_iter; ++it) {
       const int pt = pt_begin + it;
@@ -116,8 +130,9 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       const int n0 = (pt / (p.tiles_w * p.tiles_h)) * p.BNI;
       if (!mbar_wait_warp(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
       uint8_t* sa = smem + s * p.stage_bytes;
-      if (elect_one()) {
-        mbar_expect_tx(&tail->full[s], p.tx_b + cnt * p.tx_a);
+      const bool leader = elect_one();
+      if (leader && do_a) {
+        mbar_expect_tx(&tail->full[s], cnt * p.tx_a);
         for (int j = 0; j < p.rpt * cnt; ++j) {
           int g = m_tile * p.rpt + j;
           if (g >= p.total_chunks) g = p.total_chunks - 1;  // padding rows of the last tile: any finite data
@@ -126,6 +141,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           tma_load_4d(sa + j * p.a_sub_bytes, &tmX, &tail->full[s], c0, w0 * p.stride + q - p.pad,
                       h0 * p.stride + r - p.pad, n0);
         }
+      } else if (leader) {
+        mbar_expect_tx(&tail->full[s], p.tx_b);
         for (int j = 0; j < p.nb; ++j)
           tma_load_4d(sa + p.a_region + j * p.b_sub_bytes, &tmDY, &tail->full[s], n_tile * p.n_tile + j * p.scb, w0,
                       h0, n0);
@@ -212,6 +229,168 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Weight gradient of a 3x3 stride-1 convolution with tap reuse.
+//
+// K block = 128 output pixels: an 8 (w) x BH x BNI box, rows ordered (w, image, h) in both operands.
+// A "group" is a 64-channel chunk of C_in together with one kernel row r; its three taps (s = 0,1,2)
+// read x at pixels shifted by s - 1 in w.  The x box of a group is 10 pixels wide (halo of one on
+// each side), so the operand of tap s is the same box started s rows (of 128 bytes) further on; an
+// 8-pixel group of K is 8 consecutive box rows and the next one starts 10 rows later (SBO = 1280).
+// As in the forward kernel this relies on the 128-byte swizzle being a function of the address
+// bits.  A CTA holds two groups = six 64-row chunks = three 128-row accumulators in tensor memory:
+//   acc 0 = (g0,s0),(g0,s1)   acc 1 = (g0,s2),(g1,s0)   acc 2 = (g1,s1),(g1,s2)
+// The two chunks of an accumulator are the two 64-element M blocks of an MN-major operand; the
+// descriptor's leading byte offset is the distance between their first rows: 128 bytes inside a
+// box, (box size - 256) across the two boxes.  Per K block a CTA fetches 2 x boxes (40 KB) and
+// the dy tile (128 x n_tile) for 24 MMAs, against 6 sub-boxes (96 KB) without the reuse.
+// Roles as in wgrad_tc_kernel.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(224, 1)
+wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmDY,
+                  const __grid_constant__ WgradParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  WgSmemTail* tail = reinterpret_cast<WgSmemTail*>(smem + (size_t)p.stages * p.stage_bytes);
+  volatile int* abort_flag = &tail->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tile = blockIdx.x % p.m_tiles, n_tile = blockIdx.x / p.m_tiles;
+  const int g0 = 2 * m_tile;                       // groups g0 and g0 + 1 (the second may not exist)
+  const int split = blockIdx.y;
+  const int pt_begin = (int)(((long long)p.pix_tiles * split) / p.splits);
+  const int pt_end = (int)(((long long)p.pix_tiles * (split + 1)) / p.splits);
+  const int n_iter = pt_end - pt_begin;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&tail->full[s], 2);
+      mbar_init(&tail->empty[s], 1);
+    }
+    mbar_init(&tail->acc_full, 1);
+    tail->abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmX);
+    prefetch_tmap(&tmDY);
+  }
+  if (warp == 2) {
+    tmem_alloc(&tail->tmem_base, p.tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tail->tmem_base;
+  bool failed = false;
+
+  if (warp == 0 || warp == 6) {
+    const bool do_a = warp == 0;
+    uint32_t s = 0, ph = 0;
+    for (int it = 0; it < n_iter; ++it) {
+      const int pt = pt_begin + it;
+      const int w0 = (pt % p.tiles_w) * 8;
+      const int h0 = ((pt / p.tiles_w) % p.tiles_h) * p.BH;
+      const int n0 = (pt / (p.tiles_w * p.tiles_h)) * p.BNI;
+      if (!mbar_wait_warp(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
+      uint8_t* sa = smem + s * p.stage_bytes;
+      const bool leader = elect_one();
+      if (leader && do_a) {
+        mbar_expect_tx(&tail->full[s], 2 * p.tx_a);
+        for (int j = 0; j < 2; ++j) {
+          const int g = min(g0 + j, p.groups - 1);   // a missing second group: any finite data
+          const int c0 = (g / 3) * 64, r = g % 3;
+          tma_load_4d(sa + j * p.a_box_bytes, &tmX, &tail->full[s], c0, w0 - 1, n0, h0 + r - 1);
+        }
+      } else if (leader) {
+        mbar_expect_tx(&tail->full[s], p.tx_b);
+        for (int j = 0; j < p.nb; ++j)
+          tma_load_4d(sa + p.a_region + j * p.b_sub_bytes, &tmDY, &tail->full[s], n_tile * p.n_tile + j * p.scb, w0,
+                      n0, h0);
+      }
+      __syncwarp();
+      if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
+    }
+  } else if (warp == 1) {
+    uint32_t s = 0, ph = 0;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t a_kstep = p.a_kstep_bytes >> 4, b_kstep = (uint32_t)(16 * p.scb * 2) >> 4;
+    for (int it = 0; it < n_iter; ++it) {
+      if (!mbar_wait_warp(&tail->full[s], ph, abort_flag)) { failed = true; break; }
+      tc_fence_after();
+      const uint32_t a_addr = smem_base + s * p.stage_bytes;
+      const uint64_t bd = smem_desc(p.bdesc_hi, a_addr + p.a_region);
+      const uint64_t ad0 = smem_desc(p.adesc_hi3[0], a_addr + p.a_start3[0]);
+      const uint64_t ad1 = smem_desc(p.adesc_hi3[1], a_addr + p.a_start3[1]);
+      const uint64_t ad2 = smem_desc(p.adesc_hi3[2], a_addr + p.a_start3[2]);
+      if (elect_one()) {
+#pragma unroll 1
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t acc = (it | j) ? 1u : 0u;
+          mma_bf16(tmem_base, ad0 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
+          mma_bf16(tmem_base + p.acc_stride, ad1 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
+          mma_bf16(tmem_base + 2 * p.acc_stride, ad2 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
+        }
+        mma_commit(&tail->empty[s]);
+      }
+      __syncwarp();
+      if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
+    }
+    if (!failed && n_iter > 0) {
+      if (elect_one()) mma_commit(&tail->acc_full);
+      __syncwarp();
+    }
+  } else {
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const int et = threadIdx.x - 64;
+    if (et == 0) tail->epi_ok = (n_iter > 0 && mbar_wait(&tail->acc_full, 0, abort_flag)) ? 1 : 0;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (*(volatile int*)&tail->epi_ok) {
+      tc_fence_after();
+      for (int a = 0; a < 3; ++a) {
+        const int chunk = 2 * a + (row >> 6);          // 0..5: group chunk/3, kernel column chunk%3
+        const int g = g0 + chunk / 3, sx = chunk % 3;
+        const int ci_raw = (g / 3) * 64 + (row & 63);
+        const bool valid = g < p.groups && ci_raw < p.Cin;
+        const int tap = valid ? (g % 3) * 3 + sx : 0;
+        const int ci = valid ? ci_raw : 0;
+        const uint32_t taddr = tmem_base + a * p.acc_stride + ((uint32_t)(q * 32) << 16);
+        const int co0 = n_tile * p.n_tile;
+        for (int cc = 0; cc < (p.n_tile >> 4); ++cc) {
+          float v[16];
+          tmem_ld16(taddr + cc * 16, v);
+          if (valid) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int co = co0 + cc * 16 + j;
+              if (co < p.Cout) atomicAdd(&p.dw[((long long)co * 9 + tap) * p.Cin + ci], v[j]);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+    } else if (n_iter > 0) {
+      failed = true;
+    }
+  }
+
+  if (failed) {
+    *abort_flag = 1;
+    atomicExch(p.err, 1);
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && !failed) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
 }  // namespace tc
 
 typedef CUresult (*WgEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -234,9 +413,114 @@ static int wg_encode(WgEncodeFn enc, CUtensorMap* m, const void* base, int N, in
   return r == CUDA_SUCCESS ? 0 : -8;
 }
 
+// Tensor maps with the dimension order (C, W, image, H), as the halo kernel's boxes want them.
+static int wg_encode_wnh(WgEncodeFn enc, CUtensorMap* m, const void* base, int N, int H, int W, int C, int boxC, int boxW,
+                         int BNI, int BH) {
+  cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)N, (cuuint64_t)H};
+  cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)H * W * C * 2, (cuuint64_t)W * C * 2};
+  cuuint32_t box[4] = {(cuuint32_t)boxC, (cuuint32_t)boxW, (cuuint32_t)BNI, (cuuint32_t)BH};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  const int row_bytes = boxC * 2;
+  const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS ? 0 : -1;
+}
+
+// Returns 1 when the shape is not one the halo kernel takes (the caller then uses wgrad_tc_kernel).
+static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, const bf16* x, const bf16* dy, float* dw, int N, int H, int W,
+                             int Cin, int Cout, int* dev_err, cudaStream_t st) {
+  if (W % 8 || Cin < 64) return 1;
+  tc::WgradParams p;
+  memset(&p, 0, sizeof(p));
+  p.Nimg = N; p.OH = H; p.OW = W; p.stride = 1; p.pad = 1; p.R = 3;
+  p.Cin = Cin; p.Cout = Cout; p.taps = 9;
+  // pixel box: 8 x BH x BNI = 128
+  if (H >= 16) { p.BH = 16; p.BNI = 1; }
+  else if (H == 8 || H == 4 || H == 2) { p.BH = H; p.BNI = 16 / H; }
+  else return 1;
+  if (p.BNI > N) return 1;
+  p.BW = 8;
+  p.tiles_w = W / 8;
+  p.tiles_h = (H + p.BH - 1) / p.BH;
+  p.pix_tiles = p.tiles_w * p.tiles_h * ((N + p.BNI - 1) / p.BNI);
+  p.rows = p.rows_pad = 128;
+  // dy sub-boxes as in the plain kernel, one channel tile of at most 160 so that three accumulators fit
+  int best_tile = 0;
+  for (int sc : {64, 32, 16}) {
+    if (Cout % sc && sc != 16) continue;
+    const int chunks = (Cout + sc - 1) / sc;
+    int nb = 1;
+    for (int d = 1; d <= chunks && d * sc <= 160; ++d)
+      if (chunks % d == 0) nb = d;
+    if (nb * sc > best_tile) { best_tile = nb * sc; p.scb = sc; p.nb = nb; }
+  }
+  if (best_tile < 64) return 1;
+  p.n_tile = best_tile;
+  p.n_tiles = (Cout + p.n_tile - 1) / p.n_tile;
+  p.acc_stride = (p.n_tile + 31) / 32 * 32;
+  if (3 * p.acc_stride > 512) return 1;
+  p.tmem_cols = 512;
+  p.cin_chunks = (Cin + 63) / 64;
+  p.groups = 3 * p.cin_chunks;
+  p.m_tiles = (p.groups + 1) / 2;
+  const int box_rows = 10 * p.BNI * p.BH;               // 160
+  p.a_box_bytes = (uint32_t)(box_rows * 128);
+  p.a_region = 2 * p.a_box_bytes;
+  p.b_sub_bytes = (uint32_t)((128 * p.scb * 2 + 1023) / 1024 * 1024);
+  p.stage_bytes = p.a_region + p.b_sub_bytes * p.nb;
+  p.tx_a = p.a_box_bytes;
+  p.tx_b = (uint32_t)(128 * p.nb * p.scb * 2);
+  const size_t tail = sizeof(tc::WgSmemTail) + 1024;
+  int stages = (int)((220 * 1024 - tail) / p.stage_bytes);
+  stages = std::min(stages, tc::kWgMaxStages);
+  if (stages < 2) return 1;
+  p.stages = stages;
+  // A operands: rows of 128 bytes; an 8-pixel K group is 8 rows, the next group 10 rows further
+  const uint32_t sbo = 10 * 128;
+  const uint32_t lbo_in = 128, lbo_across = p.a_box_bytes - 2 * 128;
+  p.a_start3[0] = 0;                p.adesc_hi3[0] = tc::smem_desc_hi(lbo_in, sbo, 2);
+  p.a_start3[1] = 2 * 128;          p.adesc_hi3[1] = tc::smem_desc_hi(lbo_across, sbo, 2);
+  p.a_start3[2] = p.a_box_bytes + 128; p.adesc_hi3[2] = tc::smem_desc_hi(lbo_in, sbo, 2);
+  p.a_kstep_bytes = 2 * sbo;                             // 16 pixels = two groups
+  p.bdesc_hi = tc::smem_desc_hi(p.b_sub_bytes, 8 * p.scb * 2, tc::swizzle_code_for_row_bytes(p.scb * 2));
+  p.idesc = tc::instr_desc_bf16(128, p.n_tile, 1, 1);
+  const int tiles = p.m_tiles * p.n_tiles;
+  {
+    int best_s = 1;
+    double best_t = 1e30;
+    const int max_s = std::min(p.pix_tiles, 64);
+    for (int sp = 1; sp <= max_s; ++sp) {
+      const int waves = (tiles * sp + sm_count - 1) / sm_count;
+      const double t = waves * ((double)((p.pix_tiles + sp - 1) / sp) * 1.5 + 4.0);
+      if (t < best_t - 1e-9) { best_t = t; best_s = sp; }
+    }
+    p.splits = best_s;
+  }
+  p.dw = dw; p.err = dev_err;
+  CUtensorMap tmX, tmDY;
+  if (wg_encode_wnh(enc, &tmX, x, N, H, W, Cin, 64, 10, p.BNI, p.BH)) return -8;
+  if (wg_encode_wnh(enc, &tmDY, dy, N, H, W, Cout, p.scb, 8, p.BNI, p.BH)) return -8;
+  size_t smem = std::max((size_t)stages * p.stage_bytes + tail, (size_t)120 * 1024);
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(tc::wgrad_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
+      return -8;
+    attr_set = true;
+  }
+  dim3 grid(tiles, p.splits);
+  tc::wgrad_halo_kernel<<<grid, 224, smem, st>>>(tmX, tmDY, p);
+  return cudaGetLastError() == cudaSuccess ? 0 : -8;
+}
+
 static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf16* dy, float* dw, int N, int H, int W,
                            int Cin, int OH, int OW, int Cout, int R, int stride, int pad, int* dev_err,
                            cudaStream_t st) {
+  if (R == 3 && stride == 1 && pad == 1) {
+    const int rc = launch_wgrad_halo(enc, sm_count, x, dy, dw, N, H, W, Cin, Cout, dev_err, st);
+    if (rc != 1) return rc;
+  }
   tc::WgradParams p;
   memset(&p, 0, sizeof(p));
   p.Nimg = N; p.OH = OH; p.OW = OW;
@@ -327,7 +611,7 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf
     attr_set = true;
   }
   dim3 grid(tiles, p.splits);
-  tc::wgrad_tc_kernel<<<grid, 192, smem, st>>>(tmX, tmDY, p);
+  tc::wgrad_tc_kernel<<<grid, 224, smem, st>>>(tmX, tmDY, p);
   return cudaGetLastError() == cudaSuccess ? 0 : -8;
 }
 
