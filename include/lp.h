@@ -180,6 +180,17 @@ int lp_layer_parallel_step(lp_handle* h, const void* images, void* const* x_out,
 int lp_auxnet_distill(lp_handle* h, const void* images, void* const* x, const void* const* dx, float lr_lambda,
                       float lr_aux, void* const* x_new, float* loss_out, void* stream);
 
+/* Stored-auxiliary-variable mode (Section 4.1, Eq. Parallel-ResNet-Slack-Variables-Update, without
+ * an AuxNet): the caller keeps x_1..x_{K-1} for the batch, runs lp_modules_fwd_bwd_all and lp_step
+ * on them, and this call applies the correction in place,
+ *     x_k <- x_k - lr_lambda * (dx_k - seed_{k-1}),   k = 1..K-1,
+ * where seed_{k-1} is module k-1's terminal adjoint of the same batch (taken from the workspace).
+ *   x_inout[k-1] = x_k (device, K-1 pointers, updated in place); dx[k] = dx_k (K entries, entry 0
+ *   unused); norm_out: device float[K-1] or NULL, receives lr_lambda^2 ||dx_k - seed_{k-1}||^2.
+ * LP_ERR_ORDER if module k-1 has not run. */
+int lp_aux_correct(lp_handle* h, void* const* x_inout, const void* const* dx, float lr_lambda, float* norm_out,
+                   void* stream);
+
 /* Layer-serial comparator (K = 1 in the paper's notation): forward through all modules with
  * x_{k+1} := F_k(x_k); logits: device float[N][num_classes]. */
 int lp_forward_serial(lp_handle* h, const void* images, float* logits, void* stream);

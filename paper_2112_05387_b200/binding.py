@@ -12,7 +12,7 @@ __all__ = [
     "lp_get_params", "lp_get_grads", "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd",
     "lp_modules_fwd_bwd_all", "lp_step", "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual",
     "lp_last_device_status", "lp_launch_count", "lp_conv_profile", "lp_conv2d", "lp_conv2d_scratch_bytes", "lp_graph_begin", "lp_graph_end",
-    "lp_graph_launch", "lp_conv2d_fwd_noalloc", "LP_NOALLOC_SCRATCH_BYTES", "lp_layer_parallel_step", "lp_auxnet_distill", "lp_timeline", "lp_timeline_record",
+    "lp_graph_launch", "lp_conv2d_fwd_noalloc", "LP_NOALLOC_SCRATCH_BYTES", "lp_layer_parallel_step", "lp_auxnet_distill", "lp_aux_correct", "lp_timeline", "lp_timeline_record",
     "LP_PHASE_NAMES", "LP_OP_NAMES", "EXPORTED_SYMBOLS",
 ]
 
@@ -33,7 +33,7 @@ EXPORTED_SYMBOLS = [
     "lp_boundary_shape", "lp_auxnet_forward", "lp_module_fwd_bwd", "lp_modules_fwd_bwd_all", "lp_step",
     "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual", "lp_last_device_status", "lp_launch_count",
     "lp_conv_profile", "lp_conv2d_scratch_bytes", "lp_conv2d", "lp_graph_begin", "lp_graph_end", "lp_graph_launch",
-    "lp_conv2d_fwd_noalloc", "lp_layer_parallel_step", "lp_auxnet_distill", "lp_timeline",
+    "lp_conv2d_fwd_noalloc", "lp_layer_parallel_step", "lp_auxnet_distill", "lp_timeline", "lp_aux_correct",
 ]
 
 
@@ -111,6 +111,8 @@ def library():
     lib.lp_layer_parallel_step.argtypes = [vp, vp, ctypes.POINTER(vp), vp, ctypes.POINTER(vp), f32, vp,
                                            ctypes.POINTER(vp), f32, f32, f32, f32, vp]
     lib.lp_auxnet_distill.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), f32, f32, ctypes.POINTER(vp), vp, vp]
+    lib.lp_aux_correct.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), f32, vp, vp]
+    lib.lp_aux_correct.restype = i32
     lib.lp_forward_serial.argtypes = [vp, vp, vp, vp]
     lib.lp_serial_fwd_bwd.argtypes = [vp, vp, vp, vp, vp]
     lib.lp_get_residual.argtypes = [vp, i32, vp, vp, vp]
@@ -307,6 +309,12 @@ def lp_auxnet_distill(h, images, x, dx, lr_lambda, lr_aux, x_new, loss_out, stre
     na = _ptr_array(x_new, h.K - 1) if x_new is not None else None
     _check(library().lp_auxnet_distill(h.ptr, _ptr(images), xa, da, lr_lambda, lr_aux, na, _ptr(loss_out), _ptr(stream)),
            "lp_auxnet_distill")
+
+
+def lp_aux_correct(h, x_inout, dx, lr_lambda, norm_out=None, stream=None):
+    xa = _ptr_array(x_inout, h.K - 1)
+    da = _ptr_array(dx, h.K)
+    _check(library().lp_aux_correct(h.ptr, xa, da, lr_lambda, _ptr(norm_out), _ptr(stream)), "lp_aux_correct")
 
 
 def lp_forward_serial(h, images, logits, stream=None):

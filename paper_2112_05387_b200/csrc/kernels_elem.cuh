@@ -634,8 +634,8 @@ __global__ void kappa_update_kernel(T* __restrict__ kappa, const T* __restrict__
 //   g = dx_k - seed_{k-1};  x_new = x_k - lr*g (optional output);  d = 2*(x_k - x_new) = 2*lr*g;
 //   acc[0] += sum (lr*g)^2   (the distillation loss ||x_new - AuxNet(x_{k-1})||^2 before the update)
 template <typename T>
-__global__ void distill_seed_kernel(const T* __restrict__ xk, const T* __restrict__ dxk, const T* __restrict__ seed_prev,
-                                    float lr, T* __restrict__ x_new, T* __restrict__ d_out, double* __restrict__ acc,
+__global__ void distill_seed_kernel(const T* xk, const T* __restrict__ dxk, const T* __restrict__ seed_prev,
+                                    float lr, T* x_new /* may alias xk */, T* __restrict__ d_out /* nullable */, double* __restrict__ acc,
                                     long long total_vecs) {
   constexpr int V = VecT<T>::N;
   float sum = 0.f;
@@ -655,9 +655,11 @@ __global__ void distill_seed_kernel(const T* __restrict__ xk, const T* __restric
       for (int j = 0; j < V; ++j) x[j] -= a[j];
       stv(x_new + i * V, x);
     }
+    if (d_out) {
 #pragma unroll
-    for (int j = 0; j < V; ++j) a[j] *= 2.f;
-    stv(d_out + i * V, a);
+      for (int j = 0; j < V; ++j) a[j] *= 2.f;
+      stv(d_out + i * V, a);
+    }
   }
   __shared__ float red[32];
   sum = warp_sum(sum);

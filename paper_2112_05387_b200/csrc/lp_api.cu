@@ -1673,6 +1673,39 @@ int lp_auxnet_distill(lp_handle* h, const void* images, void* const* x, const vo
   return LP_OK;
 }
 
+int lp_aux_correct(lp_handle* h, void* const* x_inout, const void* const* dx, float lr_lambda, float* norm_out,
+                   void* stream) {
+  if (!h || !x_inout || !dx) return LP_ERR_NULL;
+  const int K = h->net.K;
+  for (int k = 1; k < K; ++k) {
+    if (!x_inout[k - 1] || !dx[k]) return LP_ERR_NULL;
+    if (!aligned16(x_inout[k - 1]) || !aligned16(dx[k])) return LP_ERR_ALIGN;
+    if (!h->modules[k - 1].ran_fwd_bwd) return LP_ERR_ORDER;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  for (int k = 1; k < K; ++k) {
+    Plan& A = h->auxs[k - 1];   // only its loss accumulator is used
+    const long long n = h->modules[k - 1].seed.elems();
+    TimelineScope ts(h, st, LP_AUX(k - 1), LP_OP_UPDATE, LP_PHASE_DISTILL);
+    LP_CUDA_OK(cudaMemsetAsync(A.loss_acc, 0, 2 * sizeof(double), st));
+    if (h->dtype == LP_F32)
+      distill_seed_kernel<float><<<grid_for(n / 4, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+          (const float*)x_inout[k - 1], (const float*)dx[k], (const float*)h->modules[k - 1].seed.p, lr_lambda,
+          (float*)x_inout[k - 1], nullptr, A.loss_acc, n / 4);
+    else
+      distill_seed_kernel<bf16><<<grid_for(n / 8, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+          (const bf16*)x_inout[k - 1], (const bf16*)dx[k], (const bf16*)h->modules[k - 1].seed.p, lr_lambda,
+          (bf16*)x_inout[k - 1], nullptr, A.loss_acc, n / 8);
+    h->launches++;
+    if (norm_out) {
+      distill_loss_kernel<<<1, 1, 0, st>>>(A.loss_acc, norm_out + (k - 1));
+      h->launches++;
+    }
+    LP_CUDA_OK(cudaGetLastError());
+  }
+  return LP_OK;
+}
+
 static int serial_forward(lp_handle* h, const void* images, const int32_t* labels, float* loss_out, cudaStream_t st) {
   const int K = h->net.K;
   const void* x = images;

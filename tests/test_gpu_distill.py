@@ -74,3 +74,46 @@ def test_distill_needs_module_passes_first():
         run.lp.lp_auxnet_distill(run.h, run.d_images, run.d_x[1:], run.d_dx, 0.1, 0.1, None,
                                  run.torch.zeros(1, device="cuda:0"))
     assert e.value.status == -6
+
+
+@pytest.mark.parametrize("dtype,tol", [("f32", 1e-5), ("bf16", 2e-2)])
+def test_stored_auxiliary_variables_are_corrected_in_place(dtype, tol):
+    """lp_aux_correct (no AuxNet): caller-held x_1..x_{K-1} (here random tensors, not AuxNet
+    outputs) go through the module passes, then x_k <- x_k - lr*(dx_k - seed_{k-1}) in place;
+    against the oracle's correction fed with the GPU's own dx and terminal adjoints, and against
+    the x_new output of lp_auxnet_distill on the same inputs."""
+    if dtype == "f32":
+        cfg = small_cfg("preact", N=4, H=8, W=8, stage_channels=(8, 16), stage_blocks=(2, 2), module_block_end=(1, 3, 4))
+    else:
+        cfg = small_cfg("preact", N=8, H=16, W=16, dtype="bf16", stage_channels=(16, 32), stage_blocks=(2, 2),
+                        module_block_end=(1, 3, 4), stem_channels=16, classes=10)
+    run = GpuRun(cfg)
+    net, lp, torch = run.net, run.lp, run.torch
+    K = net.K
+    run.auxnet()
+    stored = [gen.storage_round(gen.normal(7, "stored/%d" % k, net.boundary[k], std=0.5), dtype) for k in range(1, K)]
+    run.set_boundaries(stored)
+    with pytest.raises(lp.LpError):                      # module passes have not run yet
+        lp.lp_aux_correct(run.h, run.d_x[1:], run.d_dx, 0.1)
+    run.fwd_bwd_all()
+    lr = 0.1
+    seeds = []
+    for k in range(K - 1):
+        s = torch.zeros_like(run.d_x[k + 1])
+        lp.lp_get_residual(run.h, k, None, s, None)
+        seeds.append(to_host(s))
+    dxs = [None] + [to_host(run.d_dx[k]) for k in range(1, K)]
+    want = [O.aux_correction(stored[k - 1].astype(np.float64), dxs[k], seeds[k - 1], lr)[0] for k in range(1, K)]
+    d_new = [torch.zeros_like(run.d_x[k]) for k in range(1, K)]
+    d_l1 = torch.zeros(K - 1, dtype=torch.float32, device="cuda:0")
+    lp.lp_auxnet_distill(run.h, run.d_images, run.d_x[1:], run.d_dx, lr, 0.0, d_new, d_l1)
+    d_l2 = torch.zeros(K - 1, dtype=torch.float32, device="cuda:0")
+    lp.lp_aux_correct(run.h, run.d_x[1:], run.d_dx, lr, d_l2)
+    assert lp.lp_last_device_status(run.h) == 0
+    np.testing.assert_allclose(d_l2.cpu().numpy(), d_l1.cpu().numpy(), rtol=1e-5)
+    for k in range(1, K):
+        got = to_host(run.d_x[k])
+        np.testing.assert_array_equal(got, to_host(d_new[k - 1]))
+        assert rel_err(got, want[k - 1]) < tol
+        g = dxs[k].astype(np.float64) - seeds[k - 1]
+        assert abs(float(d_l2[k - 1]) - lr * lr * float((g * g).sum())) < 1e-4 * lr * lr * float((g * g).sum()) + 1e-12
