@@ -64,6 +64,7 @@ struct ConvTcParams {
   int ntaps;
   int tap_dh[9], tap_dw[9], tap_w[9];
   int Cin, KC, chunks;
+  int nk_last;                   // K = 16 slices of the last chunk that hold real channels (the rest is zero fill)
   int stages;
   int mpair;                     // pixel tiles per unit: 1 or 2
   int nslots, acc_stride;        // accumulator ring: slots and their TMEM column stride
@@ -240,6 +241,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t accum = 0;
       for (int c = 0; c < p.chunks && !failed; ++c) {
         const uint32_t a_addr = smem_base + sa * p.a_stage_bytes + me * p.a_halo_bytes;
+        const int nkc = c + 1 == p.chunks ? p.nk_last : nk;   // slices of pure zero fill are not multiplied
         for (int ti = 0; ti < 9; ++ti) {
           // The box barrier is polled together with the first weight stage and released together
           // with the last one: a separate trip (poll, election, commit) at every chunk boundary
@@ -252,7 +254,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint64_t bd = smem_desc(p.desc_hi, smem_base + p.b_ring_offset + sb * p.b_stage_bytes);
           if (elect_one()) {
             if (active) {
-              for (int j = 0; j < nk; ++j)
+              for (int j = 0; j < nkc; ++j)
                 mma_bf16(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (accum | j) ? 1u : 0u);
               mma_commit(&tail->empty_b[sb]);
               if (ti == 8) mma_commit(&tail->empty[sa]);
@@ -332,15 +334,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_after();
       }
       const uint32_t d = tmem_base + sl[me] * p.acc_stride;
+      int cc = 0;   // chunk index within the tap
       for (int k = 0; k < kiters; ++k) {
         if (!mbar_wait_warp(&tail->full[s], ph, abort_flag)) { failed = true; break; }
         tc_fence_after();
+        const int nkc = cc + 1 == p.chunks ? p.nk_last : nk;
+        if (++cc == p.chunks) cc = 0;
         const uint32_t a_addr = smem_base + s * p.stage_bytes;
         const uint64_t ad = smem_desc(p.desc_hi, a_addr + me * p.a_region_bytes);
         const uint64_t bd = smem_desc(p.desc_hi, a_addr + p.b_offset);
         if (elect_one()) {
           if (active) {
-            for (int j = 0; j < nk; ++j)  // +32 bytes (one K = 16 slice) per step, in 16-byte units
+            for (int j = 0; j < nkc; ++j)  // +32 bytes (one K = 16 slice) per step, in 16-byte units
               mma_bf16(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k | j) ? 1u : 0u);
             mma_commit(&tail->empty[s]);
           } else {
@@ -366,11 +371,30 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int rows_used = p.BW * p.BH * p.BNI;
     const int ngroups = (p.n_tile_cols + 31) >> 5;
     uint32_t slot = 0, slot_phase = 0;
+    // The residual operand was written several kernels ago and is no longer in L2.  Each thread
+    // asks for the row of the NEXT tile it will add while it works on the current one, so that the
+    // loads of the epilogue find their lines in L2 instead of waiting for DRAM.
+    auto prefetch_addend = [&](int tile) {
+      if (!p.addend || tile >= t_end) return;
+      const int pnt = tile / p.m_tiles, pm = tile % p.m_tiles;
+      const int pw = (pm % p.tiles_w) * p.BW + row % p.BW;
+      const int phh = ((pm / p.tiles_w) % p.tiles_h) * p.BH + (p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH);
+      const int pn = (pm / (p.tiles_w * p.tiles_h)) * p.BNI + (p.halo ? (row / p.BW) % p.BNI : row / (p.BW * p.BH));
+      if (row >= rows_used || pw >= p.OWl || phh >= p.OHl || pn >= p.Nimg || grp) return;
+      const long long pb =
+          (((long long)pn * p.out_H + (phh * p.os + p.oo_h)) * p.out_W + (pw * p.os + p.oo_w)) * p.out_C + pnt * p.n_tile_cols;
+      const int ncols = min(p.n_tile_cols, p.Cout - pnt * p.n_tile_cols);
+      const uintptr_t b = reinterpret_cast<uintptr_t>(p.addend + pb);
+      for (uintptr_t l = b & ~(uintptr_t)127; l < b + 2 * (uintptr_t)ncols; l += 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(l));
+    };
+    prefetch_addend(t_begin);
     for (int t = t_begin; t < t_end && !failed;) {
       const int nt = t / p.m_tiles, m0 = t % p.m_tiles;
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m0 + 1 < p.m_tiles) ? 2 : 1;
       const int col0 = nt * p.n_tile_cols;
       for (int a = 0; a < cnt && !failed; ++a) {
+        prefetch_addend(t + a + 1);
         const int m = m0 + a;
         const uint32_t buf = slot;
         const int w0 = (m % p.tiles_w) * p.BW;

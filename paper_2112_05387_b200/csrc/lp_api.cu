@@ -377,6 +377,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   p.Cin = s.aC;
   p.KC = pick_kc(s.aC);
   p.chunks = (s.aC + p.KC - 1) / p.KC;
+  p.nk_last = (s.aC - (p.chunks - 1) * p.KC + 15) / 16;
   const int row_bytes = p.KC * 2;
   p.a_region_bytes = (uint32_t)align_up((size_t)128 * row_bytes, 1024);
   const uint32_t b_region = (uint32_t)align_up((size_t)p.n_tile_cols * row_bytes, 1024);
