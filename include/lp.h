@@ -58,6 +58,13 @@ enum { LP_KIND_CONV_W = 0, LP_KIND_BN_GAMMA = 1, LP_KIND_BN_BETA = 2, LP_KIND_FC
 enum { LP_CONV_IMPL_AUTO = 0, LP_CONV_IMPL_SIMT = 1, LP_CONV_IMPL_TENSOR = 2 };
 /* May be OR-ed into conv_impl: keep one kind of convolution on the CUDA cores (diagnostics). */
 enum { LP_CONV_NO_TENSOR_FWD = 16, LP_CONV_NO_TENSOR_DGRAD = 32, LP_CONV_NO_TENSOR_WGRAD = 64 };
+/* May be OR-ed into conv_impl: pre-activation networks take the local loss of an interior module
+ * (residual against x_{k+1}, its two sums and the terminal adjoint of
+ * Eq. Parallel-ResNet-Gradient-Propagation-Equation) inside the epilogue of the module's last
+ * tensor-core convolution instead of in a pass of its own over the stored module output.  Same
+ * arithmetic, same results; with the present row-per-thread epilogue it is the slower of the two
+ * (the extra operands are read and written in 16-byte pieces), hence off by default. */
+enum { LP_CONV_LOSS_IN_EPILOGUE = 128 };
 enum { LP_CONV_FWD = 0, LP_CONV_DGRAD = 1, LP_CONV_WGRAD = 2 };
 
 #define LP_MAX_STAGES 8

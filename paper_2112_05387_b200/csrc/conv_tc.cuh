@@ -85,6 +85,14 @@ struct ConvTcParams {
   int tap_widx9[9];              // weight tap index of the nine taps in (dy, dx) order
   uint32_t tap_off9[9];          // byte offset of the tap's first row inside the box
   uint64_t desc_hi_a;            // descriptor of the activation operand (row-group stride of the box)
+  // local loss of an interior module, fused into the epilogue of the module's last convolution
+  // (kLoss instantiation): r = out - x_next, sums of r^2 and kappa*r, seed = rho*r + kappa
+  const bf16* x_next;            // same geometry as out
+  const bf16* kappa;             // nullable (penalty method)
+  bf16* r_out;
+  bf16* seed_out;
+  float rho;
+  double* loss_acc;              // [2]: sum r^2, sum kappa*r (atomically added)
 };
 
 struct TcSmemTail {
@@ -99,43 +107,15 @@ struct TcSmemTail {
   int epi_ok;
   float ssum[LP_EPI_WARPS][256];   // per epilogue warp: plain read-modify-write, no shared-memory atomics
   float ssq[LP_EPI_WARPS][256];
+  uint32_t tr[LP_EPI_WARPS][16 * 33];   // per epilogue warp: transposition scratch of the statistics
 };
-
-// Sum 16 per-lane values over the 32 lanes of a warp; lane l ends with the total of column
-// ((l>>4)&1)*8 + ((l>>3)&1)*4 + ((l>>2)&1)*2 + ((l>>1)&1).
-__device__ __forceinline__ float transpose_reduce16(const float (&v)[16], int lane) {
-  float a[8], b[4], c[2];
-  const bool h4 = lane & 16, h3 = lane & 8, h2 = lane & 4, h1 = lane & 2;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const float send = h4 ? v[j] : v[j + 8];
-    const float keep = h4 ? v[j + 8] : v[j];
-    a[j] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-  }
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const float send = h3 ? a[j] : a[j + 4];
-    const float keep = h3 ? a[j + 4] : a[j];
-    b[j] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-  }
-#pragma unroll
-  for (int j = 0; j < 2; ++j) {
-    const float send = h2 ? b[j] : b[j + 2];
-    const float keep = h2 ? b[j + 2] : b[j];
-    c[j] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-  }
-  const float send = h1 ? c[0] : c[1];
-  const float keep = h1 ? c[1] : c[0];
-  float d = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-  d += __shfl_xor_sync(0xffffffffu, d, 1);
-  return d;
-}
 
 constexpr int kEpiThreads = 32 * LP_EPI_WARPS;
 constexpr int kConvThreads = 96 + kEpiThreads;
 constexpr int kFirstEpiWarp = 3;
 constexpr int kEpiGroups = LP_EPI_WARPS / 4;
 
+template <bool kLoss>
 __global__ void __launch_bounds__(kConvThreads, LP_CONV_MIN_BLOCKS)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ ConvTcParams p) {
@@ -371,6 +351,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int rows_used = p.BW * p.BH * p.BNI;
     const int ngroups = (p.n_tile_cols + 31) >> 5;
     uint32_t slot = 0, slot_phase = 0;
+    float sum_rr = 0.f, sum_kr = 0.f;    // local-loss sums of this thread (kLoss)
     // The residual operand was written several kernels ago and is no longer in L2.  Each thread
     // asks for the row of the NEXT tile it will add while it works on the current one, so that the
     // loads of the epilogue find their lines in L2 instead of waiting for DRAM.
@@ -456,30 +437,72 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                   for (int j = 0; j < 8; ++j) v[8 * u + j] += f[j];
                 }
             }
+            // bf16 pairs as they go to memory: the store and the statistics both work from them
+            uint32_t pk[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
 #pragma unroll
             for (int u = 0; u < 4; ++u)
               if (u < nv && valid && col + 8 * u < p.Cout)
-                stv(p.out + obase + col + 8 * u, *reinterpret_cast<float(*)[8]>(&v[8 * u]));
-            if (p.stats) {
-              // statistics of the tensor as stored (bf16), so that the batch-norm that follows
-              // normalises exactly the values it reads
-              float sq[32];
+                *reinterpret_cast<uint4*>(p.out + obase + col + 8 * u) =
+                    make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+            if constexpr (kLoss) {
+              // The module output is what was just stored (bf16); the residual against the
+              // auxiliary variable, the loss sums and the terminal adjoint follow from it.
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                v[j] = valid ? round_storage<bf16>(v[j]) : 0.f;
-                sq[j] = v[j] * v[j];
-              }
-              const int cl = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+              for (int u = 0; u < 4; ++u)
+                if (u < nv && valid && col + 8 * u < p.Cout) {
+                  float xn[8], r[8], sd[8];
+                  ldv(p.x_next + obase + col + 8 * u, xn);
 #pragma unroll
-              for (int hf = 0; hf < 2; ++hf) {
-                if (hf == 1 && !wide) break;
-                const float cs = transpose_reduce16(*reinterpret_cast<float(*)[16]>(&v[16 * hf]), lane);
-                const float cq = transpose_reduce16(*reinterpret_cast<float(*)[16]>(&sq[16 * hf]), lane);
-                if ((lane & 1) == 0) {
-                  tail->ssum[warp - kFirstEpiWarp][c_in_tile + 16 * hf + cl] += cs;
-                  tail->ssq[warp - kFirstEpiWarp][c_in_tile + 16 * hf + cl] += cq;
+                  for (int j = 0; j < 8; ++j) {
+                    r[j] = round_storage<bf16>(v[8 * u + j]) - xn[j];
+                    sum_rr += r[j] * r[j];
+                  }
+                  stv(p.r_out + obase + col + 8 * u, r);
+                  if (p.kappa) {
+                    float kp[8];
+                    ldv(p.kappa + obase + col + 8 * u, kp);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                      sum_kr += kp[j] * r[j];
+                      sd[j] = p.rho * r[j] + kp[j];
+                    }
+                  } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) sd[j] = p.rho * r[j];
+                  }
+                  stv(p.seed_out + obase + col + 8 * u, sd);
                 }
+            }
+            if (p.stats) {
+              // Statistics of the tensor as stored (bf16), so that the batch-norm that follows
+              // normalises exactly the values it reads.  A thread holds one pixel and 32 channels;
+              // the sums run over pixels, so the warp transposes through shared memory: every lane
+              // writes its 16 channel pairs, then lane l sums channel pair (l & 15) over 16 of the
+              // warp's 32 pixels (both phases conflict-free with the row pitch of 33 words).
+              uint32_t* T = tail->tr[warp - kFirstEpiWarp];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) T[j * 33 + lane] = (valid && (wide || j < 8)) ? pk[j] : 0u;
+              __syncwarp();
+              const int jc = lane & 15, hh = lane >> 4;
+              const uint32_t* col_t = T + jc * 33 + hh * 16;
+              float s0 = 0.f, s1 = 0.f, q0 = 0.f, q1 = 0.f;
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const uint32_t w2 = col_t[i];
+                const float lo = __uint_as_float(w2 << 16), hi = __uint_as_float(w2 & 0xFFFF0000u);
+                s0 += lo; s1 += hi;
+                q0 = fmaf(lo, lo, q0); q1 = fmaf(hi, hi, q1);
               }
+              __syncwarp();
+              s0 += __shfl_xor_sync(0xffffffffu, s0, 16);
+              s1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+              q0 += __shfl_xor_sync(0xffffffffu, q0, 16);
+              q1 += __shfl_xor_sync(0xffffffffu, q1, 16);
+              float* dst = hh ? tail->ssq[warp - kFirstEpiWarp] : tail->ssum[warp - kFirstEpiWarp];
+              dst[c_in_tile + 2 * jc] += hh ? q0 : s0;
+              dst[c_in_tile + 2 * jc + 1] += hh ? q1 : s1;
             }
           }
         }
@@ -507,6 +530,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
       t += cnt;
+    }
+    if constexpr (kLoss) {
+      __syncwarp();
+      sum_rr = warp_sum(sum_rr);
+      sum_kr = warp_sum(sum_kr);
+      if (lane == 0 && !failed) {
+        atomicAdd(&p.loss_acc[0], (double)sum_rr);
+        atomicAdd(&p.loss_acc[1], (double)sum_kr);
+      }
     }
   }
 

@@ -64,6 +64,7 @@ struct Op {
   Tensor in, in2, addend, mask, out;
   int conv = -1, bn = -1, bn2 = -1, stats_bn = -1;
   int relu = 0;
+  int fuse_loss = 0;       // conv: its epilogue takes the module's local loss; out_loss: only the final scalars are left
   uint8_t* arg = nullptr;  // max-pool argmax
 };
 
@@ -242,6 +243,8 @@ struct TcGemmSpec {
   int ntaps; int dh[9], dw[9], widx[9];
   bf16* out; const bf16* addend; int out_H, out_W, out_C, os, oo_h, oo_w;
   double* stats;
+  // local loss fused into the epilogue (interior module's last convolution); x_next == nullptr: off
+  const bf16* x_next; const bf16* kappa; bf16* r_out; bf16* seed_out; float rho; double* loss_acc;
 };
 
 static void pick_pixel_box(int OWl, int OHl, int Nimg, int& BW, int& BH, int& BNI) {
@@ -440,6 +443,8 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   p.idesc = tc::instr_desc_bf16(128, p.n_tile_cols, 0, 0);
   p.desc_hi = tc::smem_desc_hi(16, 8 * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
   p.out = s.out; p.addend = s.addend; p.stats = s.stats; p.err = dev_err;
+  p.x_next = s.x_next; p.kappa = s.kappa; p.r_out = s.r_out; p.seed_out = s.seed_out; p.rho = s.rho;
+  p.loss_acc = s.loss_acc;
   CUtensorMap tmA, tmB;
   int rc = p.halo ? encode_act_map_halo(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, p.KC, kHaloBoxW, p.BH, p.BNI, row_bytes)
                   : encode_act_map(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, p.KC, p.BW, p.BH, p.BNI, s.in_step, row_bytes);
@@ -450,11 +455,15 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   smem = std::max(smem, kTcMinSmem);
   static bool attr_set = false;
   if (!attr_set) {
-    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcMaxSmem));
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)kTcMaxSmem));
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)kTcMaxSmem));
     attr_set = true;
   }
   const int grid = std::min(p.total_tiles, g_dev.sm_count);
-  tc::conv_tc_kernel<<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
+  if (s.x_next) tc::conv_tc_kernel<true><<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
+  else tc::conv_tc_kernel<false><<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
   if (h) h->launches++;
   LP_CUDA_OK(cudaGetLastError());
   return LP_OK;
@@ -469,6 +478,11 @@ static bool tc_dgrad_ok(const ConvDef& c) {
 static bool tc_wgrad_ok(const ConvDef& c) {
   return c.cin % 8 == 0 && c.cout % 8 == 0 && (c.R == 1 || c.R == 3) && (c.stride == 1 || c.stride == 2);
 }
+
+// Local loss of an interior module computed by the epilogue of the module's last convolution.
+struct LossFuse {
+  const void* x_next; const void* kappa; void* r_out; void* seed_out; float rho; double* acc;
+};
 
 struct ProfScope {
   lp_handle* h; cudaStream_t st; double flops; bool on = false; size_t idx = 0;
@@ -493,10 +507,12 @@ struct ProfScope {
 
 // y = conv(x, w) [+ addend]; optional per-channel statistics of y
 static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int N, const void* x, void* y,
-                        const void* addend, double* stats, bool* stats_done, int* dev_err, cudaStream_t st) {
+                        const void* addend, double* stats, bool* stats_done, int* dev_err, cudaStream_t st,
+                        const LossFuse* loss = nullptr) {
   if (stats_done) *stats_done = false;
   const bool use_tc = dtype == LP_BF16 && (impl & 15) != LP_CONV_IMPL_SIMT && !(impl & 16) && tc_fwd_ok(c) && c.wf;
   if ((impl & 15) == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
+  if (loss && !use_tc) return LP_ERR_UNSUPPORTED;  // the planner fuses the loss only into tensor-core convolutions
   if (use_tc) {
     TcGemmSpec s;
     memset(&s, 0, sizeof(s));
@@ -511,6 +527,10 @@ static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int
     s.out = (bf16*)y; s.addend = (const bf16*)addend;
     s.out_H = c.OH; s.out_W = c.OW; s.out_C = c.cout; s.os = 1; s.oo_h = s.oo_w = 0;
     s.stats = stats;
+    if (loss) {
+      s.x_next = (const bf16*)loss->x_next; s.kappa = (const bf16*)loss->kappa; s.r_out = (bf16*)loss->r_out;
+      s.seed_out = (bf16*)loss->seed_out; s.rho = loss->rho; s.loss_acc = loss->acc;
+    }
     if (stats_done) *stats_done = stats != nullptr;
     ProfScope ps(h, st, 2.0 * N * c.OH * c.OW * (double)c.cout * c.R * c.R * c.cin);
     return launch_conv_tc(h, s, dev_err, st);
@@ -888,7 +908,12 @@ struct Planner {
         const int next_bn = !final_block ? recs[i + 1].bn1 : (last ? head_bn : -1);
         Tensor out = emit_conv(P, F, r.a1, r.c2, &sc, next_bn);
         if (final_block && !last) {
+          // The module output is this convolution's accumulator plus the shortcut: on request its
+          // epilogue also takes the residual against x_{k+1}, the loss sums and the terminal adjoint.
+          const bool fuse = (net.d.conv_impl & LP_CONV_LOSS_IN_EPILOGUE) && conv_fuses_stats(P.convs[r.c2]);
+          if (fuse) F.back().fuse_loss = 1;
           Op op;
+          op.fuse_loss = fuse ? 1 : 0;
           op.type = OP_OUT_LOSS; op.addend = out; op.out = P.out;  // in undefined: output already final
           F.push_back(op);
           P.out = like(P.out, out.p);  // layer-serial mode reads the conv output directly
@@ -1057,6 +1082,12 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       double* stats = op.stats_bn >= 0 ? P.bns[op.stats_bn].stats : nullptr;
       const void* addend = op.addend.defined() ? resolve(op.addend, c) : nullptr;
       bool done = false;
+      if (op.fuse_loss && !c.serial) {
+        if (c.loss_wait) LP_CUDA_OK(cudaStreamWaitEvent(st, c.loss_wait, 0));   // x_{k+1} must exist
+        LossFuse lf{c.xnext, c.kappa, P.r.p, P.seed.p, c.rho, P.loss_acc};
+        return conv_forward(h, dtype, h->conv_impl, cv, op.in.n, resolve(op.in, c), resolve(op.out, c), addend, stats,
+                            &done, h->dev_err, st, &lf);
+      }
       return conv_forward(h, dtype, h->conv_impl, cv, op.in.n, resolve(op.in, c), resolve(op.out, c), addend, stats,
                           &done, h->dev_err, st);
     }
@@ -1111,6 +1142,11 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       if (op.in.defined()) { x = (const T*)resolve(op.in, c); A = bn_args(P.bns[op.bn], eps); }
       if (op.in2.defined()) { x2 = (const T*)resolve(op.in2, c); B2 = bn_args(P.bns[op.bn2], eps); }
       const T* addend = op.addend.defined() ? (const T*)resolve(op.addend, c) : nullptr;
+      if (op.fuse_loss && !c.serial) {   // sums, residual and seed came from the last convolution's epilogue
+        loss_finalize_kernel<<<1, 1, 0, st>>>(P.loss_acc, c.rho, c.loss_out);
+        h->launches++;
+        break;
+      }
       if (c.serial) {
         if (!x) break;  // the producing convolution already wrote the module output
         launch_bn_apply<T>(grid, threads, st, x, A, x2, B2, addend, (T*)P.out.p, vecs, C, 0);

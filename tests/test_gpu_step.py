@@ -160,6 +160,17 @@ def test_wrn28_10_reduced_batch_bf16():
     full_step_parity(scaled("wrn28_10", N=6), steps=1)
 
 
+def test_wrn28_10_loss_in_the_last_convolutions_epilogue():
+    """LP_CONV_LOSS_IN_EPILOGUE: residual, loss sums and terminal adjoint taken by the epilogue of each
+    interior module's last convolution give the same step as the separate pass (penalty and AL)."""
+    import paper_2112_05387_b200 as lp
+    full_step_parity(scaled("wrn28_10", N=6), conv_impl=lp.LP_CONV_LOSS_IN_EPILOGUE, steps=1)
+    cfg = scaled("wrn28_10", N=4)
+    cfg["loss"] = "al"
+    cfg["kappa_std"] = 0.1
+    full_step_parity(cfg, conv_impl=lp.LP_CONV_LOSS_IN_EPILOGUE, steps=1)
+
+
 def test_resnet34_reduced_bf16():
     full_step_parity(scaled("resnet34", N=2, H=64, W=64), steps=1)
 
