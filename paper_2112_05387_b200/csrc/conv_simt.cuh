@@ -140,4 +140,125 @@ __global__ void conv_wgrad_simt_kernel(const T* __restrict__ x, const T* __restr
   atomicAdd(&dw[o], acc);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Few input channels (the 3-channel stems and the first AuxNet convolution): K = R*S*Cin is tiny,
+// so the whole filter bank fits in shared memory.  A thread produces CPT output channels of one
+// pixel: one activation load and CPT/4 broadcast reads of the filter bank feed CPT multiply-adds.
+// Same operands as the generic kernels (weights rounded to the activation type, fp32 accumulation).
+// ---------------------------------------------------------------------------------------------
+template <typename T, int CPT>
+__global__ void __launch_bounds__(256)
+conv_fwd_fewch_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, ConvGeom g) {
+  constexpr int V = VecT<T>::N;
+  extern __shared__ float ws[];            // [K][Cout], K = R*S*Cin
+  const int K = g.R * g.S * g.Cin;
+  for (int i = threadIdx.x; i < K * g.Cout; i += blockDim.x) {
+    const int k = i / g.Cout, co = i % g.Cout;
+    ws[i] = round_storage<T>(w[(long long)co * K + k]);
+  }
+  __syncthreads();
+  const int CG = g.Cout / CPT;
+  const long long total = (long long)g.N * g.OH * g.OW * CG;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int cg = (int)(i % CG);
+    const long long p = i / CG;
+    const int ow = (int)(p % g.OW);
+    const long long q = p / g.OW;
+    const int oh = (int)(q % g.OH);
+    const int n = (int)(q / g.OH);
+    float acc[CPT];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) acc[j] = 0.f;
+    for (int r = 0; r < g.R; ++r) {
+      const int ih = oh * g.stride + r - g.pad;
+      if (ih < 0 || ih >= g.H) continue;
+      for (int s = 0; s < g.S; ++s) {
+        const int iw = ow * g.stride + s - g.pad;
+        if (iw < 0 || iw >= g.W) continue;
+        const T* xp = x + (((long long)n * g.H + ih) * g.W + iw) * g.Cin;
+        const float* wr = ws + (r * g.S + s) * g.Cin * g.Cout + cg * CPT;
+        for (int ci = 0; ci < g.Cin; ++ci) {
+          const float xv = to_f(xp[ci]);
+#pragma unroll
+          for (int j4 = 0; j4 < CPT; j4 += 4) {
+            const float4 wv = *reinterpret_cast<const float4*>(wr + ci * g.Cout + j4);
+            acc[j4] += xv * wv.x; acc[j4 + 1] += xv * wv.y; acc[j4 + 2] += xv * wv.z; acc[j4 + 3] += xv * wv.w;
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < CPT; j += V) stv(y + p * g.Cout + cg * CPT + j, *reinterpret_cast<float(*)[V]>(&acc[j]));
+  }
+}
+
+// Weight gradient for few input channels.  A thread owns one filter position k = (r, s, ci) and
+// CPT output channels, and walks the pixels of its block's range: per pixel one activation load
+// and CPT/V 16-byte loads of dy (the same for every thread of a channel group) feed CPT
+// multiply-adds.  With few (k, group) pairs the block's threads also split into pixel lanes, summed
+// through shared memory (threads * CPT floats, dynamic) before one atomic add per output.
+// dw must be zero before the launch.
+template <typename T, int CPT>
+__global__ void __launch_bounds__(256)
+conv_wgrad_fewch_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw, ConvGeom g,
+                        int pair_threads, long long pixels_per_block) {
+  constexpr int V = VecT<T>::N;
+  extern __shared__ float red[];
+  const int K = g.R * g.S * g.Cin;
+  const int CG = g.Cout / CPT;
+  const int npairs = K * CG;
+  const int PL = blockDim.x / pair_threads;          // pixel lanes
+  const int pl = threadIdx.x / pair_threads, pt = threadIdx.x % pair_threads;
+  const bool live = pt < npairs;
+  const int k = live ? pt / CG : 0, cg = live ? pt % CG : 0;
+  const int ci = k % g.Cin, fs = (k / g.Cin) % g.S, fr = k / (g.Cin * g.S);
+  float acc[CPT];
+#pragma unroll
+  for (int j = 0; j < CPT; ++j) acc[j] = 0.f;
+  const long long npix = (long long)g.N * g.OH * g.OW;
+  const long long p0 = (long long)blockIdx.x * pixels_per_block;
+  long long p1 = p0 + pixels_per_block;
+  if (p1 > npix) p1 = npix;
+  if (live && p0 + pl < p1) {
+    long long p = p0 + pl;
+    int ow = (int)(p % g.OW);
+    long long t = p / g.OW;
+    int oh = (int)(t % g.OH);
+    int n = (int)(t / g.OH);
+    for (; p < p1; p += PL) {
+      const int ih = oh * g.stride + fr - g.pad, iw = ow * g.stride + fs - g.pad;
+      if (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) {
+        const float xv = to_f(x[(((long long)n * g.H + ih) * g.W + iw) * g.Cin + ci]);
+        const T* dp = dy + p * g.Cout + cg * CPT;
+#pragma unroll
+        for (int j = 0; j < CPT; j += V) {
+          float f[V];
+          ldv(dp + j, f);
+#pragma unroll
+          for (int u = 0; u < V; ++u) acc[j + u] += xv * f[u];
+        }
+      }
+      ow += PL;
+      while (ow >= g.OW) {
+        ow -= g.OW;
+        if (++oh == g.OH) { oh = 0; ++n; }
+      }
+    }
+  }
+  if (PL > 1) {
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) red[threadIdx.x * CPT + j] = acc[j];
+    __syncthreads();
+    if (pl == 0)
+      for (int l = 1; l < PL; ++l)
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) acc[j] += red[(l * pair_threads + pt) * CPT + j];
+  }
+  if (pl == 0 && live) {
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) atomicAdd(&dw[(long long)(cg * CPT + j) * K + k], acc[j]);
+  }
+}
+
 }  // namespace lp

@@ -115,7 +115,9 @@ constexpr int kConvThreads = 96 + kEpiThreads;
 constexpr int kFirstEpiWarp = 3;
 constexpr int kEpiGroups = LP_EPI_WARPS / 4;
 
-template <bool kLoss>
+// kAddend: a residual operand is added in the epilogue (its loads run one channel group ahead);
+// kLoss: the epilogue also takes the local loss of an interior module (implies kAddend).
+template <bool kLoss, bool kAddend>
 __global__ void __launch_bounds__(kConvThreads, LP_CONV_MIN_BLOCKS)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ ConvTcParams p) {
@@ -356,7 +358,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // asks for the row of the NEXT tile it will add while it works on the current one, so that the
     // loads of the epilogue find their lines in L2 instead of waiting for DRAM.
     auto prefetch_addend = [&](int tile) {
-      if (!p.addend || tile >= t_end) return;
+      if (!kAddend || tile >= t_end) return;
       const int pnt = tile / p.m_tiles, pm = tile % p.m_tiles;
       const int pw = (pm % p.tiles_w) * p.BW + row % p.BW;
       const int phh = ((pm / p.tiles_w) % p.tiles_h) * p.BH + (p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH);
@@ -398,8 +400,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // Drain the accumulator into registers first (up to kBatch x 32 columns per pass) and hand
         // the TMEM slot back to the MMA warp; stores and statistics then work from registers.
         constexpr int kBatch = LP_EPI_BATCH;
+        // Residual operand of one 32-channel group, as raw 16-byte pieces (zero where nothing is added).
+        // A group's pieces are requested while the group before it is processed.
+        auto load_addend = [&](int g, uint4 (&a)[4]) {
+          const int c_in_tile = g * 32;
+          const int nv = c_in_tile + 32 <= p.n_tile_cols ? 4 : 2;
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            a[u] = (g < ngroups && u < nv && valid && col0 + c_in_tile + 8 * u < p.Cout)
+                       ? ld_raw(p.addend + obase + col0 + c_in_tile + 8 * u) : make_uint4(0u, 0u, 0u, 0u);
+        };
         for (int g0 = grp; g0 < ngroups; g0 += kBatch * kEpiGroups) {
           uint32_t raw[kBatch][32];
+          uint4 add_cur[4], add_next[4];
+          if constexpr (kAddend) load_addend(g0, add_cur);
 #pragma unroll
           for (int i = 0; i < kBatch; ++i) {
             const int g = g0 + i * kEpiGroups;
@@ -427,15 +441,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             float v[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = (wide || j < 16) ? __uint_as_float(raw[i][j]) : 0.f;
-            if (p.addend) {
+            if constexpr (kAddend) {
+              if (i + 1 < kBatch) load_addend(g + kEpiGroups, add_next);
 #pragma unroll
-              for (int u = 0; u < 4; ++u)
-                if (u < nv && valid && col + 8 * u < p.Cout) {
-                  float f[8];
-                  ldv(p.addend + obase + col + 8 * u, f);
+              for (int u = 0; u < 4; ++u) {
+                float f[8];
+                cvt_raw(add_cur[u], f);
 #pragma unroll
-                  for (int j = 0; j < 8; ++j) v[8 * u + j] += f[j];
-                }
+                for (int j = 0; j < 8; ++j) v[8 * u + j] += f[j];
+                add_cur[u] = add_next[u];
+              }
             }
             // bf16 pairs as they go to memory: the store and the statistics both work from them
             uint32_t pk[16];

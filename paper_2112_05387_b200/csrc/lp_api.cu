@@ -455,15 +455,19 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   smem = std::max(smem, kTcMinSmem);
   static bool attr_set = false;
   if (!attr_set) {
-    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kTcMaxSmem));
-    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)kTcMaxSmem));
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kTcMaxSmem));
     attr_set = true;
   }
   const int grid = std::min(p.total_tiles, g_dev.sm_count);
-  if (s.x_next) tc::conv_tc_kernel<true><<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
-  else tc::conv_tc_kernel<false><<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
+  if (s.x_next && !s.addend) return LP_ERR_UNSUPPORTED;   // the fused loss belongs to a convolution with a shortcut
+  if (s.x_next) tc::conv_tc_kernel<true, true><<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
+  else if (s.addend) tc::conv_tc_kernel<false, true><<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
+  else tc::conv_tc_kernel<false, false><<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
   if (h) h->launches++;
   LP_CUDA_OK(cudaGetLastError());
   return LP_OK;
@@ -505,6 +509,15 @@ struct ProfScope {
   }
 };
 
+// Output channels per thread of the few-input-channel kernels: the largest of 64, 32, 16, 8 that
+// divides C_out (0: not eligible).
+static int fewch_cpt(int cout, int dtype) {
+  (void)dtype;
+  for (int c : {64, 32, 16, 8})
+    if (cout % c == 0) return c;
+  return 0;
+}
+
 // y = conv(x, w) [+ addend]; optional per-channel statistics of y
 static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int N, const void* x, void* y,
                         const void* addend, double* stats, bool* stats_done, int* dev_err, cudaStream_t st,
@@ -537,6 +550,28 @@ static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int
   }
   if (c.cout % 4) return LP_ERR_UNSUPPORTED;
   ConvGeom g{N, c.H, c.W, c.cin, c.OH, c.OW, c.cout, c.R, c.R, c.stride, c.pad};
+  const size_t few_smem = (size_t)c.R * c.R * c.cin * c.cout * 4;
+  const int few_cpt = fewch_cpt(c.cout, dtype);
+  if (c.cin <= 4 && !addend && few_cpt && few_smem <= 48 * 1024) {
+    // stems and the first AuxNet convolution: filter bank in shared memory
+    const long long items = (long long)N * c.OH * c.OW * (c.cout / few_cpt);
+    const int fgrid = grid_for(items, 256, g_dev.sm_count, 8);
+#define LP_FEWCH_FWD(CPT)                                                                                      \
+    if (dtype == LP_F32)                                                                                       \
+      conv_fwd_fewch_kernel<float, CPT><<<fgrid, 256, few_smem, st>>>((const float*)x, c.w, (float*)y, g);       \
+    else                                                                                                       \
+      conv_fwd_fewch_kernel<bf16, CPT><<<fgrid, 256, few_smem, st>>>((const bf16*)x, c.w, (bf16*)y, g)
+    switch (few_cpt) {
+      case 64: LP_FEWCH_FWD(64); break;
+      case 32: LP_FEWCH_FWD(32); break;
+      case 16: LP_FEWCH_FWD(16); break;
+      default: LP_FEWCH_FWD(8); break;
+    }
+#undef LP_FEWCH_FWD
+    if (h) h->launches++;
+    LP_CUDA_OK(cudaGetLastError());
+    return LP_OK;
+  }
   const long long work = (long long)N * c.OH * c.OW * (c.cout / 4);
   const int grid = grid_for(work, 128, g_dev.sm_count, 16);
   if (dtype == LP_F32)
@@ -624,6 +659,37 @@ static int conv_wgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
   ConvGeom g{N, c.H, c.W, c.cin, c.OH, c.OW, c.cout, c.R, c.R, c.stride, c.pad};
   const int n_out = c.cout * c.R * c.R * c.cin;
   const long long npix = (long long)N * c.OH * c.OW;
+  const int few_cpt = fewch_cpt(c.cout, dtype);
+  if (c.cin <= 4 && few_cpt) {
+    const int npairs = c.R * c.R * c.cin * (c.cout / few_cpt);
+    if (npairs <= 256) {
+      const int pair_threads = (npairs + 31) / 32 * 32;
+      int lanes = 256 / pair_threads;   // pixel lanes, as many as 48 KB of reduction scratch allow
+      while (lanes > 1 && (size_t)lanes * pair_threads * few_cpt * 4 > 48 * 1024) --lanes;
+      const int threads = lanes * pair_threads;
+      const size_t red_bytes = lanes > 1 ? (size_t)threads * few_cpt * 4 : 0;
+      const long long blocks = std::min<long long>((npix + 63) / 64, 6LL * g_dev.sm_count);
+      const long long ppb = (npix + blocks - 1) / blocks;
+      const int fgrid = (int)((npix + ppb - 1) / ppb);
+#define LP_FEWCH_WGRAD(CPT)                                                                                    \
+      if (dtype == LP_F32)                                                                                     \
+        conv_wgrad_fewch_kernel<float, CPT><<<fgrid, threads, red_bytes, st>>>((const float*)x, (const float*)dy, dw, \
+                                                                               g, pair_threads, ppb);          \
+      else                                                                                                     \
+        conv_wgrad_fewch_kernel<bf16, CPT><<<fgrid, threads, red_bytes, st>>>((const bf16*)x, (const bf16*)dy, dw, g, \
+                                                                              pair_threads, ppb)
+      switch (few_cpt) {
+        case 64: LP_FEWCH_WGRAD(64); break;
+        case 32: LP_FEWCH_WGRAD(32); break;
+        case 16: LP_FEWCH_WGRAD(16); break;
+        default: LP_FEWCH_WGRAD(8); break;
+      }
+#undef LP_FEWCH_WGRAD
+      if (h) h->launches++;
+      LP_CUDA_OK(cudaGetLastError());
+      return LP_OK;
+    }
+  }
   int chunk = 256;
   while ((npix + chunk - 1) / chunk > 4096) chunk *= 2;
   dim3 grid((n_out + 127) / 128, (unsigned)((npix + chunk - 1) / chunk));
