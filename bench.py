@@ -30,6 +30,11 @@ METRIC = "images/sec per layer-parallel step"
 UNIT = "images/s"
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of the tensor-core convolution kernels of one WideResNet
+# step, divided by their launches (ncu capture summarised under profiles/).
+TC_CONV_DRAM_BYTES_PER_LAUNCH = 36.5e6
+
+
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -457,7 +462,10 @@ def run_ours(args):
                 "unit": "TFLOP/s", "frac": achieved_tf / peak_tf if peak_tf else None,
                 "frac_of_nominal_2250": achieved_tf / 2250.0,
                 "launches_timed": int(conv_launches), "avg_launch_ms": conv_ms / max(conv_launches, 1),
-                "flops_per_launch_avg": conv_flops / max(conv_launches, 1), "traffic": None,
+                "flops_per_launch_avg": conv_flops / max(conv_launches, 1),
+                "traffic": TC_CONV_DRAM_BYTES_PER_LAUNCH if args.workload == "wrn28_10" and not args.batch else None,
+                "traffic_note": "DRAM bytes read + written per tensor-core conv launch, ncu launch list of one step "
+                                "(profiles/wrn28_10_step_launch_list.md: 3355 MB in 92 launches)",
                 "timing": "CUDA events around every tensor-core conv launch, modules run back to back on one stream"}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
