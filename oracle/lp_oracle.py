@@ -394,6 +394,93 @@ def auxnet_forward(net, aux_params, images, post=None):
 
 
 # ----------------------------------------------------------------------------
+# Recursive auxiliary-variable networks  (Section 4.3, "Recursive Auxiliary-Variable Networks":
+# Eq. ReAuxNet-FP and Eq. ReAuxNet-Distill)
+#
+# ReAuxNet_k(X_0; xi_k) = AuxNet_{k-1}(AuxNet_{k-2}(... AuxNet_0(X_0) ...)) with parameters xi_k of
+# its own: a stack of k units, unit j having the architecture of AuxNet_j.  Every x_k, k = 1..K-1,
+# is generated from the input batch alone, so the K-1 stacks are independent of one another.
+# ``stacks[k-1]`` is the list of the k flat parameter blobs of stack k (unit j in AuxNet_j's layout).
+# ----------------------------------------------------------------------------
+def _aux_unit_fwd(net, j, p, x):
+    """One AuxNet-shaped unit, keeping what its backward pass needs."""
+    convs = net.aux[j]
+    c = {"x": x}
+    c["y1"] = _st(net, conv_fwd(x, _wq(net, p["conv1.w"]), convs[0]["stride"], 1))
+    c["z1"], c["bn1"] = bn_fwd(c["y1"], p["bn1.g"], p["bn1.b"], net.eps)
+    if len(convs) == 2:
+        c["h"] = _st(net, relu(c["z1"]))
+        c["y2"] = _st(net, conv_fwd(c["h"], _wq(net, p["conv2.w"]), convs[1]["stride"], 1))
+        c["z2"], c["bn2"] = bn_fwd(c["y2"], p["bn2.g"], p["bn2.b"], net.eps)
+        return _st(net, c["z2"]), c
+    return _st(net, c["z1"]), c
+
+
+def _aux_unit_bwd(net, j, p, c, d, need_dx):
+    """Adjoint d of the unit's output -> parameter gradients (dict) and, on request, the adjoint of
+    its input."""
+    convs = net.aux[j]
+    g = {}
+    if len(convs) == 2:
+        dy2, g["bn2.g"], g["bn2.b"] = bn_bwd(d, c["bn2"], p["bn2.g"])
+        dy2 = _st(net, dy2)
+        g["conv2.w"] = conv_wgrad(c["h"], dy2, p["conv2.w"].shape, convs[1]["stride"], 1)
+        dh = _st(net, conv_dgrad(dy2, _wq(net, p["conv2.w"]), convs[1]["stride"], 1, c["h"].shape))
+        d = relu_bwd(dh, c["z1"])
+    dy1, g["bn1.g"], g["bn1.b"] = bn_bwd(d, c["bn1"], p["bn1.g"])
+    dy1 = _st(net, dy1)
+    g["conv1.w"] = conv_wgrad(c["x"], dy1, p["conv1.w"].shape, convs[0]["stride"], 1)
+    dx = _st(net, conv_dgrad(dy1, _wq(net, p["conv1.w"]), convs[0]["stride"], 1, c["x"].shape)) if need_dx else None
+    return g, dx
+
+
+def reauxnet_forward(net, stacks, images):
+    """x_k = ReAuxNet_k(X_0; xi_k) for k = 1..K-1 (Eq. ReAuxNet-FP), each from the images alone."""
+    xs = []
+    for k in range(1, net.K):
+        x = np.asarray(images, dtype=F)
+        for j in range(k):
+            x, _ = _aux_unit_fwd(net, j, net.unpack(LP_AUX(j), stacks[k - 1][j]), x)
+        xs.append(x)
+    return xs
+
+
+def reauxnet_fwd_bwd(net, k, stack_params, images, target):
+    """D = ||target - ReAuxNet_k(X_0)||^2 and its gradient with respect to every unit of stack k
+    (``target`` constant).  Returns dict(out, loss, grads: list of k flat blobs)."""
+    ps = [net.unpack(LP_AUX(j), stack_params[j]) for j in range(k)]
+    x, caches = np.asarray(images, dtype=F), []
+    for j in range(k):
+        x, c = _aux_unit_fwd(net, j, ps[j], x)
+        caches.append(c)
+    diff = x - np.asarray(target, dtype=F)
+    loss = float((diff * diff).sum())
+    d = _st(net, 2.0 * diff)
+    grads = [None] * k
+    for j in range(k - 1, -1, -1):
+        g, d = _aux_unit_bwd(net, j, ps[j], caches[j], d, need_dx=j > 0)
+        grads[j] = net.pack(LP_AUX(j), g)
+    return dict(out=x, loss=loss, grads=grads)
+
+
+def reauxnet_distill_step(net, stacks, images, xs, dxs, seeds, lr_lambda, lr_aux):
+    """Knowledge distillation of the recursive networks (Eq. ReAuxNet-Distill), in the same form as
+    ``auxnet_distill_step``: the direction g_k = dx_k - seed_{k-1} (adjoint at the module input plus
+    the derivative of the penalty with respect to x_k) corrects x_k, and every unit of stack k takes
+    one SGD step on ||x_k_new - ReAuxNet_k(X_0)||^2.  With x_k just generated by the stack this
+    gradient is 2*lr_lambda * g_k dReAuxNet_k/dxi_k, the direction of the paper's update."""
+    new_stacks, new_x, losses, grads = [], [], [], []
+    for k in range(1, net.K):
+        x_new, _ = aux_correction(xs[k - 1], dxs[k - 1], seeds[k - 1], lr_lambda)
+        res = reauxnet_fwd_bwd(net, k, stacks[k - 1], images, x_new)
+        new_stacks.append([sgd_update(stacks[k - 1][j], res["grads"][j], lr_aux)[0] for j in range(k)])
+        new_x.append(x_new)
+        losses.append(res["loss"])
+        grads.append(res["grads"])
+    return new_stacks, new_x, losses, grads
+
+
+# ----------------------------------------------------------------------------
 # module forward / backward
 # ----------------------------------------------------------------------------
 def _stem_fwd(net, p, x, cache):

@@ -295,3 +295,105 @@ def test_aux_correction_direction_and_distillation_is_linear_in_the_step():
     np.testing.assert_allclose(grads[0], g1, rtol=1e-12)
     np.testing.assert_allclose(newp[0], auxs[0] - 0.01 * g1, rtol=1e-12, atol=1e-15)
     assert abs(losses[0] - 0.05 ** 2 * float((g * g).sum())) < 1e-12 * max(1.0, losses[0])
+
+
+# -- Recursive auxiliary-variable networks (Eq. ReAuxNet-FP, Eq. ReAuxNet-Distill) ------------------
+def build_stacks(net, cfg, perturb=True):
+    """Stack k (k = 1..K-1) holds k units with parameters of their own; unit j has AuxNet_j's layout."""
+    return [[gen.make_params(net.param_layout(O.LP_AUX(j)), cfg["seed"], "reaux%d/%d" % (k, j), perturb_bn=perturb)
+             for j in range(k)] for k in range(1, net.K)]
+
+
+REAUX_CFGS = [ALL_CFGS[4],
+              ("postbn-4mod", lambda: small_cfg("postbn", stage_channels=(8, 16), stage_blocks=(2, 2),
+                                                module_block_end=(1, 2, 3, 4), N=3))]
+
+
+@pytest.mark.parametrize("name,mk", REAUX_CFGS)
+def test_reauxnet_with_shared_first_parts_is_the_auxnet_chain(name, mk):
+    """The paper's remark at the end of the section: stacks whose leading units share the chain's
+    parameters degenerate to the serial AuxNet chain; and for k = 1 the stack is AuxNet_0 itself."""
+    cfg = mk()
+    net, mods, auxs = build(cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    chain = O.auxnet_forward(net, auxs, x0)
+    shared = [[auxs[j] for j in range(k)] for k in range(1, net.K)]
+    rec = O.reauxnet_forward(net, shared, x0)
+    assert len(rec) == net.K - 1
+    for a, b in zip(rec, chain):
+        np.testing.assert_array_equal(a, b)
+    target = chain[0] + 0.2 * gen.normal(5, "t", chain[0].shape)
+    r1 = O.reauxnet_fwd_bwd(net, 1, shared[0], x0, target)
+    r2 = O.auxnet_fwd_bwd(net, 0, auxs[0], x0, target)
+    assert r1["loss"] == r2["loss"]
+    np.testing.assert_array_equal(r1["grads"][0], r2["grads"])
+    # independent parameters give different variables, each of its boundary's shape
+    stacks = build_stacks(net, cfg)
+    own = O.reauxnet_forward(net, stacks, x0)
+    for k in range(1, net.K):
+        assert own[k - 1].shape == tuple(net.boundary[k])
+    assert not np.allclose(own[-1], chain[-1])
+
+
+@pytest.mark.parametrize("name,mk", REAUX_CFGS)
+def test_reauxnet_distillation_gradients_by_finite_differences(name, mk):
+    cfg = mk()
+    net, mods, auxs = build(cfg)
+    stacks = build_stacks(net, cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    xs = O.reauxnet_forward(net, stacks, x0)
+    for k in range(1, net.K):
+        target = xs[k - 1] + 0.3 * gen.normal(9, "t%d" % k, xs[k - 1].shape)
+        res = O.reauxnet_fwd_bwd(net, k, stacks[k - 1], x0, target)
+        np.testing.assert_allclose(res["out"], xs[k - 1], rtol=1e-12, atol=1e-12)
+        assert len(res["grads"]) == k
+
+        def loss_of(j, p):
+            st = list(stacks[k - 1])
+            st[j] = p
+            out = _stack_forward(net, k, st, x0)
+            return float(((out - target) ** 2).sum())
+        for j in range(k):
+            p0 = stacks[k - 1][j].astype(np.float64)
+            off = 0
+            for pname, _, shape in net.param_layout(O.LP_AUX(j)):
+                n = int(np.prod(shape))
+                for i in sorted(set([off, off + n // 2, off + n - 1])):
+                    h = 1e-5
+                    pp, pm = p0.copy(), p0.copy()
+                    pp[i] += h
+                    pm[i] -= h
+                    fd = (loss_of(j, pp) - loss_of(j, pm)) / (2 * h)
+                    assert abs(fd - res["grads"][j][i]) < 2e-6 * max(1.0, res["loss"]) + 1e-5 * abs(fd), (name, k, j, pname, i)
+                off += n
+        zero = O.reauxnet_fwd_bwd(net, k, stacks[k - 1], x0, xs[k - 1])
+        assert zero["loss"] == 0.0 and all(np.all(g == 0.0) for g in zero["grads"])
+
+
+def _stack_forward(net, k, stack, x0):
+    """Stack k alone, written with the chain's own unit function (not the stack code under test)."""
+    x = np.asarray(x0, dtype=np.float64)
+    for j in range(k):
+        x = O.auxnet_apply(net, j, net.unpack(O.LP_AUX(j), stack[j]), x)
+    return x
+
+
+def test_reauxnet_distill_step_closed_form():
+    """One distillation step: x_k_new = x_k - lr*(dx_k - seed_{k-1}); since x_k was just generated by
+    the stack, the loss is lr^2 ||g_k||^2 and the gradient is linear in lr; units take plain SGD steps."""
+    cfg = REAUX_CFGS[0][1]()
+    net, mods, auxs = build(cfg)
+    stacks = build_stacks(net, cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    xs = O.reauxnet_forward(net, stacks, x0)
+    dxs = [gen.normal(11, "dx%d" % k, xs[k - 1].shape, std=0.1) for k in range(1, net.K)]
+    seeds = [gen.normal(12, "sd%d" % k, xs[k - 1].shape, std=0.1) for k in range(1, net.K)]
+    new1, newx1, loss1, g1 = O.reauxnet_distill_step(net, stacks, x0, xs, dxs, seeds, 0.05, 0.01)
+    new2, newx2, loss2, g2 = O.reauxnet_distill_step(net, stacks, x0, xs, dxs, seeds, 0.10, 0.01)
+    for k in range(1, net.K):
+        g = dxs[k - 1] - seeds[k - 1]
+        np.testing.assert_allclose(newx1[k - 1], xs[k - 1] - 0.05 * g, rtol=1e-14)
+        assert abs(loss1[k - 1] - 0.05 ** 2 * float((g * g).sum())) < 1e-10 * max(1.0, loss1[k - 1])
+        for j in range(k):
+            np.testing.assert_allclose(g2[k - 1][j], 2 * g1[k - 1][j], rtol=1e-8, atol=1e-12)
+            np.testing.assert_allclose(new1[k - 1][j], stacks[k - 1][j] - 0.01 * g1[k - 1][j], rtol=1e-12, atol=1e-15)
