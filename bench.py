@@ -438,6 +438,45 @@ def run_ours(args):
             serial = {"value": cfg["N"] * n_ser / (g0.elapsed_time(g1) * 1e-3), "unit": UNIT,
                       "what": "layer-serial forward + back-propagation + update with the same kernels (no AuxNet)"}
 
+        # the same step with recursive AuxNets (Section 4.3): every x_k generated from the images by a
+        # stack of its own on module k's stream, no serial AuxNet chain
+        recursive = None
+        if not args.no_serial and world == 1 and K > 2:
+            rdesc = lp.desc_from_config(cfg, args.conv_impl, aux_recursive=True)
+            hr = lp.lp_create(rdesc, device=str(dev))
+            for k in range(K):
+                lp.lp_set_params(hr, k, gen.make_params(lp.lp_param_layout(rdesc, k), 0, "module%d" % k, dtype=cfg["dtype"]))
+            for k in range(1, K):
+                for j in range(k):
+                    w = lp.LP_REAUX(k, j)
+                    lp.lp_set_params(hr, w, gen.make_params(lp.lp_param_layout(rdesc, w), 0, "reaux%d/%d" % (k, j),
+                                                            dtype=cfg["dtype"]))
+
+            def step_recursive():
+                lp.lp_layer_parallel_step(hr, d_images, d_x[1:], d_labels, d_kappa, cfg["rho"], d_loss, d_dx, lr, 0.0,
+                                          0.0, kstep, sp)
+            step_recursive()
+            rgid = None
+            if not args.no_graph:
+                lp.lp_graph_begin(hr, sp)
+                step_recursive()
+                rgid = lp.lp_graph_end(hr, sp)
+            for _ in range(3):
+                lp.lp_graph_launch(hr, rgid, sp) if rgid is not None else step_recursive()
+            barrier()
+            r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_r = max(3, args.steps // 3)
+            r0.record(stream)
+            for _ in range(n_r):
+                lp.lp_graph_launch(hr, rgid, sp) if rgid is not None else step_recursive()
+            r1.record(stream)
+            barrier()
+            if lp.lp_last_device_status(hr, sp) != 0:
+                raise RuntimeError("device status in the recursive-AuxNet step")
+            recursive = {"value": cfg["N"] * n_r / (r0.elapsed_time(r1) * 1e-3), "unit": UNIT,
+                         "what": "the step with recursive AuxNets (one independent stack per boundary, K(K-1)/2 units)"}
+            lp.lp_destroy(hr)
+
     # max over ranks
     ms, ms_e2e = max_over_ranks([ms, ms_e2e], dist, dev)
     if rank != 0:
@@ -490,6 +529,8 @@ def run_ours(args):
         line["three_calls"] = three
     if distill:
         line["with_distillation"] = distill
+    if recursive:
+        line["recursive_auxnets"] = recursive
     if not args.no_cpu_baseline and world == 1:
         sb = oracle_sample_batch(cfg)
         val, dt = time_oracle_step(args.workload, sb)

@@ -54,6 +54,11 @@ enum { LP_STEM_CONV3X3 = 0, LP_STEM_CONV7X7S2_MAXPOOL = 1 };
 enum { LP_POSTBN = 0, LP_PREACT = 1 };
 /* `which` argument of the parameter calls: module k is k, AuxNet k is LP_AUX(k). */
 #define LP_AUX(k) (256 + (k))
+/* Recursive auxiliary-variable networks (aux_recursive = 1; Section 4.3, Eq. ReAuxNet-FP): x_k, k = 1..K-1,
+ * is generated from the images alone by a stack of k units with parameters of its own, unit j having
+ * the architecture of AuxNet_j.  LP_REAUX(k, j) names unit j (0 <= j < k) of stack k; the K-1 stacks
+ * do not depend on one another, so the AuxNet chain's serial dependency is gone. */
+#define LP_REAUX(k, j) LP_AUX((k) * ((k) - 1) / 2 + (j))
 enum { LP_KIND_CONV_W = 0, LP_KIND_BN_GAMMA = 1, LP_KIND_BN_BETA = 2, LP_KIND_FC_W = 3, LP_KIND_FC_B = 4 };
 enum { LP_CONV_IMPL_AUTO = 0, LP_CONV_IMPL_SIMT = 1, LP_CONV_IMPL_TENSOR = 2 };
 /* May be OR-ed into conv_impl: keep one kind of convolution on the CUDA cores (diagnostics). */
@@ -99,6 +104,7 @@ typedef struct lp_net_desc {
   int32_t aux_width_div;              /* >= 1 */
   float bn_eps;
   int32_t conv_impl;                  /* LP_CONV_IMPL_*: AUTO picks tensor cores where shapes allow */
+  int32_t aux_recursive;              /* 0: serial AuxNet chain; 1: recursive AuxNets (see LP_REAUX) */
 } lp_net_desc;
 
 typedef struct lp_param_entry {

@@ -5,7 +5,7 @@ import os
 import numpy as np
 
 __all__ = [
-    "LP_OK", "LP_F32", "LP_BF16", "LP_AUX", "LP_CONV_IMPL_AUTO", "LP_CONV_IMPL_SIMT", "LP_CONV_IMPL_TENSOR", "LP_CONV_LOSS_IN_EPILOGUE",
+    "LP_OK", "LP_F32", "LP_BF16", "LP_AUX", "LP_REAUX", "LP_CONV_IMPL_AUTO", "LP_CONV_IMPL_SIMT", "LP_CONV_IMPL_TENSOR", "LP_CONV_LOSS_IN_EPILOGUE",
     "LP_CONV_FWD", "LP_CONV_DGRAD", "LP_CONV_WGRAD", "LpError", "lp_net_desc", "lp_param_entry", "library",
     "library_path", "desc_from_config", "lp_status_string", "lp_validate_desc", "lp_workspace_bytes",
     "lp_param_layout", "lp_boundary_shape_desc", "lp_create", "lp_destroy", "lp_param_count", "lp_set_params",
@@ -42,6 +42,11 @@ def LP_AUX(k):
     return 256 + k
 
 
+def LP_REAUX(k, j):
+    """Unit j (0 <= j < k) of the recursive stack that generates x_k (descriptor aux_recursive = 1)."""
+    return LP_AUX(k * (k - 1) // 2 + j)
+
+
 class LpError(RuntimeError):
     def __init__(self, status, where):
         self.status = status
@@ -57,7 +62,7 @@ class lp_net_desc(ctypes.Structure):
         ("stage_channels", ctypes.c_int32 * LP_MAX_STAGES), ("stage_blocks", ctypes.c_int32 * LP_MAX_STAGES),
         ("stage_stride", ctypes.c_int32 * LP_MAX_STAGES), ("K", ctypes.c_int32),
         ("module_block_end", ctypes.c_int32 * LP_MAX_MODULES), ("aux_convs_per_boundary", ctypes.c_int32),
-        ("aux_width_div", ctypes.c_int32), ("bn_eps", ctypes.c_float), ("conv_impl", ctypes.c_int32),
+        ("aux_width_div", ctypes.c_int32), ("bn_eps", ctypes.c_float), ("conv_impl", ctypes.c_int32), ("aux_recursive", ctypes.c_int32),
     ]
 
 
@@ -149,7 +154,7 @@ def _check(status, where):
         raise LpError(status, where)
 
 
-def desc_from_config(cfg, conv_impl=LP_CONV_IMPL_AUTO):
+def desc_from_config(cfg, conv_impl=LP_CONV_IMPL_AUTO, aux_recursive=False):
     """Translate a workload dict (workloads/configs.py) into the C descriptor."""
     d = lp_net_desc()
     d.struct_size = ctypes.sizeof(lp_net_desc)
@@ -170,6 +175,7 @@ def desc_from_config(cfg, conv_impl=LP_CONV_IMPL_AUTO):
     d.aux_width_div = cfg["aux_width_div"]
     d.bn_eps = cfg["bn_eps"]
     d.conv_impl = conv_impl
+    d.aux_recursive = 1 if aux_recursive else 0
     return d
 
 

@@ -1065,18 +1065,43 @@ struct Planner {
     }
   }
 
+  // AuxNet_k of the serial chain: x_k (the images for k = 0) -> x_{k+1}
   void build_aux(Plan& P, int k) {
-    alloc_params(P, LP_AUX(k));
-    const auto& cv = net.aux[k];
     Tensor x;
     x.ext = k == 0 ? EXT_IMAGES : EXT_XOUT0 + (k - 1);
     const Shape4 s = net.boundary[k];
     x.n = s.n; x.h = s.h; x.w = s.w; x.c = s.c;
+    build_aux_unit(P, k, k, x, true, nullptr);
+  }
+  // Stack k of the recursive form: units j = 0..k-1, the first fed by the images, the last writing x_k;
+  // in the backward pass unit j+1 hands the adjoint of its input to unit j as its seed.
+  void build_reaux_stack(std::vector<Plan>& plans, int k) {
+    Tensor cur;
+    cur.ext = EXT_IMAGES;
+    const Shape4 s0 = net.boundary[0];
+    cur.n = s0.n; cur.h = s0.h; cur.w = s0.w; cur.c = s0.c;
+    for (int j = 0; j < k; ++j) {
+      Plan& P = plans[NetDef::reaux_index(k, j)];
+      const Tensor* dx_out = j > 0 ? &plans[NetDef::reaux_index(k, j - 1)].seed : nullptr;
+      build_aux_unit(P, NetDef::reaux_index(k, j), j, cur, false, dx_out, j == k - 1 ? k - 1 : -1);
+      cur = P.out;
+    }
+  }
+  // One AuxNet-shaped unit (architecture of AuxNet_j) as plan number `idx`.  out_slot >= 0: the output
+  // is the caller's x_{out_slot+1}; otherwise it stays in the workspace.  dx_out: where the adjoint of
+  // the unit's input goes (nullptr: not needed).
+  void build_aux_unit(Plan& P, int idx, int j, const Tensor& x, bool chain, const Tensor* dx_out, int out_slot = -1) {
+    alloc_params(P, LP_AUX(idx));
+    const int k = j;
+    if (chain) out_slot = k;
+    const auto& cv = net.aux[k];
+    const Shape4 s = net.boundary[k];
     std::vector<int> ci, bi;
     for (size_t i = 0; i < cv.size(); ++i) {
       const std::string id = std::to_string(i + 1);
       // the distillation step back-propagates through the second convolution into the first
-      ci.push_back(add_conv(P, "conv" + id + ".w", cv[i].cin, cv[i].cout, 3, cv[i].stride, 1, cv[i].hin, cv[i].win, i > 0));
+      ci.push_back(add_conv(P, "conv" + id + ".w", cv[i].cin, cv[i].cout, 3, cv[i].stride, 1, cv[i].hin, cv[i].win,
+                            i > 0 || dx_out != nullptr));
       bi.push_back(add_bn(P, "bn" + id, cv[i].cout, (long long)s.n * cv[i].hout * cv[i].wout));
     }
     finish_stats(P);
@@ -1090,9 +1115,9 @@ struct Planner {
       Tensor out;
       Op op;
       op.type = OP_BN_APPLY; op.in = y; op.bn = bi[i]; op.relu = final_conv ? 0 : 1;
-      if (final_conv) {
+      if (final_conv && out_slot >= 0) {
         const Shape4 o = net.boundary[k + 1];
-        out.ext = EXT_XOUT0 + k; out.n = o.n; out.h = o.h; out.w = o.w; out.c = o.c;
+        out.ext = EXT_XOUT0 + out_slot; out.n = o.n; out.h = o.h; out.w = o.w; out.c = o.c;
       } else {
         out = new_tensor(y.n, y.h, y.w, y.c);
       }
@@ -1111,6 +1136,7 @@ struct Planner {
       Tensor dy = emit_bn_bwd(P.bwd, d, ys[i], relu_after ? &acts[i] : nullptr, bi[i], nullptr);
       emit_wgrad(P.bwd, ins[i], dy, ci[i]);
       if (i > 0) d = emit_dgrad(P, P.bwd, dy, ci[i], nullptr, nullptr);
+      else if (dx_out) emit_dgrad(P, P.bwd, dy, ci[i], nullptr, dx_out);
     }
   }
 };
@@ -1417,8 +1443,12 @@ static int plan_all(const NetDef& net, Arena& A, std::vector<Plan>* modules, std
   *zero_labels = (int32_t*)A.alloc((size_t)net.d.N * 4);
   modules->resize(net.K);
   for (int k = 0; k < net.K; ++k) pl.build_module((*modules)[k], k);
-  auxs->resize(net.K > 1 ? net.K - 1 : 0);
-  for (int k = 0; k + 1 < net.K; ++k) pl.build_aux((*auxs)[k], k);
+  auxs->resize(net.n_aux_plans());
+  if (net.d.aux_recursive) {
+    for (int k = 1; k < net.K; ++k) pl.build_reaux_stack(*auxs, k);
+  } else {
+    for (int k = 0; k + 1 < net.K; ++k) pl.build_aux((*auxs)[k], k);
+  }
   return LP_OK;
 }
 
@@ -1580,6 +1610,13 @@ int lp_boundary_shape(lp_handle* h, int k, int shape[4]) {
   return LP_OK;
 }
 
+static int aux_plan_forward(lp_handle* h, int idx, RunCtx& c) {
+  int rc = zero_forward_state(h->auxs[idx], c.st);
+  if (rc != LP_OK) return rc;
+  c.plan_id = LP_AUX(idx); c.phase = LP_PHASE_AUX_FORWARD;
+  return run_ops(h, h->auxs[idx], h->auxs[idx].fwd, c);
+}
+
 int lp_auxnet_forward(lp_handle* h, const void* images, void* const* x_out, void* stream) {
   if (!h || !images) return LP_ERR_NULL;
   const int K = h->net.K;
@@ -1591,11 +1628,8 @@ int lp_auxnet_forward(lp_handle* h, const void* images, void* const* x_out, void
   }
   RunCtx c;
   c.st = (cudaStream_t)stream; c.images = images; c.xout = x_out;
-  for (int k = 0; k + 1 < K; ++k) {
-    int rc = zero_forward_state(h->auxs[k], c.st);
-    if (rc != LP_OK) return rc;
-    c.plan_id = LP_AUX(k); c.phase = LP_PHASE_AUX_FORWARD;
-      rc = run_ops(h, h->auxs[k], h->auxs[k].fwd, c);
+  for (size_t i = 0; i < h->auxs.size(); ++i) {   // chain order, or stack by stack (units in order)
+    int rc = aux_plan_forward(h, (int)i, c);
     if (rc != LP_OK) return rc;
   }
   return LP_OK;
@@ -1699,16 +1733,28 @@ int lp_layer_parallel_step(lp_handle* h, const void* images, void* const* x_out,
   }
   cudaStream_t st = (cudaStream_t)stream;
   LP_CUDA_OK(cudaEventRecord(h->fork, st));
-  // AuxNet chain on its own stream; aux_done[k] marks x_{k+1}
   LP_CUDA_OK(cudaStreamWaitEvent(h->aux_stream, h->fork, 0));
-  {
+  if (h->net.d.aux_recursive) {
+    // recursive form: stack k needs the images only and runs on module k's stream, right before the
+    // module it feeds; aux_done[k-1] marks x_k for module k-1's local loss
+    for (int k = 1; k < K; ++k) {
+      cudaStream_t sk = h->streams[k];
+      LP_CUDA_OK(cudaStreamWaitEvent(sk, h->fork, 0));
+      RunCtx c;
+      c.st = sk; c.images = images; c.xout = x_out;
+      for (int j = 0; j < k; ++j) {
+        int rc = aux_plan_forward(h, NetDef::reaux_index(k, j), c);
+        if (rc != LP_OK) return rc;
+      }
+      LP_CUDA_OK(cudaEventRecord(h->aux_done[k - 1], sk));
+    }
+    LP_CUDA_OK(cudaEventRecord(h->aux_end, h->aux_stream));
+  } else {
+    // AuxNet chain on its own stream; aux_done[k] marks x_{k+1}
     RunCtx c;
     c.st = h->aux_stream; c.images = images; c.xout = x_out;
     for (int k = 0; k + 1 < K; ++k) {
-      int rc = zero_forward_state(h->auxs[k], c.st);
-      if (rc != LP_OK) return rc;
-      c.plan_id = LP_AUX(k); c.phase = LP_PHASE_AUX_FORWARD;
-      rc = run_ops(h, h->auxs[k], h->auxs[k].fwd, c);
+      int rc = aux_plan_forward(h, k, c);
       if (rc != LP_OK) return rc;
       LP_CUDA_OK(cudaEventRecord(h->aux_done[k], h->aux_stream));
     }
@@ -1749,11 +1795,15 @@ int lp_auxnet_distill(lp_handle* h, const void* images, void* const* x, const vo
   cudaStream_t st = (cudaStream_t)stream;
   RunCtx c;
   c.st = st; c.images = images; c.xout = x;
+  const bool rec = h->net.d.aux_recursive != 0;
   for (int k = 1; k < K; ++k) {
-    Plan& A = h->auxs[k - 1];
+    // the network that produced x_k: AuxNet_{k-1}, or the last unit of stack k
+    const int last_idx = rec ? NetDef::reaux_index(k, k - 1) : k - 1;
+    const int first_idx = rec ? NetDef::reaux_index(k, 0) : k - 1;
+    Plan& A = h->auxs[last_idx];
     const long long n = A.seed.elems();
     LP_CUDA_OK(cudaMemsetAsync(A.loss_acc, 0, 2 * sizeof(double), st));
-    LP_CUDA_OK(cudaMemsetAsync(A.ps.g, 0, A.ps.n * 4, st));
+    for (int i = first_idx; i <= last_idx; ++i) LP_CUDA_OK(cudaMemsetAsync(h->auxs[i].ps.g, 0, h->auxs[i].ps.n * 4, st));
     void* xn = x_new ? x_new[k - 1] : nullptr;
     if (h->dtype == LP_F32)
       distill_seed_kernel<float><<<grid_for(n / 4, 256, g_dev.sm_count, 8), 256, 0, st>>>(
@@ -1766,12 +1816,18 @@ int lp_auxnet_distill(lp_handle* h, const void* images, void* const* x, const vo
     distill_loss_kernel<<<1, 1, 0, st>>>(A.loss_acc, loss_out + (k - 1));
     h->launches += 2;
     LP_CUDA_OK(cudaGetLastError());
-    c.plan_id = LP_AUX(k - 1); c.phase = LP_PHASE_DISTILL;
-    int rc = run_ops(h, A, A.bwd, c);
-    if (rc != LP_OK) return rc;
-    TimelineScope ts(h, st, LP_AUX(k - 1), LP_OP_UPDATE, LP_PHASE_DISTILL);
-    rc = sgd_update(h, A, lr_aux, 0.f, 0.f, st);
-    if (rc != LP_OK) return rc;
+    // back through the units (one in the chain form), each followed by its own SGD step
+    for (int i = last_idx; i >= first_idx; --i) {
+      Plan& U = h->auxs[i];
+      c.plan_id = LP_AUX(i); c.phase = LP_PHASE_DISTILL;
+      int rc = run_ops(h, U, U.bwd, c);
+      if (rc != LP_OK) return rc;
+    }
+    for (int i = first_idx; i <= last_idx; ++i) {
+      TimelineScope ts(h, st, LP_AUX(i), LP_OP_UPDATE, LP_PHASE_DISTILL);
+      int rc = sgd_update(h, h->auxs[i], lr_aux, 0.f, 0.f, st);
+      if (rc != LP_OK) return rc;
+    }
   }
   return LP_OK;
 }

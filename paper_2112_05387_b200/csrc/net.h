@@ -50,6 +50,7 @@ struct NetDef {
     if (d.K < 1 || d.K > LP_MAX_MODULES) return LP_ERR_BAD_DESC;
     if (d.aux_convs_per_boundary < 1 || d.aux_convs_per_boundary > 2 || d.aux_width_div < 1) return LP_ERR_BAD_DESC;
     if (!(d.bn_eps > 0.f)) return LP_ERR_BAD_DESC;
+    if (d.aux_recursive != 0 && d.aux_recursive != 1) return LP_ERR_BAD_DESC;
     if (d.conv_impl < 0 || (d.conv_impl & 15) > LP_CONV_IMPL_TENSOR || d.conv_impl > 255) return LP_ERR_BAD_DESC;
     const int vec = d.dtype == LP_F32 ? 4 : 8;
     if (d.stem_channels < vec || d.stem_channels % vec) return LP_ERR_BAD_DESC;
@@ -139,12 +140,24 @@ struct NetDef {
   }
 
   // Flat parameter layout (blob order) of module `which` or AuxNet LP_AUX(k).
+  // AuxNet plans: the K-1 networks of the chain, or (recursive form) the units of the K-1 stacks,
+  // stack k = 1..K-1 holding units j = 0..k-1 at index k(k-1)/2 + j; a unit has AuxNet_j's shape.
+  int n_aux_plans() const { return K < 2 ? 0 : (d.aux_recursive ? K * (K - 1) / 2 : K - 1); }
+  static int reaux_index(int k, int j) { return k * (k - 1) / 2 + j; }
+  int aux_unit(int idx) const {
+    if (!d.aux_recursive) return idx;
+    int k = 1;
+    while (reaux_index(k + 1, 0) <= idx) ++k;
+    return idx - reaux_index(k, 0);
+  }
+
   int layout(int which, std::vector<lp_param_entry>& L, uint64_t* total) const {
     L.clear();
     uint64_t off = 0;
     if (which >= LP_AUX(0)) {
-      const int k = which - LP_AUX(0);
-      if (k < 0 || k >= K - 1) return LP_ERR_BAD_INDEX;
+      const int idx = which - LP_AUX(0);
+      if (idx < 0 || idx >= n_aux_plans()) return LP_ERR_BAD_INDEX;
+      const int k = aux_unit(idx);
       for (size_t i = 0; i < aux[k].size(); ++i) {
         const std::string id = std::to_string(i + 1);
         push(L, off, "conv" + id + ".w", LP_KIND_CONV_W, aux[k][i].cout, 3, 3, aux[k][i].cin);

@@ -46,18 +46,27 @@ def per_tensor_errors(net, which, got_flat, ref_flat):
 class GpuRun:
     """One workload on the GPU: handle, parameters, device buffers."""
 
-    def __init__(self, cfg, conv_impl=0, perturb=True, kappa_std=None):
+    def __init__(self, cfg, conv_impl=0, perturb=True, kappa_std=None, aux_recursive=False):
         import torch
         import paper_2112_05387_b200 as lp
         self.lp, self.torch, self.cfg = lp, torch, cfg
         self.net = O.Net(cfg)
-        self.desc = lp.desc_from_config(cfg, conv_impl)
+        self.desc = lp.desc_from_config(cfg, conv_impl, aux_recursive)
         self.h = lp.lp_create(self.desc)
         self.mods, self.auxs = make_all_params(self.net, cfg, perturb)
         for k in range(self.net.K):
             lp.lp_set_params(self.h, k, self.mods[k])
-        for k in range(self.net.K - 1):
-            lp.lp_set_params(self.h, lp.LP_AUX(k), self.auxs[k])
+        self.stacks = None
+        if aux_recursive:   # stack k = 1..K-1: k units with parameters of their own
+            self.stacks = [[gen.make_params(self.net.param_layout(O.LP_AUX(j)), cfg["seed"], "reaux%d/%d" % (k, j),
+                                            perturb_bn=perturb, dtype=cfg["dtype"]) for j in range(k)]
+                           for k in range(1, self.net.K)]
+            for k in range(1, self.net.K):
+                for j in range(k):
+                    lp.lp_set_params(self.h, lp.LP_REAUX(k, j), self.stacks[k - 1][j])
+        else:
+            for k in range(self.net.K - 1):
+                lp.lp_set_params(self.h, lp.LP_AUX(k), self.auxs[k])
         self.images = gen.make_images(cfg)
         self.labels = gen.make_labels(cfg)
         self.d_images = to_dev(self.images, cfg)

@@ -101,3 +101,23 @@ def test_with_modules_splits_the_blocks_evenly_and_validates():
             assert sizes.max() - sizes.min() <= 1
             assert lp.lp_validate_desc(lp.desc_from_config(cfg)) == 0
             assert O.Net(cfg).K == K
+
+
+def test_recursive_auxnet_layouts_match_the_oracle():
+    """aux_recursive = 1: LP_REAUX(k, j) has the layout of AuxNet_j; indices past the last stack are refused."""
+    import paper_2112_05387_b200 as lp
+    from conftest import small_cfg
+    from oracle import lp_oracle as O
+    cfg = small_cfg("preact", stage_channels=(8, 16), stage_blocks=(2, 2), module_block_end=(1, 2, 3, 4), N=3)
+    net = O.Net(cfg)
+    desc = lp.desc_from_config(cfg, aux_recursive=True)
+    assert lp.lp_validate_desc(desc) == 0
+    assert lp.lp_workspace_bytes(desc) > lp.lp_workspace_bytes(lp.desc_from_config(cfg))
+    for k in range(1, net.K):
+        for j in range(k):
+            lay = lp.lp_param_layout(desc, lp.LP_REAUX(k, j))
+            assert [(n, tuple(s)) for n, _, s in lay] == [(n, tuple(s)) for n, _, s in net.param_layout(O.LP_AUX(j))]
+    with pytest.raises(lp.LpError):
+        lp.lp_param_layout(desc, lp.LP_REAUX(net.K, 0))
+    desc.aux_recursive = 2
+    assert lp.lp_validate_desc(desc) != 0
