@@ -28,6 +28,11 @@ namespace tc {
 
 constexpr int kWgMaxStages = 8;
 
+// pixels per K block of wgrad_halo_kernel (128 or 64)
+#ifndef LP_WGRAD_HALO_KBLOCK
+#define LP_WGRAD_HALO_KBLOCK 128
+#endif
+
 struct WgradParams {
   int Nimg, OH, OW;
   int BW, BH, BNI, tiles_w, tiles_h, pix_tiles;
@@ -232,7 +237,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 // ---------------------------------------------------------------------------------------------
 // Weight gradient of a 3x3 stride-1 convolution with tap reuse.
 //
-// K block = 128 output pixels: an 8 (w) x BH x BNI box, rows ordered (w, image, h) in both operands.
+// K block = 128 (or 64) output pixels: an 8 (w) x BH x BNI box, rows ordered (w, image, h) in both operands.
 // A "group" is a 64-channel chunk of C_in together with one kernel row r; its three taps (s = 0,1,2)
 // read x at pixels shifted by s - 1 in w.  The x box of a group is 10 pixels wide (halo of one on
 // each side), so the operand of tap s is the same box started s rows (of 128 bytes) further on; an
@@ -242,7 +247,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 //   acc 0 = (g0,s0),(g0,s1)   acc 1 = (g0,s2),(g1,s0)   acc 2 = (g1,s1),(g1,s2)
 // The two chunks of an accumulator are the two 64-element M blocks of an MN-major operand; the
 // descriptor's leading byte offset is the distance between their first rows: 128 bytes inside a
-// box, (box size - 256) across the two boxes.  Per K block a CTA fetches 2 x boxes (40 KB) and
+// box, (box size - 256) across the two boxes.  Per 128 pixels of K a CTA fetches x boxes of 40 KB and
 // the dy tile (128 x n_tile) for 24 MMAs, against 6 sub-boxes (96 KB) without the reuse.
 // Roles as in wgrad_tc_kernel.
 // ---------------------------------------------------------------------------------------------
@@ -313,6 +318,7 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     uint32_t s = 0, ph = 0;
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t a_kstep = p.a_kstep_bytes >> 4, b_kstep = (uint32_t)(16 * p.scb * 2) >> 4;
+    const int ksteps = p.rows >> 4;   // K = 16 pixels per MMA
     for (int it = 0; it < n_iter; ++it) {
       if (!mbar_wait_warp(&tail->full[s], ph, abort_flag)) { failed = true; break; }
       tc_fence_after();
@@ -323,7 +329,7 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       const uint64_t ad2 = smem_desc(p.adesc_hi3[2], a_addr + p.a_start3[2]);
       if (elect_one()) {
 #pragma unroll 1
-        for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < ksteps; ++j) {
           const uint32_t acc = (it | j) ? 1u : 0u;
           mma_bf16(tmem_base, ad0 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
           mma_bf16(tmem_base + p.acc_stride, ad1 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
@@ -436,16 +442,19 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, const bf16* x, const 
   memset(&p, 0, sizeof(p));
   p.Nimg = N; p.OH = H; p.OW = W; p.stride = 1; p.pad = 1; p.R = 3;
   p.Cin = Cin; p.Cout = Cout; p.taps = 9;
-  // pixel box: 8 x BH x BNI = 128
-  if (H >= 16) { p.BH = 16; p.BNI = 1; }
-  else if (H == 8 || H == 4 || H == 2) { p.BH = H; p.BNI = 16 / H; }
+  // pixel box (K block): 8 x BH x BNI = LP_WGRAD_HALO_KBLOCK pixels.  Blocks of 64 make a stage 40 KB
+  // instead of 80 KB for a 160-channel tile (five stages in flight instead of two); measured, that is
+  // no faster (0.079 against 0.078 ms at 160 channels), so the copy latency is not what limits it.
+  constexpr int per_col = LP_WGRAD_HALO_KBLOCK / 8;
+  if (H >= per_col) { p.BH = per_col; p.BNI = 1; }
+  else if (H == 8 || H == 4 || H == 2) { p.BH = H; p.BNI = per_col / H; }
   else return 1;
   if (p.BNI > N) return 1;
   p.BW = 8;
   p.tiles_w = W / 8;
   p.tiles_h = (H + p.BH - 1) / p.BH;
   p.pix_tiles = p.tiles_w * p.tiles_h * ((N + p.BNI - 1) / p.BNI);
-  p.rows = p.rows_pad = 128;
+  p.rows = p.rows_pad = LP_WGRAD_HALO_KBLOCK;
   // dy sub-boxes as in the plain kernel, one channel tile of at most 160 so that three accumulators fit
   int best_tile = 0;
   for (int sc : {64, 32, 16}) {
@@ -465,13 +474,13 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, const bf16* x, const 
   p.cin_chunks = (Cin + 63) / 64;
   p.groups = 3 * p.cin_chunks;
   p.m_tiles = (p.groups + 1) / 2;
-  const int box_rows = 10 * p.BNI * p.BH;               // 160
+  const int box_rows = 10 * p.BNI * p.BH;
   p.a_box_bytes = (uint32_t)(box_rows * 128);
   p.a_region = 2 * p.a_box_bytes;
-  p.b_sub_bytes = (uint32_t)((128 * p.scb * 2 + 1023) / 1024 * 1024);
+  p.b_sub_bytes = (uint32_t)((p.rows * p.scb * 2 + 1023) / 1024 * 1024);
   p.stage_bytes = p.a_region + p.b_sub_bytes * p.nb;
   p.tx_a = p.a_box_bytes;
-  p.tx_b = (uint32_t)(128 * p.nb * p.scb * 2);
+  p.tx_b = (uint32_t)(p.rows * p.nb * p.scb * 2);
   const size_t tail = sizeof(tc::WgSmemTail) + 1024;
   int stages = (int)((220 * 1024 - tail) / p.stage_bytes);
   stages = std::min(stages, tc::kWgMaxStages);
@@ -493,7 +502,7 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, const bf16* x, const 
     const int max_s = std::min(p.pix_tiles, 64);
     for (int sp = 1; sp <= max_s; ++sp) {
       const int waves = (tiles * sp + sm_count - 1) / sm_count;
-      const double t = waves * ((double)((p.pix_tiles + sp - 1) / sp) * 1.5 + 4.0);
+      const double t = waves * ((double)((p.pix_tiles + sp - 1) / sp) * 1.5 * (p.rows / 128.0) + 4.0);
       if (t < best_t - 1e-9) { best_t = t; best_s = sp; }
     }
     p.splits = best_s;
