@@ -289,7 +289,7 @@ __global__ void loss_finalize_kernel(const double* __restrict__ acc, float rho, 
 //   apply : dx = gamma*rstd*(dy_m - dbeta/M - xhat*dgamma/M) [+ addend]
 // ---------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(256, 2)
 bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_mask,
                                      BnArgs A, float* __restrict__ dgamma, float* __restrict__ dbeta,
                                      long long total_vecs, int C) {
@@ -309,7 +309,7 @@ bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu
     }
   }
   const long long stride = (long long)gridDim.x * blockDim.x;
-  constexpr int U = 2;
+  constexpr int U = 4;
   for (long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i0 < total_vecs; i0 += U * stride) {
     uint4 rd[U], rx[U];
 #pragma unroll
@@ -353,7 +353,7 @@ bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu
 }
 
 template <typename T>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(256, 2)
 bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_mask, BnArgs A,
                     const float* __restrict__ dgamma, const float* __restrict__ dbeta,
                     const T* __restrict__ addend, T* __restrict__ out, long long total_vecs, int C) {
@@ -389,7 +389,7 @@ bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_
     }
   }
   const long long stride = (long long)gridDim.x * blockDim.x;
-  constexpr int U = 2;
+  constexpr int U = 4;
   for (long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i0 < total_vecs; i0 += U * stride) {
     uint4 rd[U], rx[U], ra[U];
 #pragma unroll
