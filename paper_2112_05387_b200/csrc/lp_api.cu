@@ -319,6 +319,9 @@ static const size_t kTcMaxSmem = 220 * 1024;
 
 // Halo mode (one activation box per K chunk serves all nine taps, see conv_tc.cuh): a 3x3 stride-1
 // tap set, 64-channel K chunks and an output width that is a multiple of 8.
+#ifndef LP_CONV_MAX_NB
+#define LP_CONV_MAX_NB 8   // weight stages in flight (halo mode), as far as shared memory allows
+#endif
 static const int kHaloBoxW = 10;   // 8-pixel tile width plus one halo pixel on each side
 
 static bool pick_halo_box(const TcGemmSpec& s, int& BW, int& BH, int& BNI, int tapw3[3][3]) {
@@ -409,7 +412,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
          pair >= 1 && !fits; --pair) {
       const size_t a_bytes = (size_t)p.nA * pair * p.a_halo_bytes;
       if (a_bytes >= avail) continue;
-      const int nb = (int)std::min<size_t>((avail - a_bytes) / b_region, 8);
+      const int nb = (int)std::min<size_t>((avail - a_bytes) / b_region, LP_CONV_MAX_NB);
       if (nb >= 3) { p.mpair = pair; p.nB = nb; fits = true; }
     }
     if (fits) {
