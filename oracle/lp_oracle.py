@@ -194,7 +194,10 @@ class Net:
         self.K = len(cfg["module_block_end"])
         self.eps = float(cfg["bn_eps"])
         self.kind = cfg["block_kind"]
-        assert self.kind in ("postbn", "preact")
+        assert self.kind in ("postbn", "preact", "bottleneck")
+        # the bottleneck block is a post-activation block with three convolutions: stem, head and the
+        # storage of block outputs follow the post-BN form
+        self.post = self.kind in ("postbn", "bottleneck")
         # stem output geometry
         h, w = cfg["H"], cfg["W"]
         if cfg["stem_kind"] == "conv3x3":
@@ -208,7 +211,7 @@ class Net:
         for ch, nb, st in zip(cfg["stage_channels"], cfg["stage_blocks"], cfg["stage_stride"]):
             for b in range(nb):
                 s = st if b == 0 else 1
-                blk = dict(cin=c, cout=ch, stride=s, hin=h, win=w, proj=(s != 1 or c != ch))
+                blk = dict(cin=c, cout=ch, stride=s, hin=h, win=w, proj=(s != 1 or c != ch), mid=ch // 4)
                 h, w = out_size(h, 3, s, 1), out_size(w, 3, s, 1)
                 blk["hout"], blk["wout"] = h, w
                 self.blocks.append(blk)
@@ -252,14 +255,22 @@ class Net:
         if k == 0:
             R = self.stem["R"]
             L.append(("stem.conv.w", "conv_w", (cfg["stem_channels"], R, R, cfg["C_in"])))
-            if self.kind == "postbn":
+            if self.post:
                 L.append(("stem.bn.g", "bn_gamma", (cfg["stem_channels"],)))
                 L.append(("stem.bn.b", "bn_beta", (cfg["stem_channels"],)))
         for bi in self.module_blocks[k]:
             b = self.blocks[bi]
             p = "block%d." % bi
             ci, co = b["cin"], b["cout"]
-            if self.kind == "postbn":
+            if self.kind == "bottleneck":
+                m = b["mid"]
+                L += [(p + "conv1.w", "conv_w", (m, 1, 1, ci)), (p + "bn1.g", "bn_gamma", (m,)), (p + "bn1.b", "bn_beta", (m,)),
+                      (p + "conv2.w", "conv_w", (m, 3, 3, m)), (p + "bn2.g", "bn_gamma", (m,)), (p + "bn2.b", "bn_beta", (m,)),
+                      (p + "conv3.w", "conv_w", (co, 1, 1, m)), (p + "bn3.g", "bn_gamma", (co,)), (p + "bn3.b", "bn_beta", (co,))]
+                if b["proj"]:
+                    L += [(p + "sc.w", "conv_w", (co, 1, 1, ci)), (p + "bns.g", "bn_gamma", (co,)),
+                          (p + "bns.b", "bn_beta", (co,))]
+            elif self.kind == "postbn":
                 L += [(p + "conv1.w", "conv_w", (co, 3, 3, ci)), (p + "bn1.g", "bn_gamma", (co,)),
                       (p + "bn1.b", "bn_beta", (co,)),
                       (p + "conv2.w", "conv_w", (co, 3, 3, co)), (p + "bn2.g", "bn_gamma", (co,)),
@@ -487,7 +498,7 @@ def _stem_fwd(net, p, x, cache):
     st = net.stem
     y = _st(net, conv_fwd(x, _wq(net, p["stem.conv.w"]), st["stride"], st["pad"]))
     cache["stem.x"] = x
-    if net.kind == "postbn":
+    if net.post:
         z, cache["stem.bn"] = bn_fwd(y, p["stem.bn.g"], p["stem.bn.b"], net.eps)
         cache["stem.z"] = z
         y = _st(net, relu(z))
@@ -498,7 +509,7 @@ def _stem_fwd(net, p, x, cache):
 
 def _stem_bwd(net, p, d, cache, g):
     st = net.stem
-    if net.kind == "postbn":
+    if net.post:
         if st["pool"]:
             d = _st(net, maxpool_bwd(d, cache["stem.pool"]))
         d = relu_bwd(d, cache["stem.z"])
@@ -514,6 +525,23 @@ def _block_fwd(net, bi, p, x, cache):
     q = "block%d." % bi
     c = cache.setdefault(bi, {})
     c["x"] = x
+    if net.kind == "bottleneck":
+        # conv1x1 - BN - ReLU - conv3x3 (carries the stride) - BN - ReLU - conv1x1 - BN, plus shortcut
+        y1 = _st(net, conv_fwd(x, _wq(net, p[q + "conv1.w"]), 1, 0))
+        z1, c["bn1"] = bn_fwd(y1, p[q + "bn1.g"], p[q + "bn1.b"], net.eps)
+        a1 = _st(net, relu(z1))
+        y2 = _st(net, conv_fwd(a1, _wq(net, p[q + "conv2.w"]), b["stride"], 1))
+        z2, c["bn2"] = bn_fwd(y2, p[q + "bn2.g"], p[q + "bn2.b"], net.eps)
+        a2 = _st(net, relu(z2))
+        y3 = _st(net, conv_fwd(a2, _wq(net, p[q + "conv3.w"]), 1, 0))
+        z3, c["bn3"] = bn_fwd(y3, p[q + "bn3.g"], p[q + "bn3.b"], net.eps)
+        c["z1"], c["a1"], c["z2"], c["a2"] = z1, a1, z2, a2
+        if b["proj"]:
+            ys = _st(net, conv_fwd(x, _wq(net, p[q + "sc.w"]), b["stride"], 0))
+            sc, c["bns"] = bn_fwd(ys, p[q + "bns.g"], p[q + "bns.b"], net.eps)
+        else:
+            sc = x
+        return sc + z3
     if net.kind == "postbn":
         y1 = _st(net, conv_fwd(x, _wq(net, p[q + "conv1.w"]), b["stride"], 1))
         z1, c["bn1"] = bn_fwd(y1, p[q + "bn1.g"], p[q + "bn1.b"], net.eps)
@@ -545,6 +573,29 @@ def _block_bwd(net, bi, p, d, cache, g):
     q = "block%d." % bi
     c = cache[bi]
     x = c["x"]
+    if net.kind == "bottleneck":
+        dy3, g[q + "bn3.g"], g[q + "bn3.b"] = bn_bwd(d, c["bn3"], p[q + "bn3.g"])
+        dy3 = _st(net, dy3)
+        g[q + "conv3.w"] = conv_wgrad(c["a2"], dy3, p[q + "conv3.w"].shape, 1, 0)
+        da2 = _st(net, conv_dgrad(dy3, _wq(net, p[q + "conv3.w"]), 1, 0, c["a2"].shape))
+        dz2 = relu_bwd(da2, c["z2"])
+        dy2, g[q + "bn2.g"], g[q + "bn2.b"] = bn_bwd(dz2, c["bn2"], p[q + "bn2.g"])
+        dy2 = _st(net, dy2)
+        g[q + "conv2.w"] = conv_wgrad(c["a1"], dy2, p[q + "conv2.w"].shape, b["stride"], 1)
+        da1 = _st(net, conv_dgrad(dy2, _wq(net, p[q + "conv2.w"]), b["stride"], 1, c["a1"].shape))
+        dz1 = relu_bwd(da1, c["z1"])
+        dy1, g[q + "bn1.g"], g[q + "bn1.b"] = bn_bwd(dz1, c["bn1"], p[q + "bn1.g"])
+        dy1 = _st(net, dy1)
+        g[q + "conv1.w"] = conv_wgrad(x, dy1, p[q + "conv1.w"].shape, 1, 0)
+        dx = conv_dgrad(dy1, _wq(net, p[q + "conv1.w"]), 1, 0, x.shape)
+        if b["proj"]:
+            dys, g[q + "bns.g"], g[q + "bns.b"] = bn_bwd(d, c["bns"], p[q + "bns.g"])
+            dys = _st(net, dys)
+            g[q + "sc.w"] = conv_wgrad(x, dys, p[q + "sc.w"].shape, b["stride"], 0)
+            dx = _st(net, dx) + conv_dgrad(dys, _wq(net, p[q + "sc.w"]), b["stride"], 0, x.shape)
+        else:
+            dx = dx + d
+        return _st(net, dx)
     if net.kind == "postbn":
         dy2, g[q + "bn2.g"], g[q + "bn2.b"] = bn_bwd(d, c["bn2"], p[q + "bn2.g"])
         dy2 = _st(net, dy2)
@@ -614,7 +665,7 @@ def module_forward(net, k, p, x_k, cache=None):
         x = _block_fwd(net, bi, p, x, cache)
         # an interior module's final output goes straight into the local loss; every other block
         # output is kept as an activation tensor
-        if not (i == len(net.module_blocks[k]) - 1 and k < net.K - 1 and net.kind == "postbn"):
+        if not (i == len(net.module_blocks[k]) - 1 and k < net.K - 1 and net.post):
             x = _st(net, x)
     if k == net.K - 1:
         x = _head_fwd(net, p, x, cache)
@@ -683,13 +734,20 @@ def forward_serial(net, module_params, images):
     x = np.asarray(images, dtype=F)
     st = net.stem
     x = conv_fwd(x, named["stem.conv.w"], st["stride"], st["pad"])
-    if net.kind == "postbn":
+    if net.post:
         x = relu(bn_fwd(x, named["stem.bn.g"], named["stem.bn.b"], eps)[0])
         if st["pool"]:
             x = maxpool_fwd(x)[0]
     for bi, b in enumerate(net.blocks):
         q = "block%d." % bi
-        if net.kind == "postbn":
+        if net.kind == "bottleneck":
+            t = relu(bn_fwd(conv_fwd(x, named[q + "conv1.w"], 1, 0), named[q + "bn1.g"], named[q + "bn1.b"], eps)[0])
+            t = relu(bn_fwd(conv_fwd(t, named[q + "conv2.w"], b["stride"], 1), named[q + "bn2.g"], named[q + "bn2.b"], eps)[0])
+            t = bn_fwd(conv_fwd(t, named[q + "conv3.w"], 1, 0), named[q + "bn3.g"], named[q + "bn3.b"], eps)[0]
+            s = (bn_fwd(conv_fwd(x, named[q + "sc.w"], b["stride"], 0), named[q + "bns.g"], named[q + "bns.b"], eps)[0]
+                 if b["proj"] else x)
+            x = s + t
+        elif net.kind == "postbn":
             t = conv_fwd(x, named[q + "conv1.w"], b["stride"], 1)
             t = relu(bn_fwd(t, named[q + "bn1.g"], named[q + "bn1.b"], eps)[0])
             t = conv_fwd(t, named[q + "conv2.w"], 1, 1)

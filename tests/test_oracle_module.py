@@ -33,6 +33,10 @@ ALL_CFGS = [
                                      stage_channels=(8, 8), stage_stride=(1, 1))),
     ("preact-3mod", lambda: small_cfg("preact", stage_channels=(8, 16), stage_blocks=(2, 2),
                                       module_block_end=(1, 3, 4), N=3)),
+    # bottleneck blocks (1x1 - 3x3 - 1x1, the block of the paper's ResNet-50 workload): identity and
+    # projection shortcuts, a stride-2 block, a module boundary inside a stage
+    ("bottleneck", lambda: small_cfg("bottleneck", stage_channels=(16, 32), stage_blocks=(2, 2),
+                                     module_block_end=(1, 3, 4), N=3, stem_channels=16)),
 ]
 
 
