@@ -51,7 +51,7 @@ typedef enum lp_status {
 
 enum { LP_F32 = 0, LP_BF16 = 1 };
 enum { LP_STEM_CONV3X3 = 0, LP_STEM_CONV7X7S2_MAXPOOL = 1 };
-enum { LP_POSTBN = 0, LP_PREACT = 1 };
+enum { LP_POSTBN = 0, LP_PREACT = 1, LP_BOTTLENECK = 2 };
 /* `which` argument of the parameter calls: module k is k, AuxNet k is LP_AUX(k). */
 #define LP_AUX(k) (256 + (k))
 /* Recursive auxiliary-variable networks (aux_recursive = 1; Section 4.3, Eq. ReAuxNet-FP): x_k, k = 1..K-1,
@@ -81,6 +81,9 @@ enum { LP_CONV_FWD = 0, LP_CONV_DGRAD = 1, LP_CONV_WGRAD = 2 };
  * (every n-th block, Section 4.1); the stem belongs to module 0 and the head to module K-1.
  *   LP_POSTBN block: conv3x3-BN-ReLU-conv3x3-BN + shortcut (no ReLU after the sum)
  *   LP_PREACT block: BN-ReLU-conv3x3-BN-ReLU-conv3x3 + shortcut
+ *   LP_BOTTLENECK block: conv1x1-BN-ReLU-conv3x3-BN-ReLU-conv1x1-BN + shortcut, inner width C_out/4, the
+ *             block's stride in the 3x3 convolution (the block of the paper's ResNet-50 workload);
+ *             stem, head and shortcut as in LP_POSTBN
  *   shortcut: identity, or a 1x1 convolution with the block's stride where shape changes
  *             (followed by BN in LP_POSTBN; applied to the pre-activated tensor in LP_PREACT)
  *   stem: LP_POSTBN conv-BN-ReLU (7x7/2 variant adds a 3x3/2 max-pool); LP_PREACT conv only

@@ -163,7 +163,7 @@ def desc_from_config(cfg, conv_impl=LP_CONV_IMPL_AUTO, aux_recursive=False):
     d.num_classes = cfg["num_classes"]
     d.stem_kind = 0 if cfg["stem_kind"] == "conv3x3" else 1
     d.stem_channels = cfg["stem_channels"]
-    d.block_kind = 0 if cfg["block_kind"] == "postbn" else 1
+    d.block_kind = {"postbn": 0, "preact": 1, "bottleneck": 2}[cfg["block_kind"]]
     d.post_add_relu = 0
     d.num_stages = len(cfg["stage_channels"])
     for i, (c, b, s) in enumerate(zip(cfg["stage_channels"], cfg["stage_blocks"], cfg["stage_stride"])):

@@ -860,12 +860,15 @@ struct Planner {
   struct BlockRec {
     int bi;
     Tensor x, y1, a1, y2, ys, o;  // saved activations (o: pre-activated input, pre-act blocks)
+    Tensor a2, y3;                // bottleneck blocks: second activation, third convolution output
     int c1, c2, cs, bn1, bn2, bns;
+    int c3 = -1, bn3 = -1;
   };
 
   void build_module(Plan& P, int k) {
     const lp_net_desc& d = net.d;
-    const bool post = d.block_kind == LP_POSTBN;
+    const bool post = d.block_kind != LP_PREACT;
+    const bool bott = d.block_kind == LP_BOTTLENECK;
     const bool last = k == net.K - 1;
     P.interior = !last;
     alloc_params(P, k);
@@ -887,10 +890,22 @@ struct Planner {
       BlockRec r;
       r.bi = bi; r.cs = -1; r.bns = -1;
       const bool need_dx1 = true;  // every block input is either x_k (dx_k exported) or an internal tensor
-      r.c1 = add_conv(P, q + ".conv1.w", b.cin, b.cout, 3, b.stride, 1, b.hin, b.win, need_dx1);
-      r.c2 = add_conv(P, q + ".conv2.w", b.cout, b.cout, 3, 1, 1, b.hout, b.wout, true);
+      if (bott) {
+        r.c1 = add_conv(P, q + ".conv1.w", b.cin, b.mid, 1, 1, 0, b.hin, b.win, need_dx1);
+        r.c2 = add_conv(P, q + ".conv2.w", b.mid, b.mid, 3, b.stride, 1, b.hin, b.win, true);
+        r.c3 = add_conv(P, q + ".conv3.w", b.mid, b.cout, 1, 1, 0, b.hout, b.wout, true);
+      } else {
+        r.c1 = add_conv(P, q + ".conv1.w", b.cin, b.cout, 3, b.stride, 1, b.hin, b.win, need_dx1);
+        r.c2 = add_conv(P, q + ".conv2.w", b.cout, b.cout, 3, 1, 1, b.hout, b.wout, true);
+      }
       if (b.proj) r.cs = add_conv(P, q + ".sc.w", b.cin, b.cout, 1, b.stride, 0, b.hin, b.win, true);
-      if (post) {
+      if (bott) {
+        const long long cnt = (long long)d.N * b.hout * b.wout;
+        r.bn1 = add_bn(P, q + ".bn1", b.mid, (long long)d.N * b.hin * b.win);
+        r.bn2 = add_bn(P, q + ".bn2", b.mid, cnt);
+        r.bn3 = add_bn(P, q + ".bn3", b.cout, cnt);
+        if (b.proj) r.bns = add_bn(P, q + ".bns", b.cout, cnt);
+      } else if (post) {
         const long long cnt = (long long)d.N * b.hout * b.wout;
         r.bn1 = add_bn(P, q + ".bn1", b.cout, cnt);
         r.bn2 = add_bn(P, q + ".bn2", b.cout, cnt);
@@ -957,16 +972,22 @@ struct Planner {
         r.y1 = emit_conv(P, F, cur, r.c1, nullptr, r.bn1);
         r.a1 = emit_bn_apply(F, r.y1, r.bn1, nullptr, -1, nullptr, 1);
         r.y2 = emit_conv(P, F, r.a1, r.c2, nullptr, r.bn2);
+        if (bott) {
+          r.a2 = emit_bn_apply(F, r.y2, r.bn2, nullptr, -1, nullptr, 1);
+          r.y3 = emit_conv(P, F, r.a2, r.c3, nullptr, r.bn3);
+        }
+        const Tensor& ylast = bott ? r.y3 : r.y2;   // the branch's last convolution and its batch norm
+        const int bnlast = bott ? r.bn3 : r.bn2;
         if (b.proj) r.ys = emit_conv(P, F, cur, r.cs, nullptr, r.bns);
         if (final_block && !last) {
           Op op;
-          op.type = OP_OUT_LOSS; op.in = r.y2; op.bn = r.bn2; op.out = P.out;
+          op.type = OP_OUT_LOSS; op.in = ylast; op.bn = bnlast; op.out = P.out;
           if (b.proj) { op.in2 = r.ys; op.bn2 = r.bns; } else { op.addend = cur; }
           F.push_back(op);
           cur = P.out;
         } else {
-          cur = b.proj ? emit_bn_apply(F, r.y2, r.bn2, &r.ys, r.bns, nullptr, 0)
-                       : emit_bn_apply(F, r.y2, r.bn2, nullptr, -1, &cur, 0);
+          cur = b.proj ? emit_bn_apply(F, ylast, bnlast, &r.ys, r.bns, nullptr, 0)
+                       : emit_bn_apply(F, ylast, bnlast, nullptr, -1, &cur, 0);
         }
       } else {
         r.o = emit_bn_apply(F, cur, r.bn1, nullptr, -1, nullptr, 1);
@@ -1026,7 +1047,15 @@ struct Planner {
       const bool first_of_module = i == 0 && k > 0;  // its input is x_k: dx goes to the caller
       const Tensor* dx_target = first_of_module ? &dx_ext : nullptr;
       if (post) {
-        Tensor dy2 = emit_bn_bwd(Bw, dcur, r.y2, nullptr, r.bn2, nullptr);
+        Tensor dy2;
+        if (bott) {
+          Tensor dy3 = emit_bn_bwd(Bw, dcur, r.y3, nullptr, r.bn3, nullptr);
+          emit_wgrad(Bw, r.a2, dy3, r.c3);
+          Tensor da2 = emit_dgrad(P, Bw, dy3, r.c3, nullptr, nullptr);
+          dy2 = emit_bn_bwd(Bw, da2, r.y2, &r.a2, r.bn2, nullptr);
+        } else {
+          dy2 = emit_bn_bwd(Bw, dcur, r.y2, nullptr, r.bn2, nullptr);
+        }
         emit_wgrad(Bw, r.a1, dy2, r.c2);
         Tensor da1 = emit_dgrad(P, Bw, dy2, r.c2, nullptr, nullptr);
         Tensor dy1 = emit_bn_bwd(Bw, da1, r.y1, &r.a1, r.bn1, nullptr);

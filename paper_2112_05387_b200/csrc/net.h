@@ -14,6 +14,7 @@ namespace lp {
 struct BlockDef {
   int cin, cout, stride, hin, win, hout, wout;
   bool proj;
+  int mid;   // inner width of a bottleneck block (C_out / 4)
 };
 struct AuxConvDef {
   int cin, cout, stride, hin, win, hout, wout;
@@ -44,7 +45,7 @@ struct NetDef {
     if (d.dtype != LP_F32 && d.dtype != LP_BF16) return LP_ERR_BAD_DESC;
     if (d.N < 1 || d.H < 1 || d.W < 1 || d.C_in < 1 || d.num_classes < 2) return LP_ERR_BAD_DESC;
     if (d.stem_kind != LP_STEM_CONV3X3 && d.stem_kind != LP_STEM_CONV7X7S2_MAXPOOL) return LP_ERR_BAD_DESC;
-    if (d.block_kind != LP_POSTBN && d.block_kind != LP_PREACT) return LP_ERR_BAD_DESC;
+    if (d.block_kind != LP_POSTBN && d.block_kind != LP_PREACT && d.block_kind != LP_BOTTLENECK) return LP_ERR_BAD_DESC;
     if (d.post_add_relu != 0) return LP_ERR_UNSUPPORTED;
     if (d.num_stages < 1 || d.num_stages > LP_MAX_STAGES) return LP_ERR_BAD_DESC;
     if (d.K < 1 || d.K > LP_MAX_MODULES) return LP_ERR_BAD_DESC;
@@ -77,6 +78,8 @@ struct NetDef {
         bd.cin = c; bd.cout = ch; bd.stride = b == 0 ? st : 1;
         bd.hin = h; bd.win = w;
         bd.proj = bd.stride != 1 || c != ch;
+        bd.mid = ch / 4;
+        if (d.block_kind == LP_BOTTLENECK && (ch % 4 || bd.mid < vec || bd.mid % vec)) return LP_ERR_BAD_DESC;
         h = conv_out(h, 3, bd.stride, 1); w = conv_out(w, 3, bd.stride, 1);
         if (h < 1 || w < 1) return LP_ERR_BAD_DESC;
         bd.hout = h; bd.wout = w;
@@ -169,7 +172,8 @@ struct NetDef {
     }
     const int k = which;
     if (k < 0 || k >= K) return LP_ERR_BAD_INDEX;
-    const bool post = d.block_kind == LP_POSTBN;
+    const bool post = d.block_kind != LP_PREACT;
+    const bool bott = d.block_kind == LP_BOTTLENECK;
     if (k == 0) {
       push(L, off, "stem.conv.w", LP_KIND_CONV_W, d.stem_channels, stem_R, stem_R, d.C_in);
       if (post) {
@@ -180,7 +184,22 @@ struct NetDef {
     for (int bi = mod_begin[k]; bi < mod_end[k]; ++bi) {
       const BlockDef& b = blocks[bi];
       const std::string p = "block" + std::to_string(bi) + ".";
-      if (post) {
+      if (bott) {
+        push(L, off, p + "conv1.w", LP_KIND_CONV_W, b.mid, 1, 1, b.cin);
+        push(L, off, p + "bn1.g", LP_KIND_BN_GAMMA, b.mid);
+        push(L, off, p + "bn1.b", LP_KIND_BN_BETA, b.mid);
+        push(L, off, p + "conv2.w", LP_KIND_CONV_W, b.mid, 3, 3, b.mid);
+        push(L, off, p + "bn2.g", LP_KIND_BN_GAMMA, b.mid);
+        push(L, off, p + "bn2.b", LP_KIND_BN_BETA, b.mid);
+        push(L, off, p + "conv3.w", LP_KIND_CONV_W, b.cout, 1, 1, b.mid);
+        push(L, off, p + "bn3.g", LP_KIND_BN_GAMMA, b.cout);
+        push(L, off, p + "bn3.b", LP_KIND_BN_BETA, b.cout);
+        if (b.proj) {
+          push(L, off, p + "sc.w", LP_KIND_CONV_W, b.cout, 1, 1, b.cin);
+          push(L, off, p + "bns.g", LP_KIND_BN_GAMMA, b.cout);
+          push(L, off, p + "bns.b", LP_KIND_BN_BETA, b.cout);
+        }
+      } else if (post) {
         push(L, off, p + "conv1.w", LP_KIND_CONV_W, b.cout, 3, 3, b.cin);
         push(L, off, p + "bn1.g", LP_KIND_BN_GAMMA, b.cout);
         push(L, off, p + "bn1.b", LP_KIND_BN_BETA, b.cout);

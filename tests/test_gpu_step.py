@@ -171,6 +171,23 @@ def test_wrn28_10_loss_in_the_last_convolutions_epilogue():
     full_step_parity(cfg, conv_impl=lp.LP_CONV_LOSS_IN_EPILOGUE, steps=1)
 
 
+def test_bottleneck_blocks_fp32():
+    """1x1 - 3x3 - 1x1 blocks: identity and projection shortcuts, a stride-2 block, a module boundary inside a stage."""
+    cfg = small_cfg("bottleneck", N=4, H=8, W=8, stage_channels=(16, 32), stage_blocks=(2, 2), module_block_end=(1, 3, 4),
+                    stem_channels=16)
+    full_step_parity(cfg, steps=2)
+
+
+def test_bottleneck_blocks_bf16_tensor_cores():
+    cfg = small_cfg("bottleneck", N=8, H=16, W=16, dtype="bf16", stage_channels=(64, 128), stage_blocks=(2, 2),
+                    module_block_end=(1, 3, 4), stem_channels=16, classes=10)
+    full_step_parity(cfg, steps=1)
+
+
+def test_resnet50_reduced_bf16():
+    full_step_parity(scaled("resnet50", N=2, H=64, W=64), steps=1)
+
+
 def test_resnet34_reduced_bf16():
     full_step_parity(scaled("resnet34", N=2, H=64, W=64), steps=1)
 

@@ -61,6 +61,12 @@ def test_parameter_counts_of_named_networks():
     net = O.Net(cfg)
     total = sum(net.param_count(k) for k in range(net.K))
     assert 1.6e6 < total < 1.8e6
+    # ResNet-50 (bottleneck blocks, projection shortcuts with BN, 1000 classes): the textbook 25,557,032
+    cfg = get_config("resnet50")
+    net = O.Net(cfg)
+    assert sum(net.param_count(k) for k in range(net.K)) == 25557032
+    desc = lp.desc_from_config(cfg)
+    assert sum(int(np.prod(s)) for k in range(net.K) for _, _, s in lp.lp_param_layout(desc, k)) == 25557032
 
 
 def test_bad_descriptors_are_rejected():

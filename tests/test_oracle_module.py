@@ -401,3 +401,25 @@ def test_reauxnet_distill_step_closed_form():
         for j in range(k):
             np.testing.assert_allclose(g2[k - 1][j], 2 * g1[k - 1][j], rtol=1e-8, atol=1e-12)
             np.testing.assert_allclose(new1[k - 1][j], stacks[k - 1][j] - 0.01 * g1[k - 1][j], rtol=1e-12, atol=1e-15)
+
+
+def test_bottleneck_shift_before_1x1_convolutions_and_batch_norms_has_no_gradient():
+    """A per-channel shift of a tensor that only feeds 1x1 convolutions followed by batch norms is
+    removed by their mean subtraction: the local loss does not depend on bn3.beta of a bottleneck block
+    whose successor has a projection shortcut (3x3 convolutions do see it, through their zero padding)."""
+    cfg = ALL_CFGS[5][1]()
+    net, mods, auxs = build(cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    xs = [x0] + O.auxnet_forward(net, auxs, x0)
+    k = 1                                         # blocks 1 (identity shortcut) and 2 (projection, stride 2)
+    assert net.module_blocks[k] == [1, 2] and net.blocks[2]["proj"]
+    res = O.module_fwd_bwd(net, k, mods[k], xs[k], xs[k + 1], None, 0.7)
+    g = net.unpack(k, res["grads"])
+    scale = np.linalg.norm(res["grads"])
+    assert np.linalg.norm(g["block1.bn3.b"]) < 1e-10 * scale
+    assert np.linalg.norm(g["block1.bn3.g"]) > 1e-4 * scale      # the scale does matter
+    # and the loss itself does not move when that shift changes
+    p = net.unpack(k, mods[k].astype(np.float64).copy())
+    p["block1.bn3.b"] = p["block1.bn3.b"] + 0.37
+    res2 = O.module_fwd_bwd(net, k, net.pack(k, p), xs[k], xs[k + 1], None, 0.7)
+    assert abs(res2["loss"] - res["loss"]) < 1e-9 * abs(res["loss"])

@@ -12,7 +12,7 @@ N,H,W,C_in       input batch (NHWC)
 num_classes
 stem_kind        "conv3x3" | "conv7x7s2_maxpool"
 stem_channels
-block_kind       "postbn" (conv-BN-ReLU-conv-BN + shortcut)
+block_kind       "postbn" (conv-BN-ReLU-conv-BN + shortcut), "bottleneck" (1x1-3x3-1x1, inner width C_out/4)
                  | "preact" (BN-ReLU-conv-BN-ReLU-conv + shortcut)
 stage_channels / stage_blocks / stage_stride
 module_block_end cumulative block index that ends each of the K modules
@@ -61,6 +61,15 @@ CONFIGS = {
         stage_stride=[1, 2, 2, 2], module_block_end=[3, 7, 13, 16],
         aux_convs=2, aux_width_div=4,
         loss="al", rho=1.0, kappa_std=0.0, augment=False, **_COMMON),
+    # beyond the five named configurations: ImageNet-shaped ResNet-50 (bottleneck blocks), the network of
+    # the paper's ImageNet experiment; K=4 at the stage boundaries, penalty loss.
+    "resnet50": dict(
+        dtype="bf16", N=32, H=224, W=224, C_in=3, num_classes=1000,
+        stem_kind="conv7x7s2_maxpool", stem_channels=64, block_kind="bottleneck",
+        stage_channels=[256, 512, 1024, 2048], stage_blocks=[3, 4, 6, 3],
+        stage_stride=[1, 2, 2, 2], module_block_end=[3, 7, 13, 16],
+        aux_convs=2, aux_width_div=4,
+        loss="penalty", rho=1.0, kappa_std=0.0, augment=False, **_COMMON),
 }
 
 
