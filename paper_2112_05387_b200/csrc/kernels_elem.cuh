@@ -520,23 +520,40 @@ __global__ void avgpool_kernel(const T* __restrict__ x, float* __restrict__ pool
   }
 }
 
-// one block per sample; logits, softmax, loss (atomic mean), dlogits = (softmax - onehot)/N
-__global__ void head_fwd_kernel(const float* __restrict__ pooled, const float* __restrict__ Wt,
-                                const float* __restrict__ bias, const int32_t* __restrict__ labels,
-                                float* __restrict__ logits, float* __restrict__ dlogits, double* __restrict__ loss_acc,
-                                int N, int C, int classes) {
+// logits[n][j] = bias[j] + sum_c W[j][c] * pooled[n][c].  One warp per class and tile of 8 samples: the
+// weight row is read once (coalesced) for the eight dot products.
+__global__ void __launch_bounds__(128)
+head_logits_kernel(const float* __restrict__ pooled, const float* __restrict__ Wt, const float* __restrict__ bias,
+                   float* __restrict__ logits, int N, int C, int classes) {
+  const int lane = threadIdx.x & 31;
+  const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int n0 = blockIdx.y * 8;
+  if (j >= classes) return;
+  float acc[8];
+#pragma unroll
+  for (int s = 0; s < 8; ++s) acc[s] = 0.f;
+  const float* w = Wt + (long long)j * C;
+  for (int c = lane; c < C; c += 32) {
+    const float wv = w[c];
+#pragma unroll
+    for (int s = 0; s < 8; ++s)
+      if (n0 + s < N) acc[s] += wv * pooled[(long long)(n0 + s) * C + c];
+  }
+#pragma unroll
+  for (int s = 0; s < 8; ++s) {
+    const float v = warp_sum(acc[s]);
+    if (lane == 0 && n0 + s < N) logits[(long long)(n0 + s) * classes + j] = v + bias[j];
+  }
+}
+
+// one block per sample; softmax of the logits, loss (atomic mean), dlogits = (softmax - onehot)/N
+__global__ void head_fwd_kernel(const int32_t* __restrict__ labels, const float* __restrict__ logits,
+                                float* __restrict__ dlogits, double* __restrict__ loss_acc, int N, int classes) {
   extern __shared__ float sh[];  // [classes] logits, then reduction scratch [32]
   float* lg = sh;
   float* red = sh + classes;
   const int n = blockIdx.x;
-  const float* pv = pooled + (long long)n * C;
-  for (int j = threadIdx.x; j < classes; j += blockDim.x) {
-    float acc = bias[j];
-    const float* w = Wt + (long long)j * C;
-    for (int c = 0; c < C; ++c) acc += w[c] * pv[c];
-    lg[j] = acc;
-    logits[(long long)n * classes + j] = acc;
-  }
+  for (int j = threadIdx.x; j < classes; j += blockDim.x) lg[j] = logits[(long long)n * classes + j];
   __syncthreads();
   float mx = -INFINITY;
   for (int j = threadIdx.x; j < classes; j += blockDim.x) mx = fmaxf(mx, lg[j]);
@@ -590,15 +607,23 @@ template <typename T>
 __global__ void head_bwd_x_kernel(const float* __restrict__ dlogits, const float* __restrict__ Wt, T* __restrict__ d,
                                   int HW, int C, int classes) {
   const int n = blockIdx.x;
-  for (int c = threadIdx.x; c < C; c += blockDim.x) {
-    float acc = 0.f;
-    for (int j = 0; j < classes; ++j) acc += dlogits[(long long)n * classes + j] * Wt[(long long)j * C + c];
-    acc /= (float)HW;
-    T v;
-    from_f(v, acc);
-    T* p = d + (long long)n * HW * C + c;
-    for (int i = 0; i < HW; ++i) p[(long long)i * C] = v;
+  const int c = blockIdx.y * blockDim.x + threadIdx.x;   // grid.y covers the channels
+  if (c >= C) return;
+  const float* dl = dlogits + (long long)n * classes;
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+  int j = 0;
+  for (; j + 4 <= classes; j += 4) {
+    a0 += dl[j] * Wt[(long long)j * C + c];
+    a1 += dl[j + 1] * Wt[(long long)(j + 1) * C + c];
+    a2 += dl[j + 2] * Wt[(long long)(j + 2) * C + c];
+    a3 += dl[j + 3] * Wt[(long long)(j + 3) * C + c];
   }
+  for (; j < classes; ++j) a0 += dl[j] * Wt[(long long)j * C + c];
+  const float acc = ((a0 + a1) + (a2 + a3)) / (float)HW;
+  T v;
+  from_f(v, acc);
+  T* p = d + (long long)n * HW * C + c;
+  for (int i = 0; i < HW; ++i) p[(long long)i * C] = v;
 }
 
 // ---------------------------------------------------------------------------------------

@@ -1321,9 +1321,11 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       avgpool_kernel<T><<<hd.N, 256, 0, st>>>((const T*)resolve(op.in, c), hd.pooled, hd.HW, hd.C);
       h->launches++;
       const int32_t* labels = c.labels ? c.labels : h->zero_labels;  // logits-only runs use label 0
-      head_fwd_kernel<<<hd.N, 128, (size_t)(hd.classes + 32) * 4, st>>>(hd.pooled, hd.W, hd.b, labels, hd.logits,
-                                                                        hd.dlogits, P.loss_acc, hd.N, hd.C, hd.classes);
-      h->launches++;
+      head_logits_kernel<<<dim3((hd.classes + 3) / 4, (hd.N + 7) / 8), 128, 0, st>>>(hd.pooled, hd.W, hd.b, hd.logits, hd.N,
+                                                                                     hd.C, hd.classes);
+      head_fwd_kernel<<<hd.N, 128, (size_t)(hd.classes + 32) * 4, st>>>(labels, hd.logits, hd.dlogits, P.loss_acc, hd.N,
+                                                                        hd.classes);
+      h->launches += 2;
       if (c.loss_out) {
         ce_finalize_kernel<<<1, 1, 0, st>>>(P.loss_acc, c.loss_out);
         h->launches++;
@@ -1335,7 +1337,8 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       const long long total = (long long)hd.classes * hd.C;
       head_bwd_w_kernel<<<grid_for(total, 128, g_dev.sm_count, 16), 128, 0, st>>>(hd.dlogits, hd.pooled, hd.dW, hd.db,
                                                                                   hd.N, hd.C, hd.classes);
-      head_bwd_x_kernel<T><<<hd.N, 256, 0, st>>>(hd.dlogits, hd.W, (T*)resolve(op.out, c), hd.HW, hd.C, hd.classes);
+      head_bwd_x_kernel<T><<<dim3(hd.N, (hd.C + 255) / 256), 256, 0, st>>>(hd.dlogits, hd.W, (T*)resolve(op.out, c), hd.HW,
+                                                                           hd.C, hd.classes);
       h->launches += 2;
       break;
     }
