@@ -188,6 +188,59 @@ def test_resnet50_reduced_bf16():
     full_step_parity(scaled("resnet50", N=2, H=64, W=64), steps=1)
 
 
+@pytest.mark.parametrize("kind", ["postbn", "preact", "bottleneck"])
+def test_degenerate_split_one_module_is_ordinary_backpropagation(kind):
+    """K = 1: no auxiliary variable, no AuxNet, no interior loss; the step is plain BP of the cross-entropy."""
+    ch = (16, 32) if kind == "bottleneck" else (8, 16)
+    cfg = small_cfg(kind, N=4, H=8, W=8, stage_channels=ch, stage_blocks=(1, 1), module_block_end=(2,),
+                    stem_channels=ch[0])
+    run = full_step_parity(cfg, steps=2)
+    assert run.net.K == 1 and run.lp.lp_workspace_bytes(run.desc) > 0
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_batch_of_two_images(dtype):
+    """N = 2, the smallest batch whose last-module gradients do not vanish identically (with one image the
+    adjoint of the pooled head is constant over the pixels and the last batch norms remove it: an oracle
+    pin); tiles are mostly ragged."""
+    kw = dict(stem_channels=16, stage_channels=(16, 32), classes=10) if dtype == "bf16" else {}
+    cfg = small_cfg("postbn", N=2, H=16, W=16, dtype=dtype, stage_blocks=(1, 1), module_block_end=(1, 2), **kw)
+    full_step_parity(cfg, steps=1)
+
+
+def test_batch_of_one_image_runs_and_matches_in_the_forward_quantities():
+    cfg = small_cfg("postbn", N=1, H=16, W=16, stage_blocks=(1, 1), module_block_end=(1, 2))
+    run = GpuRun(cfg)
+    post = (lambda a: gen.storage_round(a, cfg["dtype"]))
+    ox = O.auxnet_forward(run.net, run.auxs, run.images, post=post)
+    gx = run.auxnet()
+    assert rel_err(gx[0], ox[0]) < 1e-4
+    run.set_boundaries(ox)
+    grads = run.fwd_bwd_all()
+    ref = oracle_modules(run, [to_host(t) for t in run.d_x[1:]])
+    loss = run.d_loss.cpu().numpy()
+    for k in range(2):
+        assert abs(loss[k, 0] - ref[k]["loss"]) < 1e-4 * abs(ref[k]["loss"])
+    errs = per_tensor_errors(run.net, 0, grads[0], ref[0]["grads"])      # the interior module is not degenerate
+    assert max(errs.values()) < 1e-4, errs
+    # last module: only the head and the shifts of the last batch norms receive a gradient
+    g = run.net.unpack(1, grads[1])
+    r = run.net.unpack(1, ref[1]["grads"])
+    for name in ("head.fc.w", "head.fc.b", "block1.bn2.b", "block1.bns.b"):
+        assert rel_err(g[name], r[name]) < 1e-4, name
+    scale = np.linalg.norm(ref[1]["grads"])
+    for name in ("block1.conv1.w", "block1.conv2.w", "block1.sc.w", "block1.bn2.g"):
+        assert np.linalg.norm(r[name]) < 1e-9 * scale and np.linalg.norm(g[name]) < 1e-5 * scale, name
+
+
+def test_every_block_its_own_module():
+    """The finest split: K = number of blocks (module boundaries at a stride-2 block's entry included)."""
+    cfg = small_cfg("preact", N=4, H=16, W=16, stage_channels=(8, 16, 32), stage_blocks=(2, 2, 2), stage_stride=(1, 2, 2),
+                    module_block_end=(1, 2, 3, 4, 5, 6))
+    run = full_step_parity(cfg, steps=1)
+    assert run.net.K == 6
+
+
 def test_resnet34_reduced_bf16():
     full_step_parity(scaled("resnet34", N=2, H=64, W=64), steps=1)
 

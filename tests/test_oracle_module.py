@@ -423,3 +423,21 @@ def test_bottleneck_shift_before_1x1_convolutions_and_batch_norms_has_no_gradien
     p["block1.bn3.b"] = p["block1.bn3.b"] + 0.37
     res2 = O.module_fwd_bwd(net, k, net.pack(k, p), xs[k], xs[k + 1], None, 0.7)
     assert abs(res2["loss"] - res["loss"]) < 1e-9 * abs(res["loss"])
+
+
+def test_one_image_cross_entropy_gradient_stops_at_the_last_batch_norms():
+    """N = 1: the adjoint of global average pooling is constant over the pixels of the only image, and the
+    backward pass of a batch norm removes a per-channel constant (its statistics run over those same
+    pixels).  In a post-BN block everything upstream of the last batch norms then has zero gradient."""
+    cfg = small_cfg("postbn", N=1, H=16, W=16, stage_blocks=(1, 1), module_block_end=(1, 2))
+    net, mods, auxs = build(cfg)
+    x0 = gen.make_images(cfg).astype(np.float64)
+    xs = [x0] + O.auxnet_forward(net, auxs, x0)
+    res = O.module_fwd_bwd(net, 1, mods[1], xs[1], gen.make_labels(cfg), None, 1.0)
+    g = net.unpack(1, res["grads"])
+    scale = np.linalg.norm(res["grads"])
+    for name in ("block1.conv1.w", "block1.conv2.w", "block1.sc.w", "block1.bn1.g", "block1.bn2.g", "block1.bns.g"):
+        assert np.linalg.norm(g[name]) < 1e-10 * scale, name
+    assert np.linalg.norm(res["dx"]) < 1e-10 * scale
+    for name in ("head.fc.w", "block1.bn2.b", "block1.bns.b"):
+        assert np.linalg.norm(g[name]) > 1e-3 * scale, name
