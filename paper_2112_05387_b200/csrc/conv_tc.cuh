@@ -93,6 +93,7 @@ struct ConvTcParams {
   bf16* seed_out;
   float rho;
   double* loss_acc;              // [2]: sum r^2, sum kappa*r (atomically added)
+  int wide32;                    // output (and residual) rows can be accessed in 32-byte pieces
 };
 
 struct TcSmemTail {
@@ -109,6 +110,19 @@ struct TcSmemTail {
   float ssq[LP_EPI_WARPS][256];
   uint32_t tr[LP_EPI_WARPS][16 * 33];   // per epilogue warp: transposition scratch of the statistics
 };
+
+// 32-byte global accesses (sm_100: 256-bit vector loads and stores); the address must be 32-byte aligned.
+__device__ __forceinline__ void st_global_32B(void* p, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+               "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+__device__ __forceinline__ void ld_global_32B(const void* p, uint4& lo, uint4& hi) {
+  asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w), "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w)
+               : "l"(p)
+               : "memory");
+}
 
 constexpr int kEpiThreads = 32 * LP_EPI_WARPS;
 constexpr int kConvThreads = 96 + kEpiThreads;
@@ -405,6 +419,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         auto load_addend = [&](int g, uint4 (&a)[4]) {
           const int c_in_tile = g * 32;
           const int nv = c_in_tile + 32 <= p.n_tile_cols ? 4 : 2;
+          if (p.wide32) {
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              if (g < ngroups && 2 * u < nv && valid && col0 + c_in_tile + 16 * u < p.Cout) {
+                ld_global_32B(p.addend + obase + col0 + c_in_tile + 16 * u, a[2 * u], a[2 * u + 1]);
+              } else {
+                a[2 * u] = a[2 * u + 1] = make_uint4(0u, 0u, 0u, 0u);
+              }
+            }
+            return;
+          }
 #pragma unroll
           for (int u = 0; u < 4; ++u)
             a[u] = (g < ngroups && u < nv && valid && col0 + c_in_tile + 8 * u < p.Cout)
@@ -456,11 +481,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t pk[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
+            if (p.wide32) {
+              // whole 32-byte sectors per lane: half as many store instructions, no partial sectors
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-              if (u < nv && valid && col + 8 * u < p.Cout)
-                *reinterpret_cast<uint4*>(p.out + obase + col + 8 * u) =
-                    make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+              for (int u = 0; u < 2; ++u)
+                if (2 * u < nv && valid && col + 16 * u < p.Cout) st_global_32B(p.out + obase + col + 16 * u, &pk[8 * u]);
+            } else {
+#pragma unroll
+              for (int u = 0; u < 4; ++u)
+                if (u < nv && valid && col + 8 * u < p.Cout)
+                  *reinterpret_cast<uint4*>(p.out + obase + col + 8 * u) =
+                      make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+            }
             if constexpr (kLoss) {
               // The module output is what was just stored (bf16); the residual against the
               // auxiliary variable, the loss sums and the terminal adjoint follow from it.

@@ -448,6 +448,11 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   p.out = s.out; p.addend = s.addend; p.stats = s.stats; p.err = dev_err;
   p.x_next = s.x_next; p.kappa = s.kappa; p.r_out = s.r_out; p.seed_out = s.seed_out; p.rho = s.rho;
   p.loss_acc = s.loss_acc;
+  // 32-byte epilogue accesses: rows and channel-group offsets are multiples of 32 bytes when the channel
+  // count is a multiple of 16 and the tensors start on a 32-byte boundary (caller buffers need only 16)
+  p.wide32 = (s.out_C % 16 == 0 && s.w_rows % 16 == 0 && p.n_tile_cols % 16 == 0 &&
+              (reinterpret_cast<uintptr_t>(s.out) & 31) == 0 &&
+              (!s.addend || (reinterpret_cast<uintptr_t>(s.addend) & 31) == 0)) ? 1 : 0;
   CUtensorMap tmA, tmB;
   int rc = p.halo ? encode_act_map_halo(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, p.KC, kHaloBoxW, p.BH, p.BNI, row_bytes)
                   : encode_act_map(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, p.KC, p.BW, p.BH, p.BNI, s.in_step, row_bytes);
