@@ -56,6 +56,8 @@ struct WgradParams {
   uint32_t a_start3[3];          // first row of the three accumulators' A operands (bytes into the A region)
   uint64_t adesc_hi3[3];         // their descriptors (the leading byte offset differs)
   uint32_t a_kstep_bytes;        // 16 pixels further along K
+  int epi_bufs;                  // 0: fp32 atomics; else number of 64-row staging buffers of the bulk-reduction epilogue
+  uint32_t epi_buf_bytes;
 };
 
 struct WgSmemTail {
@@ -253,7 +255,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(224, 1)
 wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmDY,
-                  const __grid_constant__ WgradParams p) {
+                  const __grid_constant__ CUtensorMap tmDW, const __grid_constant__ WgradParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   WgSmemTail* tail = reinterpret_cast<WgSmemTail*>(smem + (size_t)p.stages * p.stage_bytes);
@@ -350,7 +352,46 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     const int et = threadIdx.x - 64;
     if (et == 0) tail->epi_ok = (n_iter > 0 && mbar_wait(&tail->acc_full, 0, abort_flag)) ? 1 : 0;
     asm volatile("bar.sync 1, 128;" ::: "memory");
-    if (*(volatile int*)&tail->epi_ok) {
+    if (*(volatile int*)&tail->epi_ok && p.epi_bufs >= 2) {
+      // Bulk-reduction epilogue.  The operand ring is free now (every MMA has completed); each
+      // accumulator is transposed into two [channel-out][64 channel-in] fp32 tiles there, and one
+      // thread adds each tile to dw with a TMA reduction (whole 256-byte rows, asynchronous), in
+      // place of 61 440 scalar atomics per CTA.  Tiles of a later accumulator reuse a buffer once the
+      // reduction that read it has finished reading.
+      tc_fence_after();
+      const int hh = q >> 1;                       // which 64-row chunk of the accumulator this warp holds
+      const int ci_l = (q & 1) * 32 + lane;        // input channel within the chunk
+      const int rounds_in_flight = p.epi_bufs >> 1;
+      const int co0 = n_tile * p.n_tile;
+      for (int a = 0; a < 3; ++a) {
+        if (a >= rounds_in_flight) {
+          if (et == 0) bulk_wait_read(rounds_in_flight - 1);
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        const int slot = (a % rounds_in_flight) * 2;
+        float* buf = reinterpret_cast<float*>(smem + (size_t)(slot + hh) * p.epi_buf_bytes);
+        const uint32_t taddr = tmem_base + a * p.acc_stride + ((uint32_t)(q * 32) << 16);
+        for (int cc = 0; cc < (p.n_tile >> 4); ++cc) {
+          float v[16];
+          tmem_ld16(taddr + cc * 16, v);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) buf[(cc * 16 + j) * 64 + ci_l] = v[j];
+        }
+        fence_proxy_async();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et == 0) {
+          for (int h2 = 0; h2 < 2; ++h2) {
+            const int chunk = 2 * a + h2;
+            const int g = g0 + chunk / 3, sx = chunk % 3;
+            if (g < p.groups)
+              tma_reduce_add_3d(&tmDW, smem + (size_t)(slot + h2) * p.epi_buf_bytes, (g / 3) * 64, (g % 3) * 3 + sx, co0);
+          }
+          bulk_commit_group();
+        }
+      }
+      if (et == 0) bulk_wait_read(0);
+      tc_fence_before();
+    } else if (*(volatile int*)&tail->epi_ok) {
       tc_fence_after();
       for (int a = 0; a < 3; ++a) {
         const int chunk = 2 * a + (row >> 6);          // 0..5: group chunk/3, kernel column chunk%3
@@ -511,6 +552,23 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, const bf16* x, const 
   CUtensorMap tmX, tmDY;
   if (wg_encode_wnh(enc, &tmX, x, N, H, W, Cin, 64, 10, p.BNI, p.BH)) return -8;
   if (wg_encode_wnh(enc, &tmDY, dy, N, H, W, Cout, p.scb, 8, p.BNI, p.BH)) return -8;
+  // dw as a (C_in, tap, C_out) fp32 tensor for the bulk-reduction epilogue: boxes of 64 input channels
+  // of one tap and the CTA's output channels; staged in the operand ring after the main loop
+  CUtensorMap tmDW;
+  memset(&tmDW, 0, sizeof(tmDW));
+  p.epi_buf_bytes = (uint32_t)(p.n_tile * 64 * 4);
+  p.epi_bufs = 0;
+  {
+    cuuint64_t dims[3] = {(cuuint64_t)Cin, 9, (cuuint64_t)Cout};
+    cuuint64_t strides[2] = {(cuuint64_t)Cin * 4, (cuuint64_t)Cin * 9 * 4};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)p.n_tile};
+    cuuint32_t es[3] = {1, 1, 1};
+    const int fit = (int)std::min<size_t>(6, ((size_t)stages * p.stage_bytes) / p.epi_buf_bytes);
+    if (fit >= 2 && (reinterpret_cast<uintptr_t>(dw) & 15) == 0 && Cin % 4 == 0 &&
+        enc(&tmDW, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dw, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+      p.epi_bufs = fit & ~1;
+  }
   size_t smem = std::max((size_t)stages * p.stage_bytes + tail, (size_t)120 * 1024);
   static bool attr_set = false;
   if (!attr_set) {
@@ -519,7 +577,7 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, const bf16* x, const 
     attr_set = true;
   }
   dim3 grid(tiles, p.splits);
-  tc::wgrad_halo_kernel<<<grid, 224, smem, st>>>(tmX, tmDY, p);
+  tc::wgrad_halo_kernel<<<grid, 224, smem, st>>>(tmX, tmDY, tmDW, p);
   return cudaGetLastError() == cudaSuccess ? 0 : -8;
 }
 
