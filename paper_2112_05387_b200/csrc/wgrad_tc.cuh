@@ -71,7 +71,7 @@ struct WgSmemTail {
 
 __global__ void __launch_bounds__(224, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmDY,
-                const __grid_constant__ WgradParams p) {
+                const __grid_constant__ CUtensorMap tmDW, const __grid_constant__ WgradParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   WgSmemTail* tail = reinterpret_cast<WgSmemTail*>(smem + (size_t)p.stages * p.stage_bytes);
@@ -190,7 +190,40 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     const int et = threadIdx.x - 64;
     if (et == 0) tail->epi_ok = (n_iter > 0 && mbar_wait(&tail->acc_full, 0, abort_flag)) ? 1 : 0;
     asm volatile("bar.sync 1, 128;" ::: "memory");
-    if (*(volatile int*)&tail->epi_ok) {
+    if (*(volatile int*)&tail->epi_ok && p.epi_bufs) {
+      // Bulk-reduction epilogue (see wgrad_halo_kernel): an accumulator is transposed into its rpt
+      // [channel-out][sca channel-in] fp32 tiles in the free operand ring, each added to dw by a TMA
+      // reduction; the second accumulator of a pair reuses the buffers once they have been read.
+      tc_fence_after();
+      const int sub = row / p.sca, ci_l = row % p.sca;
+      const int co0 = n_tile * p.n_tile;
+      for (int a = 0; a < cnt; ++a) {
+        if (a > 0) {
+          if (et == 0) bulk_wait_read(0);
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        float* buf = reinterpret_cast<float*>(smem + (size_t)sub * p.epi_buf_bytes);
+        const uint32_t taddr = tmem_base + a * 256 + ((uint32_t)(q * 32) << 16);
+        for (int cc = 0; cc < (p.n_tile >> 4); ++cc) {
+          float v[16];
+          tmem_ld16(taddr + cc * 16, v);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) buf[(cc * 16 + j) * p.sca + ci_l] = v[j];
+        }
+        fence_proxy_async();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et == 0) {
+          for (int sb = 0; sb < p.rpt; ++sb) {
+            const int g = (m_tile + a) * p.rpt + sb;
+            if (g < p.total_chunks)
+              tma_reduce_add_3d(&tmDW, smem + (size_t)sb * p.epi_buf_bytes, (g % p.cin_chunks) * p.sca, g / p.cin_chunks, co0);
+          }
+          bulk_commit_group();
+        }
+      }
+      if (et == 0) bulk_wait_read(0);
+      tc_fence_before();
+    } else if (*(volatile int*)&tail->epi_ok) {
       tc_fence_after();
       for (int a = 0; a < cnt; ++a) {
         const int g = (m_tile + a) * p.rpt + row / p.sca;
@@ -670,6 +703,23 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf
   CUtensorMap tmX, tmDY;
   if (wg_encode(enc, &tmX, x, N, H, W, Cin, p.sca, p.BW, p.BH, p.BNI, stride)) return -8;
   if (wg_encode(enc, &tmDY, dy, N, OH, OW, Cout, p.scb, p.BW, p.BH, p.BNI, 1)) return -8;
+  // dw as a (C_in, tap, C_out) fp32 tensor for the bulk-reduction epilogue (boxes of one sub-box of
+  // input channels, one tap, the CTA's output channels), where the operand ring can hold an accumulator
+  CUtensorMap tmDW;
+  memset(&tmDW, 0, sizeof(tmDW));
+  p.epi_buf_bytes = (uint32_t)(p.n_tile * p.sca * 4);
+  p.epi_bufs = 0;
+  {
+    cuuint64_t dims[3] = {(cuuint64_t)Cin, (cuuint64_t)p.taps, (cuuint64_t)Cout};
+    cuuint64_t strides[2] = {(cuuint64_t)Cin * 4, (cuuint64_t)Cin * p.taps * 4};
+    cuuint32_t box[3] = {(cuuint32_t)p.sca, 1, (cuuint32_t)p.n_tile};
+    cuuint32_t es[3] = {1, 1, 1};
+    if ((size_t)p.rpt * p.epi_buf_bytes <= (size_t)stages * p.stage_bytes && p.epi_buf_bytes % 128 == 0 &&
+        (reinterpret_cast<uintptr_t>(dw) & 15) == 0 && Cin % 4 == 0 &&
+        enc(&tmDW, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dw, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+      p.epi_bufs = p.rpt;
+  }
   size_t smem = std::max((size_t)stages * p.stage_bytes + tail, (size_t)120 * 1024);
   static bool attr_set = false;
   if (!attr_set) {
@@ -678,7 +728,7 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf
     attr_set = true;
   }
   dim3 grid(tiles, p.splits);
-  tc::wgrad_tc_kernel<<<grid, 224, smem, st>>>(tmX, tmDY, p);
+  tc::wgrad_tc_kernel<<<grid, 224, smem, st>>>(tmX, tmDY, tmDW, p);
   return cudaGetLastError() == cudaSuccess ? 0 : -8;
 }
 
