@@ -76,10 +76,41 @@ __device__ __forceinline__ float round_storage(float v) {
   return to_f(t);
 }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialisation attribute
+// may start while the kernel before it in the stream is still draining: everything up to
+// pdl_wait() (barrier set-up, tensor-memory allocation, constants) overlaps that tail; pdl_wait()
+// returns once the preceding grid has completed and its memory is visible, so nothing that depends
+// on it may come earlier.  Every such kernel executes it unconditionally, which also keeps the
+// stream order transitive.  pdl_launch_dependents() lets the NEXT kernel begin its own prologue as
+// soon as this grid's blocks have all passed that point and resources free up.  Launched without
+// the attribute both are no-ops.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
+}
+
+// Host side: launch with programmatic stream serialisation allowed (see pdl_wait).
+#ifndef LP_PDL
+#define LP_PDL 1
+#endif
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                     Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = LP_PDL;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 }  // namespace lp

@@ -172,6 +172,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();                 // the set-up above overlapped the tail of the preceding kernel
+  pdl_launch_dependents();
   const uint32_t tmem_base = tail->tmem_base;
   const int kiters = p.ntaps * p.chunks;
   bool failed = false;

@@ -63,6 +63,8 @@ __device__ __forceinline__ void bn_load_consts(const BnArgs& a, int C, int c0, f
 // ---------------------------------------------------------------------------------------
 template <typename T>
 __global__ void bn_stats_kernel(const T* __restrict__ x, long long total_vecs, int C, double* __restrict__ stats) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int V = VecT<T>::N;
   extern __shared__ float sm[];  // [blockDim][2*V]
   const int CV = C / V;
@@ -105,6 +107,8 @@ template <typename T, bool X2, bool ADD>
 __global__ void __launch_bounds__(256, X2 ? 2 : (ADD ? 3 : 4))
 bn_apply_kernel(const T* __restrict__ x, BnArgs A, const T* __restrict__ x2, BnArgs B,
                 const T* __restrict__ addend, T* __restrict__ out, long long total_vecs, int C, int relu) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int V = VecT<T>::N;
   const int CV = C / V;
   const int c0 = (threadIdx.x % CV) * V;
@@ -172,10 +176,10 @@ bn_apply_kernel(const T* __restrict__ x, BnArgs A, const T* __restrict__ x2, BnA
 template <typename T>
 void launch_bn_apply(int grid, int threads, cudaStream_t st, const T* x, const BnArgs& A, const T* x2, const BnArgs& B,
                      const T* addend, T* out, long long total_vecs, int C, int relu) {
-  if (x2 && addend) bn_apply_kernel<T, true, true><<<grid, threads, 0, st>>>(x, A, x2, B, addend, out, total_vecs, C, relu);
-  else if (x2) bn_apply_kernel<T, true, false><<<grid, threads, 0, st>>>(x, A, x2, B, addend, out, total_vecs, C, relu);
-  else if (addend) bn_apply_kernel<T, false, true><<<grid, threads, 0, st>>>(x, A, x2, B, addend, out, total_vecs, C, relu);
-  else bn_apply_kernel<T, false, false><<<grid, threads, 0, st>>>(x, A, x2, B, addend, out, total_vecs, C, relu);
+  if (x2 && addend) launch_pdl(bn_apply_kernel<T, true, true>, dim3(grid), dim3(threads), 0, st, x, A, x2, B, addend, out, total_vecs, C, relu);
+  else if (x2) launch_pdl(bn_apply_kernel<T, true, false>, dim3(grid), dim3(threads), 0, st, x, A, x2, B, addend, out, total_vecs, C, relu);
+  else if (addend) launch_pdl(bn_apply_kernel<T, false, true>, dim3(grid), dim3(threads), 0, st, x, A, x2, B, addend, out, total_vecs, C, relu);
+  else launch_pdl(bn_apply_kernel<T, false, false>, dim3(grid), dim3(threads), 0, st, x, A, x2, B, addend, out, total_vecs, C, relu);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -293,6 +297,8 @@ __global__ void __launch_bounds__(256, 2)
 bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_mask,
                                      BnArgs A, float* __restrict__ dgamma, float* __restrict__ dbeta,
                                      long long total_vecs, int C) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int V = VecT<T>::N;
   extern __shared__ float sm[];
   const int CV = C / V;
@@ -357,6 +363,8 @@ __global__ void __launch_bounds__(256, 2)
 bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu_mask, BnArgs A,
                     const float* __restrict__ dgamma, const float* __restrict__ dbeta,
                     const T* __restrict__ addend, T* __restrict__ out, long long total_vecs, int C) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int V = VecT<T>::N;
   const int CV = C / V;
   const int c0 = (threadIdx.x % CV) * V;

@@ -473,9 +473,11 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   }
   const int grid = std::min(p.total_tiles, g_dev.sm_count);
   if (s.x_next && !s.addend) return LP_ERR_UNSUPPORTED;   // the fused loss belongs to a convolution with a shortcut
-  if (s.x_next) tc::conv_tc_kernel<true, true><<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
-  else if (s.addend) tc::conv_tc_kernel<false, true><<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
-  else tc::conv_tc_kernel<false, false><<<grid, tc::kConvThreads, smem, st>>>(tmA, tmB, p);
+  cudaError_t le;
+  if (s.x_next) le = launch_pdl(tc::conv_tc_kernel<true, true>, dim3(grid), dim3(tc::kConvThreads), smem, st, tmA, tmB, p);
+  else if (s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true>, dim3(grid), dim3(tc::kConvThreads), smem, st, tmA, tmB, p);
+  else le = launch_pdl(tc::conv_tc_kernel<false, false>, dim3(grid), dim3(tc::kConvThreads), smem, st, tmA, tmB, p);
+  LP_CUDA_OK(le);
   if (h) h->launches++;
   LP_CUDA_OK(cudaGetLastError());
   return LP_OK;
@@ -1237,8 +1239,8 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       if (!threads) return LP_ERR_UNSUPPORTED;
       const long long vecs = op.in.elems() / V;
       const int grid = grid_for(vecs, threads * 8, g_dev.sm_count, 4);
-      bn_stats_kernel<T><<<grid, threads, (size_t)threads * 2 * V * 4, st>>>((const T*)resolve(op.in, c), vecs, b.C,
-                                                                             b.stats);
+      LP_CUDA_OK(launch_pdl(bn_stats_kernel<T>, dim3(grid), dim3(threads), (size_t)threads * 2 * V * 4, st,
+                            (const T*)resolve(op.in, c), vecs, b.C, b.stats));
       h->launches++;
       break;
     }
@@ -1297,11 +1299,12 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       const int mask = op.mask.defined() ? 1 : 0;  // a ReLU followed this BN in the forward pass
       const T* addend = op.addend.defined() ? (const T*)resolve(op.addend, c) : nullptr;
       const int grid_r = grid_for(vecs, threads * 8, g_dev.sm_count, 4);
-      bn_bwd_reduce_kernel<T><<<grid_r, threads, (size_t)threads * 2 * V * 4, st>>>(
-          (const T*)resolve(op.in, c), (const T*)resolve(op.in2, c), mask, A, b.dgamma, b.dbeta, vecs, b.C);
+      LP_CUDA_OK(launch_pdl(bn_bwd_reduce_kernel<T>, dim3(grid_r), dim3(threads), (size_t)threads * 2 * V * 4, st,
+                            (const T*)resolve(op.in, c), (const T*)resolve(op.in2, c), mask, A, b.dgamma, b.dbeta, vecs, b.C));
       const int grid_a = grid_for(vecs, threads * 4, g_dev.sm_count, 8);
-      bn_bwd_apply_kernel<T><<<grid_a, threads, 0, st>>>((const T*)resolve(op.in, c), (const T*)resolve(op.in2, c), mask,
-                                                         A, b.dgamma, b.dbeta, addend, (T*)resolve(op.out, c), vecs, b.C);
+      LP_CUDA_OK(launch_pdl(bn_bwd_apply_kernel<T>, dim3(grid_a), dim3(threads), 0, st, (const T*)resolve(op.in, c),
+                            (const T*)resolve(op.in2, c), mask, A, (const float*)b.dgamma, (const float*)b.dbeta, addend,
+                            (T*)resolve(op.out, c), vecs, b.C));
       h->launches += 2;
       break;
     }

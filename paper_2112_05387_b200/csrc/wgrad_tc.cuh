@@ -121,6 +121,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();
+  pdl_launch_dependents();
   const uint32_t tmem_base = tail->tmem_base;
   bool failed = false;
 
@@ -319,6 +321,8 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();
+  pdl_launch_dependents();
   const uint32_t tmem_base = tail->tmem_base;
   bool failed = false;
 
@@ -610,8 +614,7 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, const bf16* x, const 
     attr_set = true;
   }
   dim3 grid(tiles, p.splits);
-  tc::wgrad_halo_kernel<<<grid, 224, smem, st>>>(tmX, tmDY, tmDW, p);
-  return cudaGetLastError() == cudaSuccess ? 0 : -8;
+  return launch_pdl(tc::wgrad_halo_kernel, grid, dim3(224), smem, st, tmX, tmDY, tmDW, p) == cudaSuccess ? 0 : -8;
 }
 
 static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf16* dy, float* dw, int N, int H, int W,
@@ -728,8 +731,7 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf
     attr_set = true;
   }
   dim3 grid(tiles, p.splits);
-  tc::wgrad_tc_kernel<<<grid, 224, smem, st>>>(tmX, tmDY, tmDW, p);
-  return cudaGetLastError() == cudaSuccess ? 0 : -8;
+  return launch_pdl(tc::wgrad_tc_kernel, grid, dim3(224), smem, st, tmX, tmDY, tmDW, p) == cudaSuccess ? 0 : -8;
 }
 
 }  // namespace lp
