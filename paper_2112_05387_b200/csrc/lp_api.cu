@@ -1249,7 +1249,10 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       const int threads = threads_for_channels(b.C, dtype);
       if (!threads) return LP_ERR_UNSUPPORTED;
       const long long vecs = op.in.elems() / V;
-      const int grid = grid_for(vecs, threads * 4, g_dev.sm_count, 8);
+      // one wave of blocks: as many per SM as the variant's register cap keeps resident (a second, partial
+      // wave cost a fifth of these kernels' time)
+      const int per_sm = op.in2.defined() ? 2 : (op.addend.defined() ? 3 : 4);
+      const int grid = grid_for(vecs, threads * 4, g_dev.sm_count, per_sm);
       BnArgs A = bn_args(b, eps), B2 = A;
       const T* x2 = nullptr;
       if (op.in2.defined()) { x2 = (const T*)resolve(op.in2, c); B2 = bn_args(P.bns[op.bn2], eps); }
@@ -1298,10 +1301,10 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       BnArgs A = bn_args(b, eps);
       const int mask = op.mask.defined() ? 1 : 0;  // a ReLU followed this BN in the forward pass
       const T* addend = op.addend.defined() ? (const T*)resolve(op.addend, c) : nullptr;
-      const int grid_r = grid_for(vecs, threads * 8, g_dev.sm_count, 4);
+      const int grid_r = grid_for(vecs, threads * 8, g_dev.sm_count, 2);   // one wave: two blocks stay resident per SM
       LP_CUDA_OK(launch_pdl(bn_bwd_reduce_kernel<T>, dim3(grid_r), dim3(threads), (size_t)threads * 2 * V * 4, st,
                             (const T*)resolve(op.in, c), (const T*)resolve(op.in2, c), mask, A, b.dgamma, b.dbeta, vecs, b.C));
-      const int grid_a = grid_for(vecs, threads * 4, g_dev.sm_count, 8);
+      const int grid_a = grid_for(vecs, threads * 4, g_dev.sm_count, 2);
       LP_CUDA_OK(launch_pdl(bn_bwd_apply_kernel<T>, dim3(grid_a), dim3(threads), 0, st, (const T*)resolve(op.in, c),
                             (const T*)resolve(op.in2, c), mask, A, (const float*)b.dgamma, (const float*)b.dbeta, addend,
                             (T*)resolve(op.out, c), vecs, b.C));
