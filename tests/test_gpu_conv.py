@@ -136,3 +136,38 @@ def test_unsupported_shapes_are_refused_not_faulted():
     x, w, dy = make_case(*case, "bf16")
     st, _, _ = run_conv(lp.LP_CONV_FWD, "bf16", lp.LP_CONV_IMPL_TENSOR, *case, x, w)
     assert st == -10
+
+
+@pytest.mark.parametrize("op_name", ["fwd", "dgrad"])
+def test_output_on_a_16_byte_boundary_takes_the_narrow_epilogue(op_name):
+    """The epilogue writes 32-byte pieces only when the output starts on a 32-byte boundary; a caller
+    buffer that is merely 16-byte aligned (the documented requirement) must give the same result."""
+    import torch
+    import paper_2112_05387_b200 as lp
+    case = (4, 16, 16, 64, 64, 3, 1, 1)
+    N, H, W, Cin, Cout, R, stride, pad = case
+    x, w, dy = make_case(*case, "bf16")
+    dev = "cuda:0"
+    op = lp.LP_CONV_FWD if op_name == "fwd" else lp.LP_CONV_DGRAD
+    a = x if op_name == "fwd" else dy
+    da = torch.from_numpy(a.astype(np.float32)).to(dev).to(torch.bfloat16).contiguous()
+    dw = torch.from_numpy(w.astype(np.float32)).to(dev).contiguous()
+    n_out = N * H * W * (Cout if op_name == "fwd" else Cin)
+    nbytes = lp.lp_conv2d_scratch_bytes(Cin, Cout, R)
+    scratch = torch.zeros(nbytes + 256, dtype=torch.uint8, device=dev)
+    base = (scratch.data_ptr() + 255) // 256 * 256
+    results = []
+    for shift in (0, 8):                      # elements: 0 -> 256-byte aligned, 8 -> 16 bytes further
+        buf = torch.full((n_out + 64,), 7.0, dtype=torch.bfloat16, device=dev)
+        off = (-(buf.data_ptr() // 2) % 128) + shift
+        out = buf[off:off + n_out]
+        assert out.data_ptr() % 32 == (16 if shift else 0)
+        st, _ = lp.lp_conv2d(op, lp.LP_BF16, lp.LP_CONV_IMPL_TENSOR, N, H, W, Cin, Cout, R, stride, pad, da, dw, out, None,
+                             base, nbytes)
+        assert st == 0, lp.lp_status_string(st)
+        torch.cuda.synchronize()
+        results.append(out.float().cpu().numpy().astype(np.float64))
+        assert float(buf[off - 1]) == 7.0 and float(buf[off + n_out]) == 7.0      # nothing written outside
+    np.testing.assert_array_equal(results[0], results[1])
+    ref = O.conv_fwd(x, w, stride, pad) if op_name == "fwd" else O.conv_dgrad(dy, w, stride, pad, x.shape)
+    assert rel_err(results[0], ref.reshape(-1)) < 6e-3
