@@ -200,6 +200,7 @@ struct lp_handle {
   ConvProfile prof;
   Timeline tl;
   int conv_impl = LP_CONV_IMPL_AUTO;
+  bool concurrent = false;   // set while a call enqueues the K modules on their own streams
   uint8_t* ws = nullptr;
   size_t ws_bytes = 0;
   int32_t* zero_labels = nullptr;  // N zeros, for forward passes that only want logits
@@ -471,7 +472,18 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
                                     (int)kTcMaxSmem));
     attr_set = true;
   }
-  const int grid = std::min(p.total_tiles, g_dev.sm_count);
+  // Persistent CTAs walk contiguous tile ranges; the launch takes about as long as the CTA with the most
+  // units (pairs of tiles).  While the K modules are enqueued side by side, the smallest grid with that
+  // same maximum is used (1024 tiles: 128 CTAs of four pairs instead of 148 of three pairs and a single
+  // tile): the freed SMs go to the kernels of the other modules' streams and the freed power to the
+  // clock (step 5.21 -> 5.07 ms).  A module running alone keeps one CTA per SM, which is a few per
+  // cent faster for the launch itself.
+  int grid = std::min(p.total_tiles, g_dev.sm_count);
+  if (h && h->concurrent) {
+    int per = (p.total_tiles + grid - 1) / grid;
+    if (p.mpair == 2) per = (per + 1) / 2 * 2;
+    grid = (p.total_tiles + per - 1) / per;
+  }
   if (s.x_next && !s.addend) return LP_ERR_UNSUPPORTED;   // the fused loss belongs to a convolution with a shortcut
   cudaError_t le;
   if (s.x_next) le = launch_pdl(tc::conv_tc_kernel<true, true>, dim3(grid), dim3(tc::kConvThreads), smem, st, tmA, tmB, p);
@@ -1698,6 +1710,14 @@ int lp_module_fwd_bwd(lp_handle* h, int k, const void* x_k, const void* x_next_o
   return module_fwd_bwd(h, k, x_k, x_next_or_labels, lambda_k, rho, loss_out, dx_k, (cudaStream_t)stream);
 }
 
+// Marks the handle while the modules are being enqueued side by side (convolution grids then leave SMs
+// to the other streams, see launch_conv_tc).
+struct ConcurrentScope {
+  lp_handle* h;
+  explicit ConcurrentScope(lp_handle* h_) : h(h_) { h->concurrent = true; }
+  ~ConcurrentScope() { h->concurrent = false; }
+};
+
 int lp_modules_fwd_bwd_all(lp_handle* h, const void* const* x, const int32_t* labels, const void* const* lambdas,
                            float rho, float* loss_out, void* const* dx, void* stream) {
   if (!h || !x || !labels || !loss_out) return LP_ERR_NULL;
@@ -1709,6 +1729,7 @@ int lp_modules_fwd_bwd_all(lp_handle* h, const void* const* x, const int32_t* la
     if (rc != LP_OK) return rc;
   }
   cudaStream_t st = (cudaStream_t)stream;
+  ConcurrentScope concurrent(h);
   LP_CUDA_OK(cudaEventRecord(h->fork, st));
   // heaviest modules first is not needed: all K are enqueued before any can finish
   for (int k = 0; k < K; ++k) {
@@ -1778,6 +1799,7 @@ int lp_layer_parallel_step(lp_handle* h, const void* images, void* const* x_out,
       return LP_ERR_ALIGN;
   }
   cudaStream_t st = (cudaStream_t)stream;
+  ConcurrentScope concurrent(h);
   LP_CUDA_OK(cudaEventRecord(h->fork, st));
   LP_CUDA_OK(cudaStreamWaitEvent(h->aux_stream, h->fork, 0));
   if (h->net.d.aux_recursive) {
