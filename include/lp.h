@@ -131,9 +131,10 @@ int lp_param_layout(const lp_net_desc* desc, int which, lp_param_entry* entries,
 /* Shape (NHWC) of x_k, k = 0..K-1 (x_0 is the image batch), from the descriptor alone. */
 int lp_boundary_shape_desc(const lp_net_desc* desc, int k, int shape_nhwc[4]);
 
-/* Create a handle over the caller's device workspace (zero-filled by this call on `stream`
- * order of the default stream; parameters start at zero until lp_set_params).  The handle owns
- * host memory, streams and events only. */
+/* Create a handle over the caller's device workspace.  The call zero-fills the workspace with a
+ * synchronous cudaMemset (it returns after the fill; work of the caller still running on other
+ * streams must not touch the workspace meanwhile); parameters start at zero until lp_set_params.
+ * The handle owns host memory, streams and events only. */
 int lp_create(const lp_net_desc* desc, void* dev_workspace, size_t bytes, lp_handle** out);
 int lp_destroy(lp_handle* h);
 
@@ -222,6 +223,12 @@ int lp_get_residual(lp_handle* h, int k, void* r_dst, void* seed_dst, void* stre
 
 /* Synchronise `stream` and return LP_OK, LP_ERR_DEVICE_TIMEOUT or LP_ERR_CUDA. */
 int lp_last_device_status(lp_handle* h, void* stream);
+/* Self-test of the device-side bounded wait (the mechanism behind LP_ERR_DEVICE_TIMEOUT): launches one
+ * small kernel in which a thread waits, for at most limit_ms (0 < limit_ms <= 100), on a barrier that
+ * nothing ever signals.  The wait runs out, the kernel records it the way the convolution kernels do and
+ * returns; the next lp_last_device_status reports LP_ERR_DEVICE_TIMEOUT and clears it, and the handle
+ * stays usable.  waited_ms (nullable; makes the call synchronous) receives the time the thread waited. */
+int lp_selftest_bounded_wait(lp_handle* h, double limit_ms, double* waited_ms, void* stream);
 /* Number of kernels the library launched since the counter was last reset. */
 int64_t lp_launch_count(lp_handle* h, int reset);
 /* Time (ms, CUDA events on the launching stream) spent in tensor-core convolution kernels and
@@ -302,7 +309,9 @@ int lp_conv2d(int op, int dtype, int impl, int N, int H, int W, int Cin, int Cou
  *   x: device bf16 [N,H,W,Cin]; w: device fp32 [Cout,R,R,Cin]; y: device bf16 [N,OH,OW,Cout].
  *   Same shape rules as the tensor-core path of lp_conv2d (Cin, Cout multiples of 8, R in {1,3},
  *   stride in {1,2}); LP_ERR_UNSUPPORTED otherwise.  The call is synchronous on `stream`.
- *   LP_ERR_SIZE ("size mismatch") if 2*Cout*R*R*Cin + 1024 bytes exceed the array.
+ *   LP_ERR_SIZE ("size mismatch") if the scratch does not fit the array: the call needs
+ *   512 + 2*Cout*R*R*Cin bytes, the middle term rounded up to a multiple of 256 (an error word, the
+ *   bf16 weights, a one-entry table), e.g. up to 640 -> 640 channels with a 3x3 kernel.
  *
  * The first call on a device looks up the array's device address (once per device, with that
  * device current) and sets kernel attributes: make it before any stream capture.  All calls share

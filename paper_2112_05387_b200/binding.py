@@ -13,7 +13,7 @@ __all__ = [
     "lp_modules_fwd_bwd_all", "lp_step", "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual",
     "lp_last_device_status", "lp_launch_count", "lp_conv_profile", "lp_conv2d", "lp_conv2d_scratch_bytes", "lp_graph_begin", "lp_graph_end",
     "lp_graph_launch", "lp_conv2d_fwd_noalloc", "LP_NOALLOC_SCRATCH_BYTES", "lp_layer_parallel_step", "lp_auxnet_distill", "lp_aux_correct", "lp_timeline", "lp_timeline_record",
-    "LP_PHASE_NAMES", "LP_OP_NAMES", "EXPORTED_SYMBOLS",
+    "LP_PHASE_NAMES", "LP_OP_NAMES", "EXPORTED_SYMBOLS", "lp_selftest_bounded_wait",
 ]
 
 LP_OK = 0
@@ -35,6 +35,7 @@ EXPORTED_SYMBOLS = [
     "lp_forward_serial", "lp_serial_fwd_bwd", "lp_get_residual", "lp_last_device_status", "lp_launch_count",
     "lp_conv_profile", "lp_conv2d_scratch_bytes", "lp_conv2d", "lp_graph_begin", "lp_graph_end", "lp_graph_launch",
     "lp_conv2d_fwd_noalloc", "lp_layer_parallel_step", "lp_auxnet_distill", "lp_timeline", "lp_aux_correct",
+    "lp_selftest_bounded_wait",
 ]
 
 
@@ -123,6 +124,7 @@ def library():
     lib.lp_serial_fwd_bwd.argtypes = [vp, vp, vp, vp, vp]
     lib.lp_get_residual.argtypes = [vp, i32, vp, vp, vp]
     lib.lp_last_device_status.argtypes = [vp, vp]
+    lib.lp_selftest_bounded_wait.argtypes = [vp, ctypes.c_double, ctypes.POINTER(ctypes.c_double), vp]
     lib.lp_launch_count.restype = ctypes.c_int64
     lib.lp_launch_count.argtypes = [vp, i32]
     lib.lp_timeline.argtypes = [vp, i32, i32, ctypes.POINTER(lp_timeline_record), ctypes.POINTER(ctypes.c_int)]
@@ -339,6 +341,14 @@ def lp_get_residual(h, k, r_dst, seed_dst, stream=None):
 
 def lp_last_device_status(h, stream=None):
     return library().lp_last_device_status(h.ptr, _ptr(stream))
+
+
+def lp_selftest_bounded_wait(h, limit_ms, stream=None):
+    """Launch the bounded-wait self-test; returns the milliseconds the device thread waited before giving up."""
+    w = ctypes.c_double(0.0)
+    _check(library().lp_selftest_bounded_wait(h.ptr, float(limit_ms), ctypes.byref(w), _ptr(stream)),
+           "lp_selftest_bounded_wait")
+    return w.value
 
 
 def lp_launch_count(h, reset=False):

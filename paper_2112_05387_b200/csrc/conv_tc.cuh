@@ -105,7 +105,7 @@ struct TcSmemTail {
   uint64_t tmem_empty[kMaxSlots];
   uint32_t tmem_base;
   int abort_flag;
-  int epi_ok;
+  int epi_ok[2];                   // outcome of the epilogue's wait, alternating by accumulator (see the epilogue)
   float ssum[LP_EPI_WARPS][256];   // per epilogue warp: plain read-modify-write, no shared-memory atomics
   float ssq[LP_EPI_WARPS][256];
   uint32_t tr[LP_EPI_WARPS][16 * 33];   // per epilogue warp: transposition scratch of the statistics
@@ -370,6 +370,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int ngroups = (p.n_tile_cols + 31) >> 5;
     uint32_t slot = 0, slot_phase = 0;
     float sum_rr = 0.f, sum_kr = 0.f;    // local-loss sums of this thread (kLoss)
+    int epi_turn = 0;
     // The residual operand was written several kernels ago and is no longer in L2.  Each thread
     // asks for the row of the NEXT tile it will add while it works on the current one, so that the
     // loads of the epilogue find their lines in L2 instead of waiting for DRAM.
@@ -408,9 +409,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             (((long long)n * p.out_H + (oh * p.os + p.oo_h)) * p.out_W + (ow * p.os + p.oo_w)) * p.out_C;
         // one thread waits (bounded) and all epilogue threads agree on the outcome, so that the
         // named barriers below are reached by all of them or by none
-        if (et == 0) tail->epi_ok = mbar_wait(&tail->tmem_full[buf], (slot_phase >> buf) & 1, abort_flag) ? 1 : 0;
+        // (two words used in turn: the one of the previous accumulator may still be read by a slower warp
+        // when thread 0 writes the next outcome; the barrier below separates uses two apart)
+        if (et == 0) tail->epi_ok[epi_turn] = mbar_wait(&tail->tmem_full[buf], (slot_phase >> buf) & 1, abort_flag) ? 1 : 0;
         asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-        if (!*(volatile int*)&tail->epi_ok) { failed = true; break; }
+        const int wait_ok = *(volatile int*)&tail->epi_ok[epi_turn];
+        epi_turn ^= 1;
+        if (!wait_ok) { failed = true; break; }
         tc_fence_after();
         const uint32_t taddr = tmem_base + buf * p.acc_stride + ((uint32_t)(q * 32) << 16);
         // Drain the accumulator into registers first (up to kBatch x 32 columns per pass) and hand

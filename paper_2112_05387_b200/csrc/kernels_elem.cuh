@@ -260,21 +260,21 @@ __global__ void module_out_loss_kernel(const T* __restrict__ x, BnArgs A, const 
     }
     stv(seed_out + i * V, y);
   }
-  __shared__ float red[2][32];
-  sum_rr = warp_sum(sum_rr);
-  sum_kr = warp_sum(sum_kr);
-  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
-  if (l == 0) {
-    red[0][w] = sum_rr;
-    red[1][w] = sum_kr;
-  }
+  // Block sums through shared memory: the block size follows the channel count (240 threads for 160, 320
+  // or 640 bf16 channels), so the last warp may be partial and full-mask shuffles are not available to it.
+  __shared__ float red[2][1024];
+  red[0][threadIdx.x] = sum_rr;
+  red[1][threadIdx.x] = sum_kr;
   __syncthreads();
-  if (w == 0) {
-    const int nw = (blockDim.x + 31) >> 5;
-    float a = l < nw ? red[0][l] : 0.f, b = l < nw ? red[1][l] : 0.f;
-    a = warp_sum(a);
+  if (threadIdx.x < 32) {
+    float a = 0.f, b = 0.f;
+    for (int t = threadIdx.x; t < (int)blockDim.x; t += 32) {
+      a += red[0][t];
+      b += red[1][t];
+    }
+    a = warp_sum(a);   // warp 0 is always complete: block sizes are at least 32
     b = warp_sum(b);
-    if (l == 0) {
+    if (threadIdx.x == 0) {
       atomicAdd(&acc[0], (double)a);
       atomicAdd(&acc[1], (double)b);
     }

@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -141,6 +142,8 @@ struct Device {
   bool ready = false;
   int sm_count = 148;
   EncodeTiledFn encode = nullptr;
+  // kernel attributes are per device: set on the first launch of each kernel family on that device
+  bool conv_attr = false, wgrad_attr = false, wgrad_halo_attr = false;
   int init() {
     if (ready) return LP_OK;
     int dev = 0;
@@ -158,7 +161,20 @@ struct Device {
     return LP_OK;
   }
 };
-static Device g_dev;
+// One record per device ordinal; the current device's record is looked up at every use.  The mutex
+// covers first-use initialisation from several host threads.
+static const int kMaxDevices = 64;
+static Device g_devices[kMaxDevices];
+static std::mutex g_devices_mutex;
+static inline Device& cur_dev() {
+  int d = 0;
+  if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) d = 0;
+  return g_devices[d];
+}
+static inline int init_cur_dev() {
+  std::lock_guard<std::mutex> lock(g_devices_mutex);
+  return cur_dev().init();
+}
 
 // Per-operation time line: a pair of events around every operation of every plan, on the stream
 // the operation runs on.  Events do not serialise the streams; they cannot be recorded into a graph.
@@ -295,7 +311,7 @@ static int encode_act_map(CUtensorMap* m, const void* base, int N, int H, int W,
   cuuint32_t es[4] = {1, (cuuint32_t)step, (cuuint32_t)step, 1};
   const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                 : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
-  CUresult r = g_dev.encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+  CUresult r = cur_dev().encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? LP_OK : LP_ERR_CUDA;
@@ -309,7 +325,7 @@ static int encode_mat_map(CUtensorMap* m, const void* base, long long K, int row
   cuuint32_t es[2] = {1, 1};
   const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                 : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
-  CUresult r = g_dev.encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+  CUresult r = cur_dev().encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? LP_OK : LP_ERR_CUDA;
@@ -356,7 +372,7 @@ static int encode_act_map_halo(CUtensorMap* m, const void* base, int N, int H, i
   cuuint32_t es[4] = {1, 1, 1, 1};
   const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                 : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
-  CUresult r = g_dev.encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+  CUresult r = cur_dev().encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? LP_OK : LP_ERR_CUDA;
@@ -409,7 +425,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     // two activation stages (each lasts nine weight stages), the rest of shared memory for weights
     bool fits = false;
     p.nA = 2;
-    for (int pair = (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, g_dev.sm_count)) ? 2 : 1;
+    for (int pair = (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, cur_dev().sm_count)) ? 2 : 1;
          pair >= 1 && !fits; --pair) {
       const size_t a_bytes = (size_t)p.nA * pair * p.a_halo_bytes;
       if (a_bytes >= avail) continue;
@@ -432,7 +448,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   if (!p.halo) {
     // two pixel tiles per weight tile wherever a CTA has at least two tiles and three stages still fit
     p.mpair = 1;
-    if (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, g_dev.sm_count) &&
+    if (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, cur_dev().sm_count) &&
         (kTcMaxSmem - tail) / (2 * p.a_region_bytes + b_region) >= 3)
       p.mpair = 2;
     p.b_offset = p.mpair * p.a_region_bytes;
@@ -462,7 +478,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   if (rc != LP_OK) return rc;
   size_t smem = (size_t)p.tail_offset + tail;
   smem = std::max(smem, kTcMinSmem);
-  static bool attr_set = false;
+  bool& attr_set = cur_dev().conv_attr;
   if (!attr_set) {
     LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kTcMaxSmem));
@@ -478,7 +494,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   // tile): the freed SMs go to the kernels of the other modules' streams and the freed power to the
   // clock (step 5.21 -> 5.07 ms).  A module running alone keeps one CTA per SM, which is a few per
   // cent faster for the launch itself.
-  int grid = std::min(p.total_tiles, g_dev.sm_count);
+  int grid = std::min(p.total_tiles, cur_dev().sm_count);
   if (h && h->concurrent) {
     int per = (p.total_tiles + grid - 1) / grid;
     if (p.mpair == 2) per = (per + 1) / 2 * 2;
@@ -577,7 +593,7 @@ static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int
   if (c.cin <= 4 && !addend && few_cpt && few_smem <= 48 * 1024) {
     // stems and the first AuxNet convolution: filter bank in shared memory
     const long long items = (long long)N * c.OH * c.OW * (c.cout / few_cpt);
-    const int fgrid = grid_for(items, 256, g_dev.sm_count, 8);
+    const int fgrid = grid_for(items, 256, cur_dev().sm_count, 8);
 #define LP_FEWCH_FWD(CPT)                                                                                      \
     if (dtype == LP_F32)                                                                                       \
       conv_fwd_fewch_kernel<float, CPT><<<fgrid, 256, few_smem, st>>>((const float*)x, c.w, (float*)y, g);       \
@@ -595,7 +611,7 @@ static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int
     return LP_OK;
   }
   const long long work = (long long)N * c.OH * c.OW * (c.cout / 4);
-  const int grid = grid_for(work, 128, g_dev.sm_count, 16);
+  const int grid = grid_for(work, 128, cur_dev().sm_count, 16);
   if (dtype == LP_F32)
     conv_fwd_simt_kernel<float><<<grid, 128, 0, st>>>((const float*)x, c.w, (const float*)addend, (float*)y, g);
   else
@@ -656,7 +672,7 @@ static int conv_dgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
   if (c.cin % 4) return LP_ERR_UNSUPPORTED;
   ConvGeom g{N, c.H, c.W, c.cin, c.OH, c.OW, c.cout, c.R, c.R, c.stride, c.pad};
   const long long work = (long long)N * c.H * c.W * (c.cin / 4);
-  const int grid = grid_for(work, 128, g_dev.sm_count, 16);
+  const int grid = grid_for(work, 128, cur_dev().sm_count, 16);
   if (dtype == LP_F32)
     conv_dgrad_simt_kernel<float><<<grid, 128, 0, st>>>((const float*)dy, c.w, (const float*)addend, (float*)dx, g);
   else
@@ -673,8 +689,9 @@ static int conv_wgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
   if ((impl & 15) == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
   if (use_tc) {
     ProfScope ps(h, st, 2.0 * N * c.OH * c.OW * (double)c.cout * c.R * c.R * c.cin);
-    int rc = launch_wgrad_tc(g_dev.encode, g_dev.sm_count, (const bf16*)x, (const bf16*)dy, dw, N, c.H, c.W, c.cin,
-                             c.OH, c.OW, c.cout, c.R, c.stride, c.pad, dev_err, st);
+    Device& D = cur_dev();
+    int rc = launch_wgrad_tc(D.encode, D.sm_count, &D.wgrad_attr, &D.wgrad_halo_attr, (const bf16*)x, (const bf16*)dy, dw, N,
+                             c.H, c.W, c.cin, c.OH, c.OW, c.cout, c.R, c.stride, c.pad, dev_err, st);
     if (h) h->launches++;
     return rc;
   }
@@ -690,7 +707,7 @@ static int conv_wgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
       while (lanes > 1 && (size_t)lanes * pair_threads * few_cpt * 4 > 48 * 1024) --lanes;
       const int threads = lanes * pair_threads;
       const size_t red_bytes = lanes > 1 ? (size_t)threads * few_cpt * 4 : 0;
-      const long long blocks = std::min<long long>((npix + 63) / 64, 6LL * g_dev.sm_count);
+      const long long blocks = std::min<long long>((npix + 63) / 64, 6LL * cur_dev().sm_count);
       const long long ppb = (npix + blocks - 1) / blocks;
       const int fgrid = (int)((npix + ppb - 1) / ppb);
 #define LP_FEWCH_WGRAD(CPT)                                                                                    \
@@ -1250,7 +1267,7 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       const int threads = threads_for_channels(b.C, dtype);
       if (!threads) return LP_ERR_UNSUPPORTED;
       const long long vecs = op.in.elems() / V;
-      const int grid = grid_for(vecs, threads * 8, g_dev.sm_count, 4);
+      const int grid = grid_for(vecs, threads * 8, cur_dev().sm_count, 4);
       LP_CUDA_OK(launch_pdl(bn_stats_kernel<T>, dim3(grid), dim3(threads), (size_t)threads * 2 * V * 4, st,
                             (const T*)resolve(op.in, c), vecs, b.C, b.stats));
       h->launches++;
@@ -1264,7 +1281,7 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       // one wave of blocks: as many per SM as the variant's register cap keeps resident (a second, partial
       // wave cost a fifth of these kernels' time)
       const int per_sm = op.in2.defined() ? 2 : (op.addend.defined() ? 3 : 4);
-      const int grid = grid_for(vecs, threads * 4, g_dev.sm_count, per_sm);
+      const int grid = grid_for(vecs, threads * 4, cur_dev().sm_count, per_sm);
       BnArgs A = bn_args(b, eps), B2 = A;
       const T* x2 = nullptr;
       if (op.in2.defined()) { x2 = (const T*)resolve(op.in2, c); B2 = bn_args(P.bns[op.bn2], eps); }
@@ -1280,7 +1297,7 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       const int threads = threads_for_channels(C, dtype);
       if (!threads) return LP_ERR_UNSUPPORTED;
       const long long vecs = op.out.elems() / V;
-      const int grid = grid_for(vecs, threads * 4, g_dev.sm_count, 8);
+      const int grid = grid_for(vecs, threads * 4, cur_dev().sm_count, 8);
       BnArgs A, B2;
       memset(&A, 0, sizeof(A));
       memset(&B2, 0, sizeof(B2));
@@ -1313,10 +1330,10 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       BnArgs A = bn_args(b, eps);
       const int mask = op.mask.defined() ? 1 : 0;  // a ReLU followed this BN in the forward pass
       const T* addend = op.addend.defined() ? (const T*)resolve(op.addend, c) : nullptr;
-      const int grid_r = grid_for(vecs, threads * 8, g_dev.sm_count, 2);   // one wave: two blocks stay resident per SM
+      const int grid_r = grid_for(vecs, threads * 8, cur_dev().sm_count, 2);   // one wave: two blocks stay resident per SM
       LP_CUDA_OK(launch_pdl(bn_bwd_reduce_kernel<T>, dim3(grid_r), dim3(threads), (size_t)threads * 2 * V * 4, st,
                             (const T*)resolve(op.in, c), (const T*)resolve(op.in2, c), mask, A, b.dgamma, b.dbeta, vecs, b.C));
-      const int grid_a = grid_for(vecs, threads * 4, g_dev.sm_count, 2);
+      const int grid_a = grid_for(vecs, threads * 4, cur_dev().sm_count, 2);
       LP_CUDA_OK(launch_pdl(bn_bwd_apply_kernel<T>, dim3(grid_a), dim3(threads), 0, st, (const T*)resolve(op.in, c),
                             (const T*)resolve(op.in2, c), mask, A, (const float*)b.dgamma, (const float*)b.dbeta, addend,
                             (T*)resolve(op.out, c), vecs, b.C));
@@ -1325,7 +1342,7 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
     }
     case OP_MAXPOOL_FWD: {
       const long long total = op.out.elems();
-      maxpool_fwd_kernel<T><<<grid_for(total, 256, g_dev.sm_count, 16), 256, 0, st>>>(
+      maxpool_fwd_kernel<T><<<grid_for(total, 256, cur_dev().sm_count, 16), 256, 0, st>>>(
           (const T*)resolve(op.in, c), (T*)resolve(op.out, c), op.arg, op.in.n, op.in.h, op.in.w, op.in.c, op.out.h,
           op.out.w);
       h->launches++;
@@ -1333,7 +1350,7 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
     }
     case OP_MAXPOOL_BWD: {
       const long long total = op.out.elems();
-      maxpool_bwd_kernel<T><<<grid_for(total, 256, g_dev.sm_count, 16), 256, 0, st>>>(
+      maxpool_bwd_kernel<T><<<grid_for(total, 256, cur_dev().sm_count, 16), 256, 0, st>>>(
           (const T*)resolve(op.in, c), op.arg, (T*)resolve(op.out, c), op.out.n, op.out.h, op.out.w, op.out.c, op.in.h,
           op.in.w);
       h->launches++;
@@ -1358,7 +1375,7 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
     case OP_HEAD_BWD: {
       HeadDef& hd = P.head;
       const long long total = (long long)hd.classes * hd.C;
-      head_bwd_w_kernel<<<grid_for(total, 128, g_dev.sm_count, 16), 128, 0, st>>>(hd.dlogits, hd.pooled, hd.dW, hd.db,
+      head_bwd_w_kernel<<<grid_for(total, 128, cur_dev().sm_count, 16), 128, 0, st>>>(hd.dlogits, hd.pooled, hd.dW, hd.db,
                                                                                   hd.N, hd.C, hd.classes);
       head_bwd_x_kernel<T><<<dim3(hd.N, (hd.C + 255) / 256), 256, 0, st>>>(hd.dlogits, hd.W, (T*)resolve(op.out, c), hd.HW,
                                                                            hd.C, hd.classes);
@@ -1420,7 +1437,7 @@ static int pack_weights(lp_handle* h, Plan& P, cudaStream_t st) {
 static int sgd_update(lp_handle* h, Plan& P, float lr, float momentum, float weight_decay, cudaStream_t st) {
   float* mom = momentum != 0.f ? P.ps.m : nullptr;
   if (P.ps.host_pack.empty()) {
-    sgd_kernel<<<grid_for((long long)P.ps.n, 256, g_dev.sm_count, 8), 256, 0, st>>>(P.ps.p, P.ps.g, P.ps.m,
+    sgd_kernel<<<grid_for((long long)P.ps.n, 256, cur_dev().sm_count, 8), 256, 0, st>>>(P.ps.p, P.ps.g, P.ps.m,
                                                                                     (long long)P.ps.n, lr, momentum,
                                                                                     weight_decay);
     h->launches++;
@@ -1553,7 +1570,7 @@ int lp_create(const lp_net_desc* desc, void* dev_workspace, size_t bytes, lp_han
   if (reinterpret_cast<uintptr_t>(dev_workspace) & 255) return LP_ERR_WORKSPACE;
   const size_t need = lp_workspace_bytes(desc);
   if (bytes < need) return LP_ERR_WORKSPACE;
-  rc = g_dev.init();
+  rc = init_cur_dev();
   if (rc != LP_OK) return rc;
   lp_handle* h = new lp_handle();
   h->net = net;
@@ -1605,6 +1622,7 @@ int lp_destroy(lp_handle* h) {
   if (h->aux_end) cudaEventDestroy(h->aux_end);
   for (auto e : h->aux_done) if (e) cudaEventDestroy(e);
   for (auto& pr : h->prof.events) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
+  for (auto& r : h->tl.recs) { if (r.a) cudaEventDestroy(r.a); if (r.b) cudaEventDestroy(r.b); }
   for (auto g : h->graphs) cudaGraphExecDestroy(g);
   delete h;
   return LP_OK;
@@ -1732,16 +1750,22 @@ int lp_modules_fwd_bwd_all(lp_handle* h, const void* const* x, const int32_t* la
   ConcurrentScope concurrent(h);
   LP_CUDA_OK(cudaEventRecord(h->fork, st));
   // heaviest modules first is not needed: all K are enqueued before any can finish
-  for (int k = 0; k < K; ++k) {
-    LP_CUDA_OK(cudaStreamWaitEvent(h->streams[k], h->fork, 0));
+  // A failure part-way still joins every stream that was forked back into the caller's (a stream left
+  // unjoined would invalidate a capture in progress); the first error is what the call returns.
+  int first_err = LP_OK;
+  int forked = 0;
+  for (int k = 0; k < K && first_err == LP_OK; ++k) {
+    if (cudaStreamWaitEvent(h->streams[k], h->fork, 0) != cudaSuccess) { first_err = LP_ERR_CUDA; break; }
+    forked = k + 1;
     const void* tgt = k == K - 1 ? (const void*)labels : x[k + 1];
-    int rc = module_fwd_bwd(h, k, x[k], tgt, (lambdas && k < K - 1) ? lambdas[k] : nullptr, rho, loss_out + 2 * k,
-                            dx ? dx[k] : nullptr, h->streams[k]);
-    if (rc != LP_OK) return rc;
-    LP_CUDA_OK(cudaEventRecord(h->done[k], h->streams[k]));
+    first_err = module_fwd_bwd(h, k, x[k], tgt, (lambdas && k < K - 1) ? lambdas[k] : nullptr, rho, loss_out + 2 * k,
+                               dx ? dx[k] : nullptr, h->streams[k]);
   }
-  for (int k = 0; k < K; ++k) LP_CUDA_OK(cudaStreamWaitEvent(st, h->done[k], 0));
-  return LP_OK;
+  for (int k = 0; k < forked; ++k) {
+    if (cudaEventRecord(h->done[k], h->streams[k]) != cudaSuccess || cudaStreamWaitEvent(st, h->done[k], 0) != cudaSuccess)
+      if (first_err == LP_OK) first_err = LP_ERR_CUDA;
+  }
+  return first_err;
 }
 
 static int update_module(lp_handle* h, int k, float lr, float momentum, float weight_decay, float kappa_step,
@@ -1754,10 +1778,10 @@ static int update_module(lp_handle* h, int k, float lr, float momentum, float we
   if (lambda_inout && k + 1 < h->net.K) {
     const long long n = P.r.elems();
     if (h->dtype == LP_F32)
-      kappa_update_kernel<float><<<grid_for(n / 4, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+      kappa_update_kernel<float><<<grid_for(n / 4, 256, cur_dev().sm_count, 8), 256, 0, st>>>(
           (float*)lambda_inout, (const float*)P.r.p, kappa_step, n / 4);
     else
-      kappa_update_kernel<bf16><<<grid_for(n / 8, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+      kappa_update_kernel<bf16><<<grid_for(n / 8, 256, cur_dev().sm_count, 8), 256, 0, st>>>(
           (bf16*)lambda_inout, (const bf16*)P.r.p, kappa_step, n / 8);
     h->launches++;
     LP_CUDA_OK(cudaGetLastError());
@@ -1801,53 +1825,75 @@ int lp_layer_parallel_step(lp_handle* h, const void* images, void* const* x_out,
   cudaStream_t st = (cudaStream_t)stream;
   ConcurrentScope concurrent(h);
   LP_CUDA_OK(cudaEventRecord(h->fork, st));
-  LP_CUDA_OK(cudaStreamWaitEvent(h->aux_stream, h->fork, 0));
-  if (h->net.d.aux_recursive) {
-    // recursive form: stack k needs the images only and runs on module k's stream, right before the
-    // module it feeds; aux_done[k-1] marks x_k for module k-1's local loss
-    for (int k = 1; k < K; ++k) {
-      cudaStream_t sk = h->streams[k];
-      LP_CUDA_OK(cudaStreamWaitEvent(sk, h->fork, 0));
-      RunCtx c;
-      c.st = sk; c.images = images; c.xout = x_out;
-      for (int j = 0; j < k; ++j) {
-        int rc = aux_plan_forward(h, NetDef::reaux_index(k, j), c);
-        if (rc != LP_OK) return rc;
+  // Streams forked from the caller's so far; whatever happens below, each is joined back before the
+  // call returns (a stream left unjoined would invalidate a capture in progress).
+  bool aux_forked = false;
+  std::vector<bool> forked(K, false);
+  auto fork = [&](cudaStream_t s, bool* flag) -> int {
+    if (*flag) return LP_OK;
+    LP_CUDA_OK(cudaStreamWaitEvent(s, h->fork, 0));
+    *flag = true;
+    return LP_OK;
+  };
+  auto fork_module = [&](int k) -> int {
+    bool f = forked[k];
+    int rc = fork(h->streams[k], &f);
+    forked[k] = f;
+    return rc;
+  };
+  auto enqueue = [&]() -> int {
+    int rc = fork(h->aux_stream, &aux_forked);
+    if (rc != LP_OK) return rc;
+    if (h->net.d.aux_recursive) {
+      // recursive form: stack k needs the images only and runs on module k's stream, right before the
+      // module it feeds; aux_done[k-1] marks x_k for module k-1's local loss
+      for (int k = 1; k < K; ++k) {
+        cudaStream_t sk = h->streams[k];
+        if ((rc = fork_module(k)) != LP_OK) return rc;
+        RunCtx c;
+        c.st = sk; c.images = images; c.xout = x_out;
+        for (int j = 0; j < k; ++j)
+          if ((rc = aux_plan_forward(h, NetDef::reaux_index(k, j), c)) != LP_OK) return rc;
+        LP_CUDA_OK(cudaEventRecord(h->aux_done[k - 1], sk));
       }
-      LP_CUDA_OK(cudaEventRecord(h->aux_done[k - 1], sk));
+    } else {
+      // AuxNet chain on its own stream; aux_done[k] marks x_{k+1}
+      RunCtx c;
+      c.st = h->aux_stream; c.images = images; c.xout = x_out;
+      for (int k = 0; k + 1 < K; ++k) {
+        if ((rc = aux_plan_forward(h, k, c)) != LP_OK) return rc;
+        LP_CUDA_OK(cudaEventRecord(h->aux_done[k], h->aux_stream));
+      }
     }
-    LP_CUDA_OK(cudaEventRecord(h->aux_end, h->aux_stream));
-  } else {
-    // AuxNet chain on its own stream; aux_done[k] marks x_{k+1}
-    RunCtx c;
-    c.st = h->aux_stream; c.images = images; c.xout = x_out;
-    for (int k = 0; k + 1 < K; ++k) {
-      int rc = aux_plan_forward(h, k, c);
+    // module k starts as soon as x_k exists, takes its local loss as soon as x_{k+1} exists, and
+    // updates its own parameters right after its own backward pass
+    for (int k = 0; k < K; ++k) {
+      cudaStream_t sk = h->streams[k];
+      if ((rc = fork_module(k)) != LP_OK) return rc;
+      if (k > 0) LP_CUDA_OK(cudaStreamWaitEvent(sk, h->aux_done[k - 1], 0));
+      const bool last = k == K - 1;
+      const void* xk = k == 0 ? images : x_out[k - 1];
+      const void* tgt = last ? (const void*)labels : (const void*)x_out[k];
+      void* lam = (lambdas_inout && !last) ? lambdas_inout[k] : nullptr;
+      rc = module_fwd_bwd(h, k, xk, tgt, lam, rho, loss_out + 2 * k, dx ? dx[k] : nullptr, sk,
+                          last ? nullptr : h->aux_done[k]);
       if (rc != LP_OK) return rc;
-      LP_CUDA_OK(cudaEventRecord(h->aux_done[k], h->aux_stream));
+      rc = update_module(h, k, lr, momentum, weight_decay, kappa_step, lam, sk);
+      if (rc != LP_OK) return rc;
     }
-    LP_CUDA_OK(cudaEventRecord(h->aux_end, h->aux_stream));
+    return LP_OK;
+  };
+  int first_err = enqueue();
+  if (aux_forked) {
+    if (cudaEventRecord(h->aux_end, h->aux_stream) != cudaSuccess || cudaStreamWaitEvent(st, h->aux_end, 0) != cudaSuccess)
+      if (first_err == LP_OK) first_err = LP_ERR_CUDA;
   }
-  // module k starts as soon as x_k exists, takes its local loss as soon as x_{k+1} exists, and
-  // updates its own parameters right after its own backward pass
   for (int k = 0; k < K; ++k) {
-    cudaStream_t sk = h->streams[k];
-    LP_CUDA_OK(cudaStreamWaitEvent(sk, h->fork, 0));
-    if (k > 0) LP_CUDA_OK(cudaStreamWaitEvent(sk, h->aux_done[k - 1], 0));
-    const bool last = k == K - 1;
-    const void* xk = k == 0 ? images : x_out[k - 1];
-    const void* tgt = last ? (const void*)labels : (const void*)x_out[k];
-    void* lam = (lambdas_inout && !last) ? lambdas_inout[k] : nullptr;
-    int rc = module_fwd_bwd(h, k, xk, tgt, lam, rho, loss_out + 2 * k, dx ? dx[k] : nullptr, sk,
-                            last ? nullptr : h->aux_done[k]);
-    if (rc != LP_OK) return rc;
-    rc = update_module(h, k, lr, momentum, weight_decay, kappa_step, lam, sk);
-    if (rc != LP_OK) return rc;
-    LP_CUDA_OK(cudaEventRecord(h->done[k], sk));
+    if (!forked[k]) continue;
+    if (cudaEventRecord(h->done[k], h->streams[k]) != cudaSuccess || cudaStreamWaitEvent(st, h->done[k], 0) != cudaSuccess)
+      if (first_err == LP_OK) first_err = LP_ERR_CUDA;
   }
-  LP_CUDA_OK(cudaStreamWaitEvent(st, h->aux_end, 0));
-  for (int k = 0; k < K; ++k) LP_CUDA_OK(cudaStreamWaitEvent(st, h->done[k], 0));
-  return LP_OK;
+  return first_err;
 }
 
 int lp_auxnet_distill(lp_handle* h, const void* images, void* const* x, const void* const* dx, float lr_lambda,
@@ -1874,11 +1920,11 @@ int lp_auxnet_distill(lp_handle* h, const void* images, void* const* x, const vo
     for (int i = first_idx; i <= last_idx; ++i) LP_CUDA_OK(cudaMemsetAsync(h->auxs[i].ps.g, 0, h->auxs[i].ps.n * 4, st));
     void* xn = x_new ? x_new[k - 1] : nullptr;
     if (h->dtype == LP_F32)
-      distill_seed_kernel<float><<<grid_for(n / 4, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+      distill_seed_kernel<float><<<grid_for(n / 4, 256, cur_dev().sm_count, 8), 256, 0, st>>>(
           (const float*)x[k - 1], (const float*)dx[k], (const float*)h->modules[k - 1].seed.p, lr_lambda,
           (float*)xn, (float*)A.seed.p, A.loss_acc, n / 4);
     else
-      distill_seed_kernel<bf16><<<grid_for(n / 8, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+      distill_seed_kernel<bf16><<<grid_for(n / 8, 256, cur_dev().sm_count, 8), 256, 0, st>>>(
           (const bf16*)x[k - 1], (const bf16*)dx[k], (const bf16*)h->modules[k - 1].seed.p, lr_lambda, (bf16*)xn,
           (bf16*)A.seed.p, A.loss_acc, n / 8);
     distill_loss_kernel<<<1, 1, 0, st>>>(A.loss_acc, loss_out + (k - 1));
@@ -1916,11 +1962,11 @@ int lp_aux_correct(lp_handle* h, void* const* x_inout, const void* const* dx, fl
     TimelineScope ts(h, st, LP_AUX(k - 1), LP_OP_UPDATE, LP_PHASE_DISTILL);
     LP_CUDA_OK(cudaMemsetAsync(A.loss_acc, 0, 2 * sizeof(double), st));
     if (h->dtype == LP_F32)
-      distill_seed_kernel<float><<<grid_for(n / 4, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+      distill_seed_kernel<float><<<grid_for(n / 4, 256, cur_dev().sm_count, 8), 256, 0, st>>>(
           (const float*)x_inout[k - 1], (const float*)dx[k], (const float*)h->modules[k - 1].seed.p, lr_lambda,
           (float*)x_inout[k - 1], nullptr, A.loss_acc, n / 4);
     else
-      distill_seed_kernel<bf16><<<grid_for(n / 8, 256, g_dev.sm_count, 8), 256, 0, st>>>(
+      distill_seed_kernel<bf16><<<grid_for(n / 8, 256, cur_dev().sm_count, 8), 256, 0, st>>>(
           (const bf16*)x_inout[k - 1], (const bf16*)dx[k], (const bf16*)h->modules[k - 1].seed.p, lr_lambda,
           (bf16*)x_inout[k - 1], nullptr, A.loss_acc, n / 8);
     h->launches++;
@@ -2005,6 +2051,27 @@ int lp_last_device_status(lp_handle* h, void* stream) {
   if (e) {
     cudaMemset(h->dev_err, 0, sizeof(int));
     return LP_ERR_DEVICE_TIMEOUT;
+  }
+  return LP_OK;
+}
+
+int lp_selftest_bounded_wait(lp_handle* h, double limit_ms, double* waited_ms, void* stream) {
+  if (!h) return LP_ERR_NULL;
+  if (!(limit_ms > 0.0) || limit_ms > 100.0) return LP_ERR_SIZE;
+  int dev = 0, khz = 0;
+  LP_CUDA_OK(cudaGetDevice(&dev));
+  LP_CUDA_OK(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev));
+  const long long limit_cycles = (long long)(limit_ms * (double)khz);
+  cudaStream_t st = (cudaStream_t)stream;
+  long long* waited = reinterpret_cast<long long*>(h->dev_err + 2);   // the error word's 256-byte slot
+  tc::bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(limit_cycles, h->dev_err, waited);
+  h->launches++;
+  LP_CUDA_OK(cudaGetLastError());
+  if (waited_ms) {
+    LP_CUDA_OK(cudaStreamSynchronize(st));
+    long long w = 0;
+    LP_CUDA_OK(cudaMemcpy(&w, waited, sizeof(w), cudaMemcpyDeviceToHost));
+    *waited_ms = (double)w / (double)khz;
   }
   return LP_OK;
 }
@@ -2110,7 +2177,7 @@ int lp_conv2d(int op, int dtype, int impl, int N, int H, int W, int Cin, int Cou
   if (N < 1 || H < 1 || W < 1 || Cin < 1 || Cout < 1 || R < 1 || stride < 1 || pad < 0) return LP_ERR_SIZE;
   if (scratch_bytes < lp_conv2d_scratch_bytes(Cin, Cout, R)) return LP_ERR_WORKSPACE;
   if (!aligned16(a) || !aligned16(b) || !aligned16(out) || (reinterpret_cast<uintptr_t>(scratch) & 255)) return LP_ERR_ALIGN;
-  int rc = g_dev.init();
+  int rc = init_cur_dev();
   if (rc != LP_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   ConvDef c;
@@ -2133,7 +2200,7 @@ int lp_conv2d(int op, int dtype, int impl, int N, int H, int W, int Cin, int Cou
       PackEntry* dpe = (PackEntry*)(sp + 256 + 2 * align_up(n * 2, 256));
       LP_CUDA_OK(cudaMemcpyAsync(dpe, &pe, sizeof(pe), cudaMemcpyHostToDevice, st));
       LP_CUDA_OK(cudaStreamSynchronize(st));
-      pack_weights_kernel<<<grid_for((long long)n, 256, g_dev.sm_count, 8), 256, 0, st>>>(dpe, 1, (long long)n);
+      pack_weights_kernel<<<grid_for((long long)n, 256, cur_dev().sm_count, 8), 256, 0, st>>>(dpe, 1, (long long)n);
       LP_CUDA_OK(cudaGetLastError());
     } else {
       c.wf = nullptr; c.wt = nullptr;
@@ -2155,10 +2222,10 @@ int lp_conv2d(int op, int dtype, int impl, int N, int H, int W, int Cin, int Cou
       const long long elems = (long long)N * c.OH * c.OW * Cout;
       if (!threads) rc = LP_ERR_UNSUPPORTED;
       else if (dtype == LP_F32)
-        bn_stats_kernel<float><<<grid_for(elems / 4, threads * 8, g_dev.sm_count, 4), threads, (size_t)threads * 8 * 4, st>>>(
+        bn_stats_kernel<float><<<grid_for(elems / 4, threads * 8, cur_dev().sm_count, 4), threads, (size_t)threads * 8 * 4, st>>>(
             (const float*)out, elems / 4, Cout, stats);
       else
-        bn_stats_kernel<bf16><<<grid_for(elems / 8, threads * 8, g_dev.sm_count, 4), threads, (size_t)threads * 16 * 4, st>>>(
+        bn_stats_kernel<bf16><<<grid_for(elems / 8, threads * 8, cur_dev().sm_count, 4), threads, (size_t)threads * 16 * 4, st>>>(
             (const bf16*)out, elems / 8, Cout, stats);
     }
   } else if (op == LP_CONV_DGRAD) {
@@ -2200,7 +2267,7 @@ int lp_conv2d_fwd_noalloc(int N, int H, int W, int Cin, int Cout, int R, int str
   const size_t n = (size_t)Cin * Cout * R * R;
   const size_t need = 256 + align_up(n * 2, 256) + 256;  // error word | bf16 weights | one-entry table
   if (need > (size_t)LP_NOALLOC_SCRATCH_BYTES) return LP_ERR_SIZE;
-  int rc = g_dev.init();
+  int rc = init_cur_dev();
   if (rc != LP_OK) return rc;
   int dev = 0;
   LP_CUDA_OK(cudaGetDevice(&dev));
@@ -2227,7 +2294,7 @@ int lp_conv2d_fwd_noalloc(int N, int H, int W, int Cin, int Cout, int R, int str
   LP_CUDA_OK(cudaMemsetAsync(dev_err, 0, 4, st));  // the only word that must start at zero
   LP_CUDA_OK(cudaMemcpyAsync(dpe, &pe, sizeof(pe), cudaMemcpyHostToDevice, st));
   LP_CUDA_OK(cudaStreamSynchronize(st));
-  pack_weights_kernel<<<grid_for((long long)n, 256, g_dev.sm_count, 8), 256, 0, st>>>(dpe, 1, (long long)n);
+  pack_weights_kernel<<<grid_for((long long)n, 256, cur_dev().sm_count, 8), 256, 0, st>>>(dpe, 1, (long long)n);
   LP_CUDA_OK(cudaGetLastError());
   bool done = false;
   rc = conv_forward(nullptr, LP_BF16, LP_CONV_IMPL_TENSOR, c, N, x, y, nullptr, nullptr, &done, dev_err, st);

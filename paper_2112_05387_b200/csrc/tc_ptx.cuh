@@ -34,14 +34,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 
 // Bounded wait.  `abort_flag` (shared) lets one role's failure release the others quickly.
 constexpr long long kWaitLimitCycles = 600000000LL;  // about 0.3 s at 1.9 GHz
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   int polls = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++polls & 63) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) return false;
+      if (clock64() - t0 > limit_cycles) return false;
     }
   }
   return true;
@@ -208,6 +209,26 @@ __host__ __device__ __forceinline__ uint32_t instr_desc_bf16(int M, int N, int a
 }
 __host__ __device__ __forceinline__ uint32_t swizzle_code_for_row_bytes(int row_bytes) {
   return row_bytes == 128 ? 2u : (row_bytes == 64 ? 4u : 6u);
+}
+
+// Self-test of the bounded wait: one thread waits, for at most `limit_cycles`, on a barrier that nothing
+// ever arrives on; the wait runs out, the kernel records that in *err exactly as the convolution kernels
+// do, and returns.  *waited receives the cycles spent.
+__global__ void bounded_wait_selftest_kernel(long long limit_cycles, int* err, long long* waited) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const long long t0 = clock64();
+    const bool ok = mbar_wait(&bar, 0, &abort_flag, limit_cycles);
+    if (waited) *waited = clock64() - t0;
+    if (!ok) atomicExch(err, 1);
+  }
 }
 
 }  // namespace tc

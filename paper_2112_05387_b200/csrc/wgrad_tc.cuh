@@ -513,7 +513,7 @@ static int wg_encode_wnh(WgEncodeFn enc, CUtensorMap* m, const void* base, int N
 }
 
 // Returns 1 when the shape is not one the halo kernel takes (the caller then uses wgrad_tc_kernel).
-static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, const bf16* x, const bf16* dy, float* dw, int N, int H, int W,
+static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, bool* attr_done, const bf16* x, const bf16* dy, float* dw, int N, int H, int W,
                              int Cin, int Cout, int* dev_err, cudaStream_t st) {
   if (W % 8 || Cin < 64) return 1;
   tc::WgradParams p;
@@ -607,21 +607,20 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, const bf16* x, const 
       p.epi_bufs = fit & ~1;
   }
   size_t smem = std::max((size_t)stages * p.stage_bytes + tail, (size_t)120 * 1024);
-  static bool attr_set = false;
-  if (!attr_set) {
+  if (!*attr_done) {   // per device
     if (cudaFuncSetAttribute(tc::wgrad_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
       return -8;
-    attr_set = true;
+    *attr_done = true;
   }
   dim3 grid(tiles, p.splits);
   return launch_pdl(tc::wgrad_halo_kernel, grid, dim3(224), smem, st, tmX, tmDY, tmDW, p) == cudaSuccess ? 0 : -8;
 }
 
-static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf16* dy, float* dw, int N, int H, int W,
-                           int Cin, int OH, int OW, int Cout, int R, int stride, int pad, int* dev_err,
-                           cudaStream_t st) {
+static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, bool* attr_done, bool* halo_attr_done, const bf16* x,
+                           const bf16* dy, float* dw, int N, int H, int W, int Cin, int OH, int OW, int Cout, int R,
+                           int stride, int pad, int* dev_err, cudaStream_t st) {
   if (R == 3 && stride == 1 && pad == 1) {
-    const int rc = launch_wgrad_halo(enc, sm_count, x, dy, dw, N, H, W, Cin, Cout, dev_err, st);
+    const int rc = launch_wgrad_halo(enc, sm_count, halo_attr_done, x, dy, dw, N, H, W, Cin, Cout, dev_err, st);
     if (rc != 1) return rc;
   }
   tc::WgradParams p;
@@ -724,11 +723,10 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, const bf16* x, const bf
       p.epi_bufs = p.rpt;
   }
   size_t smem = std::max((size_t)stages * p.stage_bytes + tail, (size_t)120 * 1024);
-  static bool attr_set = false;
-  if (!attr_set) {
+  if (!*attr_done) {   // per device
     if (cudaFuncSetAttribute(tc::wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
       return -8;
-    attr_set = true;
+    *attr_done = true;
   }
   dim3 grid(tiles, p.splits);
   return launch_pdl(tc::wgrad_tc_kernel, grid, dim3(224), smem, st, tmX, tmDY, tmDW, p) == cudaSuccess ? 0 : -8;

@@ -1,4 +1,7 @@
 """Helpers shared by the GPU parity tests: run a workload through the C ABI and through the oracle."""
+import json
+import os
+
 import numpy as np
 
 from oracle import lp_oracle as O
@@ -138,6 +141,46 @@ def noisy_bf16_store(seed=1234, eps=1e-7):
         a = np.asarray(a, dtype=np.float64)
         return gen.round_bf16(a * (1.0 + eps * rng.standard_normal(a.shape)))
     return store
+
+
+# Noise seeds of the floor: the floor of a tensor is the LARGEST change over these runs.
+NOISE_SEEDS = (1234, 4321, 777)
+# No tensor of a bf16 workload may be further from the oracle than this, whatever its floor.
+ALLOWANCE_CAP = 0.10
+
+
+def allowance(tol, floor):
+    """Largest relative L2 error accepted for a tensor of a bf16 workload: the stated tolerance, widened to
+    twice the tensor's own noise floor where that is larger, and never beyond ALLOWANCE_CAP."""
+    return max(tol, min(2.0 * floor, ALLOWANCE_CAP))
+
+
+def log_parity(**rec):
+    """Append one record (tensor, error, floor, allowance) to the file named by LP_PARITY_LOG, if set."""
+    path = os.environ.get("LP_PARITY_LOG")
+    if not path:
+        return
+    rec["test"] = os.environ.get("PYTEST_CURRENT_TEST", "").split(" ")[0]
+    with open(path, "a") as f:
+        f.write(json.dumps(rec) + "\n")
+
+
+def noise_floors(run, xs_host, ref, kappas=None, params=None):
+    """Per module: the noise floor of every gradient tensor, of the whole gradient and of dx -- the largest
+    relative change between the storage-model oracle `ref` and runs of the same oracle that differ only by
+    rounding-level noise before each bf16 rounding (one run per seed in NOISE_SEEDS)."""
+    net = run.net
+    floors = [dict(grads={}, whole=0.0, dx=0.0) for _ in range(net.K)]
+    for seed in NOISE_SEEDS:
+        noisy = oracle_modules(run, xs_host, kappas=kappas, params=params, store=noisy_bf16_store(seed))
+        for k in range(net.K):
+            per = per_tensor_errors(net, k, noisy[k]["grads"], ref[k]["grads"])
+            for n, e in per.items():
+                floors[k]["grads"][n] = max(floors[k]["grads"].get(n, 0.0), e)
+            floors[k]["whole"] = max(floors[k]["whole"], rel_err(noisy[k]["grads"], ref[k]["grads"]))
+            if ref[k]["dx"] is not None:
+                floors[k]["dx"] = max(floors[k]["dx"], rel_err(noisy[k]["dx"], ref[k]["dx"]))
+    return floors
 
 
 def oracle_modules(run, xs_host, kappas=None, params=None, exact=False, store=None):

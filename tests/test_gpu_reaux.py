@@ -5,7 +5,8 @@ import numpy as np
 import pytest
 
 from conftest import small_cfg
-from harness import GpuRun, oracle_modules, per_tensor_errors, rel_err, to_host
+from harness import (GpuRun, NOISE_SEEDS, allowance, log_parity, noisy_bf16_store, oracle_modules, per_tensor_errors, rel_err,
+                     to_dev, to_host)
 from oracle import lp_oracle as O
 from workloads import gen
 
@@ -94,31 +95,58 @@ def test_reauxnet_distillation_matches_oracle(mk, tol, lr_lambda=0.05, lr_aux=0.
             assert rel_err(after, newp[k - 1][j]) < tol, (k, j)
 
 
-def test_reauxnet_distillation_bf16_runs_and_updates_every_unit():
+def test_reauxnet_distillation_bf16_matches_the_storage_model_oracle():
+    """bf16: boundaries from the oracle's stacks, dx from the oracle's module passes; losses within 2e-2 (twice
+    that for the squared distillation loss), every gradient tensor of every unit within max(2e-2, min(2 x floor,
+    0.10)), the floor taken from noisy runs of the oracle's own distillation pass."""
     cfg = cfg_bf16()
     run = GpuRun(cfg, aux_recursive=True)
     net, lp, torch = run.net, run.lp, run.torch
     K = net.K
-    xs_host = run.auxnet()
+    images = run.images.astype(np.float64)
+    net.store = gen.round_bf16
+    ox = O.reauxnet_forward(net, run.stacks, images)
+    net.store = None
+    gx = run.auxnet()                   # the stacks' kept activations
+    for k in range(1, K):
+        assert rel_err(gx[k - 1], ox[k - 1]) < 2e-2
+    run.set_boundaries(ox)
+    xs_host = [to_host(t) for t in run.d_x[1:]]
     run.fwd_bwd_all()
     ref = oracle_modules(run, xs_host)
+    d_dx = [None] + [to_dev(ref[k]["dx"], cfg) for k in range(1, K)]
     d_loss = torch.zeros(K - 1, dtype=torch.float32, device="cuda:0")
-    lp.lp_auxnet_distill(run.h, run.d_images, run.d_x[1:], run.d_dx, 0.05, 0.01, None, d_loss)
+    lr_lambda, lr_aux = 0.05, 0.01
+    lp.lp_auxnet_distill(run.h, run.d_images, run.d_x[1:], d_dx, lr_lambda, lr_aux, None, d_loss)
     assert lp.lp_last_device_status(run.h) == 0
     net.store = gen.round_bf16
-    _, _, losses, grads = O.reauxnet_distill_step(net, run.stacks, run.images.astype(np.float64), xs_host,
-                                                 [r["dx"] for r in ref[1:]], [r["seed"] for r in ref[:-1]], 0.05, 0.01)
+    _, newx, losses, grads = O.reauxnet_distill_step(net, run.stacks, images, xs_host, [r["dx"] for r in ref[1:]],
+                                                    [r["seed"] for r in ref[:-1]], lr_lambda, lr_aux)
     net.store = None
+    floors = {}
+    for seed in NOISE_SEEDS:
+        net.store = noisy_bf16_store(seed)
+        try:
+            for k in range(1, K):
+                res = O.reauxnet_fwd_bwd(net, k, run.stacks[k - 1], images, newx[k - 1])
+                for j in range(k):
+                    for n, e in per_tensor_errors(net, O.LP_AUX(j), res["grads"][j], grads[k - 1][j]).items():
+                        floors[(k, j, n)] = max(floors.get((k, j, n), 0.0), e)
+        finally:
+            net.store = None
     got_loss = d_loss.cpu().numpy()
+    bad = []
     for k in range(1, K):
-        # the loss depends on dx and the seeds of the modules, both compared elsewhere at 2e-2 plus their noise floor
-        assert abs(got_loss[k - 1] - losses[k - 1]) < 0.15 * losses[k - 1], (k, got_loss[k - 1], losses[k - 1])
+        assert abs(got_loss[k - 1] - losses[k - 1]) < 4e-2 * losses[k - 1], (k, got_loss[k - 1], losses[k - 1])
         for j in range(k):
             g = lp.lp_get_grads(run.h, lp.LP_REAUX(k, j)).astype(np.float64)
-            assert np.all(np.isfinite(g)) and np.linalg.norm(g) > 0
-            # direction of the whole-unit gradient against the storage-model oracle
-            cos = float(g @ grads[k - 1][j]) / (np.linalg.norm(g) * np.linalg.norm(grads[k - 1][j]))
-            assert cos > 0.9, (k, j, cos)
+            for n, e in per_tensor_errors(net, O.LP_AUX(j), g, grads[k - 1][j]).items():
+                a = allowance(2e-2, floors[(k, j, n)])
+                log_parity(workload=cfg["name"] + " (recursive distillation)", dtype="bf16", module="stack%d/unit%d" % (k, j),
+                           tensor=n, err=e, floor=floors[(k, j, n)], allowed=a)
+                if not e < a:
+                    bad.append((k, j, n, e, floors[(k, j, n)], a))
+    assert not bad, bad
 
 
 def test_fused_step_in_recursive_form_equals_separate_calls():

@@ -46,7 +46,7 @@ def test_single_rank_is_identity():
     assert bench.whole_job_images_per_s(64, 10, 1, 100.0) == 6400.0
 
 
-def test_flop_accounting_matches_survey_figures():
+def test_flop_accounting_of_the_named_workloads():
     """Forward conv FLOPs per image: 10.49 G (WRN-28-10), 0.2515 G (ResNet-56), 7.33 G (ResNet-34)."""
     import bench
     from workloads import get_config

@@ -47,6 +47,25 @@ def test_noalloc_forward_matches_lp_conv2d_twice_in_a_row():
     assert _both((2, 8, 8, 128, 64, 1, 1, 0), seed=3) < 6e-3
 
 
+def test_noalloc_forward_matches_the_cpu_oracle():
+    """One case against the plain definition of the convolution (the oracle), not only against lp_conv2d."""
+    import torch
+    import paper_2112_05387_b200 as lp
+    from oracle import lp_oracle as O
+    from workloads import gen
+    N, H, W, Cin, Cout, R, stride, pad = 3, 12, 12, 32, 48, 3, 1, 1
+    x = gen.round_bf16(gen.normal(11, "x", (N, H, W, Cin)))
+    w = gen.round_bf16(gen.normal(11, "w", (Cout, R, R, Cin), std=(2.0 / (R * R * Cin)) ** 0.5))
+    dx = torch.from_numpy(x).to("cuda:0").to(torch.bfloat16)
+    dw = torch.from_numpy(w).to("cuda:0")
+    y = torch.zeros(N, H, W, Cout, device="cuda:0", dtype=torch.bfloat16)
+    assert lp.lp_conv2d_fwd_noalloc(N, H, W, Cin, Cout, R, stride, pad, dx, dw, y) == 0
+    torch.cuda.synchronize()
+    ref = O.conv_fwd(x.astype(np.float64), w.astype(np.float64), stride, pad)
+    got = y.float().cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < 6e-3
+
+
 def test_noalloc_rejects_what_does_not_fit_or_is_not_supported():
     import torch
     import paper_2112_05387_b200 as lp
