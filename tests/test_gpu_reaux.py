@@ -98,7 +98,7 @@ def test_reauxnet_distillation_matches_oracle(mk, tol, lr_lambda=0.05, lr_aux=0.
 def test_reauxnet_distillation_bf16_matches_the_storage_model_oracle():
     """bf16: boundaries from the oracle's stacks, dx from the oracle's module passes; losses within 2e-2 (twice
     that for the squared distillation loss), every gradient tensor of every unit within max(2e-2, min(2 x floor,
-    0.10)), the floor taken from noisy runs of the oracle's own distillation pass."""
+    0.20)), the floor taken from noisy runs of the oracle's own distillation pass."""
     cfg = cfg_bf16()
     run = GpuRun(cfg, aux_recursive=True)
     net, lp, torch = run.net, run.lp, run.torch
