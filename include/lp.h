@@ -70,6 +70,13 @@ enum { LP_CONV_NO_TENSOR_FWD = 16, LP_CONV_NO_TENSOR_DGRAD = 32, LP_CONV_NO_TENS
  * arithmetic, same results; with the present row-per-thread epilogue it is the slower of the two
  * (the extra operands are read and written in 16-byte pieces), hence off by default. */
 enum { LP_CONV_LOSS_IN_EPILOGUE = 128 };
+/* The tensor-core forward / input-gradient kernel has two epilogues with the same results: "direct" (bf16
+ * stores from registers) and "staged" (the tile goes through shared memory and leaves by TMA tile stores;
+ * a residual operand arrives by TMA loads a tile ahead and is added in place).  By default a convolution
+ * with a residual operand takes the staged one where it applies (measured faster there: the residual is no
+ * longer read in 16-byte pieces 2*C_out bytes apart) and every other convolution the direct one.  These
+ * flags, OR-ed into conv_impl, force one or the other wherever it applies (comparisons, tests). */
+enum { LP_CONV_DIRECT_EPILOGUE = 256, LP_CONV_STAGED_EPILOGUE = 512 };
 enum { LP_CONV_FWD = 0, LP_CONV_DGRAD = 1, LP_CONV_WGRAD = 2 };
 
 #define LP_MAX_STAGES 8

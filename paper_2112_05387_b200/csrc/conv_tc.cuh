@@ -94,6 +94,8 @@ struct ConvTcParams {
   float rho;
   double* loss_acc;              // [2]: sum r^2, sum kappa*r (atomically added)
   int wide32;                    // output (and residual) rows can be accessed in 32-byte pieces
+  // staged epilogue (kStaged instantiations): the output tile goes through shared memory and leaves by TMA
+  uint32_t stage_offset;         // staging region: one 128-row x 64-byte group per 32 output channels of the tile
 };
 
 struct TcSmemTail {
@@ -103,13 +105,19 @@ struct TcSmemTail {
   uint64_t empty_b[kMaxStages];
   uint64_t tmem_full[kMaxSlots];
   uint64_t tmem_empty[kMaxSlots];
+  uint64_t add_full;               // staged epilogue: the residual tile has landed in the staging region
   uint32_t tmem_base;
   int abort_flag;
   int epi_ok[2];                   // outcome of the epilogue's wait, alternating by accumulator (see the epilogue)
+};
+// Scratch of the direct (register -> global) epilogue's statistics, placed right after the tail.
+struct TcStatScratch {
   float ssum[LP_EPI_WARPS][256];   // per epilogue warp: plain read-modify-write, no shared-memory atomics
   float ssq[LP_EPI_WARPS][256];
   uint32_t tr[LP_EPI_WARPS][16 * 33];   // per epilogue warp: transposition scratch of the statistics
 };
+constexpr uint32_t kTailBytes = (uint32_t)((sizeof(TcSmemTail) + 127) / 128 * 128);
+constexpr uint32_t kStageGroupBytes = 128 * 64;   // staging: 128 tile rows x 32 bf16 channels
 
 // 32-byte global accesses (sm_100: 256-bit vector loads and stores); the address must be 32-byte aligned.
 __device__ __forceinline__ void st_global_32B(void* p, const uint32_t* v) {
@@ -130,14 +138,23 @@ constexpr int kFirstEpiWarp = 3;
 constexpr int kEpiGroups = LP_EPI_WARPS / 4;
 
 // kAddend: a residual operand is added in the epilogue (its loads run one channel group ahead);
-// kLoss: the epilogue also takes the local loss of an interior module (implies kAddend).
-template <bool kLoss, bool kAddend>
+// kLoss: the epilogue also takes the local loss of an interior module (implies kAddend);
+// kStaged: the epilogue writes the bf16 tile into shared memory (64-byte swizzled rows of 32 channels)
+//   and one thread sends it to global memory with TMA tile stores; the residual tile, when there is
+//   one, arrives in the same region by TMA loads issued a tile ahead and is added in place.  Global
+//   memory then sees whole 64-byte row pieces written by the copy engine instead of 16- or 32-byte
+//   stores 2 x C_out bytes apart across the lanes of a warp, and the per-channel statistics are column
+//   sums over the staged tile.  tmOut / tmAdd are only read by these instantiations.
+template <bool kLoss, bool kAddend, bool kStaged>
 __global__ void __launch_bounds__(kConvThreads, LP_CONV_MIN_BLOCKS)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmAdd,
                const __grid_constant__ ConvTcParams p) {
+  static_assert(!(kStaged && kLoss), "the fused local loss uses the direct epilogue");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   TcSmemTail* tail = reinterpret_cast<TcSmemTail*>(smem + p.tail_offset);
+  TcStatScratch* scratch = reinterpret_cast<TcStatScratch*>(smem + p.tail_offset + kTailBytes);
   volatile int* abort_flag = &tail->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -156,14 +173,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(&tail->tmem_full[b], 1);
       mbar_init(&tail->tmem_empty[b], kEpiThreads / 32);
     }
+    mbar_init(&tail->add_full, 1);
     tail->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
+    if constexpr (kStaged) {
+      prefetch_tmap(&tmOut);
+      if constexpr (kAddend) prefetch_tmap(&tmAdd);
+    }
   }
-  for (int i = threadIdx.x; i < LP_EPI_WARPS * 256; i += blockDim.x) {
-    (&tail->ssum[0][0])[i] = 0.f;
-    (&tail->ssq[0][0])[i] = 0.f;
+  if constexpr (!kStaged) {
+    for (int i = threadIdx.x; i < LP_EPI_WARPS * 256; i += blockDim.x) {
+      (&scratch->ssum[0][0])[i] = 0.f;
+      (&scratch->ssq[0][0])[i] = 0.f;
+    }
   }
   if (warp == kFirstEpiWarp) {
     tmem_alloc(&tail->tmem_base, kTmemCols);
@@ -361,6 +385,168 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       t += cnt;
     }
   } else {
+    if constexpr (kStaged) {
+    // ------------------------------- epilogue, staged through shared memory -------------
+    // Requires (checked by the launcher): output grid = logical grid (os = 1), channel tile a multiple
+    // of 32, kEpiThreads = 128.  Thread `row` owns tile row `row` (one pixel) as in the direct epilogue.
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const int et = threadIdx.x - 32 * kFirstEpiWarp;
+    const int rows_used = p.BW * p.BH * p.BNI;
+    const int ngroups = p.n_tile_cols >> 5;
+    uint8_t* stg = smem + p.stage_offset;
+    // 64-byte swizzle of the staging rows, as the TMA unit applies it: 16-byte piece index ^= address bits 7..8
+    uint8_t* my_row = stg + row * 64;
+    const uint32_t swz = (uint32_t)((row >> 1) & 3);
+    uint32_t slot = 0, slot_phase = 0, add_phase = 0;
+    int epi_turn = 0;
+    // per-channel statistics: thread (group sg, word sw) owns two channels and sums them over the rows
+    const int sg = et >> 4, sw = et & 15;
+    const bool stat_owner = p.stats != nullptr && sg < ngroups;
+    float st_s0 = 0.f, st_s1 = 0.f, st_q0 = 0.f, st_q1 = 0.f;
+    auto tile_origin = [&](int tile, int& col0, int& c1, int& c2, int& c3) {
+      const int nt = tile / p.m_tiles, m = tile % p.m_tiles;
+      const int w0 = (m % p.tiles_w) * p.BW;
+      const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
+      const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
+      col0 = nt * p.n_tile_cols;
+      c1 = w0;
+      c2 = p.halo ? n0 : h0;      // box dimension order (C, W, image, H) in halo mode, (C, W, H, image) otherwise
+      c3 = p.halo ? h0 : n0;
+    };
+    auto load_addend_tile = [&](int tile) {   // elected thread only
+      int col0, c1, c2, c3;
+      tile_origin(tile, col0, c1, c2, c3);
+      mbar_expect_tx(&tail->add_full, (uint32_t)(ngroups * rows_used * 64));
+      for (int g = 0; g < ngroups; ++g)
+        tma_load_4d(stg + g * kStageGroupBytes, &tmAdd, &tail->add_full, col0 + 32 * g, c1, c2, c3);
+    };
+    auto flush_stats = [&](int col0) {
+      if (stat_owner) {
+        const int c = col0 + sg * 32 + 2 * sw;
+        if (c < p.Cout) {
+          atomicAdd(&p.stats[c], (double)st_s0);
+          atomicAdd(&p.stats[p.Cout + c], (double)st_q0);
+        }
+        if (c + 1 < p.Cout) {
+          atomicAdd(&p.stats[c + 1], (double)st_s1);
+          atomicAdd(&p.stats[p.Cout + c + 1], (double)st_q1);
+        }
+      }
+      st_s0 = st_s1 = st_q0 = st_q1 = 0.f;
+    };
+    if constexpr (kAddend) {
+      if (et == 0 && t_begin < t_end) load_addend_tile(t_begin);
+    }
+    for (int t = t_begin; t < t_end && !failed;) {
+      const int nt = t / p.m_tiles, m0 = t % p.m_tiles;
+      const int cnt = (p.mpair == 2 && t + 1 < t_end && m0 + 1 < p.m_tiles) ? 2 : 1;
+      for (int a = 0; a < cnt && !failed; ++a) {
+        const int tile = t + a;
+        const int m = m0 + a;
+        const uint32_t buf = slot;
+        const int w0 = (m % p.tiles_w) * p.BW;
+        const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
+        const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
+        const int ow = w0 + row % p.BW;
+        const int oh = h0 + (p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH);
+        const int n = n0 + (p.halo ? (row / p.BW) % p.BNI : row / (p.BW * p.BH));
+        const bool valid = row < rows_used && ow < p.OWl && oh < p.OHl && n < p.Nimg;
+        // One thread waits (bounded) for the accumulator, for the residual tile, and until the stores of
+        // the previous tile have read the staging region; all epilogue threads then agree on the outcome.
+        if (et == 0) {
+          bool ok = mbar_wait(&tail->tmem_full[buf], (slot_phase >> buf) & 1, abort_flag);
+          if constexpr (kAddend) ok = mbar_wait(&tail->add_full, add_phase, abort_flag) && ok;
+          else bulk_wait_read(0);
+          tail->epi_ok[epi_turn] = ok ? 1 : 0;
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+        const int wait_ok = *(volatile int*)&tail->epi_ok[epi_turn];
+        epi_turn ^= 1;
+        add_phase ^= 1;
+        if (!wait_ok) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + buf * p.acc_stride + ((uint32_t)(q * 32) << 16);
+        constexpr int kBatch = LP_EPI_BATCH;
+        for (int g0 = 0; g0 < ngroups; g0 += kBatch) {
+          uint32_t raw[kBatch][32];
+#pragma unroll
+          for (int i = 0; i < kBatch; ++i)
+            if (g0 + i < ngroups) tmem_ld32_issue(taddr + (g0 + i) * 32, raw[i]);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < kBatch; ++i) tmem_ld_fence(raw[i]);
+          if (g0 + kBatch >= ngroups) {      // the accumulator is in registers: hand the slot back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tail->tmem_empty[buf]);
+          }
+#pragma unroll
+          for (int i = 0; i < kBatch; ++i) {
+            const int g = g0 + i;
+            if (g >= ngroups) continue;
+            uint8_t* grow = my_row + g * kStageGroupBytes;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              uint4* dst = reinterpret_cast<uint4*>(grow + ((u ^ swz) << 4));
+              float v[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) v[j] = valid ? __uint_as_float(raw[i][8 * u + j]) : 0.f;
+              if constexpr (kAddend) {
+                float f[8];
+                cvt_raw(*dst, f);     // residual piece (zero where the tile leaves the tensor)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] += f[j];
+              }
+              if (row < rows_used)
+                *dst = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+                                  pack_bf16x2(v[6], v[7]));
+            }
+          }
+        }
+        fence_proxy_async();     // the staged tile is read by the copy engine
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+        if (et == 0) {
+          int col0, c1, c2, c3;
+          tile_origin(tile, col0, c1, c2, c3);
+          for (int g = 0; g < ngroups; ++g)
+            tma_store_4d(&tmOut, stg + g * kStageGroupBytes, col0 + 32 * g, c1, c2, c3);
+          bulk_commit_group();
+        }
+        if (stat_owner) {
+          // Statistics of the tensor as stored (bf16).  Lanes 0-15 and 16-31 of a warp read different
+          // groups at the same offset: the second half walks the rows in swapped pairs so that the two
+          // halves touch different 64-byte halves of a 128-byte line of banks.
+          const uint8_t* gbase = stg + sg * kStageGroupBytes;
+          const int flip = sg & 1;
+          for (int r = 0; r < rows_used; ++r) {
+            int rr = r ^ flip;
+            if (rr >= rows_used) rr = r;
+            const uint32_t w2 = *reinterpret_cast<const uint32_t*>(
+                gbase + rr * 64 + ((((uint32_t)sw >> 2) ^ ((uint32_t)(rr >> 1) & 3)) << 4) + ((sw & 3) << 2));
+            const float lo = __uint_as_float(w2 << 16), hi = __uint_as_float(w2 & 0xFFFF0000u);
+            st_s0 += lo; st_s1 += hi;
+            st_q0 = fmaf(lo, lo, st_q0); st_q1 = fmaf(hi, hi, st_q1);
+          }
+        }
+        if constexpr (kAddend) {
+          // the next residual tile may overwrite the staging region once the stores have read it and the
+          // statistics above are done with it
+          if (p.stats) asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+          if (et == 0) {
+            bulk_wait_read(0);
+            if (tile + 1 < t_end) load_addend_tile(tile + 1);
+          }
+        }
+        slot_phase ^= 1u << buf;
+        slot = slot + 1 == (uint32_t)p.nslots ? 0 : slot + 1;
+        const bool last_of_unit = a + 1 == cnt;
+        if (p.stats && last_of_unit && (t + cnt >= t_end || (t + cnt) / p.m_tiles != nt)) flush_stats(nt * p.n_tile_cols);
+      }
+      t += cnt;
+    }
+    if (et == 0) bulk_wait_read(0);   // shared memory must outlive the last stores' reads
+    } else {
     // ------------------------------- epilogue -----------------------------------------
     const int q = warp & 3;              // TMEM lane quarter this warp may read
     const int grp = (warp - kFirstEpiWarp) >> 2;  // which warp of the quarter (more than four epilogue warps)
@@ -535,7 +721,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               // the sums run over pixels, so the warp transposes through shared memory: every lane
               // writes its 16 channel pairs, then lane l sums channel pair (l & 15) over 16 of the
               // warp's 32 pixels (both phases conflict-free with the row pitch of 33 words).
-              uint32_t* T = tail->tr[warp - kFirstEpiWarp];
+              uint32_t* T = scratch->tr[warp - kFirstEpiWarp];
 #pragma unroll
               for (int j = 0; j < 16; ++j) T[j * 33 + lane] = (valid && (wide || j < 8)) ? pk[j] : 0u;
               __syncwarp();
@@ -554,7 +740,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               s1 += __shfl_xor_sync(0xffffffffu, s1, 16);
               q0 += __shfl_xor_sync(0xffffffffu, q0, 16);
               q1 += __shfl_xor_sync(0xffffffffu, q1, 16);
-              float* dst = hh ? tail->ssq[warp - kFirstEpiWarp] : tail->ssum[warp - kFirstEpiWarp];
+              float* dst = hh ? scratch->ssq[warp - kFirstEpiWarp] : scratch->ssum[warp - kFirstEpiWarp];
               dst[c_in_tile + 2 * jc] += hh ? q0 : s0;
               dst[c_in_tile + 2 * jc + 1] += hh ? q1 : s1;
             }
@@ -570,10 +756,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int c = et; c < p.n_tile_cols; c += kEpiThreads) {
             float a_s = 0.f, a_q = 0.f;
             for (int wi = 0; wi < kEpiThreads / 32; ++wi) {
-              a_s += tail->ssum[wi][c];
-              a_q += tail->ssq[wi][c];
-              tail->ssum[wi][c] = 0.f;
-              tail->ssq[wi][c] = 0.f;
+              a_s += scratch->ssum[wi][c];
+              a_q += scratch->ssq[wi][c];
+              scratch->ssum[wi][c] = 0.f;
+              scratch->ssq[wi][c] = 0.f;
             }
             if (col0 + c < p.Cout) {
               atomicAdd(&p.stats[col0 + c], (double)a_s);
@@ -594,6 +780,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         atomicAdd(&p.loss_acc[1], (double)sum_kr);
       }
     }
+    }   // direct epilogue
   }
 
   if (failed) {

@@ -68,7 +68,6 @@ __global__ void bn_stats_kernel(const T* __restrict__ x, long long total_vecs, i
   constexpr int V = VecT<T>::N;
   extern __shared__ float sm[];  // [blockDim][2*V]
   const int CV = C / V;
-  const int cg = threadIdx.x % CV;
   float s[V], q[V];
 #pragma unroll
   for (int j = 0; j < V; ++j) s[j] = q[j] = 0.f;

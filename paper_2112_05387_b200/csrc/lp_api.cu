@@ -262,6 +262,7 @@ struct TcGemmSpec {
   double* stats;
   // local loss fused into the epilogue (interior module's last convolution); x_next == nullptr: off
   const bf16* x_next; const bf16* kappa; bf16* r_out; bf16* seed_out; float rho; double* loss_acc;
+  int epilogue;          // 0: default (staged where a residual operand exists), 1: direct, 2: staged wherever it applies
 };
 
 static void pick_pixel_box(int OWl, int OHl, int Nimg, int& BW, int& BH, int& BNI) {
@@ -328,6 +329,21 @@ static int encode_mat_map(CUtensorMap* m, const void* base, long long K, int row
   CUresult r = cur_dev().encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LP_OK : LP_ERR_CUDA;
+}
+
+// Tensor map of an NHWC bf16 tensor for the staged epilogue: boxes of 32 channels x one pixel tile, 64-byte
+// swizzled rows; `wnh` selects the dimension order (C, W, image, H) of the halo-mode tiles.
+static int encode_tile32_map(CUtensorMap* m, const void* base, int N, int H, int W, int C, int BW, int BH, int BNI,
+                             bool wnh) {
+  cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)(wnh ? N : H), (cuuint64_t)(wnh ? H : N)};
+  cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)(wnh ? (size_t)H * W * C * 2 : (size_t)W * C * 2),
+                           (cuuint64_t)(wnh ? (size_t)W * C * 2 : (size_t)H * W * C * 2)};
+  cuuint32_t box[4] = {32, (cuuint32_t)BW, (cuuint32_t)(wnh ? BNI : BH), (cuuint32_t)(wnh ? BH : BNI)};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  CUresult r = cur_dev().encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? LP_OK : LP_ERR_CUDA;
 }
 
@@ -404,7 +420,14 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   const int row_bytes = p.KC * 2;
   p.a_region_bytes = (uint32_t)align_up((size_t)128 * row_bytes, 1024);
   const uint32_t b_region = (uint32_t)align_up((size_t)p.n_tile_cols * row_bytes, 1024);
-  const size_t tail = sizeof(tc::TcSmemTail) + 1024;
+  // Staged epilogue (output tile through shared memory, TMA stores, TMA-loaded residual): where the output
+  // grid is the logical grid, the channel tile is a multiple of 32 and the tensors start on 16-byte boundaries.
+  const bool staged = (s.epilogue == 2 || (s.epilogue == 0 && s.addend != nullptr)) && !s.x_next && s.os == 1 && s.oo_h == 0 && s.oo_w == 0 &&
+                      p.n_tile_cols % 32 == 0 && s.out_C % 8 == 0 && tc::kEpiThreads == 128 &&
+                      (reinterpret_cast<uintptr_t>(s.out) & 15) == 0 &&
+                      (!s.addend || (reinterpret_cast<uintptr_t>(s.addend) & 15) == 0);
+  const size_t stage_bytes = staged ? (size_t)(p.n_tile_cols / 32) * tc::kStageGroupBytes : 0;
+  const size_t tail = tc::kTailBytes + (staged ? 0 : sizeof(tc::TcStatScratch)) + stage_bytes + 1024;
   p.tx_b = (uint32_t)(p.n_tile_cols * row_bytes);
   p.acc_stride = (p.n_tile_cols + 31) / 32 * 32;
   p.nslots = std::min(tc::kMaxSlots, tc::kTmemCols / p.acc_stride);
@@ -435,7 +458,8 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     if (fits) {
       p.a_stage_bytes = p.mpair * p.a_halo_bytes;
       p.b_ring_offset = p.nA * p.a_stage_bytes;
-      p.tail_offset = p.b_ring_offset + p.nB * p.b_stage_bytes;
+      p.stage_offset = p.b_ring_offset + p.nB * p.b_stage_bytes;
+      p.tail_offset = p.stage_offset + (uint32_t)stage_bytes;
     } else {
       p.halo = 0;
       pick_pixel_box(s.OWl, s.OHl, s.aN, p.BW, p.BH, p.BNI);
@@ -458,7 +482,8 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     stages = std::min(stages, tc::kMaxStages);
     if (stages < 2) return LP_ERR_UNSUPPORTED;
     p.stages = stages;
-    p.tail_offset = (uint32_t)(stages * p.stage_bytes);
+    p.stage_offset = (uint32_t)(stages * p.stage_bytes);
+    p.tail_offset = p.stage_offset + (uint32_t)stage_bytes;
   }
   p.idesc = tc::instr_desc_bf16(128, p.n_tile_cols, 0, 0);
   p.desc_hi = tc::smem_desc_hi(16, 8 * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
@@ -476,15 +501,30 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   if (rc != LP_OK) return rc;
   rc = encode_mat_map(&tmB, s.wmat, s.w_K, s.w_rows, p.KC, p.n_tile_cols, row_bytes);
   if (rc != LP_OK) return rc;
-  size_t smem = (size_t)p.tail_offset + tail;
+  CUtensorMap tmOut, tmAdd;
+  memset(&tmOut, 0, sizeof(tmOut));
+  memset(&tmAdd, 0, sizeof(tmAdd));
+  if (staged) {
+    rc = encode_tile32_map(&tmOut, s.out, s.aN, s.out_H, s.out_W, s.out_C, p.BW, p.BH, p.BNI, p.halo != 0);
+    if (rc != LP_OK) return rc;
+    if (s.addend) {
+      rc = encode_tile32_map(&tmAdd, s.addend, s.aN, s.out_H, s.out_W, s.out_C, p.BW, p.BH, p.BNI, p.halo != 0);
+      if (rc != LP_OK) return rc;
+    }
+  }
+  size_t smem = (size_t)p.tail_offset + (tail - stage_bytes);
   smem = std::max(smem, kTcMinSmem);
   bool& attr_set = cur_dev().conv_attr;
   if (!attr_set) {
-    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kTcMaxSmem));
-    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kTcMaxSmem));
-    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)kTcMaxSmem));
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)kTcMaxSmem));
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kTcMaxSmem));
     attr_set = true;
   }
@@ -502,9 +542,12 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   }
   if (s.x_next && !s.addend) return LP_ERR_UNSUPPORTED;   // the fused loss belongs to a convolution with a shortcut
   cudaError_t le;
-  if (s.x_next) le = launch_pdl(tc::conv_tc_kernel<true, true>, dim3(grid), dim3(tc::kConvThreads), smem, st, tmA, tmB, p);
-  else if (s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true>, dim3(grid), dim3(tc::kConvThreads), smem, st, tmA, tmB, p);
-  else le = launch_pdl(tc::conv_tc_kernel<false, false>, dim3(grid), dim3(tc::kConvThreads), smem, st, tmA, tmB, p);
+  const dim3 g3(grid), b3(tc::kConvThreads);
+  if (s.x_next) le = launch_pdl(tc::conv_tc_kernel<true, true, false>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
+  else if (staged && s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true, true>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
+  else if (staged) le = launch_pdl(tc::conv_tc_kernel<false, false, true>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
+  else if (s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true, false>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
+  else le = launch_pdl(tc::conv_tc_kernel<false, false, false>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
   LP_CUDA_OK(le);
   if (h) h->launches++;
   LP_CUDA_OK(cudaGetLastError());
@@ -578,6 +621,7 @@ static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int
     s.out = (bf16*)y; s.addend = (const bf16*)addend;
     s.out_H = c.OH; s.out_W = c.OW; s.out_C = c.cout; s.os = 1; s.oo_h = s.oo_w = 0;
     s.stats = stats;
+    s.epilogue = (impl & LP_CONV_DIRECT_EPILOGUE) ? 1 : ((impl & LP_CONV_STAGED_EPILOGUE) ? 2 : 0);
     if (loss) {
       s.x_next = (const bf16*)loss->x_next; s.kappa = (const bf16*)loss->kappa; s.r_out = (bf16*)loss->r_out;
       s.seed_out = (bf16*)loss->seed_out; s.rho = loss->rho; s.loss_acc = loss->acc;
@@ -664,6 +708,7 @@ static int conv_dgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
       s.out = (bf16*)dx; s.addend = (const bf16*)addend;
       s.out_H = c.H; s.out_W = c.W; s.out_C = c.cin; s.os = st2; s.oo_h = ph; s.oo_w = pw;
       s.stats = nullptr;
+      s.epilogue = (impl & LP_CONV_DIRECT_EPILOGUE) ? 1 : ((impl & LP_CONV_STAGED_EPILOGUE) ? 2 : 0);
       int rc = launch_conv_tc(h, s, dev_err, st);
       if (rc != LP_OK) return rc;
     }

@@ -94,15 +94,23 @@ TC_CASES = [
     (2, 56, 56, 64, 64, 3, 1, 1),     # 56-wide boxes of 2 rows
     (9, 4, 4, 64, 32, 3, 1, 1),       # 4x4 images, eight per tile, ragged last tile
     (40, 32, 32, 160, 160, 3, 1, 1),  # 320 halo tiles of 16x8 pixels: pairs, three K chunks with zero fill
+    (5, 12, 20, 64, 256, 3, 1, 1),    # 256-channel tile: eight staging groups, two passes over the accumulator; ragged boxes
+    (3, 9, 9, 32, 96, 1, 1, 0),       # odd image size, 81-pixel boxes, three staging groups
 ]
 
 
+# both epilogues of the forward / input-gradient kernel, each forced wherever it applies: tile staged in
+# shared memory and stored by TMA, and stores from registers
+EPILOGUES = {"staged": 512, "direct": 256}
+
+
+@pytest.mark.parametrize("epilogue", list(EPILOGUES))
 @pytest.mark.parametrize("case", TC_CASES)
-def test_tensor_conv_forward_matches_oracle(case):
+def test_tensor_conv_forward_matches_oracle(case, epilogue):
     import paper_2112_05387_b200 as lp
     N, H, W, Cin, Cout, R, stride, pad = case
     x, w, dy = make_case(*case, "bf16")
-    st, y, stats = run_conv(lp.LP_CONV_FWD, "bf16", lp.LP_CONV_IMPL_TENSOR, *case, x, w, want_stats=True)
+    st, y, stats = run_conv(lp.LP_CONV_FWD, "bf16", lp.LP_CONV_IMPL_TENSOR | EPILOGUES[epilogue], *case, x, w, want_stats=True)
     assert st == 0, lp.lp_status_string(st)
     ref = O.conv_fwd(x, w, stride, pad)
     assert rel_err(y, ref) < 6e-3
@@ -110,12 +118,13 @@ def test_tensor_conv_forward_matches_oracle(case):
     np.testing.assert_allclose(stats[Cout:], (ref ** 2).reshape(-1, Cout).sum(0), rtol=5e-3)
 
 
+@pytest.mark.parametrize("epilogue", list(EPILOGUES))
 @pytest.mark.parametrize("case", [c for c in TC_CASES if c[3] % 8 == 0 and (c[6] == 1 or (c[1] % 2 == 0 and c[2] % 2 == 0))])
-def test_tensor_conv_dgrad_matches_oracle(case):
+def test_tensor_conv_dgrad_matches_oracle(case, epilogue):
     import paper_2112_05387_b200 as lp
     N, H, W, Cin, Cout, R, stride, pad = case
     x, w, dy = make_case(*case, "bf16")
-    st, dx, _ = run_conv(lp.LP_CONV_DGRAD, "bf16", lp.LP_CONV_IMPL_TENSOR, *case, dy, w)
+    st, dx, _ = run_conv(lp.LP_CONV_DGRAD, "bf16", lp.LP_CONV_IMPL_TENSOR | EPILOGUES[epilogue], *case, dy, w)
     assert st == 0, lp.lp_status_string(st)
     assert rel_err(dx, O.conv_dgrad(dy, w, stride, pad, x.shape)) < 6e-3
 

@@ -158,7 +158,7 @@ def test_small_fp32_block_kinds(kind, stem):
     full_step_parity(cfg, steps=1)
 
 
-@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("impl", [1, 0, 256, 512])     # CUDA cores; tensor cores; direct / staged epilogue everywhere
 @pytest.mark.parametrize("kind", ["postbn", "preact"])
 def test_small_bf16_block_kinds(kind, impl):
     cfg = small_cfg(kind, N=8, H=16, W=16, dtype="bf16", stage_channels=(16, 32), stage_blocks=(2, 2),
