@@ -277,6 +277,8 @@ typedef struct lp_timeline_record {
   int32_t op;     /* LP_OP_* */
   int32_t phase;  /* LP_PHASE_* */
   float start_ms, end_ms;
+  double bytes;   /* algorithmic global-memory bytes of the operation: every operand read once, every result
+                     written once (batch-norm backward: its two passes; update: parameters, gradients, copies) */
 } lp_timeline_record;
 int lp_timeline(lp_handle* h, int enable, int max_records, lp_timeline_record* records, int* n_records);
 

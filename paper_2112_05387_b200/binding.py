@@ -75,7 +75,7 @@ class lp_param_entry(ctypes.Structure):
 
 class lp_timeline_record(ctypes.Structure):
     _fields_ = [("plan", ctypes.c_int32), ("op", ctypes.c_int32), ("phase", ctypes.c_int32),
-                ("start_ms", ctypes.c_float), ("end_ms", ctypes.c_float)]
+                ("start_ms", ctypes.c_float), ("end_ms", ctypes.c_float), ("bytes", ctypes.c_double)]
 
 
 _LIB = None
@@ -375,7 +375,8 @@ def lp_timeline(h, enable, read=True, max_records=4096):
     recs = (lp_timeline_record * max_records)()
     n = ctypes.c_int(0)
     _check(library().lp_timeline(h.ptr, 1 if enable else 0, max_records, recs, ctypes.byref(n)), "lp_timeline")
-    return [dict(plan=r.plan, op=LP_OP_NAMES[r.op], phase=LP_PHASE_NAMES[r.phase], start_ms=r.start_ms, end_ms=r.end_ms)
+    return [dict(plan=r.plan, op=LP_OP_NAMES[r.op], phase=LP_PHASE_NAMES[r.phase], start_ms=r.start_ms, end_ms=r.end_ms,
+                 bytes=r.bytes)
             for r in recs[:min(n.value, max_records)]]
 
 

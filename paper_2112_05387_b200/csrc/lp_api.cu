@@ -181,6 +181,7 @@ static inline int init_cur_dev() {
 struct TimelineRec {
   cudaEvent_t a = nullptr, b = nullptr;
   int plan = 0, op_type = 0, phase = 0;
+  double bytes = 0.0;
 };
 struct Timeline {
   bool enabled = false;
@@ -1436,7 +1437,7 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
 
 struct TimelineScope {
   lp_handle* h; cudaStream_t st; TimelineRec* r = nullptr;
-  TimelineScope(lp_handle* h_, cudaStream_t st_, int plan, int op_type, int phase) : h(h_), st(st_) {
+  TimelineScope(lp_handle* h_, cudaStream_t st_, int plan, int op_type, int phase, double bytes = 0.0) : h(h_), st(st_) {
     if (!h || !h->tl.enabled) return;
     Timeline& tl = h->tl;
     if (tl.used == tl.recs.size()) {
@@ -1445,7 +1446,7 @@ struct TimelineScope {
       tl.recs.push_back(n);
     }
     r = &tl.recs[tl.used++];
-    r->plan = plan; r->op_type = op_type; r->phase = phase;
+    r->plan = plan; r->op_type = op_type; r->phase = phase; r->bytes = bytes;
     cudaEventRecord(r->a, st);
   }
   ~TimelineScope() {
@@ -1453,9 +1454,40 @@ struct TimelineScope {
   }
 };
 
+// Algorithmic global-memory traffic of one operation: every operand read once, every result written once.
+static double op_bytes(const lp_handle* h, const Plan& P, const Op& op) {
+  const double e = (double)esize(h->dtype);
+  auto sz = [&](const Tensor& t) { return t.defined() ? (double)t.elems() * e : 0.0; };
+  switch (op.type) {
+    case OP_CONV_FWD: {
+      const ConvDef& c = P.convs[op.conv];
+      return sz(op.in) + sz(op.out) + sz(op.addend) + (double)c.cout * c.R * c.R * c.cin * e;
+    }
+    case OP_CONV_DGRAD: {
+      const ConvDef& c = P.convs[op.conv];
+      return sz(op.in) + sz(op.out) + sz(op.addend) + (double)c.cout * c.R * c.R * c.cin * e;
+    }
+    case OP_CONV_WGRAD: {
+      const ConvDef& c = P.convs[op.conv];
+      return sz(op.in) + sz(op.in2) + (double)c.cout * c.R * c.R * c.cin * 4.0;
+    }
+    case OP_BN_STATS: return sz(op.in);
+    case OP_BN_APPLY: return sz(op.in) + sz(op.in2) + sz(op.addend) + sz(op.out);
+    case OP_OUT_LOSS:   // operands of the output, x_next, [kappa,] residual and terminal adjoint
+      return op.fuse_loss ? 0.0 : sz(op.in) + sz(op.in2) + sz(op.addend) + 3.0 * sz(op.out);
+    case OP_BN_BWD:     // reduction pass (dy, x) and apply pass (dy, x, [addend] -> dx)
+      return 2.0 * (sz(op.in) + sz(op.in2)) + sz(op.addend) + sz(op.out);
+    case OP_MAXPOOL_FWD: return sz(op.in) + sz(op.out) + (double)op.out.elems();
+    case OP_MAXPOOL_BWD: return sz(op.in) + sz(op.out) + (double)op.in.elems();
+    case OP_HEAD_FWD: return sz(op.in);
+    case OP_HEAD_BWD: return sz(op.out);
+    default: return 0.0;
+  }
+}
+
 static int run_ops(lp_handle* h, Plan& P, const std::vector<Op>& ops, const RunCtx& c) {
   for (const Op& op : ops) {
-    TimelineScope ts(h, c.st, c.plan_id, (int)op.type, c.phase);
+    TimelineScope ts(h, c.st, c.plan_id, (int)op.type, c.phase, h->tl.enabled ? op_bytes(h, P, op) : 0.0);
     int rc = h->dtype == LP_F32 ? run_op_t<float>(h, P, op, c) : run_op_t<bf16>(h, P, op, c);
     if (rc != LP_OK) return rc;
   }
@@ -1816,7 +1848,8 @@ int lp_modules_fwd_bwd_all(lp_handle* h, const void* const* x, const int32_t* la
 static int update_module(lp_handle* h, int k, float lr, float momentum, float weight_decay, float kappa_step,
                          void* lambda_inout, cudaStream_t st) {
   Plan& P = h->modules[k];
-  TimelineScope ts(h, st, k, LP_OP_UPDATE, LP_PHASE_UPDATE);
+  // parameters read and written, gradients read, both bf16 copies of the packed weights written
+  TimelineScope ts(h, st, k, LP_OP_UPDATE, LP_PHASE_UPDATE, 12.0 * (double)P.ps.n + 4.0 * (double)P.ps.pack_total);
   int rc = sgd_update(h, P, lr, momentum, weight_decay, st);
   if (rc != LP_OK) return rc;
   P.ps.grads_fresh = false;
@@ -2166,7 +2199,7 @@ int lp_timeline(lp_handle* h, int enable, int max_records, lp_timeline_record* r
       if (cudaEventElapsedTime(&t1[i], tl.recs[first].a, tl.recs[i].b) != cudaSuccess) return LP_ERR_CUDA;
       if (records && n < max_records) {
         records[n].plan = tl.recs[i].plan; records[n].op = tl.recs[i].op_type; records[n].phase = tl.recs[i].phase;
-        records[n].start_ms = t0[i]; records[n].end_ms = t1[i];
+        records[n].start_ms = t0[i]; records[n].end_ms = t1[i]; records[n].bytes = tl.recs[i].bytes;
       }
       ++n;
     }
