@@ -77,6 +77,10 @@ enum { LP_CONV_LOSS_IN_EPILOGUE = 128 };
  * longer read in 16-byte pieces 2*C_out bytes apart) and every other convolution the direct one.  These
  * flags, OR-ed into conv_impl, force one or the other wherever it applies (comparisons, tests). */
 enum { LP_CONV_DIRECT_EPILOGUE = 256, LP_CONV_STAGED_EPILOGUE = 512 };
+/* May be OR-ed into conv_impl: 3x3 stride-1 tensor-core convolutions (forward and input gradient) with
+ * 64-channel K chunks run on pairs of CTAs (tcgen05 cta_group::2: two pixel tiles per instruction, each CTA
+ * fetching half of every weight stage).  Same results as the one-CTA kernel. */
+enum { LP_CONV_TWO_CTA = 1024 };
 enum { LP_CONV_FWD = 0, LP_CONV_DGRAD = 1, LP_CONV_WGRAD = 2 };
 
 #define LP_MAX_STAGES 8

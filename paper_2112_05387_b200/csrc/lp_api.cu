@@ -14,6 +14,7 @@
 #include "../../include/lp.h"
 #include "conv_simt.cuh"
 #include "conv_tc.cuh"
+#include "conv_tc2.cuh"
 #include "kernels_elem.cuh"
 #include "net.h"
 #include "wgrad_tc.cuh"
@@ -143,7 +144,8 @@ struct Device {
   int sm_count = 148;
   EncodeTiledFn encode = nullptr;
   // kernel attributes are per device: set on the first launch of each kernel family on that device
-  bool conv_attr = false, wgrad_attr = false, wgrad_halo_attr = false;
+  bool conv_attr = false, wgrad_attr = false, wgrad_halo_attr = false, conv2_attr = false;
+  int max_pairs = 0;   // CTA pairs of conv_tc2_kernel that can be resident at once (0: not usable)
   int init() {
     if (ready) return LP_OK;
     int dev = 0;
@@ -264,6 +266,7 @@ struct TcGemmSpec {
   // local loss fused into the epilogue (interior module's last convolution); x_next == nullptr: off
   const bf16* x_next; const bf16* kappa; bf16* r_out; bf16* seed_out; float rho; double* loss_acc;
   int epilogue;          // 0: default (staged where a residual operand exists), 1: direct, 2: staged wherever it applies
+  int two_cta;           // 1: 3x3 stride-1 convolutions take the CTA-pair kernel where it applies
 };
 
 static void pick_pixel_box(int OWl, int OHl, int Nimg, int& BW, int& BH, int& BNI) {
@@ -395,7 +398,138 @@ static int encode_act_map_halo(CUtensorMap* m, const void* base, int N, int H, i
   return r == CUDA_SUCCESS ? LP_OK : LP_ERR_CUDA;
 }
 
+// Launch with a cluster of two CTAs and programmatic stream serialisation allowed.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl_pair(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                          Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = LP_PDL;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// 3x3 stride-1 convolutions with 64-channel K chunks on CTA pairs (conv_tc2.cuh).  Returns LP_ERR_UNSUPPORTED
+// when the shape is not one this kernel takes (the caller then uses the one-CTA kernel).
+static int launch_conv_tc2(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaStream_t st) {
+  Device& D = cur_dev();
+  tc::ConvTcParams p;
+  memset(&p, 0, sizeof(p));
+  p.Nimg = s.aN; p.OHl = s.OHl; p.OWl = s.OWl;
+  int tapw3[3][3];
+  if (s.x_next || s.os != 1 || s.oo_h || s.oo_w || pick_kc(s.aC) != 64 || !pick_halo_box(s, p.BW, p.BH, p.BNI, tapw3))
+    return LP_ERR_UNSUPPORTED;
+  p.halo = 1;
+  p.tiles_w = (s.OWl + p.BW - 1) / p.BW;
+  p.tiles_h = (s.OHl + p.BH - 1) / p.BH;
+  p.m_tiles = p.tiles_w * p.tiles_h * ((s.aN + p.BNI - 1) / p.BNI);
+  pick_n_tile(s.w_rows, p.n_tile_cols, p.n_tiles);
+  if (p.n_tile_cols % 16 || p.n_tile_cols < 32) return LP_ERR_UNSUPPORTED;
+  p.total_tiles = p.m_tiles * p.n_tiles;
+  if (p.m_tiles < 4) return LP_ERR_UNSUPPORTED;     // too few pixel tiles to form units
+  p.in_step = 1;
+  p.out_H = s.out_H; p.out_W = s.out_W; p.out_C = s.out_C;
+  p.os = 1;
+  p.Cout = s.w_rows;
+  p.ntaps = 9;
+  p.Cin = s.aC;
+  p.KC = 64;
+  p.chunks = (s.aC + 63) / 64;
+  p.nk_last = (s.aC - (p.chunks - 1) * 64 + 15) / 16;
+  const int row_bytes = 128;
+  const int n_half = p.n_tile_cols / 2;
+  const uint32_t b_half = (uint32_t)align_up((size_t)n_half * row_bytes, 1024);
+  const size_t tail = tc::kTailBytes + sizeof(tc::TcStatScratch) + 1024;
+  p.tx_b = (uint32_t)(n_half * row_bytes);
+  p.acc_stride = (p.n_tile_cols + 31) / 32 * 32;
+  p.nslots = std::min(tc::kMaxSlots, tc::kTmemCols / p.acc_stride);
+  if (p.nslots < 2) return LP_ERR_UNSUPPORTED;
+  const int halo_rows = kHaloBoxW * p.BNI * (p.BH + 2);
+  p.a_halo_bytes = (uint32_t)align_up((size_t)halo_rows * row_bytes, 1024);
+  for (int dy = 0; dy < 3; ++dy)
+    for (int dx = 0; dx < 3; ++dx) {
+      p.tap_widx9[dy * 3 + dx] = tapw3[dx][dy];
+      p.tap_off9[dy * 3 + dx] = (uint32_t)((dy * kHaloBoxW * p.BNI + dx) * row_bytes);
+    }
+  p.desc_hi_a = tc::smem_desc_hi(16, kHaloBoxW * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
+  p.desc_hi = tc::smem_desc_hi(16, 8 * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
+  p.b_stage_bytes = b_half;
+  p.tx_a = (uint32_t)(halo_rows * row_bytes);
+  p.nA = 2;
+  p.mpair = 2;
+  p.a_stage_bytes = 2 * p.a_halo_bytes;
+  const size_t a_bytes = (size_t)p.nA * p.a_stage_bytes;
+  if (a_bytes + 3 * (size_t)b_half + tail > kTcMaxSmem) return LP_ERR_UNSUPPORTED;
+  p.nB = (int)std::min<size_t>((kTcMaxSmem - tail - a_bytes) / b_half, tc::kMaxStages);
+  p.b_ring_offset = (uint32_t)a_bytes;
+  p.tail_offset = p.b_ring_offset + p.nB * p.b_stage_bytes;
+  p.stage_offset = p.tail_offset;
+  p.idesc = tc::instr_desc_bf16(256, p.n_tile_cols, 0, 0);
+  p.out = s.out; p.addend = s.addend; p.stats = s.stats; p.err = dev_err;
+  p.wide32 = (s.out_C % 16 == 0 && s.w_rows % 16 == 0 && p.n_tile_cols % 16 == 0 &&
+              (reinterpret_cast<uintptr_t>(s.out) & 31) == 0 &&
+              (!s.addend || (reinterpret_cast<uintptr_t>(s.addend) & 31) == 0)) ? 1 : 0;
+  CUtensorMap tmA, tmB;
+  int rc = encode_act_map_halo(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, 64, kHaloBoxW, p.BH, p.BNI, row_bytes);
+  if (rc != LP_OK) return rc;
+  rc = encode_mat_map(&tmB, s.wmat, s.w_K, s.w_rows, 64, n_half, row_bytes);
+  if (rc != LP_OK) return rc;
+  const size_t smem = std::max((size_t)p.tail_offset + tail, kTcMinSmem);
+  if (!D.conv2_attr) {
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcMaxSmem));
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcMaxSmem));
+    // how many CTA pairs fit the device at once (persistent kernel: never more pairs than that)
+    cudaLaunchConfig_t q = {};
+    q.gridDim = dim3(2 * D.sm_count);
+    q.blockDim = dim3(tc::kConvThreads);
+    q.dynamicSmemBytes = kTcMaxSmem;
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeClusterDimension;
+    qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+    q.attrs = qa;
+    q.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, tc::conv_tc2_kernel<false>, &q) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    D.max_pairs = n;
+    D.conv2_attr = true;
+  }
+  if (D.max_pairs < 1) return LP_ERR_UNSUPPORTED;
+  // persistent CTA pairs over contiguous tile ranges; side by side with other modules the smallest number of
+  // pairs whose busiest one has no more units of four tiles (see launch_conv_tc)
+  int pairs = std::max(1, std::min(D.max_pairs, p.total_tiles / 2));
+  // a pair whose tile range crosses a channel-tile boundary works on two short units instead of one: with
+  // several channel tiles, a number of pairs that the channel tiles divide keeps every range inside one
+  if (p.n_tiles > 1 && pairs >= p.n_tiles) pairs = pairs / p.n_tiles * p.n_tiles;
+  if (h && h->concurrent) {
+    int per = (p.total_tiles + pairs - 1) / pairs;
+    per = (per + 3) / 4 * 4;
+    pairs = (p.total_tiles + per - 1) / per;
+  }
+  cudaError_t le;
+  const dim3 g3(2 * pairs), b3(tc::kConvThreads);
+  if (s.addend) le = launch_pdl_pair(tc::conv_tc2_kernel<true>, g3, b3, smem, st, tmA, tmB, p);
+  else le = launch_pdl_pair(tc::conv_tc2_kernel<false>, g3, b3, smem, st, tmA, tmB, p);
+  LP_CUDA_OK(le);
+  if (h) h->launches++;
+  LP_CUDA_OK(cudaGetLastError());
+  return LP_OK;
+}
+
 static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaStream_t st) {
+  if (s.two_cta) {
+    const int rc2 = launch_conv_tc2(h, s, dev_err, st);
+    if (rc2 != LP_ERR_UNSUPPORTED) return rc2;
+  }
   tc::ConvTcParams p;
   memset(&p, 0, sizeof(p));
   p.Nimg = s.aN; p.OHl = s.OHl; p.OWl = s.OWl;
@@ -623,6 +757,7 @@ static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int
     s.out_H = c.OH; s.out_W = c.OW; s.out_C = c.cout; s.os = 1; s.oo_h = s.oo_w = 0;
     s.stats = stats;
     s.epilogue = (impl & LP_CONV_DIRECT_EPILOGUE) ? 1 : ((impl & LP_CONV_STAGED_EPILOGUE) ? 2 : 0);
+    s.two_cta = (impl & LP_CONV_TWO_CTA) ? 1 : 0;
     if (loss) {
       s.x_next = (const bf16*)loss->x_next; s.kappa = (const bf16*)loss->kappa; s.r_out = (bf16*)loss->r_out;
       s.seed_out = (bf16*)loss->seed_out; s.rho = loss->rho; s.loss_acc = loss->acc;
@@ -710,6 +845,7 @@ static int conv_dgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
       s.out_H = c.H; s.out_W = c.W; s.out_C = c.cin; s.os = st2; s.oo_h = ph; s.oo_w = pw;
       s.stats = nullptr;
       s.epilogue = (impl & LP_CONV_DIRECT_EPILOGUE) ? 1 : ((impl & LP_CONV_STAGED_EPILOGUE) ? 2 : 0);
+    s.two_cta = (impl & LP_CONV_TWO_CTA) ? 1 : 0;
       int rc = launch_conv_tc(h, s, dev_err, st);
       if (rc != LP_OK) return rc;
     }

@@ -99,9 +99,9 @@ TC_CASES = [
 ]
 
 
-# both epilogues of the forward / input-gradient kernel, each forced wherever it applies: tile staged in
-# shared memory and stored by TMA, and stores from registers
-EPILOGUES = {"staged": 512, "direct": 256}
+# variants of the forward / input-gradient kernel, each forced wherever it applies: tile staged in shared
+# memory and stored by TMA; stores from registers; 3x3 stride-1 layers on pairs of CTAs (cta_group::2)
+EPILOGUES = {"staged": 512, "direct": 256, "cta-pairs": 1024}   # the last: the CTA-pair kernel where it applies
 
 
 @pytest.mark.parametrize("epilogue", list(EPILOGUES))

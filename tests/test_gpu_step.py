@@ -239,6 +239,13 @@ def test_wrn28_10_reduced_batch_bf16():
     full_step_parity(scaled("wrn28_10", N=6), steps=1)
 
 
+def test_wrn28_10_reduced_batch_bf16_on_cta_pairs():
+    """LP_CONV_TWO_CTA: the 3x3 stride-1 layers (forward and input gradient, with and without a residual operand,
+    with statistics) on pairs of CTAs give the same step."""
+    import paper_2112_05387_b200 as lp
+    full_step_parity(scaled("wrn28_10", N=6), conv_impl=lp.LP_CONV_TWO_CTA, steps=1)
+
+
 def test_wrn28_10_loss_in_the_last_convolutions_epilogue():
     """LP_CONV_LOSS_IN_EPILOGUE: residual, loss sums and terminal adjoint taken by the epilogue of each
     interior module's last convolution give the same step as the separate pass (penalty and AL)."""
