@@ -66,6 +66,10 @@ struct ConvTcParams {
   int Cin, KC, chunks;
   int nk_last;                   // K = 16 slices of the last chunk that hold real channels (the rest is zero fill)
   int stages;
+  int ips;                       // (tap, K chunk) items per pipeline stage (plain mode): thin layers (few channels) put
+                                 // several taps into one stage, so that the fixed cost of a stage -- a barrier round
+                                 // trip, several hundred cycles -- is paid once per `ips` items instead of once each
+  uint32_t item_bytes;           // one item: mpair activation tiles + the weight tile
   int mpair;                     // pixel tiles per unit: 1 or 2
   int nslots, acc_stride;        // accumulator ring: slots and their TMEM column stride
   uint32_t stage_bytes, a_region_bytes, b_offset, tx_a, tx_b;
@@ -81,6 +85,10 @@ struct ConvTcParams {
   uint32_t a_halo_bytes;         // one activation box (1024-aligned)
   uint32_t a_stage_bytes;        // mpair boxes
   uint32_t b_stage_bytes, b_ring_offset;
+  int tps;                       // halo mode: taps per weight stage.  A stage costs roughly 450 cycles plus 12 per KB
+                                 // whatever it holds: with one tap (20 KB; 640 cycles of tensor work for a pair of
+                                 // tiles) that is more than the tensor work, with two taps per stage it is less
+  uint32_t b_tile_bytes;         // weights of one tap inside a weight stage
   uint32_t tail_offset;          // barriers and scratch after the rings
   int tap_widx9[9];              // weight tap index of the nine taps in (dy, dx) order
   uint32_t tap_off9[9];          // byte offset of the tap's first row inside the box
@@ -183,7 +191,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if constexpr (kAddend) prefetch_tmap(&tmAdd);
     }
   }
-  if constexpr (!kStaged) {
+  if (!kStaged && p.stats) {   // (without statistics the scratch is not part of the allocation)
     for (int i = threadIdx.x; i < LP_EPI_WARPS * 256; i += blockDim.x) {
       (&scratch->ssum[0][0])[i] = 0.f;
       (&scratch->ssq[0][0])[i] = 0.f;
@@ -229,11 +237,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         __syncwarp();
         if (++sa == (uint32_t)p.nA) { sa = 0; pha ^= 1; }
-        for (int ti = 0; ti < 9; ++ti) {
+        for (int ti0 = 0; ti0 < 9; ti0 += p.tps) {
+          const int n_taps = min(p.tps, 9 - ti0);
           if (!mbar_wait_warp(&tail->empty_b[sb], phb ^ 1, abort_flag)) { failed = true; break; }
           if (elect_one()) {
-            mbar_expect_tx(&tail->full_b[sb], p.tx_b);
-            tma_load_2d(b_ring + sb * p.b_stage_bytes, &tmB, &tail->full_b[sb], p.tap_widx9[ti] * p.Cin + c * p.KC, col0);
+            mbar_expect_tx(&tail->full_b[sb], n_taps * p.tx_b);
+            for (int i = 0; i < n_taps; ++i)
+              tma_load_2d(b_ring + sb * p.b_stage_bytes + i * p.b_tile_bytes, &tmB, &tail->full_b[sb],
+                          p.tap_widx9[ti0 + i] * p.Cin + c * p.KC, col0);
           }
           __syncwarp();
           if (++sb == (uint32_t)p.nB) { sb = 0; phb ^= 1; }
@@ -264,25 +275,30 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int c = 0; c < p.chunks && !failed; ++c) {
         const uint32_t a_addr = smem_base + sa * p.a_stage_bytes + me * p.a_halo_bytes;
         const int nkc = c + 1 == p.chunks ? p.nk_last : nk;   // slices of pure zero fill are not multiplied
-        for (int ti = 0; ti < 9; ++ti) {
+        for (int ti0 = 0; ti0 < 9; ti0 += p.tps) {
+          const int n_taps = min(p.tps, 9 - ti0);
+          const bool last_of_chunk = ti0 + n_taps == 9;
           // The box barrier is polled together with the first weight stage and released together
           // with the last one: a separate trip (poll, election, commit) at every chunk boundary
           // costs about 500 cycles in which the tensor pipe runs dry.
-          bool ok = ti ? true : mbar_wait(&tail->full[sa], pha, abort_flag);
+          bool ok = ti0 ? true : mbar_wait(&tail->full[sa], pha, abort_flag);
           ok = mbar_wait(&tail->full_b[sb], phb, abort_flag) && ok;
           if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
           tc_fence_after();
-          const uint64_t ad = smem_desc(p.desc_hi_a, a_addr + p.tap_off9[ti]);
-          const uint64_t bd = smem_desc(p.desc_hi, smem_base + p.b_ring_offset + sb * p.b_stage_bytes);
+          const uint32_t b_addr = smem_base + p.b_ring_offset + sb * p.b_stage_bytes;
           if (elect_one()) {
             if (active) {
-              for (int j = 0; j < nkc; ++j)
-                mma_bf16(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (accum | j) ? 1u : 0u);
+              for (int i = 0; i < n_taps; ++i) {
+                const uint64_t ad = smem_desc(p.desc_hi_a, a_addr + p.tap_off9[ti0 + i]);
+                const uint64_t bd = smem_desc(p.desc_hi, b_addr + i * p.b_tile_bytes);
+                for (int j = 0; j < nkc; ++j)
+                  mma_bf16(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (accum | i | j) ? 1u : 0u);
+              }
               mma_commit(&tail->empty_b[sb]);
-              if (ti == 8) mma_commit(&tail->empty[sa]);
+              if (last_of_chunk) mma_commit(&tail->empty[sa]);
             } else {
               mbar_arrive(&tail->empty_b[sb]);
-              if (ti == 8) mbar_arrive(&tail->empty[sa]);
+              if (last_of_chunk) mbar_arrive(&tail->empty[sa]);
             }
           }
           __syncwarp();
@@ -314,23 +330,26 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
       const int col0 = nt * p.n_tile_cols;
       const uint32_t tx = p.tx_b + cnt * p.tx_a;
-      for (int tap = 0; tap < p.ntaps && !failed; ++tap) {
-        const int kb = p.tap_w[tap] * p.Cin;
-        for (int c = 0; c < p.chunks; ++c) {
-          if (!mbar_wait_warp(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
-          uint8_t* sa = smem + s * p.stage_bytes;
-          if (elect_one()) {
-            mbar_expect_tx(&tail->full[s], tx);
-            tma_load_4d(sa, &tmA, &tail->full[s], c * p.KC, w0[0] * p.in_step + p.tap_dw[tap],
+      for (int k0 = 0; k0 < kiters && !failed; k0 += p.ips) {
+        const int n_items = min(p.ips, kiters - k0);
+        if (!mbar_wait_warp(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
+        uint8_t* sa = smem + s * p.stage_bytes;
+        if (elect_one()) {
+          mbar_expect_tx(&tail->full[s], n_items * tx);
+          for (int i = 0; i < n_items; ++i) {
+            const int tap = (k0 + i) / p.chunks, c = (k0 + i) % p.chunks;
+            const int kb = p.tap_w[tap] * p.Cin;
+            uint8_t* si = sa + i * p.item_bytes;
+            tma_load_4d(si, &tmA, &tail->full[s], c * p.KC, w0[0] * p.in_step + p.tap_dw[tap],
                         h0[0] * p.in_step + p.tap_dh[tap], n0[0]);
             if (cnt == 2)
-              tma_load_4d(sa + p.a_region_bytes, &tmA, &tail->full[s], c * p.KC, w0[1] * p.in_step + p.tap_dw[tap],
+              tma_load_4d(si + p.a_region_bytes, &tmA, &tail->full[s], c * p.KC, w0[1] * p.in_step + p.tap_dw[tap],
                           h0[1] * p.in_step + p.tap_dh[tap], n0[1]);
-            tma_load_2d(sa + p.b_offset, &tmB, &tail->full[s], kb + c * p.KC, col0);
+            tma_load_2d(si + p.b_offset, &tmB, &tail->full[s], kb + c * p.KC, col0);
           }
-          __syncwarp();
-          if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
         }
+        __syncwarp();
+        if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
       }
       t += cnt;
     }
@@ -356,19 +375,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_after();
       }
       const uint32_t d = tmem_base + sl[me] * p.acc_stride;
-      int cc = 0;   // chunk index within the tap
-      for (int k = 0; k < kiters; ++k) {
+      for (int k0 = 0; k0 < kiters; k0 += p.ips) {
+        const int n_items = min(p.ips, kiters - k0);
         if (!mbar_wait_warp(&tail->full[s], ph, abort_flag)) { failed = true; break; }
         tc_fence_after();
-        const int nkc = cc + 1 == p.chunks ? p.nk_last : nk;
-        if (++cc == p.chunks) cc = 0;
         const uint32_t a_addr = smem_base + s * p.stage_bytes;
-        const uint64_t ad = smem_desc(p.desc_hi, a_addr + me * p.a_region_bytes);
-        const uint64_t bd = smem_desc(p.desc_hi, a_addr + p.b_offset);
         if (elect_one()) {
           if (active) {
-            for (int j = 0; j < nkc; ++j)  // +32 bytes (one K = 16 slice) per step, in 16-byte units
-              mma_bf16(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k | j) ? 1u : 0u);
+            for (int i = 0; i < n_items; ++i) {
+              const int nkc = (k0 + i) % p.chunks + 1 == p.chunks ? p.nk_last : nk;
+              const uint64_t ad = smem_desc(p.desc_hi, a_addr + i * p.item_bytes + me * p.a_region_bytes);
+              const uint64_t bd = smem_desc(p.desc_hi, a_addr + i * p.item_bytes + p.b_offset);
+              for (int j = 0; j < nkc; ++j)  // +32 bytes (one K = 16 slice) per step, in 16-byte units
+                mma_bf16(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (k0 | i | j) ? 1u : 0u);
+            }
             mma_commit(&tail->empty[s]);
           } else {
             mbar_arrive(&tail->empty[s]);

@@ -137,9 +137,11 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
   }
-  for (int i = threadIdx.x; i < LP_EPI_WARPS * 256; i += blockDim.x) {
-    (&scratch->ssum[0][0])[i] = 0.f;
-    (&scratch->ssq[0][0])[i] = 0.f;
+  if (p.stats) {   // (without statistics the scratch is not part of the allocation)
+    for (int i = threadIdx.x; i < LP_EPI_WARPS * 256; i += blockDim.x) {
+      (&scratch->ssum[0][0])[i] = 0.f;
+      (&scratch->ssq[0][0])[i] = 0.f;
+    }
   }
   if (warp == kFirstEpiWarp) {
     tmem2_alloc(&tail->tmem_base, kTmemCols);

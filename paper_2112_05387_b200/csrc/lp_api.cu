@@ -359,6 +359,9 @@ static const size_t kTcMaxSmem = 220 * 1024;
 #ifndef LP_CONV_MAX_NB
 #define LP_CONV_MAX_NB 8   // weight stages in flight (halo mode), as far as shared memory allows
 #endif
+#ifndef LP_CONV_TAPS_PER_STAGE
+#define LP_CONV_TAPS_PER_STAGE 2   // taps per weight stage (halo mode), as far as three stages still fit
+#endif
 static const int kHaloBoxW = 10;   // 8-pixel tile width plus one halo pixel on each side
 
 static bool pick_halo_box(const TcGemmSpec& s, int& BW, int& BH, int& BNI, int tapw3[3][3]) {
@@ -449,7 +452,7 @@ static int launch_conv_tc2(lp_handle* h, const TcGemmSpec& s, int* dev_err, cuda
   const int row_bytes = 128;
   const int n_half = p.n_tile_cols / 2;
   const uint32_t b_half = (uint32_t)align_up((size_t)n_half * row_bytes, 1024);
-  const size_t tail = tc::kTailBytes + sizeof(tc::TcStatScratch) + 1024;
+  const size_t tail = tc::kTailBytes + (s.stats ? sizeof(tc::TcStatScratch) : 0) + 1024;
   p.tx_b = (uint32_t)(n_half * row_bytes);
   p.acc_stride = (p.n_tile_cols + 31) / 32 * 32;
   p.nslots = std::min(tc::kMaxSlots, tc::kTmemCols / p.acc_stride);
@@ -562,7 +565,8 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
                       (reinterpret_cast<uintptr_t>(s.out) & 15) == 0 &&
                       (!s.addend || (reinterpret_cast<uintptr_t>(s.addend) & 15) == 0);
   const size_t stage_bytes = staged ? (size_t)(p.n_tile_cols / 32) * tc::kStageGroupBytes : 0;
-  const size_t tail = tc::kTailBytes + (staged ? 0 : sizeof(tc::TcStatScratch)) + stage_bytes + 1024;
+  // the direct epilogue's statistics scratch is only there when statistics are asked for
+  const size_t tail = tc::kTailBytes + ((staged || !s.stats) ? 0 : sizeof(tc::TcStatScratch)) + stage_bytes + 1024;
   p.tx_b = (uint32_t)(p.n_tile_cols * row_bytes);
   p.acc_stride = (p.n_tile_cols + 31) / 32 * 32;
   p.nslots = std::min(tc::kMaxSlots, tc::kTmemCols / p.acc_stride);
@@ -577,19 +581,23 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
       }
     // 8-row groups of the operand are one box row (kHaloBoxW pixels) apart
     p.desc_hi_a = tc::smem_desc_hi(16, kHaloBoxW * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
-    p.b_stage_bytes = b_region;
+    p.b_tile_bytes = b_region;
     p.tx_a = (uint32_t)(halo_rows * row_bytes);
     const size_t avail = kTcMaxSmem - tail;
-    // two activation stages (each lasts nine weight stages), the rest of shared memory for weights
+    // two activation stages (each lasts all nine taps), the rest of shared memory for weights: stages of
+    // LP_CONV_TAPS_PER_STAGE taps where three of them fit, else of fewer taps
     bool fits = false;
     p.nA = 2;
     for (int pair = (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, cur_dev().sm_count)) ? 2 : 1;
          pair >= 1 && !fits; --pair) {
       const size_t a_bytes = (size_t)p.nA * pair * p.a_halo_bytes;
       if (a_bytes >= avail) continue;
-      const int nb = (int)std::min<size_t>((avail - a_bytes) / b_region, LP_CONV_MAX_NB);
-      if (nb >= 3) { p.mpair = pair; p.nB = nb; fits = true; }
+      for (int tps = LP_CONV_TAPS_PER_STAGE; tps >= 1 && !fits; --tps) {
+        const int nb = (int)std::min<size_t>((avail - a_bytes) / ((size_t)tps * b_region), LP_CONV_MAX_NB);
+        if (nb >= 3) { p.mpair = pair; p.nB = nb; p.tps = tps; fits = true; }
+      }
     }
+    p.b_stage_bytes = p.tps * b_region;
     if (fits) {
       p.a_stage_bytes = p.mpair * p.a_halo_bytes;
       p.b_ring_offset = p.nA * p.a_stage_bytes;
@@ -611,8 +619,19 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
         (kTcMaxSmem - tail) / (2 * p.a_region_bytes + b_region) >= 3)
       p.mpair = 2;
     p.b_offset = p.mpair * p.a_region_bytes;
-    p.stage_bytes = p.b_offset + b_region;
+    p.item_bytes = p.b_offset + b_region;
     p.tx_a = (uint32_t)(p.BW * p.BH * p.BNI * row_bytes);
+    // Items (one tap of one K chunk) per pipeline stage: as many as leave three stages, spread evenly over the
+    // stages of a tile.  Layers with few channels (16 or 32: an item is one or two instructions) then pay the
+    // fixed cost of a stage once per several taps; wide layers keep one item per stage.
+    {
+      const int kiters = p.ntaps * p.chunks;
+      int ips = (int)std::min<size_t>((size_t)kiters, (kTcMaxSmem - tail) / 3 / p.item_bytes);
+      ips = std::max(ips, 1);
+      const int n_st = (kiters + ips - 1) / ips;
+      p.ips = (kiters + n_st - 1) / n_st;
+    }
+    p.stage_bytes = p.ips * p.item_bytes;
     int stages = (int)((kTcMaxSmem - tail) / p.stage_bytes);
     stages = std::min(stages, tc::kMaxStages);
     if (stages < 2) return LP_ERR_UNSUPPORTED;
