@@ -62,7 +62,7 @@ struct ConvTcParams {
   int os, oo_h, oo_w;            // physical pixel = logical * os + oo
   int n_tile_cols, Cout;
   int ntaps;
-  int tap_dh[9], tap_dw[9], tap_w[9];
+  int tap_dh[16], tap_dw[16], tap_w[16];   // up to 16 taps (plain mode; the space-to-depth stem has 4x4)
   int Cin, KC, chunks;
   int nk_last;                   // K = 16 slices of the last chunk that hold real channels (the rest is zero fill)
   int stages;

@@ -449,51 +449,64 @@ __global__ void add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* 
 // ---------------------------------------------------------------------------------------
 // 3x3 / stride 2 / pad 1 max-pool; the first maximum in (r,s) scan order wins (stored as 0..8).
 // ---------------------------------------------------------------------------------------
+// A thread handles VecT<T>::N consecutive channels of one pixel (16-byte accesses; C is a multiple of that).
 template <typename T>
 __global__ void maxpool_fwd_kernel(const T* __restrict__ x, T* __restrict__ y, uint8_t* __restrict__ arg, int N,
                                    int H, int W, int C, int OH, int OW) {
-  const long long total = (long long)N * OH * OW * C;
+  constexpr int V = VecT<T>::N;
+  const int CV = C / V;
+  const long long total = (long long)N * OH * OW * CV;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
-    const int c = (int)(i % C);
-    long long p = i / C;
+    const int cg = (int)(i % CV);
+    long long p = i / CV;
     const int ow = (int)(p % OW);
     p /= OW;
     const int oh = (int)(p % OH);
     const int n = (int)(p / OH);
-    float best = -INFINITY;
-    int ba = 0;
+    float best[V];
+    int ba[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) { best[j] = -INFINITY; ba[j] = 0; }
     for (int r = 0; r < 3; ++r) {
       const int ih = oh * 2 + r - 1;
       if (ih < 0 || ih >= H) continue;
       for (int s = 0; s < 3; ++s) {
         const int iw = ow * 2 + s - 1;
         if (iw < 0 || iw >= W) continue;
-        const float v = to_f(x[(((long long)n * H + ih) * W + iw) * C + c]);
-        if (v > best) {
-          best = v;
-          ba = r * 3 + s;
-        }
+        float v[V];
+        ldv(x + (((long long)n * H + ih) * W + iw) * C + cg * V, v);
+#pragma unroll
+        for (int j = 0; j < V; ++j)
+          if (v[j] > best[j]) { best[j] = v[j]; ba[j] = r * 3 + s; }
       }
     }
-    from_f(y[i], best);
-    arg[i] = (uint8_t)ba;
+    stv(y + i * V, best);
+    uint8_t* ap = arg + i * V;
+#pragma unroll
+    for (int j = 0; j < V; j += 4)
+      *reinterpret_cast<uint32_t*>(ap + j) = (uint32_t)ba[j] | ((uint32_t)ba[j + 1] << 8) | ((uint32_t)ba[j + 2] << 16) |
+                                             ((uint32_t)ba[j + 3] << 24);
   }
 }
 
 template <typename T>
 __global__ void maxpool_bwd_kernel(const T* __restrict__ dy, const uint8_t* __restrict__ arg, T* __restrict__ dx,
                                    int N, int H, int W, int C, int OH, int OW) {
-  const long long total = (long long)N * H * W * C;
+  constexpr int V = VecT<T>::N;
+  const int CV = C / V;
+  const long long total = (long long)N * H * W * CV;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
-    const int c = (int)(i % C);
-    long long p = i / C;
+    const int cg = (int)(i % CV);
+    long long p = i / CV;
     const int iw = (int)(p % W);
     p /= W;
     const int ih = (int)(p % H);
     const int n = (int)(p / H);
-    float acc = 0.f;
+    float acc[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[j] = 0.f;
     for (int r = 0; r < 3; ++r) {
       const int t = ih + 1 - r;
       if (t < 0 || (t & 1)) continue;
@@ -504,11 +517,21 @@ __global__ void maxpool_bwd_kernel(const T* __restrict__ dy, const uint8_t* __re
         if (u < 0 || (u & 1)) continue;
         const int ow = u >> 1;
         if (ow >= OW) continue;
-        const long long o = (((long long)n * OH + oh) * OW + ow) * C + c;
-        if (arg[o] == r * 3 + s) acc += to_f(dy[o]);
+        const long long o = ((((long long)n * OH + oh) * OW + ow) * CV + cg) * V;
+        float d[V];
+        ldv(dy + o, d);
+        const uint8_t* ap = arg + o;
+        const int want = r * 3 + s;
+#pragma unroll
+        for (int j = 0; j < V; j += 4) {
+          const uint32_t a4 = *reinterpret_cast<const uint32_t*>(ap + j);
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if ((int)((a4 >> (8 * q)) & 255u) == want) acc[j + q] += d[j + q];
+        }
       }
     }
-    from_f(dx[i], acc);
+    stv(dx + i * V, acc);
   }
 }
 
@@ -823,6 +846,72 @@ __global__ void sgd_pack_tiled_kernel(const PackEntry* __restrict__ tab, int n_e
   for (int i = ty; i < 32; i += 8) {
     const int ci = ci0 + i, co = co0 + tx;
     if (co < e.cout && ci < e.cin) e.wt[((long long)ci * e.taps + t) * e.cout + co] = __float2bfloat16_rn(tile[tx][i]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// 7x7 / stride 2 / pad 3 stem convolution on the tensor cores by space-to-depth.
+// The image x[N][H][W][C] (C <= 4, H and W even) is regrouped as xs[N][H/2][W/2][16]: channel (by*2 + bx)*C + c of
+// pixel (i, j) is x[2i + by][2j + bx][c] (channels 4C..15 are zero).  Since input row 2*oh + r - 3 = 2*(oh + a) + by
+// with a = floor((r - 3) / 2) in {-2..1}, the convolution becomes a 4x4 stride-1 convolution over xs with taps
+// a_h, a_w in {-2..1} (tap index (a_h + 2)*4 + (a_w + 2)) and weights
+//   ws[co][tap][(by*2 + bx)*C + c] = w[co][2*a_h + by + 3][2*a_w + bx + 3][c]   (zero where that row or column is not 0..6).
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void s2d_input_kernel(const T* __restrict__ x, bf16* __restrict__ xs, int N, int H, int W, int C) {
+  const int OH = H >> 1, OW = W >> 1;
+  const long long total = (long long)N * OH * OW;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int ow = (int)(i % OW);
+    long long q = i / OW;
+    const int oh = (int)(q % OH);
+    const int n = (int)(q / OH);
+    float v[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = 0.f;
+    for (int by = 0; by < 2; ++by)
+      for (int bx = 0; bx < 2; ++bx) {
+        const T* px = x + (((long long)n * H + 2 * oh + by) * W + 2 * ow + bx) * C;
+        for (int c = 0; c < C; ++c) v[(by * 2 + bx) * C + c] = to_f(px[c]);
+      }
+    uint4 lo, hi;
+    lo.x = pack_bf16x2(v[0], v[1]); lo.y = pack_bf16x2(v[2], v[3]); lo.z = pack_bf16x2(v[4], v[5]); lo.w = pack_bf16x2(v[6], v[7]);
+    hi.x = pack_bf16x2(v[8], v[9]); hi.y = pack_bf16x2(v[10], v[11]); hi.z = pack_bf16x2(v[12], v[13]); hi.w = pack_bf16x2(v[14], v[15]);
+    uint4* dst = reinterpret_cast<uint4*>(xs + i * 16);
+    dst[0] = lo;
+    dst[1] = hi;
+  }
+}
+
+// ws[co][16 taps][16 channels] (bf16) from w[co][7][7][C] (fp32)
+__global__ void s2d_pack_weights_kernel(const float* __restrict__ w, bf16* __restrict__ ws, int Cout, int C) {
+  const int total = Cout * 256;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    const int ch = i & 15, tap = (i >> 4) & 15, co = i >> 8;
+    float v = 0.f;
+    if (ch < 4 * C) {
+      const int blk = ch / C, c = ch % C;
+      const int by = blk >> 1, bx = blk & 1;
+      const int r = 2 * ((tap >> 2) - 2) + by + 3, q = 2 * ((tap & 3) - 2) + bx + 3;
+      if (r >= 0 && r < 7 && q >= 0 && q < 7) v = w[(((long long)co * 7 + r) * 7 + q) * C + c];
+    }
+    ws[i] = __float2bfloat16_rn(v);
+  }
+}
+
+// gw[co][7][7][C] = the entries of dws[co][16 taps][16 channels] that correspond to real filter positions
+__global__ void s2d_unpack_wgrad_kernel(const float* __restrict__ dws, float* __restrict__ gw, int Cout, int C) {
+  const int total = Cout * 49 * C;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    const int c = i % C;
+    int t = i / C;
+    const int q = t % 7;
+    t /= 7;
+    const int r = t % 7, co = t / 7;
+    const int by = (r + 1) & 1, bx = (q + 1) & 1;            // r - 3 = 2a + by with by in {0, 1}
+    const int ah = (r - 3 - by) / 2, aw = (q - 3 - bx) / 2;   // exact: the numerators are even
+    const int tap = (ah + 2) * 4 + (aw + 2);
+    gw[i] = dws[((long long)co * 16 + tap) * 16 + (by * 2 + bx) * C + c];
   }
 }
 

@@ -45,6 +45,11 @@ struct ConvDef {
   bf16* wf = nullptr;        // bf16 [cout][R*R*cin]
   bf16* wt = nullptr;        // bf16 [cin][R*R*cout] (input-gradient operand), optional
   bool need_dgrad = true;
+  // 7x7 / stride-2 stem on the tensor cores by space-to-depth (see kernels_elem.cuh): the regrouped input,
+  // the regrouped bf16 weights [cout][16 taps][16] (in wf) and the weight gradient in that layout
+  bool s2d = false;
+  bf16* xs = nullptr;        // [N][H/2][W/2][16]
+  float* dws = nullptr;      // [cout][16][16]
 };
 struct BnDef {
   int C;
@@ -260,7 +265,7 @@ struct TcGemmSpec {
   const bf16* wmat; int w_rows; long long w_K;
   int in_step;
   int OHl, OWl;
-  int ntaps; int dh[9], dw[9], widx[9];
+  int ntaps; int dh[16], dw[16], widx[16];
   bf16* out; const bf16* addend; int out_H, out_W, out_C, os, oo_h, oo_w;
   double* stats;
   // local loss fused into the epilogue (interior module's last convolution); x_next == nullptr: off
@@ -718,6 +723,11 @@ static bool tc_wgrad_ok(const ConvDef& c) {
   return c.cin % 8 == 0 && c.cout % 8 == 0 && (c.R == 1 || c.R == 3) && (c.stride == 1 || c.stride == 2);
 }
 
+static bool s2d_stem_ok(const ConvDef& c) {
+  return c.R == 7 && c.stride == 2 && c.pad == 3 && c.cin >= 1 && c.cin <= 4 && c.cout % 8 == 0 && c.H % 2 == 0 &&
+         c.W % 2 == 0 && c.H >= 8 && c.W >= 8;
+}
+
 // Local loss of an interior module computed by the epilogue of the module's last convolution.
 struct LossFuse {
   const void* x_next; const void* kappa; void* r_out; void* seed_out; float rho; double* acc;
@@ -758,6 +768,28 @@ static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int
                         const void* addend, double* stats, bool* stats_done, int* dev_err, cudaStream_t st,
                         const LossFuse* loss = nullptr) {
   if (stats_done) *stats_done = false;
+  if (c.s2d) {
+    // 7x7 / stride-2 stem: regroup the image, then a 4x4 stride-1 tensor-core convolution over 16 channels
+    const int H2 = c.H / 2, W2 = c.W / 2;
+    const long long pix = (long long)N * H2 * W2;
+    s2d_input_kernel<bf16><<<grid_for(pix, 256, cur_dev().sm_count, 8), 256, 0, st>>>((const bf16*)x, c.xs, N, c.H, c.W, c.cin);
+    if (h) h->launches++;
+    LP_CUDA_OK(cudaGetLastError());
+    TcGemmSpec s;
+    memset(&s, 0, sizeof(s));
+    s.act = c.xs; s.aN = N; s.aH = H2; s.aW = W2; s.aC = 16;
+    s.wmat = c.wf; s.w_rows = c.cout; s.w_K = 256;
+    s.in_step = 1; s.OHl = c.OH; s.OWl = c.OW;
+    s.ntaps = 16;
+    for (int i = 0; i < 16; ++i) { s.dh[i] = i / 4 - 2; s.dw[i] = i % 4 - 2; s.widx[i] = i; }
+    s.out = (bf16*)y; s.addend = (const bf16*)addend;
+    s.out_H = c.OH; s.out_W = c.OW; s.out_C = c.cout; s.os = 1;
+    s.stats = stats;
+    s.epilogue = (impl & LP_CONV_DIRECT_EPILOGUE) ? 1 : ((impl & LP_CONV_STAGED_EPILOGUE) ? 2 : 0);
+    if (stats_done) *stats_done = stats != nullptr;
+    ProfScope ps(h, st, 2.0 * N * c.OH * c.OW * (double)c.cout * c.R * c.R * c.cin);
+    return launch_conv_tc(h, s, dev_err, st);
+  }
   const bool use_tc = dtype == LP_BF16 && (impl & 15) != LP_CONV_IMPL_SIMT && !(impl & 16) && tc_fwd_ok(c) && c.wf;
   if ((impl & 15) == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
   if (loss && !use_tc) return LP_ERR_UNSUPPORTED;  // the planner fuses the loss only into tensor-core convolutions
@@ -886,6 +918,24 @@ static int conv_dgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
 // dw += x (*) dy     (dw zeroed by the caller beforehand)
 static int conv_wgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N, const void* x, const void* dy,
                       float* dw, int* dev_err, cudaStream_t st) {
+  if (c.s2d) {
+    // weight gradient of the regrouped 4x4 convolution (x is the image: its regrouped copy was kept by the
+    // forward pass), then the real filter positions are picked out of it
+    LP_CUDA_OK(cudaMemsetAsync(c.dws, 0, (size_t)c.cout * 256 * 4, st));
+    Device& D = cur_dev();
+    {
+      ProfScope ps(h, st, 2.0 * N * c.OH * c.OW * (double)c.cout * c.R * c.R * c.cin);
+      int rc = launch_wgrad_tc(D.encode, D.sm_count, &D.wgrad_attr, &D.wgrad_halo_attr, c.xs, (const bf16*)dy, c.dws, N, c.H / 2,
+                               c.W / 2, 16, c.OH, c.OW, c.cout, 4, 1, 2, dev_err, st);
+      if (h) h->launches++;
+      if (rc != LP_OK) return rc;
+    }
+    const int total = c.cout * 49 * c.cin;
+    s2d_unpack_wgrad_kernel<<<grid_for(total, 256, D.sm_count, 8), 256, 0, st>>>(c.dws, dw, c.cout, c.cin);
+    if (h) h->launches++;
+    LP_CUDA_OK(cudaGetLastError());
+    return LP_OK;
+  }
   const bool use_tc = dtype == LP_BF16 && (impl & 15) != LP_CONV_IMPL_SIMT && !(impl & 64) && tc_wgrad_ok(c);
   if ((impl & 15) == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
   if (use_tc) {
@@ -997,6 +1047,12 @@ struct Planner {
       P.ps.pack_total += (long long)n;
       P.ps.pack_tiles += (long long)R * R * ((cin + 31) / 32) * ((cout + 31) / 32);
       P.ps.host_pack.push_back(pe);
+    } else if (dtype == LP_BF16 && impl != LP_CONV_IMPL_SIMT && !(net.d.conv_impl & 16) && !(net.d.conv_impl & 64) &&
+               !need_dgrad && s2d_stem_ok(c)) {
+      c.s2d = true;
+      c.wf = (bf16*)A.alloc((size_t)cout * 256 * 2);
+      c.dws = (float*)A.alloc((size_t)cout * 256 * 4);
+      c.xs = (bf16*)A.alloc((size_t)net.d.N * (H / 2) * (W / 2) * 16 * 2);
     }
     P.convs.push_back(c);
     return (int)P.convs.size() - 1;
@@ -1038,7 +1094,7 @@ struct Planner {
   }
 
   bool conv_fuses_stats(const ConvDef& c) const {
-    return dtype == LP_BF16 && impl != LP_CONV_IMPL_SIMT && !(net.d.conv_impl & 16) && tc_fwd_ok(c) && c.wf;
+    return dtype == LP_BF16 && impl != LP_CONV_IMPL_SIMT && !(net.d.conv_impl & 16) && (tc_fwd_ok(c) || c.s2d) && c.wf;
   }
   Tensor emit_conv(Plan& P, std::vector<Op>& ops, const Tensor& in, int conv, const Tensor* addend, int stats_bn) {
     const ConvDef& c = P.convs[conv];
@@ -1542,7 +1598,8 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       break;
     }
     case OP_MAXPOOL_FWD: {
-      const long long total = op.out.elems();
+      if (op.out.c % V) return LP_ERR_UNSUPPORTED;
+      const long long total = op.out.elems() / V;
       maxpool_fwd_kernel<T><<<grid_for(total, 256, cur_dev().sm_count, 16), 256, 0, st>>>(
           (const T*)resolve(op.in, c), (T*)resolve(op.out, c), op.arg, op.in.n, op.in.h, op.in.w, op.in.c, op.out.h,
           op.out.w);
@@ -1550,7 +1607,8 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       break;
     }
     case OP_MAXPOOL_BWD: {
-      const long long total = op.out.elems();
+      if (op.out.c % V) return LP_ERR_UNSUPPORTED;
+      const long long total = op.out.elems() / V;
       maxpool_bwd_kernel<T><<<grid_for(total, 256, cur_dev().sm_count, 16), 256, 0, st>>>(
           (const T*)resolve(op.in, c), op.arg, (T*)resolve(op.out, c), op.out.n, op.out.h, op.out.w, op.out.c, op.in.h,
           op.in.w);
@@ -1655,7 +1713,23 @@ static int zero_forward_state(Plan& P, cudaStream_t st) {
   return LP_OK;
 }
 
+// bf16 copies of the regrouped stem weights (space-to-depth stems), after every change of the master weights
+static int pack_s2d_weights(lp_handle* h, Plan& P, cudaStream_t st) {
+  for (const ConvDef& c : P.convs) {
+    if (!c.s2d) continue;
+    s2d_pack_weights_kernel<<<grid_for((long long)c.cout * 256, 256, cur_dev().sm_count, 8), 256, 0, st>>>(c.w, c.wf, c.cout,
+                                                                                                          c.cin);
+    h->launches++;
+    LP_CUDA_OK(cudaGetLastError());
+  }
+  return LP_OK;
+}
+
 static int pack_weights(lp_handle* h, Plan& P, cudaStream_t st) {
+  {
+    int rc = pack_s2d_weights(h, P, st);
+    if (rc != LP_OK) return rc;
+  }
   if (P.ps.host_pack.empty()) return LP_OK;
   pack_weights_tiled_kernel<<<(unsigned)P.ps.pack_tiles, dim3(32, 8), 0, st>>>(P.ps.dev_pack,
                                                                               (int)P.ps.host_pack.size());
@@ -1666,7 +1740,13 @@ static int pack_weights(lp_handle* h, Plan& P, cudaStream_t st) {
 
 // theta <- theta - lr*(g + wd*theta [momentum]) and, for the tensor-core path, fresh bf16 copies of
 // the convolution weights: one fused pass over the packed weights plus a small one over the rest.
+static int sgd_update_inner(lp_handle* h, Plan& P, float lr, float momentum, float weight_decay, cudaStream_t st);
 static int sgd_update(lp_handle* h, Plan& P, float lr, float momentum, float weight_decay, cudaStream_t st) {
+  int rc = sgd_update_inner(h, P, lr, momentum, weight_decay, st);
+  if (rc != LP_OK) return rc;
+  return pack_s2d_weights(h, P, st);
+}
+static int sgd_update_inner(lp_handle* h, Plan& P, float lr, float momentum, float weight_decay, cudaStream_t st) {
   float* mom = momentum != 0.f ? P.ps.m : nullptr;
   if (P.ps.host_pack.empty()) {
     sgd_kernel<<<grid_for((long long)P.ps.n, 256, cur_dev().sm_count, 8), 256, 0, st>>>(P.ps.p, P.ps.g, P.ps.m,

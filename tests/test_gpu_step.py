@@ -227,6 +227,17 @@ def test_local_loss_sums_with_160_channels_match_a_host_sum(loss):
     assert abs(loss_dev[0, 0] - want) < 2e-3 * abs(want)
 
 
+@pytest.mark.parametrize("impl", [0, 64])
+def test_bf16_stem_7x7_stride_2_on_tensor_cores(impl):
+    """The ImageNet-shaped stem (7x7 / stride 2 / pad 3, 3 input channels, max-pool) of a bf16 network runs on
+    the tensor cores by space-to-depth (a 4x4 stride-1 convolution over 2x2 pixel blocks): module 0's
+    gradients, stem weights included, at a flat 2e-2 against the storage-model oracle.  impl = 64 keeps the
+    weight gradients on the CUDA cores (the stem then takes the plain kernels): same bound."""
+    cfg = small_cfg("postbn", stem="conv7x7s2_maxpool", N=6, H=48, W=40, dtype="bf16", stem_channels=16,
+                    stage_channels=(16, 32), stage_blocks=(1, 1), module_block_end=(1, 2), classes=10)
+    flat_module_parity(cfg, impl, 2e-2)
+
+
 def test_resnet56_reduced_batch_bf16():
     full_step_parity(scaled("resnet56", N=16), steps=1)
 
