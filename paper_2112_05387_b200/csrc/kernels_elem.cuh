@@ -72,13 +72,22 @@ __global__ void bn_stats_kernel(const T* __restrict__ x, long long total_vecs, i
 #pragma unroll
   for (int j = 0; j < V; ++j) s[j] = q[j] = 0.f;
   const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_vecs; i += stride) {
-    float f[V];
-    ldv(x + i * V, f);
+  constexpr int U = 4;   // loads of a trip issued before the first use (see bn_apply_kernel)
+  for (long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i0 < total_vecs; i0 += U * stride) {
+    uint4 rf[U];
 #pragma unroll
-    for (int j = 0; j < V; ++j) {
-      s[j] += f[j];
-      q[j] += f[j] * f[j];
+    for (int u = 0; u < U; ++u)
+      if (i0 + u * stride < total_vecs) rf[u] = ld_raw(x + (i0 + u * stride) * V);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (i0 + u * stride >= total_vecs) break;
+      float f[V];
+      cvt_raw(rf[u], f);
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        s[j] += f[j];
+        q[j] += f[j] * f[j];
+      }
     }
   }
 #pragma unroll
@@ -824,15 +833,31 @@ __global__ void sgd_pack_tiled_kernel(const PackEntry* __restrict__ tab, int n_e
   const int co0 = (r % tiles_co) << 5;
   const int t = r / tiles_co;
   const int tx = threadIdx.x, ty = threadIdx.y;
-  for (int i = ty; i < 32; i += 8) {
-    const int co = co0 + i, ci = ci0 + tx;
+  // all loads of the thread's four elements first (independent requests in flight), then the arithmetic and stores
+  float pv[4], gv[4], mv[4];
+  const int ci = ci0 + tx;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int co = co0 + ty + 8 * q;
+    pv[q] = gv[q] = mv[q] = 0.f;
+    if (co < e.cout && ci < e.cin) {
+      const long long j = base + ((long long)co * e.taps + t) * e.cin + ci;
+      pv[q] = p_base[j];
+      gv[q] = g_base[j];
+      if (momentum != 0.f) mv[q] = m_base[j];
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int i = ty + 8 * q;
+    const int co = co0 + i;
     float v = 0.f;
     if (co < e.cout && ci < e.cin) {
       const long long j = ((long long)co * e.taps + t) * e.cin + ci;
-      v = p_base[base + j];
-      float gi = g_base[base + j] + wd * v;
+      v = pv[q];
+      float gi = gv[q] + wd * v;
       if (momentum != 0.f) {
-        gi = momentum * m_base[base + j] + gi;
+        gi = momentum * mv[q] + gi;
         m_base[base + j] = gi;
       }
       v -= lr * gi;
@@ -844,8 +869,8 @@ __global__ void sgd_pack_tiled_kernel(const PackEntry* __restrict__ tab, int n_e
   if (!e.wt) return;
   __syncthreads();
   for (int i = ty; i < 32; i += 8) {
-    const int ci = ci0 + i, co = co0 + tx;
-    if (co < e.cout && ci < e.cin) e.wt[((long long)ci * e.taps + t) * e.cout + co] = __float2bfloat16_rn(tile[tx][i]);
+    const int ci2 = ci0 + i, co = co0 + tx;
+    if (co < e.cout && ci2 < e.cin) e.wt[((long long)ci2 * e.taps + t) * e.cout + co] = __float2bfloat16_rn(tile[tx][i]);
   }
 }
 

@@ -364,6 +364,9 @@ static const size_t kTcMaxSmem = 220 * 1024;
 #ifndef LP_CONV_MAX_NB
 #define LP_CONV_MAX_NB 8   // weight stages in flight (halo mode), as far as shared memory allows
 #endif
+#ifndef LP_CONV_MAX_ITEMS_PER_STAGE
+#define LP_CONV_MAX_ITEMS_PER_STAGE 16   // (tap, chunk) items per pipeline stage of the plain mode, at most
+#endif
 #ifndef LP_CONV_TAPS_PER_STAGE
 #define LP_CONV_TAPS_PER_STAGE 2   // taps per weight stage (halo mode), as far as three stages still fit
 #endif
@@ -631,7 +634,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     // fixed cost of a stage once per several taps; wide layers keep one item per stage.
     {
       const int kiters = p.ntaps * p.chunks;
-      int ips = (int)std::min<size_t>((size_t)kiters, (kTcMaxSmem - tail) / 3 / p.item_bytes);
+      int ips = (int)std::min<size_t>((size_t)std::min(kiters, LP_CONV_MAX_ITEMS_PER_STAGE), (kTcMaxSmem - tail) / 3 / p.item_bytes);
       ips = std::max(ips, 1);
       const int n_st = (kiters + ips - 1) / ips;
       p.ips = (kiters + n_st - 1) / n_st;
