@@ -15,7 +15,7 @@
 // three taps of one kernel row read the same x pixels shifted by one pixel each, so ONE x box with
 // a one-pixel halo in w serves all three (see that kernel), which halves the bytes per MMA.
 //
-// Roles (224 threads): warps 0 and 6 = TMA producers (x and dy), warp 1 = MMA issuer, warps 2..5 =
+// Roles (256 threads): warps 0 and 6 = TMA producers (x and dy), warps 1 and 7 = MMA issuers, warps 2..5 =
 // epilogue.
 #pragma once
 #include <algorithm>
@@ -69,7 +69,7 @@ struct WgSmemTail {
   int epi_ok;
 };
 
-__global__ void __launch_bounds__(224, 1)
+__global__ void __launch_bounds__(256, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmDY,
                 const __grid_constant__ CUtensorMap tmDW, const __grid_constant__ WgradParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -88,9 +88,9 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(&tail->full[s], 2);    // one expect_tx arrival per producer warp
-      mbar_init(&tail->empty[s], 1);
+      mbar_init(&tail->empty[s], 2);   // one arrival per MMA warp
     }
-    mbar_init(&tail->acc_full, 1);
+    mbar_init(&tail->acc_full, 2);
     tail->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmX);
@@ -159,7 +159,12 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       __syncwarp();
       if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 || warp == 7) {
+    // Two MMA-issuing warps (one thread cannot keep the tensor pipe full): warp 1 owns the first row tile of
+    // the CTA, warp 7 the second one of a pair.  Both wait for every stage and both arrive on its "empty"
+    // barrier: with a commit after their MMAs, or (warp 7 with a single row tile) with a plain arrive.
+    const bool active = warp == 1 || cnt == 2;
+    const uint32_t acc_col = warp == 1 ? 0u : 256u;
     uint32_t s = 0, ph = 0;
     const uint32_t smem_base = smem_u32(smem);
     const int ksteps = p.rows_pad >> 4;
@@ -168,22 +173,25 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       if (!mbar_wait_warp(&tail->full[s], ph, abort_flag)) { failed = true; break; }
       tc_fence_after();
       const uint32_t a_addr = smem_base + s * p.stage_bytes;
-      const uint64_t ad = smem_desc(p.adesc_hi, a_addr), bd = smem_desc(p.bdesc_hi, a_addr + p.a_region);
-      const uint64_t ad1 = smem_desc(p.adesc_hi, a_addr + p.rpt * p.a_sub_bytes);
+      const uint64_t bd = smem_desc(p.bdesc_hi, a_addr + p.a_region);
+      const uint64_t ad = smem_desc(p.adesc_hi, a_addr + (warp == 1 ? 0u : (uint32_t)(p.rpt * p.a_sub_bytes)));
       if (elect_one()) {
-        for (int j = 0; j < ksteps; ++j) {
-          mma_bf16(tmem_base, ad + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, (it | j) ? 1u : 0u);
-          if (cnt == 2)
-            mma_bf16(tmem_base + 256, ad1 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc,
-                     (it | j) ? 1u : 0u);
+        if (active) {
+          for (int j = 0; j < ksteps; ++j)
+            mma_bf16(tmem_base + acc_col, ad + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, (it | j) ? 1u : 0u);
+          mma_commit(&tail->empty[s]);
+        } else {
+          mbar_arrive(&tail->empty[s]);
         }
-        mma_commit(&tail->empty[s]);
       }
       __syncwarp();
       if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
     }
     if (!failed && n_iter > 0) {
-      if (elect_one()) mma_commit(&tail->acc_full);
+      if (elect_one()) {
+        if (active) mma_commit(&tail->acc_full);
+        else mbar_arrive(&tail->acc_full);
+      }
       __syncwarp();
     }
   } else {
@@ -286,9 +294,9 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 // descriptor's leading byte offset is the distance between their first rows: 128 bytes inside a
 // box, (box size - 256) across the two boxes.  Per 128 pixels of K a CTA fetches x boxes of 40 KB and
 // the dy tile (128 x n_tile) for 24 MMAs, against 6 sub-boxes (96 KB) without the reuse.
-// Roles as in wgrad_tc_kernel.
+// Roles as in wgrad_tc_kernel, plus a second MMA-issuing warp (warp 7; 256 threads).
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(224, 1)
+__global__ void __launch_bounds__(256, 1)
 wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmDY,
                   const __grid_constant__ CUtensorMap tmDW, const __grid_constant__ WgradParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -306,9 +314,9 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(&tail->full[s], 2);
-      mbar_init(&tail->empty[s], 1);
+      mbar_init(&tail->empty[s], 2);     // one commit per MMA-issuing warp
     }
-    mbar_init(&tail->acc_full, 1);
+    mbar_init(&tail->acc_full, 2);
     tail->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmX);
@@ -353,7 +361,11 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       __syncwarp();
       if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 || warp == 7) {
+    // Two MMA-issuing warps: a tcgen05.mma costs its issuing thread nearly as long as the tensor pipe works on
+    // it, so one thread cannot keep the pipe full.  Warp 1 owns accumulators 0 and 1, warp 7 accumulator 2;
+    // both wait for every stage and both commit on its "empty" barrier.
+    const bool first = warp == 1;
     uint32_t s = 0, ph = 0;
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t a_kstep = p.a_kstep_bytes >> 4, b_kstep = (uint32_t)(16 * p.scb * 2) >> 4;
@@ -370,9 +382,12 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 #pragma unroll 1
         for (int j = 0; j < ksteps; ++j) {
           const uint32_t acc = (it | j) ? 1u : 0u;
-          mma_bf16(tmem_base, ad0 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
-          mma_bf16(tmem_base + p.acc_stride, ad1 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
-          mma_bf16(tmem_base + 2 * p.acc_stride, ad2 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
+          if (first) {
+            mma_bf16(tmem_base, ad0 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
+            mma_bf16(tmem_base + p.acc_stride, ad1 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
+          } else {
+            mma_bf16(tmem_base + 2 * p.acc_stride, ad2 + (uint64_t)(j * a_kstep), bd + (uint64_t)(j * b_kstep), p.idesc, acc);
+          }
         }
         mma_commit(&tail->empty[s]);
       }
@@ -613,7 +628,7 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, bool* attr_done, cons
     *attr_done = true;
   }
   dim3 grid(tiles, p.splits);
-  return launch_pdl(tc::wgrad_halo_kernel, grid, dim3(224), smem, st, tmX, tmDY, tmDW, p) == cudaSuccess ? 0 : -8;
+  return launch_pdl(tc::wgrad_halo_kernel, grid, dim3(256), smem, st, tmX, tmDY, tmDW, p) == cudaSuccess ? 0 : -8;
 }
 
 static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, bool* attr_done, bool* halo_attr_done, const bf16* x,
@@ -729,7 +744,7 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, bool* attr_done, bool* 
     *attr_done = true;
   }
   dim3 grid(tiles, p.splits);
-  return launch_pdl(tc::wgrad_tc_kernel, grid, dim3(224), smem, st, tmX, tmDY, tmDW, p) == cudaSuccess ? 0 : -8;
+  return launch_pdl(tc::wgrad_tc_kernel, grid, dim3(256), smem, st, tmX, tmDY, tmDW, p) == cudaSuccess ? 0 : -8;
 }
 
 }  // namespace lp
