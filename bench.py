@@ -366,17 +366,24 @@ def run_ours(args):
             step()
             loss_host.copy_(d_loss, non_blocking=True)
         barrier()
-        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        f0.record(stream)
-        for _ in range(args.steps):
-            d_images.copy_(images_host, non_blocking=True)
-            d_labels.copy_(labels_host, non_blocking=True)
-            step()
-            loss_host.copy_(d_loss, non_blocking=True)
-            stream.synchronize()             # the caller reads the losses before the next step
-        f1.record(stream)
-        barrier()
-        ms_e2e = f0.elapsed_time(f1)
+        # same scheme as above: the region of `steps` steps is repeated until half of --min-seconds has been
+        # measured, and the median repeat is reported
+        e2e_reps = []
+        while True:
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0.record(stream)
+            for _ in range(args.steps):
+                d_images.copy_(images_host, non_blocking=True)
+                d_labels.copy_(labels_host, non_blocking=True)
+                step()
+                loss_host.copy_(d_loss, non_blocking=True)
+                stream.synchronize()             # the caller reads the losses before the next step
+            f1.record(stream)
+            barrier()
+            e2e_reps.append(f0.elapsed_time(f1))
+            if sum(e2e_reps) >= 0.5 * args.min_seconds * 1e3 or len(e2e_reps) >= 1000:
+                break
+        ms_e2e = float(np.median(e2e_reps))
         losses = loss_host.clone().numpy()
 
         # per-kernel timing of the tensor-core convolutions: modules one after another on one
