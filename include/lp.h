@@ -81,6 +81,13 @@ enum { LP_CONV_DIRECT_EPILOGUE = 256, LP_CONV_STAGED_EPILOGUE = 512 };
  * 64-channel K chunks run on pairs of CTAs (tcgen05 cta_group::2: two pixel tiles per instruction, each CTA
  * fetching half of every weight stage).  Same results as the one-CTA kernel. */
 enum { LP_CONV_TWO_CTA = 1024 };
+/* May be OR-ed into conv_impl: a tensor-core input-gradient convolution whose output is the dy of a batch norm
+ * takes the reduction pass of that batch norm's backward (sum dy_m, sum dy_m * xhat) in its epilogue, and only the
+ * apply pass is left to run (Eq. Parallel-ResNet-Backpropagation: a module's backward pass is the chain
+ * conv^T -> BN' -> conv^T ...; the sums are taken where dy is produced).  Same gradients up to the order of fp32
+ * additions.  Not the default: the epilogue's extra shared-memory traffic costs the convolution more than the
+ * separate kernel takes. */
+enum { LP_CONV_BN_REDUCE_IN_EPILOGUE = 2048 };
 enum { LP_CONV_FWD = 0, LP_CONV_DGRAD = 1, LP_CONV_WGRAD = 2 };
 
 #define LP_MAX_STAGES 8

@@ -76,6 +76,29 @@ __device__ __forceinline__ float round_storage(float v) {
   return to_f(t);
 }
 
+// Training-mode batch norm of one tensor: per-channel sums of the batch and the affine parameters.
+struct BnArgs {
+  const double* stats;  // [2*C]: per-channel sum, sum of squares
+  const float* gamma;
+  const float* beta;
+  double inv_count;     // 1 / (N*H*W)
+  float eps;
+};
+
+// Mean and 1/sqrt(var + eps) of one channel from its sums.  Every kernel that normalises, or that
+// recomputes a ReLU mask from a normalised value, goes through this function, so that all of them
+// see the same two numbers.
+__device__ __forceinline__ void bn_mean_rstd(double s1, double s2, double inv_count, float eps, float& mean, float& rstd) {
+  const double m = s1 * inv_count;
+  const double var = fma(-m, m, s2 * inv_count);
+  mean = (float)m;
+  const float v = fmaxf((float)var, 0.f) + eps;
+  float r = rsqrtf(v);
+  r = r * fmaf(-0.5f * v * r, r, 1.5f);
+  rstd = r;
+}
+
+
 // Programmatic dependent launch.  A kernel launched with the programmatic-serialisation attribute
 // may start while the kernel before it in the stream is still draining: everything up to
 // pdl_wait() (barrier set-up, tensor-memory allocation, constants) overlaps that tail; pdl_wait()

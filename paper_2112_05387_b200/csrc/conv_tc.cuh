@@ -104,6 +104,16 @@ struct ConvTcParams {
   int wide32;                    // output (and residual) rows can be accessed in 32-byte pieces
   // staged epilogue (kStaged instantiations): the output tile goes through shared memory and leaves by TMA
   uint32_t stage_offset;         // staging region: one 128-row x 64-byte group per 32 output channels of the tile
+  // Reduction pass of a batch-norm backward, fused into the epilogue (kBnBwd instantiations).  The
+  // output of this convolution is dy, the gradient with respect to the result of y = [relu](bn(x));
+  // the epilogue adds  sum dy_m  to dbeta and  rstd * sum dy_m (x - mean)  to dgamma, with
+  // dy_m = dy where the ReLU let the value pass (recomputed from x as the forward kernel did), so
+  // that only the apply pass of the batch-norm backward is left to run afterwards.
+  const bf16* bwd_x;             // the tensor the batch norm normalised; same geometry as out
+  BnArgs bwd_bn;                 // its statistics and affine parameters
+  float* bwd_dgamma;             // [Cout], atomically added
+  float* bwd_dbeta;
+  int bwd_relu;                  // 1: a ReLU followed the batch norm
 };
 
 struct TcSmemTail {
@@ -123,6 +133,11 @@ struct TcStatScratch {
   float ssum[LP_EPI_WARPS][256];   // per epilogue warp: plain read-modify-write, no shared-memory atomics
   float ssq[LP_EPI_WARPS][256];
   uint32_t tr[LP_EPI_WARPS][16 * 33];   // per epilogue warp: transposition scratch of the statistics
+};
+// Additional scratch of the fused batch-norm-backward sums, placed right after TcStatScratch.
+struct TcBnBwdScratch {
+  uint32_t tr2[LP_EPI_WARPS][16 * 33];  // transposition scratch of the normalised tensor's tile
+  float4 consts[256];                   // per channel of the current channel tile: scale, shift, mean, rstd
 };
 constexpr uint32_t kTailBytes = (uint32_t)((sizeof(TcSmemTail) + 127) / 128 * 128);
 constexpr uint32_t kStageGroupBytes = 128 * 64;   // staging: 128 tile rows x 32 bf16 channels
@@ -153,16 +168,20 @@ constexpr int kEpiGroups = LP_EPI_WARPS / 4;
 //   memory then sees whole 64-byte row pieces written by the copy engine instead of 16- or 32-byte
 //   stores 2 x C_out bytes apart across the lanes of a warp, and the per-channel statistics are column
 //   sums over the staged tile.  tmOut / tmAdd are only read by these instantiations.
-template <bool kLoss, bool kAddend, bool kStaged>
+// kBnBwd: the direct epilogue also takes the reduction pass of the batch-norm backward that consumes
+//   this convolution's output (see ConvTcParams::bwd_x).
+template <bool kLoss, bool kAddend, bool kStaged, bool kBnBwd = false>
 __global__ void __launch_bounds__(kConvThreads, LP_CONV_MIN_BLOCKS)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmAdd,
                const __grid_constant__ ConvTcParams p) {
   static_assert(!(kStaged && kLoss), "the fused local loss uses the direct epilogue");
+  static_assert(!(kBnBwd && (kStaged || kLoss)), "the fused batch-norm sums use the plain direct epilogue");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   TcSmemTail* tail = reinterpret_cast<TcSmemTail*>(smem + p.tail_offset);
   TcStatScratch* scratch = reinterpret_cast<TcStatScratch*>(smem + p.tail_offset + kTailBytes);
+  TcBnBwdScratch* bscratch = reinterpret_cast<TcBnBwdScratch*>(smem + p.tail_offset + kTailBytes + sizeof(TcStatScratch));
   volatile int* abort_flag = &tail->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -191,7 +210,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if constexpr (kAddend) prefetch_tmap(&tmAdd);
     }
   }
-  if (!kStaged && p.stats) {   // (without statistics the scratch is not part of the allocation)
+  if (!kStaged && (p.stats || kBnBwd)) {   // (without statistics the scratch is not part of the allocation)
     for (int i = threadIdx.x; i < LP_EPI_WARPS * 256; i += blockDim.x) {
       (&scratch->ssum[0][0])[i] = 0.f;
       (&scratch->ssq[0][0])[i] = 0.f;
@@ -577,11 +596,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint32_t slot = 0, slot_phase = 0;
     float sum_rr = 0.f, sum_kr = 0.f;    // local-loss sums of this thread (kLoss)
     int epi_turn = 0;
-    // The residual operand was written several kernels ago and is no longer in L2.  Each thread
-    // asks for the row of the NEXT tile it will add while it works on the current one, so that the
-    // loads of the epilogue find their lines in L2 instead of waiting for DRAM.
-    auto prefetch_addend = [&](int tile) {
-      if (!kAddend || tile >= t_end) return;
+    // The residual operand (and the tensor of a fused batch-norm backward) was written several kernels
+    // ago and is no longer in L2.  Each thread asks for the row of the NEXT tile it will read while it
+    // works on the current one, so that the loads of the epilogue find their lines in L2 instead of
+    // waiting for DRAM.
+    auto prefetch_rows = [&](const bf16* base, int tile) {
+      if (tile >= t_end) return;
       const int pnt = tile / p.m_tiles, pm = tile % p.m_tiles;
       const int pw = (pm % p.tiles_w) * p.BW + row % p.BW;
       const int phh = ((pm / p.tiles_w) % p.tiles_h) * p.BH + (p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH);
@@ -590,15 +610,39 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const long long pb =
           (((long long)pn * p.out_H + (phh * p.os + p.oo_h)) * p.out_W + (pw * p.os + p.oo_w)) * p.out_C + pnt * p.n_tile_cols;
       const int ncols = min(p.n_tile_cols, p.Cout - pnt * p.n_tile_cols);
-      const uintptr_t b = reinterpret_cast<uintptr_t>(p.addend + pb);
+      const uintptr_t b = reinterpret_cast<uintptr_t>(base + pb);
       for (uintptr_t l = b & ~(uintptr_t)127; l < b + 2 * (uintptr_t)ncols; l += 128)
         asm volatile("prefetch.global.L2 [%0];" ::"l"(l));
     };
+    auto prefetch_addend = [&](int tile) {
+      if constexpr (kAddend) prefetch_rows(p.addend, tile);
+      if constexpr (kBnBwd) prefetch_rows(p.bwd_x, tile);
+    };
     prefetch_addend(t_begin);
+    int consts_nt = -1;                  // channel tile whose batch-norm constants are in shared memory (kBnBwd)
     for (int t = t_begin; t < t_end && !failed;) {
       const int nt = t / p.m_tiles, m0 = t % p.m_tiles;
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m0 + 1 < p.m_tiles) ? 2 : 1;
       const int col0 = nt * p.n_tile_cols;
+      if constexpr (kBnBwd) {
+        if (nt != consts_nt) {
+          // scale, shift (the forward kernel's, for the ReLU mask), mean and rstd of this channel tile
+          asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+          for (int c = et; c < 256; c += kEpiThreads) {
+            float4 k4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c < p.n_tile_cols && col0 + c < p.Cout) {
+              float mean, rstd;
+              bn_mean_rstd(p.bwd_bn.stats[col0 + c], p.bwd_bn.stats[p.Cout + col0 + c], p.bwd_bn.inv_count, p.bwd_bn.eps,
+                           mean, rstd);
+              const float sa = p.bwd_bn.gamma[col0 + c] * rstd;
+              k4 = make_float4(sa, p.bwd_bn.beta[col0 + c] - mean * sa, mean, rstd);
+            }
+            bscratch->consts[c] = k4;
+          }
+          asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+          consts_nt = nt;
+        }
+      }
       for (int a = 0; a < cnt && !failed; ++a) {
         prefetch_addend(t + a + 1);
         const int m = m0 + a;
@@ -679,6 +723,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             float v[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = (wide || j < 16) ? __uint_as_float(raw[i][j]) : 0.f;
+            // this pixel's 32 channels of the tensor the batch norm normalised, asked for before the
+            // stores so that they have arrived when the sums need them
+            uint4 xr[kBnBwd ? 4 : 1];
+            if constexpr (kBnBwd) {
+#pragma unroll
+              for (int u = 0; u < 4; ++u)
+                xr[u] = (u < nv && valid && col + 8 * u < p.Cout) ? ld_raw(p.bwd_x + obase + col + 8 * u)
+                                                                  : make_uint4(0u, 0u, 0u, 0u);
+            }
             if constexpr (kAddend) {
               if (i + 1 < kBatch) load_addend(g + kEpiGroups, add_next);
 #pragma unroll
@@ -735,25 +788,56 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                   stv(p.seed_out + obase + col + 8 * u, sd);
                 }
             }
-            if (p.stats) {
+            if (kBnBwd || p.stats) {
               // Statistics of the tensor as stored (bf16), so that the batch-norm that follows
               // normalises exactly the values it reads.  A thread holds one pixel and 32 channels;
               // the sums run over pixels, so the warp transposes through shared memory: every lane
               // writes its 16 channel pairs, then lane l sums channel pair (l & 15) over 16 of the
               // warp's 32 pixels (both phases conflict-free with the row pitch of 33 words).
+              // kBnBwd: the two sums are those of a batch-norm backward, sum dy_m and
+              // sum dy_m (x - mean), and the tile of x is transposed beside the tile of dy.
               uint32_t* T = scratch->tr[warp - kFirstEpiWarp];
 #pragma unroll
               for (int j = 0; j < 16; ++j) T[j * 33 + lane] = (valid && (wide || j < 8)) ? pk[j] : 0u;
+              if constexpr (kBnBwd) {
+                uint32_t* T2 = bscratch->tr2[warp - kFirstEpiWarp];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                  const bool on = valid && (wide || u < 2);
+                  T2[(4 * u + 0) * 33 + lane] = on ? xr[u].x : 0u;
+                  T2[(4 * u + 1) * 33 + lane] = on ? xr[u].y : 0u;
+                  T2[(4 * u + 2) * 33 + lane] = on ? xr[u].z : 0u;
+                  T2[(4 * u + 3) * 33 + lane] = on ? xr[u].w : 0u;
+                }
+              }
               __syncwarp();
               const int jc = lane & 15, hh = lane >> 4;
               const uint32_t* col_t = T + jc * 33 + hh * 16;
               float s0 = 0.f, s1 = 0.f, q0 = 0.f, q1 = 0.f;
+              if constexpr (kBnBwd) {
+                const uint32_t* col_x = bscratch->tr2[warp - kFirstEpiWarp] + jc * 33 + hh * 16;
+                const float4 k0 = bscratch->consts[c_in_tile + 2 * jc], k1 = bscratch->consts[c_in_tile + 2 * jc + 1];
+                const bool relu = p.bwd_relu != 0;
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const uint32_t w2 = col_t[i];
-                const float lo = __uint_as_float(w2 << 16), hi = __uint_as_float(w2 & 0xFFFF0000u);
-                s0 += lo; s1 += hi;
-                q0 = fmaf(lo, lo, q0); q1 = fmaf(hi, hi, q1);
+                for (int i2 = 0; i2 < 16; ++i2) {
+                  const uint32_t w2 = col_t[i2], x2 = col_x[i2];
+                  float dlo = __uint_as_float(w2 << 16), dhi = __uint_as_float(w2 & 0xFFFF0000u);
+                  const float xlo = __uint_as_float(x2 << 16), xhi = __uint_as_float(x2 & 0xFFFF0000u);
+                  if (relu) {
+                    dlo = fmaf(xlo, k0.x, k0.y) > 0.f ? dlo : 0.f;
+                    dhi = fmaf(xhi, k1.x, k1.y) > 0.f ? dhi : 0.f;
+                  }
+                  s0 += dlo; s1 += dhi;
+                  q0 = fmaf(dlo, xlo - k0.z, q0); q1 = fmaf(dhi, xhi - k1.z, q1);
+                }
+              } else {
+#pragma unroll
+                for (int i2 = 0; i2 < 16; ++i2) {
+                  const uint32_t w2 = col_t[i2];
+                  const float lo = __uint_as_float(w2 << 16), hi = __uint_as_float(w2 & 0xFFFF0000u);
+                  s0 += lo; s1 += hi;
+                  q0 = fmaf(lo, lo, q0); q1 = fmaf(hi, hi, q1);
+                }
               }
               __syncwarp();
               s0 += __shfl_xor_sync(0xffffffffu, s0, 16);
@@ -770,7 +854,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         slot = slot + 1 == (uint32_t)p.nslots ? 0 : slot + 1;
         // flush the column sums when the channel tile is about to change (or at the very end)
         const bool last_of_unit = a + 1 == cnt;
-        const bool flush = p.stats && last_of_unit && (t + cnt >= t_end || (t + cnt) / p.m_tiles != nt);
+        const bool flush = (kBnBwd || p.stats) && last_of_unit && (t + cnt >= t_end || (t + cnt) / p.m_tiles != nt);
         if (flush) {
           asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
           for (int c = et; c < p.n_tile_cols; c += kEpiThreads) {
@@ -782,8 +866,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               scratch->ssq[wi][c] = 0.f;
             }
             if (col0 + c < p.Cout) {
-              atomicAdd(&p.stats[col0 + c], (double)a_s);
-              atomicAdd(&p.stats[p.Cout + col0 + c], (double)a_q);
+              if constexpr (kBnBwd) {
+                atomicAdd(&p.bwd_dbeta[col0 + c], a_s);
+                atomicAdd(&p.bwd_dgamma[col0 + c], a_q * bscratch->consts[c].w);
+              } else {
+                atomicAdd(&p.stats[col0 + c], (double)a_s);
+                atomicAdd(&p.stats[p.Cout + col0 + c], (double)a_q);
+              }
             }
           }
           asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");

@@ -7,14 +7,6 @@
 
 namespace lp {
 
-struct BnArgs {
-  const double* stats;  // [2*C]: per-channel sum, sum of squares
-  const float* gamma;
-  const float* beta;
-  double inv_count;     // 1 / (N*H*W)
-  float eps;
-};
-
 // The constants of V consecutive channels c0..c0+V-1 (V = 4 or 8, c0 a multiple of V): mean,
 // 1/sqrt(var+eps), gamma, beta.  16-byte loads wherever the pointers allow: every thread of every
 // block runs this prologue, and scalar loads at a stride of V channels between neighbouring
@@ -47,15 +39,7 @@ __device__ __forceinline__ void bn_load_consts(const BnArgs& a, int C, int c0, f
     for (int j = 0; j < V; ++j) { gamma[j] = a.gamma[c0 + j]; beta[j] = a.beta[c0 + j]; }
   }
 #pragma unroll
-  for (int j = 0; j < V; ++j) {
-    const double m = s1[j] * a.inv_count;
-    const double var = fma(-m, m, s2[j] * a.inv_count);
-    mean[j] = (float)m;
-    const float v = fmaxf((float)var, 0.f) + a.eps;
-    float r = rsqrtf(v);
-    r = r * fmaf(-0.5f * v * r, r, 1.5f);
-    rstd[j] = r;
-  }
+  for (int j = 0; j < V; ++j) bn_mean_rstd(s1[j], s2[j], a.inv_count, a.eps, mean[j], rstd[j]);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -72,6 +72,12 @@ struct Op {
   int conv = -1, bn = -1, bn2 = -1, stats_bn = -1;
   int relu = 0;
   int fuse_loss = 0;       // conv: its epilogue takes the module's local loss; out_loss: only the final scalars are left
+  // Reduction pass of a batch-norm backward taken by the epilogue of the input-gradient convolution
+  // that writes its dy.  On the convolution: bwd_bn >= 0 names the batch norm, bwd_x the tensor it
+  // normalised, bwd_relu whether a ReLU followed.  On the batch-norm backward: reduce_fused = 1,
+  // only the apply pass is left.
+  int bwd_bn = -1, bwd_relu = 0, reduce_fused = 0;
+  Tensor bwd_x;
   uint8_t* arg = nullptr;  // max-pool argmax
 };
 
@@ -272,6 +278,8 @@ struct TcGemmSpec {
   const bf16* x_next; const bf16* kappa; bf16* r_out; bf16* seed_out; float rho; double* loss_acc;
   int epilogue;          // 0: default (staged where a residual operand exists), 1: direct, 2: staged wherever it applies
   int two_cta;           // 1: 3x3 stride-1 convolutions take the CTA-pair kernel where it applies
+  // reduction pass of a batch-norm backward fused into the epilogue; bwd_x == nullptr: off
+  const bf16* bwd_x; BnArgs bwd_bn; float* bwd_dgamma; float* bwd_dbeta; int bwd_relu;
 };
 
 static void pick_pixel_box(int OWl, int OHl, int Nimg, int& BW, int& BH, int& BNI) {
@@ -537,7 +545,9 @@ static int launch_conv_tc2(lp_handle* h, const TcGemmSpec& s, int* dev_err, cuda
 }
 
 static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaStream_t st) {
-  if (s.two_cta) {
+  const bool bnbwd = s.bwd_x != nullptr;
+  if (bnbwd && (s.stats || s.x_next)) return LP_ERR_UNSUPPORTED;
+  if (s.two_cta && !bnbwd) {
     const int rc2 = launch_conv_tc2(h, s, dev_err, st);
     if (rc2 != LP_ERR_UNSUPPORTED) return rc2;
   }
@@ -568,13 +578,14 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   const uint32_t b_region = (uint32_t)align_up((size_t)p.n_tile_cols * row_bytes, 1024);
   // Staged epilogue (output tile through shared memory, TMA stores, TMA-loaded residual): where the output
   // grid is the logical grid, the channel tile is a multiple of 32 and the tensors start on 16-byte boundaries.
-  const bool staged = (s.epilogue == 2 || (s.epilogue == 0 && s.addend != nullptr)) && !s.x_next && s.os == 1 && s.oo_h == 0 && s.oo_w == 0 &&
+  const bool staged = !bnbwd && (s.epilogue == 2 || (s.epilogue == 0 && s.addend != nullptr)) && !s.x_next && s.os == 1 && s.oo_h == 0 && s.oo_w == 0 &&
                       p.n_tile_cols % 32 == 0 && s.out_C % 8 == 0 && tc::kEpiThreads == 128 &&
                       (reinterpret_cast<uintptr_t>(s.out) & 15) == 0 &&
                       (!s.addend || (reinterpret_cast<uintptr_t>(s.addend) & 15) == 0);
   const size_t stage_bytes = staged ? (size_t)(p.n_tile_cols / 32) * tc::kStageGroupBytes : 0;
   // the direct epilogue's statistics scratch is only there when statistics are asked for
-  const size_t tail = tc::kTailBytes + ((staged || !s.stats) ? 0 : sizeof(tc::TcStatScratch)) + stage_bytes + 1024;
+  const size_t tail = tc::kTailBytes + ((staged || !(s.stats || bnbwd)) ? 0 : sizeof(tc::TcStatScratch)) +
+                      (bnbwd ? sizeof(tc::TcBnBwdScratch) : 0) + stage_bytes + 1024;
   p.tx_b = (uint32_t)(p.n_tile_cols * row_bytes);
   p.acc_stride = (p.n_tile_cols + 31) / 32 * 32;
   p.nslots = std::min(tc::kMaxSlots, tc::kTmemCols / p.acc_stride);
@@ -652,6 +663,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   p.out = s.out; p.addend = s.addend; p.stats = s.stats; p.err = dev_err;
   p.x_next = s.x_next; p.kappa = s.kappa; p.r_out = s.r_out; p.seed_out = s.seed_out; p.rho = s.rho;
   p.loss_acc = s.loss_acc;
+  p.bwd_x = s.bwd_x; p.bwd_bn = s.bwd_bn; p.bwd_dgamma = s.bwd_dgamma; p.bwd_dbeta = s.bwd_dbeta; p.bwd_relu = s.bwd_relu;
   // 32-byte epilogue accesses: rows and channel-group offsets are multiples of 32 bytes when the channel
   // count is a multiple of 16 and the tensors start on a 32-byte boundary (caller buffers need only 16)
   p.wide32 = (s.out_C % 16 == 0 && s.w_rows % 16 == 0 && p.n_tile_cols % 16 == 0 &&
@@ -688,6 +700,10 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
                                     (int)kTcMaxSmem));
     LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kTcMaxSmem));
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, false, false, true>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcMaxSmem));
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, true, false, true>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcMaxSmem));
     attr_set = true;
   }
   // Persistent CTAs walk contiguous tile ranges; the launch takes about as long as the CTA with the most
@@ -705,7 +721,9 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   if (s.x_next && !s.addend) return LP_ERR_UNSUPPORTED;   // the fused loss belongs to a convolution with a shortcut
   cudaError_t le;
   const dim3 g3(grid), b3(tc::kConvThreads);
-  if (s.x_next) le = launch_pdl(tc::conv_tc_kernel<true, true, false>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
+  if (bnbwd && s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true, false, true>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
+  else if (bnbwd) le = launch_pdl(tc::conv_tc_kernel<false, false, false, true>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
+  else if (s.x_next) le = launch_pdl(tc::conv_tc_kernel<true, true, false>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
   else if (staged && s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true, true>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
   else if (staged) le = launch_pdl(tc::conv_tc_kernel<false, false, true>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
   else if (s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true, false>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
@@ -722,6 +740,16 @@ static bool tc_fwd_ok(const ConvDef& c) {
 static bool tc_dgrad_ok(const ConvDef& c) {
   return tc_fwd_ok(c) && (c.stride == 1 || (c.H % 2 == 0 && c.W % 2 == 0));
 }
+// A stride-2 input gradient runs as one launch per parity class of the input pixels; a class that no
+// filter tap reaches (1x1 filters) is not written by any epilogue.
+static bool dgrad_has_empty_class(const ConvDef& c) {
+  for (int ph = 0; ph < c.stride; ++ph) {
+    int cnt = 0;
+    for (int r = 0; r < c.R; ++r) cnt += ((ph + c.pad - r) % c.stride == 0) ? 1 : 0;
+    if (cnt == 0) return true;
+  }
+  return false;
+}
 static bool tc_wgrad_ok(const ConvDef& c) {
   return c.cin % 8 == 0 && c.cout % 8 == 0 && (c.R == 1 || c.R == 3) && (c.stride == 1 || c.stride == 2);
 }
@@ -734,6 +762,12 @@ static bool s2d_stem_ok(const ConvDef& c) {
 // Local loss of an interior module computed by the epilogue of the module's last convolution.
 struct LossFuse {
   const void* x_next; const void* kappa; void* r_out; void* seed_out; float rho; double* acc;
+};
+
+// Reduction pass of the batch-norm backward that consumes an input gradient, taken by the epilogue
+// of the convolution that writes it.
+struct BnBwdFuse {
+  const void* x; BnArgs bn; float* dgamma; float* dbeta; int relu;
 };
 
 struct ProfScope {
@@ -857,9 +891,10 @@ static int conv_forward(lp_handle* h, int dtype, int impl, const ConvDef& c, int
 
 // dx = conv^T(dy, w) [+ addend]   (addend may alias dx)
 static int conv_dgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N, const void* dy, void* dx,
-                      const void* addend, int* dev_err, cudaStream_t st) {
+                      const void* addend, int* dev_err, cudaStream_t st, const BnBwdFuse* bnf = nullptr) {
   const bool use_tc = dtype == LP_BF16 && (impl & 15) != LP_CONV_IMPL_SIMT && !(impl & 32) && tc_dgrad_ok(c) && c.wt;
   if ((impl & 15) == LP_CONV_IMPL_TENSOR && !use_tc) return LP_ERR_UNSUPPORTED;
+  if (bnf && (!use_tc || dgrad_has_empty_class(c))) return LP_ERR_UNSUPPORTED;  // the planner fuses only where every pixel passes an epilogue
   if (use_tc) {
     const int st2 = c.stride;
     const int classes = st2 * st2;
@@ -899,7 +934,11 @@ static int conv_dgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
       s.out_H = c.H; s.out_W = c.W; s.out_C = c.cin; s.os = st2; s.oo_h = ph; s.oo_w = pw;
       s.stats = nullptr;
       s.epilogue = (impl & LP_CONV_DIRECT_EPILOGUE) ? 1 : ((impl & LP_CONV_STAGED_EPILOGUE) ? 2 : 0);
-    s.two_cta = (impl & LP_CONV_TWO_CTA) ? 1 : 0;
+      s.two_cta = (impl & LP_CONV_TWO_CTA) ? 1 : 0;
+      if (bnf) {
+        s.bwd_x = (const bf16*)bnf->x; s.bwd_bn = bnf->bn; s.bwd_dgamma = bnf->dgamma; s.bwd_dbeta = bnf->dbeta;
+        s.bwd_relu = bnf->relu;
+      }
       int rc = launch_conv_tc(h, s, dev_err, st);
       if (rc != LP_OK) return rc;
     }
@@ -1127,11 +1166,26 @@ struct Planner {
     return out;
   }
   // backward of y = bn(x) (dy optionally masked by a stored post-ReLU tensor); returns dx
-  Tensor emit_bn_bwd(std::vector<Op>& ops, const Tensor& dy, const Tensor& x, const Tensor* mask, int bn,
+  bool dgrad_fuses_bn_bwd(const ConvDef& c) const {
+    return (net.d.conv_impl & LP_CONV_BN_REDUCE_IN_EPILOGUE) && dtype == LP_BF16 && impl != LP_CONV_IMPL_SIMT &&
+           !(net.d.conv_impl & 32) && tc_dgrad_ok(c) && c.wt && !dgrad_has_empty_class(c);
+  }
+  Tensor emit_bn_bwd(Plan& P, std::vector<Op>& ops, const Tensor& dy, const Tensor& x, const Tensor* mask, int bn,
                      const Tensor* addend, const Tensor* out_override = nullptr) {
     Tensor out = out_override ? *out_override : new_tensor(x.n, x.h, x.w, x.c);
     Op op;
     op.type = OP_BN_BWD; op.in = dy; op.in2 = x; op.bn = bn; op.out = out;
+    // On request (LP_CONV_BN_REDUCE_IN_EPILOGUE): where the last kernel to write dy is a tensor-core input
+    // gradient, its epilogue takes this batch norm's reduction pass (one such consumer per convolution).
+    for (int i = (int)ops.size() - 1; i >= 0; --i) {
+      Op& w = ops[i];
+      if (!(w.out.p == dy.p && w.out.ext == dy.ext) || !w.out.defined()) continue;
+      if (w.type == OP_CONV_DGRAD && w.bwd_bn < 0 && dgrad_fuses_bn_bwd(P.convs[w.conv])) {
+        w.bwd_bn = bn; w.bwd_x = x; w.bwd_relu = mask ? 1 : 0;
+        op.reduce_fused = 1;
+      }
+      break;
+    }
     if (mask) op.mask = *mask;
     if (addend) op.addend = *addend;
     ops.push_back(op);
@@ -1327,7 +1381,7 @@ struct Planner {
       op.type = OP_HEAD_BWD; op.out = dh;
       Bw.push_back(op);
       dcur = dh;
-      if (!post) dcur = emit_bn_bwd(Bw, dh, cur, &head_o, head_bn, nullptr);
+      if (!post) dcur = emit_bn_bwd(P, Bw, dh, cur, &head_o, head_bn, nullptr);
     } else {
       dcur = P.seed;
     }
@@ -1345,19 +1399,19 @@ struct Planner {
       if (post) {
         Tensor dy2;
         if (bott) {
-          Tensor dy3 = emit_bn_bwd(Bw, dcur, r.y3, nullptr, r.bn3, nullptr);
+          Tensor dy3 = emit_bn_bwd(P, Bw, dcur, r.y3, nullptr, r.bn3, nullptr);
           emit_wgrad(Bw, r.a2, dy3, r.c3);
           Tensor da2 = emit_dgrad(P, Bw, dy3, r.c3, nullptr, nullptr);
-          dy2 = emit_bn_bwd(Bw, da2, r.y2, &r.a2, r.bn2, nullptr);
+          dy2 = emit_bn_bwd(P, Bw, da2, r.y2, &r.a2, r.bn2, nullptr);
         } else {
-          dy2 = emit_bn_bwd(Bw, dcur, r.y2, nullptr, r.bn2, nullptr);
+          dy2 = emit_bn_bwd(P, Bw, dcur, r.y2, nullptr, r.bn2, nullptr);
         }
         emit_wgrad(Bw, r.a1, dy2, r.c2);
         Tensor da1 = emit_dgrad(P, Bw, dy2, r.c2, nullptr, nullptr);
-        Tensor dy1 = emit_bn_bwd(Bw, da1, r.y1, &r.a1, r.bn1, nullptr);
+        Tensor dy1 = emit_bn_bwd(P, Bw, da1, r.y1, &r.a1, r.bn1, nullptr);
         emit_wgrad(Bw, r.x, dy1, r.c1);
         if (b.proj) {
-          Tensor dys = emit_bn_bwd(Bw, dcur, r.ys, nullptr, r.bns, nullptr);
+          Tensor dys = emit_bn_bwd(P, Bw, dcur, r.ys, nullptr, r.bns, nullptr);
           emit_wgrad(Bw, r.x, dys, r.cs);
           Tensor dx = emit_dgrad(P, Bw, dy1, r.c1, nullptr, dx_target);
           dcur = emit_dgrad(P, Bw, dys, r.cs, &dx, &dx);
@@ -1367,14 +1421,14 @@ struct Planner {
       } else {
         emit_wgrad(Bw, r.a1, dcur, r.c2);
         Tensor da1 = emit_dgrad(P, Bw, dcur, r.c2, nullptr, nullptr);
-        Tensor dy1 = emit_bn_bwd(Bw, da1, r.y1, &r.a1, r.bn2, nullptr);
+        Tensor dy1 = emit_bn_bwd(P, Bw, da1, r.y1, &r.a1, r.bn2, nullptr);
         emit_wgrad(Bw, r.o, dy1, r.c1);
         Tensor dO = emit_dgrad(P, Bw, dy1, r.c1, nullptr, nullptr);
         if (b.proj) {
           emit_wgrad(Bw, r.o, dcur, r.cs);
           dO = emit_dgrad(P, Bw, dcur, r.cs, &dO, &dO);
         }
-        dcur = emit_bn_bwd(Bw, dO, r.x, &r.o, r.bn1, b.proj ? nullptr : &dcur, dx_target);
+        dcur = emit_bn_bwd(P, Bw, dO, r.x, &r.o, r.bn1, b.proj ? nullptr : &dcur, dx_target);
       }
     }
     if (k == 0) {
@@ -1387,7 +1441,7 @@ struct Planner {
           Bw.push_back(op);
           dstem = dpool;
         }
-        dstem = emit_bn_bwd(Bw, dstem, stem_y, &stem_a, stem_bn, nullptr);
+        dstem = emit_bn_bwd(P, Bw, dstem, stem_y, &stem_a, stem_bn, nullptr);
       }
       emit_wgrad(Bw, x, dstem, stem_conv);
     }
@@ -1461,7 +1515,7 @@ struct Planner {
     Tensor d = P.seed;
     for (int i = (int)cv.size() - 1; i >= 0; --i) {
       const bool relu_after = i + 1 < (int)cv.size();
-      Tensor dy = emit_bn_bwd(P.bwd, d, ys[i], relu_after ? &acts[i] : nullptr, bi[i], nullptr);
+      Tensor dy = emit_bn_bwd(P, P.bwd, d, ys[i], relu_after ? &acts[i] : nullptr, bi[i], nullptr);
       emit_wgrad(P.bwd, ins[i], dy, ci[i]);
       if (i > 0) d = emit_dgrad(P, P.bwd, dy, ci[i], nullptr, nullptr);
       else if (dx_out) emit_dgrad(P, P.bwd, dy, ci[i], nullptr, dx_out);
@@ -1514,8 +1568,15 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
     case OP_CONV_DGRAD: {
       const ConvDef& cv = P.convs[op.conv];
       const void* addend = op.addend.defined() ? resolve(op.addend, c) : nullptr;
+      BnBwdFuse bf;
+      const BnBwdFuse* bfp = nullptr;
+      if (op.bwd_bn >= 0) {
+        const BnDef& b = P.bns[op.bwd_bn];
+        bf.x = resolve(op.bwd_x, c); bf.bn = bn_args(b, eps); bf.dgamma = b.dgamma; bf.dbeta = b.dbeta; bf.relu = op.bwd_relu;
+        bfp = &bf;
+      }
       return conv_dgrad(h, dtype, h->conv_impl, cv, op.in.n, resolve(op.in, c), resolve(op.out, c), addend, h->dev_err,
-                        st);
+                        st, bfp);
     }
     case OP_CONV_WGRAD: {
       const ConvDef& cv = P.convs[op.conv];
@@ -1590,14 +1651,17 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
       BnArgs A = bn_args(b, eps);
       const int mask = op.mask.defined() ? 1 : 0;  // a ReLU followed this BN in the forward pass
       const T* addend = op.addend.defined() ? (const T*)resolve(op.addend, c) : nullptr;
-      const int grid_r = grid_for(vecs, threads * 8, cur_dev().sm_count, 2);   // one wave: two blocks stay resident per SM
-      LP_CUDA_OK(launch_pdl(bn_bwd_reduce_kernel<T>, dim3(grid_r), dim3(threads), (size_t)threads * 2 * V * 4, st,
-                            (const T*)resolve(op.in, c), (const T*)resolve(op.in2, c), mask, A, b.dgamma, b.dbeta, vecs, b.C));
+      if (!op.reduce_fused) {   // (otherwise the convolution that wrote dy has left the two sums in dgamma, dbeta)
+        const int grid_r = grid_for(vecs, threads * 8, cur_dev().sm_count, 2);   // one wave: two blocks stay resident per SM
+        LP_CUDA_OK(launch_pdl(bn_bwd_reduce_kernel<T>, dim3(grid_r), dim3(threads), (size_t)threads * 2 * V * 4, st,
+                              (const T*)resolve(op.in, c), (const T*)resolve(op.in2, c), mask, A, b.dgamma, b.dbeta, vecs, b.C));
+        h->launches++;
+      }
       const int grid_a = grid_for(vecs, threads * 4, cur_dev().sm_count, 2);
       LP_CUDA_OK(launch_pdl(bn_bwd_apply_kernel<T>, dim3(grid_a), dim3(threads), 0, st, (const T*)resolve(op.in, c),
                             (const T*)resolve(op.in2, c), mask, A, (const float*)b.dgamma, (const float*)b.dbeta, addend,
                             (T*)resolve(op.out, c), vecs, b.C));
-      h->launches += 2;
+      h->launches++;
       break;
     }
     case OP_MAXPOOL_FWD: {
@@ -1681,7 +1745,8 @@ static double op_bytes(const lp_handle* h, const Plan& P, const Op& op) {
     }
     case OP_CONV_DGRAD: {
       const ConvDef& c = P.convs[op.conv];
-      return sz(op.in) + sz(op.out) + sz(op.addend) + (double)c.cout * c.R * c.R * c.cin * e;
+      return sz(op.in) + sz(op.out) + sz(op.addend) + (op.bwd_bn >= 0 ? sz(op.bwd_x) : 0.0) +
+             (double)c.cout * c.R * c.R * c.cin * e;
     }
     case OP_CONV_WGRAD: {
       const ConvDef& c = P.convs[op.conv];
@@ -1691,8 +1756,8 @@ static double op_bytes(const lp_handle* h, const Plan& P, const Op& op) {
     case OP_BN_APPLY: return sz(op.in) + sz(op.in2) + sz(op.addend) + sz(op.out);
     case OP_OUT_LOSS:   // operands of the output, x_next, [kappa,] residual and terminal adjoint
       return op.fuse_loss ? 0.0 : sz(op.in) + sz(op.in2) + sz(op.addend) + 3.0 * sz(op.out);
-    case OP_BN_BWD:     // reduction pass (dy, x) and apply pass (dy, x, [addend] -> dx)
-      return 2.0 * (sz(op.in) + sz(op.in2)) + sz(op.addend) + sz(op.out);
+    case OP_BN_BWD:     // reduction pass (dy, x; not where a convolution took it) and apply pass (dy, x, [addend] -> dx)
+      return (op.reduce_fused ? 1.0 : 2.0) * (sz(op.in) + sz(op.in2)) + sz(op.addend) + sz(op.out);
     case OP_MAXPOOL_FWD: return sz(op.in) + sz(op.out) + (double)op.out.elems();
     case OP_MAXPOOL_BWD: return sz(op.in) + sz(op.out) + (double)op.in.elems();
     case OP_HEAD_FWD: return sz(op.in);

@@ -158,12 +158,41 @@ def test_small_fp32_block_kinds(kind, stem):
     full_step_parity(cfg, steps=1)
 
 
-@pytest.mark.parametrize("impl", [1, 0, 256, 512])     # CUDA cores; tensor cores; direct / staged epilogue everywhere
+# CUDA cores; tensor cores; direct / staged epilogue everywhere; batch-norm backward sums in the conv epilogue
+@pytest.mark.parametrize("impl", [1, 0, 256, 512, 2048])
 @pytest.mark.parametrize("kind", ["postbn", "preact"])
 def test_small_bf16_block_kinds(kind, impl):
     cfg = small_cfg(kind, N=8, H=16, W=16, dtype="bf16", stage_channels=(16, 32), stage_blocks=(2, 2),
                     module_block_end=(1, 3, 4), stem_channels=16, classes=10)
     full_step_parity(cfg, conv_impl=impl, steps=2)
+
+
+@pytest.mark.parametrize("kind", ["postbn", "preact", "bottleneck"])
+def test_bn_backward_sums_in_the_conv_epilogue_equal_the_separate_kernel(kind):
+    """The reduction pass of a batch-norm backward taken by the epilogue of the input-gradient convolution
+    (LP_CONV_BN_REDUCE_IN_EPILOGUE) against the same pass as its own kernel (default): the same bf16 values are
+    summed, only the order of the fp32 additions differs, so the gradients agree far inside the parity
+    tolerance; the launch count shows that the kernels are really gone."""
+    import paper_2112_05387_b200 as lp
+    cfg = small_cfg(kind, N=8, H=16, W=16, dtype="bf16", stage_channels=(16, 32) if kind != "bottleneck" else (64, 128),
+                    stage_blocks=(2, 2), module_block_end=(1, 3, 4), stem_channels=16, classes=10)
+    out = {}
+    for impl in (lp.LP_CONV_BN_REDUCE_IN_EPILOGUE, 0):
+        run = GpuRun(cfg, conv_impl=impl)
+        run.auxnet()
+        run.lp.lp_launch_count(run.h, reset=True)
+        grads = run.fwd_bwd_all()
+        out[impl] = (grads, [to_host(t) for t in run.d_dx[1:]], run.d_loss.cpu().numpy().copy(),
+                     run.lp.lp_last_device_status(run.h), run.lp.lp_launch_count(run.h))
+        run.lp.lp_destroy(run.h)
+    (g0, dx0, l0, s0, n0), (g1, dx1, l1, s1, n1) = out[lp.LP_CONV_BN_REDUCE_IN_EPILOGUE], out[0]
+    assert s0 == 0 and s1 == 0
+    assert n0 <= n1 - 4, (n0, n1)                         # at least one reduction kernel per block is gone
+    np.testing.assert_array_equal(l0, l1)                 # the forward pass is untouched
+    for k in range(len(g0)):
+        assert rel_err(g0[k], g1[k]) < 2e-3, k
+    for a, b in zip(dx0, dx1):
+        assert rel_err(a, b) < 2e-3
 
 
 def flat_module_parity(cfg, conv_impl, tol_grad):
