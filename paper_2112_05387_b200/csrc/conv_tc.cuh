@@ -72,6 +72,7 @@ struct ConvTcParams {
   uint32_t item_bytes;           // one item: mpair activation tiles + the weight tile
   int mpair;                     // pixel tiles per unit: 1 or 2
   int nslots, acc_stride;        // accumulator ring: slots and their TMEM column stride
+  int tmem_cols;                 // tensor-memory columns the CTA allocates: a power of two >= nslots * acc_stride
   uint32_t stage_bytes, a_region_bytes, b_offset, tx_a, tx_b;
   uint32_t idesc;
   uint64_t desc_hi;
@@ -170,8 +171,12 @@ constexpr int kEpiGroups = LP_EPI_WARPS / 4;
 //   sums over the staged tile.  tmOut / tmAdd are only read by these instantiations.
 // kBnBwd: the direct epilogue also takes the reduction pass of the batch-norm backward that consumes
 //   this convolution's output (see ConvTcParams::bwd_x).
-template <bool kLoss, bool kAddend, bool kStaged, bool kBnBwd = false>
-__global__ void __launch_bounds__(kConvThreads, LP_CONV_MIN_BLOCKS)
+// kMinBlocks: CTAs of this kernel that must fit on one SM.  Layers of few channels (a channel tile of at most
+//   64 columns) are launched as the two-per-SM instantiation -- registers capped accordingly (the epilogue
+//   drains 64 accumulator columns per pass instead of 160), tensor memory and shared memory sized to need --
+//   so that the kernels of several modules, each bound by latency rather than by any unit, share the SMs.
+template <bool kLoss, bool kAddend, bool kStaged, bool kBnBwd = false, int kMinBlocks = LP_CONV_MIN_BLOCKS>
+__global__ void __launch_bounds__(kConvThreads, kMinBlocks)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmAdd,
                const __grid_constant__ ConvTcParams p) {
@@ -217,7 +222,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   }
   if (warp == kFirstEpiWarp) {
-    tmem_alloc(&tail->tmem_base, kTmemCols);
+    tmem_alloc(&tail->tmem_base, (uint32_t)p.tmem_cols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -670,7 +675,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t taddr = tmem_base + buf * p.acc_stride + ((uint32_t)(q * 32) << 16);
         // Drain the accumulator into registers first (up to kBatch x 32 columns per pass) and hand
         // the TMEM slot back to the MMA warp; stores and statistics then work from registers.
-        constexpr int kBatch = LP_EPI_BATCH;
+        constexpr int kBatch = kMinBlocks > 1 ? 2 : LP_EPI_BATCH;
         // Residual operand of one 32-channel group, as raw 16-byte pieces (zero where nothing is added).
         // A group's pieces are requested while the group before it is processed.
         auto load_addend = [&](int g, uint4 (&a)[4]) {
@@ -907,7 +912,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   if (warp == kFirstEpiWarp) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
   }
 }
 

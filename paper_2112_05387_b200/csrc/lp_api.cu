@@ -366,6 +366,11 @@ static int encode_tile32_map(CUtensorMap* m, const void* base, int N, int H, int
 
 static const size_t kTcMinSmem = 120 * 1024;   // more than half an SM: one CTA (and one TMEM owner) per SM
 static const size_t kTcMaxSmem = 220 * 1024;
+// A convolution of fewer FLOPs than this (and at most 64 channels) cannot fill the machine whatever its launch
+// shape: a few microseconds of fixed cost dominate.  While several modules are enqueued side by side such
+// launches are sized to share the SMs with the other modules' kernels instead of taking them whole.
+static const double kSmallConvFlops = 4e9;
+static const size_t kTcThinSmem = 100 * 1024;  // two CTAs of the few-channel instantiation (or other kernels) per SM
 
 // Halo mode (one activation box per K chunk serves all nine taps, see conv_tc.cuh): a 3x3 stride-1
 // tap set, 64-channel K chunks and an output width that is a multiple of 8.
@@ -544,7 +549,7 @@ static int launch_conv_tc2(lp_handle* h, const TcGemmSpec& s, int* dev_err, cuda
   return LP_OK;
 }
 
-static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaStream_t st) {
+static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaStream_t st, bool allow_thin = true) {
   const bool bnbwd = s.bwd_x != nullptr;
   if (bnbwd && (s.stats || s.x_next)) return LP_ERR_UNSUPPORTED;
   if (s.two_cta && !bnbwd) {
@@ -578,17 +583,29 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   const uint32_t b_region = (uint32_t)align_up((size_t)p.n_tile_cols * row_bytes, 1024);
   // Staged epilogue (output tile through shared memory, TMA stores, TMA-loaded residual): where the output
   // grid is the logical grid, the channel tile is a multiple of 32 and the tensors start on 16-byte boundaries.
-  const bool staged = !bnbwd && (s.epilogue == 2 || (s.epilogue == 0 && s.addend != nullptr)) && !s.x_next && s.os == 1 && s.oo_h == 0 && s.oo_w == 0 &&
+  const bool staged0 = !bnbwd && (s.epilogue == 2 || (s.epilogue == 0 && s.addend != nullptr)) && !s.x_next && s.os == 1 && s.oo_h == 0 && s.oo_w == 0 &&
                       p.n_tile_cols % 32 == 0 && s.out_C % 8 == 0 && tc::kEpiThreads == 128 &&
                       (reinterpret_cast<uintptr_t>(s.out) & 15) == 0 &&
                       (!s.addend || (reinterpret_cast<uintptr_t>(s.addend) & 15) == 0);
+  // Layers of few channels, while the modules are enqueued side by side: the two-per-SM instantiation with
+  // half an SM's shared memory at most and tensor memory sized to need, so that kernels of several modules share
+  // the SMs (each such kernel is bound by latency: a few hundred MFLOP and a few MB per launch).
+  const bool thin = allow_thin && h && h->concurrent && !bnbwd && !s.x_next && p.n_tile_cols <= 64 &&
+                    2.0 * s.aN * s.OHl * s.OWl * (double)s.w_rows * s.ntaps * s.aC < kSmallConvFlops;
+  const bool staged = staged0 && !thin;
+  const size_t max_smem = thin ? kTcThinSmem : kTcMaxSmem;
   const size_t stage_bytes = staged ? (size_t)(p.n_tile_cols / 32) * tc::kStageGroupBytes : 0;
   // the direct epilogue's statistics scratch is only there when statistics are asked for
   const size_t tail = tc::kTailBytes + ((staged || !(s.stats || bnbwd)) ? 0 : sizeof(tc::TcStatScratch)) +
                       (bnbwd ? sizeof(tc::TcBnBwdScratch) : 0) + stage_bytes + 1024;
   p.tx_b = (uint32_t)(p.n_tile_cols * row_bytes);
   p.acc_stride = (p.n_tile_cols + 31) / 32 * 32;
-  p.nslots = std::min(tc::kMaxSlots, tc::kTmemCols / p.acc_stride);
+  p.nslots = std::min(tc::kMaxSlots, (thin ? 256 : tc::kTmemCols) / p.acc_stride);
+  p.tmem_cols = tc::kTmemCols;
+  if (thin) {
+    p.tmem_cols = 32;
+    while (p.tmem_cols < p.nslots * p.acc_stride) p.tmem_cols *= 2;
+  }
   if (p.halo) {
     // activation ring: three boxes deep if at least three weight stages still fit, else two
     const int halo_rows = kHaloBoxW * p.BNI * (p.BH + 2);
@@ -602,7 +619,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     p.desc_hi_a = tc::smem_desc_hi(16, kHaloBoxW * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
     p.b_tile_bytes = b_region;
     p.tx_a = (uint32_t)(halo_rows * row_bytes);
-    const size_t avail = kTcMaxSmem - tail;
+    const size_t avail = max_smem - tail;
     // two activation stages (each lasts all nine taps), the rest of shared memory for weights: stages of
     // LP_CONV_TAPS_PER_STAGE taps where three of them fit, else of fewer taps
     bool fits = false;
@@ -635,7 +652,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     // two pixel tiles per weight tile wherever a CTA has at least two tiles and three stages still fit
     p.mpair = 1;
     if (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, cur_dev().sm_count) &&
-        (kTcMaxSmem - tail) / (2 * p.a_region_bytes + b_region) >= 3)
+        (max_smem - tail) / (2 * p.a_region_bytes + b_region) >= 3)
       p.mpair = 2;
     p.b_offset = p.mpair * p.a_region_bytes;
     p.item_bytes = p.b_offset + b_region;
@@ -645,15 +662,15 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     // fixed cost of a stage once per several taps; wide layers keep one item per stage.
     {
       const int kiters = p.ntaps * p.chunks;
-      int ips = (int)std::min<size_t>((size_t)std::min(kiters, LP_CONV_MAX_ITEMS_PER_STAGE), (kTcMaxSmem - tail) / 3 / p.item_bytes);
+      int ips = (int)std::min<size_t>((size_t)std::min(kiters, LP_CONV_MAX_ITEMS_PER_STAGE), (max_smem - tail) / 3 / p.item_bytes);
       ips = std::max(ips, 1);
       const int n_st = (kiters + ips - 1) / ips;
       p.ips = (kiters + n_st - 1) / n_st;
     }
     p.stage_bytes = p.ips * p.item_bytes;
-    int stages = (int)((kTcMaxSmem - tail) / p.stage_bytes);
+    int stages = (int)((max_smem - tail) / p.stage_bytes);
     stages = std::min(stages, tc::kMaxStages);
-    if (stages < 2) return LP_ERR_UNSUPPORTED;
+    if (stages < 2) return thin ? launch_conv_tc(h, s, dev_err, st, false) : LP_ERR_UNSUPPORTED;
     p.stages = stages;
     p.stage_offset = (uint32_t)(stages * p.stage_bytes);
     p.tail_offset = p.stage_offset + (uint32_t)stage_bytes;
@@ -687,7 +704,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     }
   }
   size_t smem = (size_t)p.tail_offset + (tail - stage_bytes);
-  smem = std::max(smem, kTcMinSmem);
+  if (!thin) smem = std::max(smem, kTcMinSmem);
   bool& attr_set = cur_dev().conv_attr;
   if (!attr_set) {
     LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -700,6 +717,10 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
                                     (int)kTcMaxSmem));
     LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kTcMaxSmem));
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, false, false, false, 2>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcThinSmem));
+    LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, true, false, false, 2>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcThinSmem));
     LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, false, false, true>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcMaxSmem));
     LP_CUDA_OK(cudaFuncSetAttribute(tc::conv_tc_kernel<false, true, false, true>,
@@ -721,7 +742,9 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   if (s.x_next && !s.addend) return LP_ERR_UNSUPPORTED;   // the fused loss belongs to a convolution with a shortcut
   cudaError_t le;
   const dim3 g3(grid), b3(tc::kConvThreads);
-  if (bnbwd && s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true, false, true>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
+  if (thin && s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true, false, false, 2>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
+  else if (thin) le = launch_pdl(tc::conv_tc_kernel<false, false, false, false, 2>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
+  else if (bnbwd && s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true, false, true>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
   else if (bnbwd) le = launch_pdl(tc::conv_tc_kernel<false, false, false, true>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
   else if (s.x_next) le = launch_pdl(tc::conv_tc_kernel<true, true, false>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
   else if (staged && s.addend) le = launch_pdl(tc::conv_tc_kernel<false, true, true>, g3, b3, smem, st, tmA, tmB, tmOut, tmAdd, p);
@@ -983,8 +1006,11 @@ static int conv_wgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
   if (use_tc) {
     ProfScope ps(h, st, 2.0 * N * c.OH * c.OW * (double)c.cout * c.R * c.R * c.cin);
     Device& D = cur_dev();
+    // small layers of modules that run side by side share the SMs (see kSmallConvFlops)
+    const bool shared_sm = h && h->concurrent && c.cin <= 64 && c.cout <= 64 &&
+                           2.0 * N * c.OH * c.OW * (double)c.cout * c.R * c.R * c.cin < kSmallConvFlops;
     int rc = launch_wgrad_tc(D.encode, D.sm_count, &D.wgrad_attr, &D.wgrad_halo_attr, (const bf16*)x, (const bf16*)dy, dw, N,
-                             c.H, c.W, c.cin, c.OH, c.OW, c.cout, c.R, c.stride, c.pad, dev_err, st);
+                             c.H, c.W, c.cin, c.OH, c.OW, c.cout, c.R, c.stride, c.pad, dev_err, st, shared_sm);
     if (h) h->launches++;
     return rc;
   }

@@ -528,8 +528,12 @@ static int wg_encode_wnh(WgEncodeFn enc, CUtensorMap* m, const void* base, int N
 }
 
 // Returns 1 when the shape is not one the halo kernel takes (the caller then uses wgrad_tc_kernel).
+// shared_sm: the launch is sized to share an SM with other kernels (tensor memory to need, at most
+// kWgSharedSmem of shared memory) instead of taking the SM for itself; for small layers that several
+// modules run at the same time.
+static const size_t kWgSharedSmem = 100 * 1024;
 static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, bool* attr_done, const bf16* x, const bf16* dy, float* dw, int N, int H, int W,
-                             int Cin, int Cout, int* dev_err, cudaStream_t st) {
+                             int Cin, int Cout, int* dev_err, cudaStream_t st, bool shared_sm) {
   if (W % 8 || Cin < 64) return 1;
   tc::WgradParams p;
   memset(&p, 0, sizeof(p));
@@ -564,6 +568,11 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, bool* attr_done, cons
   p.acc_stride = (p.n_tile + 31) / 32 * 32;
   if (3 * p.acc_stride > 512) return 1;
   p.tmem_cols = 512;
+  if (shared_sm) {
+    p.tmem_cols = 32;
+    while ((int)p.tmem_cols < 3 * p.acc_stride) p.tmem_cols *= 2;
+  }
+  const size_t max_smem = shared_sm ? kWgSharedSmem : (size_t)220 * 1024;
   p.cin_chunks = (Cin + 63) / 64;
   p.groups = 3 * p.cin_chunks;
   p.m_tiles = (p.groups + 1) / 2;
@@ -575,7 +584,7 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, bool* attr_done, cons
   p.tx_a = p.a_box_bytes;
   p.tx_b = (uint32_t)(p.rows * p.nb * p.scb * 2);
   const size_t tail = sizeof(tc::WgSmemTail) + 1024;
-  int stages = (int)((220 * 1024 - tail) / p.stage_bytes);
+  int stages = (int)((max_smem - tail) / p.stage_bytes);
   stages = std::min(stages, tc::kWgMaxStages);
   if (stages < 2) return 1;
   p.stages = stages;
@@ -621,7 +630,8 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, bool* attr_done, cons
             CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
       p.epi_bufs = fit & ~1;
   }
-  size_t smem = std::max((size_t)stages * p.stage_bytes + tail, (size_t)120 * 1024);
+  size_t smem = (size_t)stages * p.stage_bytes + tail;
+  if (!shared_sm) smem = std::max(smem, (size_t)120 * 1024);   // one CTA, and one owner of all tensor memory, per SM
   if (!*attr_done) {   // per device
     if (cudaFuncSetAttribute(tc::wgrad_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
       return -8;
@@ -633,11 +643,12 @@ static int launch_wgrad_halo(WgEncodeFn enc, int sm_count, bool* attr_done, cons
 
 static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, bool* attr_done, bool* halo_attr_done, const bf16* x,
                            const bf16* dy, float* dw, int N, int H, int W, int Cin, int OH, int OW, int Cout, int R,
-                           int stride, int pad, int* dev_err, cudaStream_t st) {
+                           int stride, int pad, int* dev_err, cudaStream_t st, bool shared_sm = false) {
   if (R == 3 && stride == 1 && pad == 1) {
-    const int rc = launch_wgrad_halo(enc, sm_count, halo_attr_done, x, dy, dw, N, H, W, Cin, Cout, dev_err, st);
+    const int rc = launch_wgrad_halo(enc, sm_count, halo_attr_done, x, dy, dw, N, H, W, Cin, Cout, dev_err, st, shared_sm);
     if (rc != 1) return rc;
   }
+  const size_t max_smem = shared_sm ? kWgSharedSmem : (size_t)220 * 1024;
   tc::WgradParams p;
   memset(&p, 0, sizeof(p));
   p.Nimg = N; p.OH = OH; p.OW = OW;
@@ -666,12 +677,12 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, bool* attr_done, bool* 
   p.n_tiles = (Cout + p.n_tile - 1) / p.n_tile;
   // two row tiles per CTA pay off with 64-channel sub-boxes (few, large copies per stage); with
   // narrower sub-boxes the two pipeline stages that still fit do not hide the copy latency
-  p.mpair = (p.m_tiles >= 2 && p.sca == 64) ? 2 : 1;
+  p.mpair = (p.m_tiles >= 2 && p.sca == 64 && !shared_sm) ? 2 : 1;
   p.pair_tiles = (p.m_tiles + p.mpair - 1) / p.mpair;
   const size_t tail = sizeof(tc::WgSmemTail) + 1024;
   // pixel box (K block): 128 output pixels, or 64 where three stages of 128 would not fit
   int target_rows = 128;
-  if ((220 * 1024 - tail) / ((size_t)128 * 2 * (p.mpair * 128 + p.n_tile)) < 2) target_rows = 64;
+  if ((max_smem - tail) / ((size_t)128 * 2 * (p.mpair * 128 + p.n_tile)) < 2) target_rows = 64;
   p.BW = std::min(OW, target_rows);
   int bh = std::min(std::max(1, target_rows / p.BW), OH);
   const int th = (OH + bh - 1) / bh;
@@ -706,9 +717,11 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, bool* attr_done, bool* 
   p.stage_bytes = p.a_region + p.b_sub_bytes * p.nb;
   p.tx_a = (uint32_t)(p.rows * p.rpt * p.sca * 2);
   p.tx_b = (uint32_t)(p.rows * p.nb * p.scb * 2);
-  int stages = (int)((220 * 1024 - tail) / p.stage_bytes);
+  int stages = (int)((max_smem - tail) / p.stage_bytes);
   stages = std::min(stages, tc::kWgMaxStages);
-  if (stages < 2) return -10;
+  if (stages < 2) return shared_sm ? launch_wgrad_tc(enc, sm_count, attr_done, halo_attr_done, x, dy, dw, N, H, W, Cin, OH, OW, Cout,
+                                                     R, stride, pad, dev_err, st, false)
+                                   : -10;
   p.stages = stages;
   p.idesc = tc::instr_desc_bf16(128, p.n_tile, 1, 1);
   p.adesc_hi = tc::smem_desc_hi(p.a_sub_bytes, 8 * p.sca * 2, tc::swizzle_code_for_row_bytes(p.sca * 2));
@@ -737,7 +750,8 @@ static int launch_wgrad_tc(WgEncodeFn enc, int sm_count, bool* attr_done, bool* 
             CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
       p.epi_bufs = p.rpt;
   }
-  size_t smem = std::max((size_t)stages * p.stage_bytes + tail, (size_t)120 * 1024);
+  size_t smem = (size_t)stages * p.stage_bytes + tail;
+  if (!shared_sm) smem = std::max(smem, (size_t)120 * 1024);   // one CTA, and one owner of all tensor memory, per SM
   if (!*attr_done) {   // per device
     if (cudaFuncSetAttribute(tc::wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
       return -8;
