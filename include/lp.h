@@ -88,6 +88,10 @@ enum { LP_CONV_TWO_CTA = 1024 };
  * additions.  Not the default: the epilogue's extra shared-memory traffic costs the convolution more than the
  * separate kernel takes. */
 enum { LP_CONV_BN_REDUCE_IN_EPILOGUE = 2048 };
+/* May be OR-ed into conv_impl: the weight gradients of a module stay in its stream, in the order of the
+ * backward pass.  By default each module has a second stream for them (they feed nothing but the update), so
+ * that the chain of input gradients and batch-norm backward passes does not wait for them. */
+enum { LP_CONV_WGRAD_IN_CHAIN = 4096 };
 enum { LP_CONV_FWD = 0, LP_CONV_DGRAD = 1, LP_CONV_WGRAD = 2 };
 
 #define LP_MAX_STAGES 8

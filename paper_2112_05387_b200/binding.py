@@ -5,7 +5,7 @@ import os
 import numpy as np
 
 __all__ = [
-    "LP_OK", "LP_F32", "LP_BF16", "LP_AUX", "LP_REAUX", "LP_CONV_IMPL_AUTO", "LP_CONV_IMPL_SIMT", "LP_CONV_IMPL_TENSOR", "LP_CONV_LOSS_IN_EPILOGUE", "LP_CONV_DIRECT_EPILOGUE", "LP_CONV_STAGED_EPILOGUE", "LP_CONV_TWO_CTA", "LP_CONV_BN_REDUCE_IN_EPILOGUE",
+    "LP_OK", "LP_F32", "LP_BF16", "LP_AUX", "LP_REAUX", "LP_CONV_IMPL_AUTO", "LP_CONV_IMPL_SIMT", "LP_CONV_IMPL_TENSOR", "LP_CONV_LOSS_IN_EPILOGUE", "LP_CONV_DIRECT_EPILOGUE", "LP_CONV_STAGED_EPILOGUE", "LP_CONV_TWO_CTA", "LP_CONV_BN_REDUCE_IN_EPILOGUE", "LP_CONV_WGRAD_IN_CHAIN",
     "LP_CONV_FWD", "LP_CONV_DGRAD", "LP_CONV_WGRAD", "LpError", "lp_net_desc", "lp_param_entry", "library",
     "library_path", "desc_from_config", "lp_status_string", "lp_validate_desc", "lp_workspace_bytes",
     "lp_param_layout", "lp_boundary_shape_desc", "lp_create", "lp_destroy", "lp_param_count", "lp_set_params",
@@ -23,6 +23,7 @@ LP_CONV_LOSS_IN_EPILOGUE = 128
 LP_CONV_DIRECT_EPILOGUE, LP_CONV_STAGED_EPILOGUE = 256, 512
 LP_CONV_TWO_CTA = 1024
 LP_CONV_BN_REDUCE_IN_EPILOGUE = 2048
+LP_CONV_WGRAD_IN_CHAIN = 4096
 LP_CONV_FWD, LP_CONV_DGRAD, LP_CONV_WGRAD = 0, 1, 2
 LP_MAX_STAGES, LP_MAX_MODULES = 8, 16
 LP_NOALLOC_SCRATCH_BYTES = 8 << 20

@@ -116,6 +116,12 @@ struct Plan {  // one module or one AuxNet
   void* dx_fallback = nullptr;
   bool interior = false;
   bool ran_fwd_bwd = false;
+  // Weight gradients feed nothing but the update, so in the backward pass they leave the chain
+  // dy -> BN' -> dx -> ... : each is enqueued on this second stream right after the kernel that wrote its dy
+  // (one event per weight gradient), and the pass joins the stream back at its end.
+  cudaStream_t side = nullptr;
+  std::vector<cudaEvent_t> side_ev;
+  cudaEvent_t side_done = nullptr;
 };
 
 struct Arena {
@@ -1793,12 +1799,28 @@ static double op_bytes(const lp_handle* h, const Plan& P, const Op& op) {
 }
 
 static int run_ops(lp_handle* h, Plan& P, const std::vector<Op>& ops, const RunCtx& c) {
+  // (per-operation timing wants one stream: the time line and the convolution profile keep everything in order)
+  const bool use_side = P.side && !h->tl.enabled && !h->prof.enabled;
+  size_t nside = 0;
+  int rc = LP_OK;
   for (const Op& op : ops) {
-    TimelineScope ts(h, c.st, c.plan_id, (int)op.type, c.phase, h->tl.enabled ? op_bytes(h, P, op) : 0.0);
-    int rc = h->dtype == LP_F32 ? run_op_t<float>(h, P, op, c) : run_op_t<bf16>(h, P, op, c);
-    if (rc != LP_OK) return rc;
+    if (use_side && op.type == OP_CONV_WGRAD && nside < P.side_ev.size()) {
+      if (cudaEventRecord(P.side_ev[nside], c.st) != cudaSuccess ||
+          cudaStreamWaitEvent(P.side, P.side_ev[nside], 0) != cudaSuccess) { rc = LP_ERR_CUDA; break; }
+      ++nside;
+      RunCtx c2 = c;
+      c2.st = P.side;
+      rc = h->dtype == LP_F32 ? run_op_t<float>(h, P, op, c2) : run_op_t<bf16>(h, P, op, c2);
+    } else {
+      TimelineScope ts(h, c.st, c.plan_id, (int)op.type, c.phase, h->tl.enabled ? op_bytes(h, P, op) : 0.0);
+      rc = h->dtype == LP_F32 ? run_op_t<float>(h, P, op, c) : run_op_t<bf16>(h, P, op, c);
+    }
+    if (rc != LP_OK) break;
   }
-  return LP_OK;
+  // joined whatever happened: a stream left unjoined would invalidate a capture in progress
+  if (nside && (cudaEventRecord(P.side_done, P.side) != cudaSuccess || cudaStreamWaitEvent(c.st, P.side_done, 0) != cudaSuccess))
+    if (rc == LP_OK) rc = LP_ERR_CUDA;
+  return rc;
 }
 
 static int zero_forward_state(Plan& P, cudaStream_t st) {
@@ -2008,6 +2030,18 @@ int lp_create(const lp_net_desc* desc, void* dev_workspace, size_t bytes, lp_han
       return LP_ERR_CUDA;
     }
   }
+  if (!(net.d.conv_impl & LP_CONV_WGRAD_IN_CHAIN)) {
+    for (auto& P : h->modules) {
+      size_t n_wgrad = 0;
+      for (const Op& op : P.bwd) n_wgrad += op.type == OP_CONV_WGRAD ? 1 : 0;
+      if (!n_wgrad) continue;
+      if (cudaStreamCreateWithFlags(&P.side, cudaStreamNonBlocking) != cudaSuccess ||
+          cudaEventCreateWithFlags(&P.side_done, cudaEventDisableTiming) != cudaSuccess) { delete h; return LP_ERR_CUDA; }
+      P.side_ev.assign(n_wgrad, nullptr);
+      for (auto& e : P.side_ev)
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { delete h; return LP_ERR_CUDA; }
+    }
+  }
   if (cudaEventCreateWithFlags(&h->fork, cudaEventDisableTiming) != cudaSuccess) { delete h; return LP_ERR_CUDA; }
   if (cudaStreamCreateWithFlags(&h->aux_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&h->aux_end, cudaEventDisableTiming) != cudaSuccess) { delete h; return LP_ERR_CUDA; }
@@ -2030,6 +2064,11 @@ int lp_destroy(lp_handle* h) {
   for (auto& pr : h->prof.events) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
   for (auto& r : h->tl.recs) { if (r.a) cudaEventDestroy(r.a); if (r.b) cudaEventDestroy(r.b); }
   for (auto g : h->graphs) cudaGraphExecDestroy(g);
+  for (auto& P : h->modules) {
+    if (P.side) cudaStreamDestroy(P.side);
+    if (P.side_done) cudaEventDestroy(P.side_done);
+    for (auto e : P.side_ev) if (e) cudaEventDestroy(e);
+  }
   delete h;
   return LP_OK;
 }

@@ -52,7 +52,7 @@ struct NetDef {
     if (d.aux_convs_per_boundary < 1 || d.aux_convs_per_boundary > 2 || d.aux_width_div < 1) return LP_ERR_BAD_DESC;
     if (!(d.bn_eps > 0.f)) return LP_ERR_BAD_DESC;
     if (d.aux_recursive != 0 && d.aux_recursive != 1) return LP_ERR_BAD_DESC;
-    if (d.conv_impl < 0 || (d.conv_impl & 15) > LP_CONV_IMPL_TENSOR || d.conv_impl > 4095) return LP_ERR_BAD_DESC;
+    if (d.conv_impl < 0 || (d.conv_impl & 15) > LP_CONV_IMPL_TENSOR || d.conv_impl > 8191) return LP_ERR_BAD_DESC;
     const int vec = d.dtype == LP_F32 ? 4 : 8;
     if (d.stem_channels < vec || d.stem_channels % vec) return LP_ERR_BAD_DESC;
     if (d.stem_kind == LP_STEM_CONV7X7S2_MAXPOOL && d.block_kind == LP_PREACT) return LP_ERR_UNSUPPORTED;
