@@ -13,7 +13,9 @@
 // tensor memory (3 for N_TILE = 160), so the epilogue of one unit overlaps the MMAs of the next
 // as far as slots are free.
 //
-// Tap reuse ("halo" mode, 3x3 stride-1 convolutions with 64-channel K chunks): all nine taps of
+// Tap reuse ("halo" mode, 3x3 stride-1 convolutions; described for 64-channel K chunks, i.e. rows of
+// 128 bytes -- chunks of 32 and 16 channels work the same way with 64- and 32-byte rows and their
+// swizzles): all nine taps of
 // a K chunk read the same activations, shifted by whole pixels.  The tile is 8 pixels wide and its
 // rows are ordered (w, image, h); ONE box with a one-pixel halo all round, (8+2) x BNI x (BH+2)
 // rows of 128 bytes, is fetched per K chunk and tile.  An 8-row group of the A operand (one image
@@ -24,7 +26,8 @@
 // swizzle is a function of the shared-memory address bits (16-byte chunk index ^= address bits
 // 7..9), for the TMA write and for the MMA read alike, so any row of the box can be the first row
 // of an operand (checked against the CPU oracle by the parity tests).  Activations and weights
-// travel in separate rings: an activation stage per K chunk (nine taps), a weight stage per tap.
+// travel in separate rings: an activation stage per K chunk (nine taps), a weight stage per group of
+// taps (as many taps as leave three stages: all nine for 16 or 32 channels, two for 160).
 // This cuts the bytes fetched per MMA from 52 KB to 25 KB per eight instructions.
 //
 // Roles: warp 0 = TMA producer; warps 1 and 2 = MMA issuers, one per accumulator of a pair (a

@@ -387,7 +387,7 @@ static const size_t kTcThinSmem = 100 * 1024;  // two CTAs of the few-channel in
 #define LP_CONV_MAX_ITEMS_PER_STAGE 16   // (tap, chunk) items per pipeline stage of the plain mode, at most
 #endif
 #ifndef LP_CONV_TAPS_PER_STAGE
-#define LP_CONV_TAPS_PER_STAGE 2   // taps per weight stage (halo mode), as far as three stages still fit
+#define LP_CONV_TAPS_PER_STAGE 9   // taps per weight stage (halo mode), at most: as many as leave three stages
 #endif
 static const int kHaloBoxW = 10;   // 8-pixel tile width plus one halo pixel on each side
 
@@ -566,7 +566,9 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   memset(&p, 0, sizeof(p));
   p.Nimg = s.aN; p.OHl = s.OHl; p.OWl = s.OWl;
   int tapw3[3][3];
-  p.halo = (pick_kc(s.aC) == 64 && pick_halo_box(s, p.BW, p.BH, p.BNI, tapw3)) ? 1 : 0;
+  // (any K chunk width: the row-shifted operand descriptors only need the swizzle to be a function of the
+  // shared-memory address, which holds for 32-, 64- and 128-byte rows alike)
+  p.halo = pick_halo_box(s, p.BW, p.BH, p.BNI, tapw3) ? 1 : 0;
   if (!p.halo) pick_pixel_box(s.OWl, s.OHl, s.aN, p.BW, p.BH, p.BNI);
   p.tiles_w = (s.OWl + p.BW - 1) / p.BW;
   p.tiles_h = (s.OHl + p.BH - 1) / p.BH;
@@ -627,7 +629,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     p.tx_a = (uint32_t)(halo_rows * row_bytes);
     const size_t avail = max_smem - tail;
     // two activation stages (each lasts all nine taps), the rest of shared memory for weights: stages of
-    // LP_CONV_TAPS_PER_STAGE taps where three of them fit, else of fewer taps
+    // as many taps as leave three of them (all nine for layers of 16 or 32 channels, two at 160)
     bool fits = false;
     p.nA = 2;
     for (int pair = (p.m_tiles >= 2 && 2 * p.total_tiles >= 3 * std::min(p.total_tiles, cur_dev().sm_count)) ? 2 : 1;
