@@ -195,6 +195,27 @@ def test_bn_backward_sums_in_the_conv_epilogue_equal_the_separate_kernel(kind):
         assert rel_err(a, b) < 2e-3
 
 
+def test_weight_gradients_on_their_own_stream_equal_those_in_the_chain():
+    """A module's weight gradients run on a second stream by default and inside the module's stream with
+    LP_CONV_WGRAD_IN_CHAIN: the same kernels on the same operands, so losses are identical and gradients agree
+    to the order of the fp32 reductions; run twice to show that nothing races between the two streams."""
+    import paper_2112_05387_b200 as lp
+    cfg = small_cfg("postbn", N=8, H=16, W=16, dtype="bf16", stage_channels=(16, 32), stage_blocks=(2, 2),
+                    module_block_end=(1, 3, 4), stem_channels=16, classes=10)
+    out = []
+    for impl in (0, 0, lp.LP_CONV_WGRAD_IN_CHAIN):
+        run = GpuRun(cfg, conv_impl=impl)
+        run.auxnet()
+        grads = run.fwd_bwd_all()
+        out.append((grads, run.d_loss.cpu().numpy().copy(), run.lp.lp_last_device_status(run.h)))
+        run.lp.lp_destroy(run.h)
+    for g, l, st in out:
+        assert st == 0
+        np.testing.assert_array_equal(l, out[0][1])
+        for k in range(len(g)):
+            assert rel_err(g[k], out[0][0][k]) < 1e-5, k
+
+
 def flat_module_parity(cfg, conv_impl, tol_grad):
     """Module passes of a bf16 network against the storage-model oracle with ONE tolerance for every
     gradient tensor and dx, no noise floor: for networks shallow enough that rounding-level differences
