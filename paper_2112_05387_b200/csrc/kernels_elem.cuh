@@ -42,6 +42,52 @@ __device__ __forceinline__ void bn_load_consts(const BnArgs& a, int C, int c0, f
   for (int j = 0; j < V; ++j) bn_mean_rstd(s1[j], s2[j], a.inv_count, a.eps, mean[j], rstd[j]);
 }
 
+// Block-level tail of the per-channel reductions.  Every thread holds V sums of each of two kinds (a, b) for its
+// fixed channel group (threadIdx.x % CV).  block_channel_partials() leaves partial sums in shared memory and
+// returns how many there are per channel; block_channel_sum() adds them up for one (kind, channel) column.
+// Where the channel groups line up with the lanes of a warp (CV divides 32), lanes of the same group are first
+// added by shuffles, which leaves blockDim/32 partial sums per channel instead of blockDim/CV (8 instead of 120
+// at 16 channels: that serial loop took longer than the pass over a small tensor).
+template <int V>
+__device__ __forceinline__ int block_channel_partials(float (&a)[V], float (&b)[V], float* sm, int C) {
+  const int CV = C / V;
+  if (CV <= 32 && (32 % CV) == 0 && (blockDim.x & 31) == 0) {
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      for (int o = CV; o < 32; o <<= 1) {
+        a[j] += __shfl_xor_sync(0xffffffffu, a[j], o);
+        b[j] += __shfl_xor_sync(0xffffffffu, b[j], o);
+      }
+    }
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane < CV) {
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        sm[(w * CV + lane) * 2 * V + j] = a[j];
+        sm[(w * CV + lane) * 2 * V + V + j] = b[j];
+      }
+    }
+    __syncthreads();
+    return (int)(blockDim.x >> 5);
+  }
+#pragma unroll
+  for (int j = 0; j < V; ++j) {
+    sm[threadIdx.x * 2 * V + j] = a[j];
+    sm[threadIdx.x * 2 * V + V + j] = b[j];
+  }
+  __syncthreads();
+  return (int)blockDim.x / CV;
+}
+// kind 0: the a sums, kind 1: the b sums; c: channel.  Partial p of channel group g sits at row p*CV + g.
+template <int V>
+__device__ __forceinline__ float block_channel_sum(const float* sm, int C, int n_partials, int kind, int c) {
+  const int CV = C / V;
+  const int g = c / V, j = c % V;
+  float acc = 0.f;
+  for (int p = 0; p < n_partials; ++p) acc += sm[(p * CV + g) * 2 * V + kind * V + j];
+  return acc;
+}
+
 // ---------------------------------------------------------------------------------------
 // per-channel sum / sum of squares  ->  stats[2C] (double atomics, one per block and channel)
 // ---------------------------------------------------------------------------------------
@@ -51,7 +97,6 @@ __global__ void bn_stats_kernel(const T* __restrict__ x, long long total_vecs, i
   pdl_launch_dependents();
   constexpr int V = VecT<T>::N;
   extern __shared__ float sm[];  // [blockDim][2*V]
-  const int CV = C / V;
   float s[V], q[V];
 #pragma unroll
   for (int j = 0; j < V; ++j) s[j] = q[j] = 0.f;
@@ -74,20 +119,10 @@ __global__ void bn_stats_kernel(const T* __restrict__ x, long long total_vecs, i
       }
     }
   }
-#pragma unroll
-  for (int j = 0; j < V; ++j) {
-    sm[threadIdx.x * 2 * V + j] = s[j];
-    sm[threadIdx.x * 2 * V + V + j] = q[j];
-  }
-  __syncthreads();
-  // thread t < 2*C sums one (channel, moment) column over the threads sharing its channel group
-  for (int t = threadIdx.x; t < 2 * C; t += blockDim.x) {
-    const int moment = t / C, c = t % C;
-    const int g = c / V, j = c % V;
-    float acc = 0.f;
-    for (int th = g; th < blockDim.x; th += CV) acc += sm[th * 2 * V + moment * V + j];
-    atomicAdd(&stats[moment * C + c], (double)acc);
-  }
+  // thread t < 2*C sums one (moment, channel) column of the block's partial sums
+  const int n_partials = block_channel_partials<V>(s, q, sm, C);
+  for (int t = threadIdx.x; t < 2 * C; t += blockDim.x)
+    atomicAdd(&stats[t], (double)block_channel_sum<V>(sm, C, n_partials, t / C, t % C));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -335,18 +370,10 @@ bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ x, int relu
       }
     }
   }
-#pragma unroll
-  for (int j = 0; j < V; ++j) {
-    sm[threadIdx.x * 2 * V + j] = sb[j];
-    sm[threadIdx.x * 2 * V + V + j] = sg[j];
-  }
-  __syncthreads();
+  const int n_partials = block_channel_partials<V>(sb, sg, sm, C);
   for (int t = threadIdx.x; t < 2 * C; t += blockDim.x) {
-    const int which = t / C, c = t % C;
-    const int g = c / V, j = c % V;
-    float acc = 0.f;
-    for (int th = g; th < blockDim.x; th += CV) acc += sm[th * 2 * V + which * V + j];
-    atomicAdd(which ? &dgamma[c] : &dbeta[c], acc);
+    const float acc = block_channel_sum<V>(sm, C, n_partials, t / C, t % C);
+    atomicAdd(t / C ? &dgamma[t % C] : &dbeta[t % C], acc);
   }
 }
 
