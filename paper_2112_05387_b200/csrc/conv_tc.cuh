@@ -94,8 +94,9 @@ struct ConvTcParams {
                                  // tiles) that is more than the tensor work, with two taps per stage it is less
   uint32_t b_tile_bytes;         // weights of one tap inside a weight stage
   uint32_t tail_offset;          // barriers and scratch after the rings
-  int tap_widx9[9];              // weight tap index of the nine taps in (dy, dx) order
-  uint32_t tap_off9[9];          // byte offset of the tap's first row inside the box
+  int tap_widx9[16];             // weight tap index of the taps in (dy, dx) order (nine for 3x3, sixteen for 4x4)
+  uint32_t tap_off9[16];         // byte offset of the tap's first row inside the box
+  int halo_dw0, halo_dh0;        // offset of the first tap: the box starts that many pixels from the tile (-1 for 3x3)
   uint64_t desc_hi_a;            // descriptor of the activation operand (row-group stride of the box)
   // local loss of an interior module, fused into the epilogue of the module's last convolution
   // (kLoss instantiation): r = out - x_next, sums of r^2 and kappa*r, seed = rho*r + kappa
@@ -259,13 +260,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint8_t* pa = smem + sa * p.a_stage_bytes;
         if (elect_one()) {
           mbar_expect_tx(&tail->full[sa], cnt * p.tx_a);
-          tma_load_4d(pa, &tmA, &tail->full[sa], c * p.KC, w0[0] - 1, n0[0], h0[0] - 1);
-          if (cnt == 2) tma_load_4d(pa + p.a_halo_bytes, &tmA, &tail->full[sa], c * p.KC, w0[1] - 1, n0[1], h0[1] - 1);
+          tma_load_4d(pa, &tmA, &tail->full[sa], c * p.KC, w0[0] + p.halo_dw0, n0[0], h0[0] + p.halo_dh0);
+          if (cnt == 2) tma_load_4d(pa + p.a_halo_bytes, &tmA, &tail->full[sa], c * p.KC, w0[1] + p.halo_dw0, n0[1], h0[1] + p.halo_dh0);
         }
         __syncwarp();
         if (++sa == (uint32_t)p.nA) { sa = 0; pha ^= 1; }
-        for (int ti0 = 0; ti0 < 9; ti0 += p.tps) {
-          const int n_taps = min(p.tps, 9 - ti0);
+        for (int ti0 = 0; ti0 < p.ntaps; ti0 += p.tps) {
+          const int n_taps = min(p.tps, p.ntaps - ti0);
           if (!mbar_wait_warp(&tail->empty_b[sb], phb ^ 1, abort_flag)) { failed = true; break; }
           if (elect_one()) {
             mbar_expect_tx(&tail->full_b[sb], n_taps * p.tx_b);
@@ -302,9 +303,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int c = 0; c < p.chunks && !failed; ++c) {
         const uint32_t a_addr = smem_base + sa * p.a_stage_bytes + me * p.a_halo_bytes;
         const int nkc = c + 1 == p.chunks ? p.nk_last : nk;   // slices of pure zero fill are not multiplied
-        for (int ti0 = 0; ti0 < 9; ti0 += p.tps) {
-          const int n_taps = min(p.tps, 9 - ti0);
-          const bool last_of_chunk = ti0 + n_taps == 9;
+        for (int ti0 = 0; ti0 < p.ntaps; ti0 += p.tps) {
+          const int n_taps = min(p.tps, p.ntaps - ti0);
+          const bool last_of_chunk = ti0 + n_taps == p.ntaps;
           // The box barrier is polled together with the first weight stage and released together
           // with the last one: a separate trip (poll, election, commit) at every chunk boundary
           // costs about 500 cycles in which the tensor pipe runs dry.

@@ -387,18 +387,23 @@ static const size_t kTcThinSmem = 100 * 1024;  // two CTAs of the few-channel in
 #define LP_CONV_MAX_ITEMS_PER_STAGE 16   // (tap, chunk) items per pipeline stage of the plain mode, at most
 #endif
 #ifndef LP_CONV_TAPS_PER_STAGE
-#define LP_CONV_TAPS_PER_STAGE 9   // taps per weight stage (halo mode), at most: as many as leave three stages
+#define LP_CONV_TAPS_PER_STAGE 16  // taps per weight stage (halo mode), at most: as many as leave three stages
 #endif
 static const int kHaloBoxW = 10;   // 8-pixel tile width plus one halo pixel on each side
 
-static bool pick_halo_box(const TcGemmSpec& s, int& BW, int& BH, int& BNI, int tapw3[3][3]) {
-  if (s.ntaps != 9 || s.in_step != 1 || s.os != 1 || s.OWl % 8) return false;
-  bool seen[3][3] = {};
-  for (int i = 0; i < 9; ++i) {
-    const int dx = s.dw[i] + 1, dy = s.dh[i] + 1;
-    if (dx < 0 || dx > 2 || dy < 0 || dy > 2 || seen[dx][dy]) return false;
-    seen[dx][dy] = true;
-    tapw3[dx][dy] = s.widx[i];
+// Halo mode: the taps form a full R x R grid of whole-pixel offsets (3x3 convolutions; the 4x4 grid of a
+// space-to-depth stem), stride 1.  R: grid size; dw0, dh0: offset of the first tap; tapw[dy*R + dx]: weight index.
+static bool pick_halo_box_r(const TcGemmSpec& s, int& BW, int& BH, int& BNI, int& R, int& dw0, int& dh0, int tapw[16]) {
+  R = s.ntaps == 9 ? 3 : (s.ntaps == 16 ? 4 : 0);
+  if (!R || s.in_step != 1 || s.os != 1 || s.OWl % 8) return false;
+  dw0 = dh0 = 1 << 20;
+  for (int i = 0; i < s.ntaps; ++i) { dw0 = std::min(dw0, s.dw[i]); dh0 = std::min(dh0, s.dh[i]); }
+  bool seen[16] = {};
+  for (int i = 0; i < s.ntaps; ++i) {
+    const int dx = s.dw[i] - dw0, dy = s.dh[i] - dh0;
+    if (dx < 0 || dx >= R || dy < 0 || dy >= R || seen[dy * R + dx]) return false;
+    seen[dy * R + dx] = true;
+    tapw[dy * R + dx] = s.widx[i];
   }
   BW = 8;
   if (8 * s.OHl <= 64) {
@@ -412,13 +417,20 @@ static bool pick_halo_box(const TcGemmSpec& s, int& BW, int& BH, int& BNI, int t
   }
   return BH >= 2 && 8 * BH * BNI >= 96;
 }
+static bool pick_halo_box(const TcGemmSpec& s, int& BW, int& BH, int& BNI, int tapw3[3][3]) {
+  int R, dw0, dh0, tapw[16];
+  if (!pick_halo_box_r(s, BW, BH, BNI, R, dw0, dh0, tapw) || R != 3 || dw0 != -1 || dh0 != -1) return false;
+  for (int dy = 0; dy < 3; ++dy)
+    for (int dx = 0; dx < 3; ++dx) tapw3[dx][dy] = tapw[dy * 3 + dx];
+  return true;
+}
 
 static int encode_act_map_halo(CUtensorMap* m, const void* base, int N, int H, int W, int C, int boxC, int boxW, int BH,
-                               int BNI, int row_bytes) {
+                               int BNI, int row_bytes, int halo = 2) {
   // dimension order (C, W, image, H): the image row is the slowest coordinate of the box
   cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)N, (cuuint64_t)H};
   cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)H * W * C * 2, (cuuint64_t)W * C * 2};
-  cuuint32_t box[4] = {(cuuint32_t)boxC, (cuuint32_t)boxW, (cuuint32_t)BNI, (cuuint32_t)(BH + 2)};
+  cuuint32_t box[4] = {(cuuint32_t)boxC, (cuuint32_t)boxW, (cuuint32_t)BNI, (cuuint32_t)(BH + halo)};
   cuuint32_t es[4] = {1, 1, 1, 1};
   const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                 : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
@@ -565,10 +577,11 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   tc::ConvTcParams p;
   memset(&p, 0, sizeof(p));
   p.Nimg = s.aN; p.OHl = s.OHl; p.OWl = s.OWl;
-  int tapw3[3][3];
+  int tapw[16], halo_R = 3;
   // (any K chunk width: the row-shifted operand descriptors only need the swizzle to be a function of the
   // shared-memory address, which holds for 32-, 64- and 128-byte rows alike)
-  p.halo = pick_halo_box(s, p.BW, p.BH, p.BNI, tapw3) ? 1 : 0;
+  p.halo = pick_halo_box_r(s, p.BW, p.BH, p.BNI, halo_R, p.halo_dw0, p.halo_dh0, tapw) ? 1 : 0;
+  const int halo_w = 8 + halo_R - 1;   // box width: the 8-pixel tile plus the taps' reach
   if (!p.halo) pick_pixel_box(s.OWl, s.OHl, s.aN, p.BW, p.BH, p.BNI);
   p.tiles_w = (s.OWl + p.BW - 1) / p.BW;
   p.tiles_h = (s.OHl + p.BH - 1) / p.BH;
@@ -616,15 +629,15 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   }
   if (p.halo) {
     // activation ring: three boxes deep if at least three weight stages still fit, else two
-    const int halo_rows = kHaloBoxW * p.BNI * (p.BH + 2);
+    const int halo_rows = halo_w * p.BNI * (p.BH + halo_R - 1);
     p.a_halo_bytes = (uint32_t)align_up((size_t)halo_rows * row_bytes, 1024);
-    for (int dy = 0; dy < 3; ++dy)
-      for (int dx = 0; dx < 3; ++dx) {
-        p.tap_widx9[dy * 3 + dx] = tapw3[dx][dy];
-        p.tap_off9[dy * 3 + dx] = (uint32_t)((dy * kHaloBoxW * p.BNI + dx) * row_bytes);
+    for (int dy = 0; dy < halo_R; ++dy)
+      for (int dx = 0; dx < halo_R; ++dx) {
+        p.tap_widx9[dy * halo_R + dx] = tapw[dy * halo_R + dx];
+        p.tap_off9[dy * halo_R + dx] = (uint32_t)((dy * halo_w * p.BNI + dx) * row_bytes);
       }
-    // 8-row groups of the operand are one box row (kHaloBoxW pixels) apart
-    p.desc_hi_a = tc::smem_desc_hi(16, kHaloBoxW * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
+    // 8-row groups of the operand are one box row (halo_w pixels) apart
+    p.desc_hi_a = tc::smem_desc_hi(16, halo_w * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
     p.b_tile_bytes = b_region;
     p.tx_a = (uint32_t)(halo_rows * row_bytes);
     const size_t avail = max_smem - tail;
@@ -636,7 +649,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
          pair >= 1 && !fits; --pair) {
       const size_t a_bytes = (size_t)p.nA * pair * p.a_halo_bytes;
       if (a_bytes >= avail) continue;
-      for (int tps = LP_CONV_TAPS_PER_STAGE; tps >= 1 && !fits; --tps) {
+      for (int tps = std::min(LP_CONV_TAPS_PER_STAGE, s.ntaps); tps >= 1 && !fits; --tps) {
         const int nb = (int)std::min<size_t>((avail - a_bytes) / ((size_t)tps * b_region), LP_CONV_MAX_NB);
         if (nb >= 3) { p.mpair = pair; p.nB = nb; p.tps = tps; fits = true; }
       }
@@ -695,7 +708,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
               (reinterpret_cast<uintptr_t>(s.out) & 31) == 0 &&
               (!s.addend || (reinterpret_cast<uintptr_t>(s.addend) & 31) == 0)) ? 1 : 0;
   CUtensorMap tmA, tmB;
-  int rc = p.halo ? encode_act_map_halo(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, p.KC, kHaloBoxW, p.BH, p.BNI, row_bytes)
+  int rc = p.halo ? encode_act_map_halo(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, p.KC, halo_w, p.BH, p.BNI, row_bytes, halo_R - 1)
                   : encode_act_map(&tmA, s.act, s.aN, s.aH, s.aW, s.aC, p.KC, p.BW, p.BH, p.BNI, s.in_step, row_bytes);
   if (rc != LP_OK) return rc;
   rc = encode_mat_map(&tmB, s.wmat, s.w_K, s.w_rows, p.KC, p.n_tile_cols, row_bytes);
