@@ -183,12 +183,15 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         __syncwarp();
         if (++sa == (uint32_t)p.nA) { sa = 0; pha ^= 1; }
-        for (int ti = 0; ti < 9; ++ti) {
+        for (int ti0 = 0; ti0 < 9; ti0 += p.tps) {      // a weight stage holds this CTA's half of p.tps taps
+          const int n_taps = min(p.tps, 9 - ti0);
           if (!mbar_wait_warp(&tail->empty_b[sb], phb ^ 1, abort_flag)) { failed = true; break; }
           if (elect_one()) {
             const uint32_t fb = mapa_u32(smem_u32(&tail->full_b[sb]), 0);
-            if (leader) mbar_expect_tx(&tail->full_b[sb], 2 * p.tx_b);
-            tma2_load_2d(b_ring + sb * p.b_stage_bytes, &tmB, fb, p.tap_widx9[ti] * p.Cin + c * p.KC, col0);
+            if (leader) mbar_expect_tx(&tail->full_b[sb], 2 * (uint32_t)n_taps * p.tx_b);
+            for (int i = 0; i < n_taps; ++i)
+              tma2_load_2d(b_ring + sb * p.b_stage_bytes + i * p.b_tile_bytes, &tmB, fb,
+                           p.tap_widx9[ti0 + i] * p.Cin + c * p.KC, col0);
           }
           __syncwarp();
           if (++sb == (uint32_t)p.nB) { sb = 0; phb ^= 1; }
@@ -215,7 +218,7 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       if (!active) {
         // nothing for the second warp in a unit of one accumulator: it only advances its ring positions (a
         // second warp polling the barriers slowed the active one down), and the active warp signals twice
-        const uint32_t tb = sb + (uint32_t)(p.chunks * 9), ta = sa + (uint32_t)p.chunks;
+        const uint32_t tb = sb + (uint32_t)(p.chunks * ((9 + p.tps - 1) / p.tps)), ta = sa + (uint32_t)p.chunks;
         phb ^= (tb / (uint32_t)p.nB) & 1; sb = tb % (uint32_t)p.nB;
         pha ^= (ta / (uint32_t)p.nA) & 1; sa = ta % (uint32_t)p.nA;
         slot_phase ^= 1u << sl[0];
@@ -231,19 +234,23 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       for (int c = 0; c < p.chunks && !failed; ++c) {
         const uint32_t a_addr = smem_base + sa * p.a_stage_bytes + me * p.a_halo_bytes;
         const int nkc = c + 1 == p.chunks ? p.nk_last : nk;
-        for (int ti = 0; ti < 9; ++ti) {
-          bool ok = ti ? true : mbar_wait(&tail->full[sa], pha, abort_flag);
+        for (int ti0 = 0; ti0 < 9; ti0 += p.tps) {
+          const int n_taps = min(p.tps, 9 - ti0);
+          bool ok = ti0 ? true : mbar_wait(&tail->full[sa], pha, abort_flag);
           ok = mbar_wait(&tail->full_b[sb], phb, abort_flag) && ok;
           if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
           tc_fence_after();
-          const uint64_t ad = smem_desc(p.desc_hi_a, a_addr + p.tap_off9[ti]);
-          const uint64_t bd = smem_desc(p.desc_hi, smem_base + p.b_ring_offset + sb * p.b_stage_bytes);
+          const uint32_t b_addr = smem_base + p.b_ring_offset + sb * p.b_stage_bytes;
           if (elect_one()) {
-            for (int j = 0; j < nkc; ++j)
-              mma2_bf16(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (accum | j) ? 1u : 0u);
+            for (int i = 0; i < n_taps; ++i) {
+              const uint64_t ad = smem_desc(p.desc_hi_a, a_addr + p.tap_off9[ti0 + i]);
+              const uint64_t bd = smem_desc(p.desc_hi, b_addr + i * p.b_tile_bytes);
+              for (int j = 0; j < nkc; ++j)
+                mma2_bf16(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), p.idesc, (accum | i | j) ? 1u : 0u);
+            }
             mma2_commit_both(&tail->empty_b[sb]);
             if (alone) mma2_commit_both(&tail->empty_b[sb]);
-            if (ti == 8) {
+            if (ti0 + n_taps == 9) {
               mma2_commit_both(&tail->empty[sa]);
               if (alone) mma2_commit_both(&tail->empty[sa]);
             }

@@ -386,6 +386,9 @@ static const size_t kTcThinSmem = 100 * 1024;  // two CTAs of the few-channel in
 #ifndef LP_CONV_MAX_ITEMS_PER_STAGE
 #define LP_CONV_MAX_ITEMS_PER_STAGE 16   // (tap, chunk) items per pipeline stage of the plain mode, at most
 #endif
+#ifndef LP_CONV2_TAPS_PER_STAGE
+#define LP_CONV2_TAPS_PER_STAGE 3  // the same for the CTA-pair kernel (a stage holds each CTA's half of the taps' weights)
+#endif
 #ifndef LP_CONV_TAPS_PER_STAGE
 #define LP_CONV_TAPS_PER_STAGE 16  // taps per weight stage (halo mode), at most: as many as leave three stages
 #endif
@@ -505,14 +508,19 @@ static int launch_conv_tc2(lp_handle* h, const TcGemmSpec& s, int* dev_err, cuda
     }
   p.desc_hi_a = tc::smem_desc_hi(16, kHaloBoxW * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
   p.desc_hi = tc::smem_desc_hi(16, 8 * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
-  p.b_stage_bytes = b_half;
   p.tx_a = (uint32_t)(halo_rows * row_bytes);
   p.nA = 2;
   p.mpair = 2;
   p.a_stage_bytes = 2 * p.a_halo_bytes;
   const size_t a_bytes = (size_t)p.nA * p.a_stage_bytes;
   if (a_bytes + 3 * (size_t)b_half + tail > kTcMaxSmem) return LP_ERR_UNSUPPORTED;
-  p.nB = (int)std::min<size_t>((kTcMaxSmem - tail - a_bytes) / b_half, tc::kMaxStages);
+  // taps per weight stage: as many (of at most LP_CONV2_TAPS_PER_STAGE) as leave three stages, as in the one-CTA kernel
+  p.b_tile_bytes = b_half;
+  p.tps = 1;
+  for (int tps = LP_CONV2_TAPS_PER_STAGE; tps > 1; --tps)
+    if ((kTcMaxSmem - tail - a_bytes) / ((size_t)tps * b_half) >= 3) { p.tps = tps; break; }
+  p.b_stage_bytes = p.tps * b_half;
+  p.nB = (int)std::min<size_t>((kTcMaxSmem - tail - a_bytes) / p.b_stage_bytes, tc::kMaxStages);
   p.b_ring_offset = (uint32_t)a_bytes;
   p.tail_offset = p.b_ring_offset + p.nB * p.b_stage_bytes;
   p.stage_offset = p.tail_offset;
