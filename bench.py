@@ -400,6 +400,22 @@ def run_ours(args):
         conv_ms, conv_flops, conv_launches = lp.lp_conv_profile(h, False, read=True)
         barrier()
 
+        # what an event pair costs around a launch that does nothing: the part of every per-launch time above that
+        # is not the kernel's own work (the stream is kept busy before each pair so that the host is ahead)
+        busy = torch.empty(64 << 20, dtype=torch.uint8, device=dev)
+        tiny = torch.zeros(1, dtype=torch.float32, device=dev)
+        floors = []
+        for _ in range(24):
+            busy.zero_()
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0.record(stream)
+            tiny.zero_()
+            f1.record(stream)
+            stream.synchronize()
+            floors.append(f0.elapsed_time(f1))
+        event_pair_floor_ms = float(np.median(floors[4:]))
+        del busy
+
         # per-operation time line of the same serial pass: achieved GB/s of the HBM-bound kernels
         # (algorithmic bytes of the operation / its CUDA-event time)
         lp.lp_timeline(h, True, read=False)
@@ -568,7 +584,10 @@ def run_ours(args):
                 "traffic": traffic,
                 "traffic_note": ("DRAM bytes read + written per launch, " + traffic_src) if traffic_src else
                                 "no profiler record for this workload at the present kernels",
-                "timing": "CUDA events around every tensor-core conv launch, modules run back to back on one stream"}
+                "timing": "CUDA events around every tensor-core conv launch, modules run back to back on one stream",
+                "event_pair_floor_ms": event_pair_floor_ms,
+                "event_pair_floor_note": "a one-element fill between two CUDA events on the busy stream: this much of "
+                                         "avg_launch_ms is launch and event latency, which a graph replay does not pay"}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32",
