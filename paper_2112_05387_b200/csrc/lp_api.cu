@@ -398,7 +398,11 @@ static const int kHaloBoxW = 10;   // 8-pixel tile width plus one halo pixel on 
 // space-to-depth stem), stride 1.  R: grid size; dw0, dh0: offset of the first tap; tapw[dy*R + dx]: weight index.
 static bool pick_halo_box_r(const TcGemmSpec& s, int& BW, int& BH, int& BNI, int& R, int& dw0, int& dh0, int tapw[16]) {
   R = s.ntaps == 9 ? 3 : (s.ntaps == 16 ? 4 : 0);
-  if (!R || s.in_step != 1 || s.os != 1 || s.OWl % 8) return false;
+  // tiles are 8 pixels wide; a width that is not a multiple of 8 leaves the last tile column ragged (rows past the
+  // image read zero fill and are masked in the epilogue): taken where at most an eighth of the columns is wasted
+  // (7, 14, 28, ...), since the alternative is nine shifted boxes per K chunk instead of one
+  const int tiles_w8 = (s.OWl + 7) / 8;
+  if (!R || s.in_step != 1 || s.os != 1 || s.OWl * 8 < 7 * 8 * tiles_w8) return false;
   dw0 = dh0 = 1 << 20;
   for (int i = 0; i < s.ntaps; ++i) { dw0 = std::min(dw0, s.dw[i]); dh0 = std::min(dh0, s.dh[i]); }
   bool seen[16] = {};
