@@ -81,8 +81,8 @@ TC_CASES = [
     (2, 16, 16, 64, 128, 3, 2, 1),    # stride 2
     (2, 16, 16, 64, 128, 1, 2, 0),    # 1x1 stride-2 projection
     (2, 8, 8, 128, 64, 1, 1, 0),      # 1x1
-    (2, 14, 14, 64, 64, 3, 1, 1),     # 14x14: 98-pixel boxes
-    (3, 7, 7, 128, 128, 3, 1, 1),     # 7x7 pairs of images, odd batch
+    (2, 14, 14, 64, 64, 3, 1, 1),     # 14x14: two tile columns, the second ragged
+    (3, 7, 7, 128, 128, 3, 1, 1),     # 7x7: one ragged tile column, pairs of images, odd batch
     (2, 32, 32, 40, 160, 3, 1, 1),    # AuxNet hidden width (C_in = 40)
     (2, 32, 32, 160, 80, 3, 2, 1),    # AuxNet strided
     (2, 32, 32, 160, 40, 3, 1, 1),    # AuxNet hidden width as C_out (weight gradient: 32 + 16 channel sub-boxes)
@@ -96,6 +96,7 @@ TC_CASES = [
     (40, 32, 32, 160, 160, 3, 1, 1),  # 320 halo tiles of 16x8 pixels: pairs, three K chunks with zero fill
     (5, 12, 20, 64, 256, 3, 1, 1),    # 256-channel tile: eight staging groups, two passes over the accumulator; ragged boxes
     (3, 9, 9, 32, 96, 1, 1, 0),       # odd image size, 81-pixel boxes, three staging groups
+    (3, 28, 28, 64, 128, 3, 1, 1),    # width 28: four 8-pixel tile columns, the last one half outside the image
 ]
 
 
