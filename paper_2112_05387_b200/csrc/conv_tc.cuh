@@ -66,6 +66,13 @@ struct ConvTcParams {
   int n_tile_cols, Cout;
   int ntaps;
   int tap_dh[16], tap_dw[16], tap_w[16];   // up to 16 taps (plain mode; the space-to-depth stem has 4x4)
+  // Tile classes (plain mode, direct epilogue): a stride-2 input gradient is one convolution per parity class of
+  // the input pixels -- same logical grid and tiles, but its own subset of the taps and its own offset into the
+  // physical output -- and one launch walks the classes one after another: tile t belongs to class
+  // (t / m_tiles) / n_tiles and to channel tile (t / m_tiles) % n_tiles.  Every other launch has one class.
+  int n_cls;
+  int cls_ntaps[4], cls_tap0[4];           // taps of the class: tap_*[cls_tap0 .. cls_tap0 + cls_ntaps)
+  int cls_oo_h[4], cls_oo_w[4];            // physical pixel = logical * os + cls_oo
   int Cin, KC, chunks;
   int nk_last;                   // K = 16 slices of the last chunk that hold real channels (the rest is zero fill)
   int stages;
@@ -235,7 +242,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   pdl_wait();                 // the set-up above overlapped the tail of the preceding kernel
   pdl_launch_dependents();
   const uint32_t tmem_base = tail->tmem_base;
-  const int kiters = p.ntaps * p.chunks;
   bool failed = false;
 
   // All three roles walk the same sequence of units: a unit is one pixel tile, or two consecutive
@@ -347,7 +353,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------- TMA producer (warp-uniform loop, elected issue) ----
     uint32_t s = 0, ph = 0;
     for (int t = t_begin; t < t_end && !failed;) {
-      const int nt = t / p.m_tiles, m = t % p.m_tiles;
+      const int ntg = t / p.m_tiles, m = t % p.m_tiles;
+      const int cls = ntg / p.n_tiles, nt = ntg % p.n_tiles;
+      const int kiters = p.cls_ntaps[cls] * p.chunks;
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m + 1 < p.m_tiles) ? 2 : 1;
       int w0[2], h0[2], n0[2];
       for (int a = 0; a < 2; ++a) {
@@ -365,7 +373,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (elect_one()) {
           mbar_expect_tx(&tail->full[s], n_items * tx);
           for (int i = 0; i < n_items; ++i) {
-            const int tap = (k0 + i) / p.chunks, c = (k0 + i) % p.chunks;
+            const int tap = p.cls_tap0[cls] + (k0 + i) / p.chunks, c = (k0 + i) % p.chunks;
             const int kb = p.tap_w[tap] * p.Cin;
             uint8_t* si = sa + i * p.item_bytes;
             tma_load_4d(si, &tmA, &tail->full[s], c * p.KC, w0[0] * p.in_step + p.tap_dw[tap],
@@ -393,6 +401,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint32_t slot = 0, slot_phase = 0;  // bit b of slot_phase: parity of the number of uses of slot b
     for (int t = t_begin; t < t_end && !failed;) {
       const int m = t % p.m_tiles;
+      const int kiters = p.cls_ntaps[(t / p.m_tiles) / p.n_tiles] * p.chunks;
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m + 1 < p.m_tiles) ? 2 : 1;
       uint32_t sl[2];
       sl[0] = slot;
@@ -611,13 +620,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // waiting for DRAM.
     auto prefetch_rows = [&](const bf16* base, int tile) {
       if (tile >= t_end) return;
-      const int pnt = tile / p.m_tiles, pm = tile % p.m_tiles;
+      const int pntg = tile / p.m_tiles, pm = tile % p.m_tiles;
+      const int pcls = pntg / p.n_tiles, pnt = pntg % p.n_tiles;
       const int pw = (pm % p.tiles_w) * p.BW + row % p.BW;
       const int phh = ((pm / p.tiles_w) % p.tiles_h) * p.BH + (p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH);
       const int pn = (pm / (p.tiles_w * p.tiles_h)) * p.BNI + (p.halo ? (row / p.BW) % p.BNI : row / (p.BW * p.BH));
       if (row >= rows_used || pw >= p.OWl || phh >= p.OHl || pn >= p.Nimg || grp) return;
       const long long pb =
-          (((long long)pn * p.out_H + (phh * p.os + p.oo_h)) * p.out_W + (pw * p.os + p.oo_w)) * p.out_C + pnt * p.n_tile_cols;
+          (((long long)pn * p.out_H + (phh * p.os + p.cls_oo_h[pcls])) * p.out_W + (pw * p.os + p.cls_oo_w[pcls])) * p.out_C +
+          pnt * p.n_tile_cols;
       const int ncols = min(p.n_tile_cols, p.Cout - pnt * p.n_tile_cols);
       const uintptr_t b = reinterpret_cast<uintptr_t>(base + pb);
       for (uintptr_t l = b & ~(uintptr_t)127; l < b + 2 * (uintptr_t)ncols; l += 128)
@@ -630,9 +641,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     prefetch_addend(t_begin);
     int consts_nt = -1;                  // channel tile whose batch-norm constants are in shared memory (kBnBwd)
     for (int t = t_begin; t < t_end && !failed;) {
-      const int nt = t / p.m_tiles, m0 = t % p.m_tiles;
+      const int nt = t / p.m_tiles, m0 = t % p.m_tiles;     // nt counts (class, channel tile) pairs
+      const int cls = nt / p.n_tiles;
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m0 + 1 < p.m_tiles) ? 2 : 1;
-      const int col0 = nt * p.n_tile_cols;
+      const int col0 = (nt % p.n_tiles) * p.n_tile_cols;
       if constexpr (kBnBwd) {
         if (nt != consts_nt) {
           // scale, shift (the forward kernel's, for the ReLU mask), mean and rstd of this channel tile
@@ -665,7 +677,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int n = n0 + (p.halo ? (row / p.BW) % p.BNI : row / (p.BW * p.BH));
         const bool valid = row < rows_used && ow < p.OWl && oh < p.OHl && n < p.Nimg;
         const long long obase =
-            (((long long)n * p.out_H + (oh * p.os + p.oo_h)) * p.out_W + (ow * p.os + p.oo_w)) * p.out_C;
+            (((long long)n * p.out_H + (oh * p.os + p.cls_oo_h[cls])) * p.out_W + (ow * p.os + p.cls_oo_w[cls])) * p.out_C;
         // one thread waits (bounded) and all epilogue threads agree on the outcome, so that the
         // named barriers below are reached by all of them or by none
         // (two words used in turn: the one of the previous accumulator may still be read by a slower warp

@@ -286,6 +286,9 @@ struct TcGemmSpec {
   int two_cta;           // 1: 3x3 stride-1 convolutions take the CTA-pair kernel where it applies
   // reduction pass of a batch-norm backward fused into the epilogue; bwd_x == nullptr: off
   const bf16* bwd_x; BnArgs bwd_bn; float* bwd_dgamma; float* bwd_dbeta; int bwd_relu;
+  // tile classes (see ConvTcParams): n_cls > 1 for the parity classes of a stride-2 input gradient in one launch;
+  // the taps of class i are dh/dw/widx[cls_tap0[i] .. +cls_ntaps[i]), its output offset (cls_oo_h[i], cls_oo_w[i])
+  int n_cls; int cls_ntaps[4], cls_tap0[4], cls_oo_h[4], cls_oo_w[4];
 };
 
 static void pick_pixel_box(int OWl, int OHl, int Nimg, int& BW, int& BH, int& BNI) {
@@ -592,7 +595,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   int tapw[16], halo_R = 3;
   // (any K chunk width: the row-shifted operand descriptors only need the swizzle to be a function of the
   // shared-memory address, which holds for 32-, 64- and 128-byte rows alike)
-  p.halo = pick_halo_box_r(s, p.BW, p.BH, p.BNI, halo_R, p.halo_dw0, p.halo_dh0, tapw) ? 1 : 0;
+  p.halo = (s.n_cls <= 1 && pick_halo_box_r(s, p.BW, p.BH, p.BNI, halo_R, p.halo_dw0, p.halo_dh0, tapw)) ? 1 : 0;
   const int halo_w = 8 + halo_R - 1;   // box width: the 8-pixel tile plus the taps' reach
   if (!p.halo) pick_pixel_box(s.OWl, s.OHl, s.aN, p.BW, p.BH, p.BNI);
   p.tiles_w = (s.OWl + p.BW - 1) / p.BW;
@@ -600,7 +603,19 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
   const int tiles_n = (s.aN + p.BNI - 1) / p.BNI;
   p.m_tiles = p.tiles_w * p.tiles_h * tiles_n;
   pick_n_tile(s.w_rows, p.n_tile_cols, p.n_tiles);
-  p.total_tiles = p.m_tiles * p.n_tiles;
+  p.n_cls = std::max(1, s.n_cls);
+  int max_cls_taps = s.ntaps;
+  if (s.n_cls > 1) {
+    max_cls_taps = 0;
+    for (int i = 0; i < s.n_cls; ++i) {
+      p.cls_ntaps[i] = s.cls_ntaps[i]; p.cls_tap0[i] = s.cls_tap0[i];
+      p.cls_oo_h[i] = s.cls_oo_h[i]; p.cls_oo_w[i] = s.cls_oo_w[i];
+      max_cls_taps = std::max(max_cls_taps, s.cls_ntaps[i]);
+    }
+  } else {
+    p.cls_ntaps[0] = s.ntaps; p.cls_tap0[0] = 0; p.cls_oo_h[0] = s.oo_h; p.cls_oo_w[0] = s.oo_w;
+  }
+  p.total_tiles = p.m_tiles * p.n_tiles * p.n_cls;
   p.in_step = s.in_step;
   p.out_H = s.out_H; p.out_W = s.out_W; p.out_C = s.out_C;
   p.os = s.os; p.oo_h = s.oo_h; p.oo_w = s.oo_w;
@@ -678,7 +693,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
       p.tiles_w = (s.OWl + p.BW - 1) / p.BW;
       p.tiles_h = (s.OHl + p.BH - 1) / p.BH;
       p.m_tiles = p.tiles_w * p.tiles_h * ((s.aN + p.BNI - 1) / p.BNI);
-      p.total_tiles = p.m_tiles * p.n_tiles;
+      p.total_tiles = p.m_tiles * p.n_tiles * p.n_cls;
     }
   }
   if (!p.halo) {
@@ -694,7 +709,7 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     // stages of a tile.  Layers with few channels (16 or 32: an item is one or two instructions) then pay the
     // fixed cost of a stage once per several taps; wide layers keep one item per stage.
     {
-      const int kiters = p.ntaps * p.chunks;
+      const int kiters = max_cls_taps * p.chunks;   // (of the class with the most taps)
       int ips = (int)std::min<size_t>((size_t)std::min(kiters, LP_CONV_MAX_ITEMS_PER_STAGE), (max_smem - tail) / 3 / p.item_bytes);
       ips = std::max(ips, 1);
       const int n_st = (kiters + ips - 1) / ips;
@@ -966,6 +981,40 @@ static int conv_dgrad(lp_handle* h, int dtype, int impl, const ConvDef& c, int N
       if (!addend) LP_CUDA_OK(cudaMemsetAsync(dx, 0, (size_t)N * c.H * c.W * c.cin * 2, st));
     }
     ProfScope ps(h, st, 2.0 * N * c.OH * c.OW * (double)c.cout * c.R * c.R * c.cin);
+    if (st2 == 2 && !any_empty && c.H % 2 == 0 && c.W % 2 == 0 && c.R * c.R <= 16) {
+      // every parity class has the same logical grid (H/2 x W/2) and only its taps and its offset into dx differ:
+      // one launch walks the four classes (tile classes of the kernel) instead of four quarter-size launches
+      TcGemmSpec s;
+      memset(&s, 0, sizeof(s));
+      s.act = (const bf16*)dy; s.aN = N; s.aH = c.OH; s.aW = c.OW; s.aC = c.cout;
+      s.wmat = c.wt; s.w_rows = c.cin; s.w_K = (long long)c.R * c.R * c.cout;
+      s.in_step = 1;
+      s.OHl = c.H / 2; s.OWl = c.W / 2;
+      s.n_cls = 4;
+      for (int cls = 0; cls < 4; ++cls) {
+        const int ph = cls / 2, pw = cls % 2;
+        s.cls_tap0[cls] = s.ntaps; s.cls_oo_h[cls] = ph; s.cls_oo_w[cls] = pw;
+        for (int r = 0; r < c.R; ++r) {
+          if ((ph + c.pad - r) % 2) continue;
+          for (int q = 0; q < c.R; ++q) {
+            if ((pw + c.pad - q) % 2) continue;
+            s.dh[s.ntaps] = (ph + c.pad - r) / 2;
+            s.dw[s.ntaps] = (pw + c.pad - q) / 2;
+            s.widx[s.ntaps] = r * c.R + q;
+            s.ntaps++;
+          }
+        }
+        s.cls_ntaps[cls] = s.ntaps - s.cls_tap0[cls];
+      }
+      s.out = (bf16*)dx; s.addend = (const bf16*)addend;
+      s.out_H = c.H; s.out_W = c.W; s.out_C = c.cin; s.os = 2; s.oo_h = 0; s.oo_w = 0;
+      s.epilogue = 1;   // (the staged epilogue needs the output grid to be the logical grid)
+      if (bnf) {
+        s.bwd_x = (const bf16*)bnf->x; s.bwd_bn = bnf->bn; s.bwd_dgamma = bnf->dgamma; s.bwd_dbeta = bnf->dbeta;
+        s.bwd_relu = bnf->relu;
+      }
+      return launch_conv_tc(h, s, dev_err, st);
+    }
     for (int cls = 0; cls < classes; ++cls) {
       const int ph = cls / st2, pw = cls % st2;
       TcGemmSpec s;
