@@ -56,10 +56,38 @@ constexpr int kMaxSlots = 4;     // accumulator slots in tensor memory
 #define LP_EPI_BATCH 5
 #endif
 
+// Division by a run-time constant without the divide instruction (Granlund-Montgomery): for 0 <= n < 2^31,
+// n / d = (umulhi(n, mul) + n) >> shift with shift = ceil(log2 d), mul = floor(2^32 (2^shift - d) / d) + 1.
+// The tile loops of all roles split tile numbers several times per tile; with divide instructions that was a
+// quarter of the life of a CTA on small layers.
+struct FastDiv {
+  uint32_t d, mul, shift;
+};
+__host__ inline FastDiv make_fastdiv(int d) {
+  FastDiv f;
+  f.d = (uint32_t)d; f.mul = 0; f.shift = 0;
+  if (d > 1) {
+    uint32_t s = 0;
+    while ((1u << s) < (uint32_t)d) ++s;
+    f.shift = s;
+    f.mul = (uint32_t)((((uint64_t)1 << 32) * (((uint64_t)1 << s) - (uint64_t)d)) / (uint64_t)d + 1);
+  }
+  return f;
+}
+__device__ __forceinline__ int fd_div(int n, const FastDiv& f) {
+  return f.d == 1 ? n : (int)((__umulhi((uint32_t)n, f.mul) + (uint32_t)n) >> f.shift);
+}
+// q = n / d, r = n % d
+__device__ __forceinline__ void fd_divmod(int n, const FastDiv& f, int& q, int& r) {
+  q = fd_div(n, f);
+  r = n - q * (int)f.d;
+}
+
 struct ConvTcParams {
   int Nimg, OHl, OWl;            // logical output grid
   int BW, BH, BNI;               // tile box (logical pixels), BW*BH*BNI <= 128
   int tiles_w, tiles_h, m_tiles, n_tiles, total_tiles;
+  FastDiv fd_tiles_w, fd_tiles_h, fd_m_tiles, fd_n_tiles, fd_chunks;   // the same numbers as divisors
   int in_step;                   // input coordinate = logical * in_step + tap offset
   int out_H, out_W, out_C;       // physical output tensor
   int os, oo_h, oo_w;            // physical pixel = logical * os + oo
@@ -167,6 +195,14 @@ __device__ __forceinline__ void ld_global_32B(const void* p, uint4& lo, uint4& h
                : "memory");
 }
 
+// first pixel (w0, h0) and first image n0 of pixel tile m
+__device__ __forceinline__ void tile_first_pixel(const ConvTcParams& p, int m, int& w0, int& h0, int& n0) {
+  int q1, r1, q2, r2;
+  fd_divmod(m, p.fd_tiles_w, q1, r1);
+  fd_divmod(q1, p.fd_tiles_h, q2, r2);
+  w0 = r1 * p.BW; h0 = r2 * p.BH; n0 = q2 * p.BNI;
+}
+
 constexpr int kEpiThreads = 32 * LP_EPI_WARPS;
 constexpr int kConvThreads = 96 + kEpiThreads;
 constexpr int kFirstEpiWarp = 3;
@@ -251,15 +287,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint32_t sa = 0, pha = 0, sb = 0, phb = 0;
     uint8_t* b_ring = smem + p.b_ring_offset;
     for (int t = t_begin; t < t_end && !failed;) {
-      const int nt = t / p.m_tiles, m = t % p.m_tiles;
+      int nt, m;
+      fd_divmod(t, p.fd_m_tiles, nt, m);
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m + 1 < p.m_tiles) ? 2 : 1;
       int w0[2], h0[2], n0[2];
-      for (int a = 0; a < 2; ++a) {
-        const int mm = m + a;
-        w0[a] = (mm % p.tiles_w) * p.BW;
-        h0[a] = ((mm / p.tiles_w) % p.tiles_h) * p.BH;
-        n0[a] = (mm / (p.tiles_w * p.tiles_h)) * p.BNI;
-      }
+      for (int a = 0; a < 2; ++a) tile_first_pixel(p, m + a, w0[a], h0[a], n0[a]);
       const int col0 = nt * p.n_tile_cols;
       for (int c = 0; c < p.chunks && !failed; ++c) {
         if (!mbar_wait_warp(&tail->empty[sa], pha ^ 1, abort_flag)) { failed = true; break; }
@@ -294,7 +326,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int nk = p.KC >> 4;
     uint32_t slot = 0, slot_phase = 0;
     for (int t = t_begin; t < t_end && !failed;) {
-      const int m = t % p.m_tiles;
+      const int m = t - fd_div(t, p.fd_m_tiles) * p.m_tiles;
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m + 1 < p.m_tiles) ? 2 : 1;
       uint32_t sl[2];
       sl[0] = slot;
@@ -353,17 +385,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------- TMA producer (warp-uniform loop, elected issue) ----
     uint32_t s = 0, ph = 0;
     for (int t = t_begin; t < t_end && !failed;) {
-      const int ntg = t / p.m_tiles, m = t % p.m_tiles;
-      const int cls = ntg / p.n_tiles, nt = ntg % p.n_tiles;
+      int ntg, m, cls, nt;
+      fd_divmod(t, p.fd_m_tiles, ntg, m);
+      fd_divmod(ntg, p.fd_n_tiles, cls, nt);
       const int kiters = p.cls_ntaps[cls] * p.chunks;
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m + 1 < p.m_tiles) ? 2 : 1;
       int w0[2], h0[2], n0[2];
-      for (int a = 0; a < 2; ++a) {
-        const int mm = m + a;
-        w0[a] = (mm % p.tiles_w) * p.BW;
-        h0[a] = ((mm / p.tiles_w) % p.tiles_h) * p.BH;
-        n0[a] = (mm / (p.tiles_w * p.tiles_h)) * p.BNI;
-      }
+      for (int a = 0; a < 2; ++a) tile_first_pixel(p, m + a, w0[a], h0[a], n0[a]);
       const int col0 = nt * p.n_tile_cols;
       const uint32_t tx = p.tx_b + cnt * p.tx_a;
       for (int k0 = 0; k0 < kiters && !failed; k0 += p.ips) {
@@ -373,7 +401,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (elect_one()) {
           mbar_expect_tx(&tail->full[s], n_items * tx);
           for (int i = 0; i < n_items; ++i) {
-            const int tap = p.cls_tap0[cls] + (k0 + i) / p.chunks, c = (k0 + i) % p.chunks;
+            int tap, c;
+            fd_divmod(k0 + i, p.fd_chunks, tap, c);
+            tap += p.cls_tap0[cls];
             const int kb = p.tap_w[tap] * p.Cin;
             uint8_t* si = sa + i * p.item_bytes;
             tma_load_4d(si, &tmA, &tail->full[s], c * p.KC, w0[0] * p.in_step + p.tap_dw[tap],
@@ -400,8 +430,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int nk = p.KC >> 4;
     uint32_t slot = 0, slot_phase = 0;  // bit b of slot_phase: parity of the number of uses of slot b
     for (int t = t_begin; t < t_end && !failed;) {
-      const int m = t % p.m_tiles;
-      const int kiters = p.cls_ntaps[(t / p.m_tiles) / p.n_tiles] * p.chunks;
+      int ntg, m;
+      fd_divmod(t, p.fd_m_tiles, ntg, m);
+      const int kiters = p.cls_ntaps[fd_div(ntg, p.fd_n_tiles)] * p.chunks;
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m + 1 < p.m_tiles) ? 2 : 1;
       uint32_t sl[2];
       sl[0] = slot;
@@ -420,7 +451,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (elect_one()) {
           if (active) {
             for (int i = 0; i < n_items; ++i) {
-              const int nkc = (k0 + i) % p.chunks + 1 == p.chunks ? p.nk_last : nk;
+              const int kc = k0 + i - fd_div(k0 + i, p.fd_chunks) * p.chunks;
+              const int nkc = kc + 1 == p.chunks ? p.nk_last : nk;
               const uint64_t ad = smem_desc(p.desc_hi, a_addr + i * p.item_bytes + me * p.a_region_bytes);
               const uint64_t bd = smem_desc(p.desc_hi, a_addr + i * p.item_bytes + p.b_offset);
               for (int j = 0; j < nkc; ++j)  // +32 bytes (one K = 16 slice) per step, in 16-byte units
@@ -450,6 +482,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int row = q * 32 + lane;
     const int et = threadIdx.x - 32 * kFirstEpiWarp;
     const int rows_used = p.BW * p.BH * p.BNI;
+    // rows of a tile are ordered (w, h, image), or (w, image, h) in halo mode: this thread's place in every tile
+    const int row_w = row % p.BW;
+    const int row_h = p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH;
+    const int row_n = p.halo ? (row / p.BW) % p.BNI : row / (p.BW * p.BH);
     const int ngroups = p.n_tile_cols >> 5;
     uint8_t* stg = smem + p.stage_offset;
     // 64-byte swizzle of the staging rows, as the TMA unit applies it: 16-byte piece index ^= address bits 7..8
@@ -462,10 +498,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool stat_owner = p.stats != nullptr && sg < ngroups;
     float st_s0 = 0.f, st_s1 = 0.f, st_q0 = 0.f, st_q1 = 0.f;
     auto tile_origin = [&](int tile, int& col0, int& c1, int& c2, int& c3) {
-      const int nt = tile / p.m_tiles, m = tile % p.m_tiles;
-      const int w0 = (m % p.tiles_w) * p.BW;
-      const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
-      const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
+      int nt, m, w0, h0, n0;
+      fd_divmod(tile, p.fd_m_tiles, nt, m);
+      tile_first_pixel(p, m, w0, h0, n0);
       col0 = nt * p.n_tile_cols;
       c1 = w0;
       c2 = p.halo ? n0 : h0;      // box dimension order (C, W, image, H) in halo mode, (C, W, H, image) otherwise
@@ -496,18 +531,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (et == 0 && t_begin < t_end) load_addend_tile(t_begin);
     }
     for (int t = t_begin; t < t_end && !failed;) {
-      const int nt = t / p.m_tiles, m0 = t % p.m_tiles;
+      int nt, m0;
+      fd_divmod(t, p.fd_m_tiles, nt, m0);
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m0 + 1 < p.m_tiles) ? 2 : 1;
       for (int a = 0; a < cnt && !failed; ++a) {
         const int tile = t + a;
         const int m = m0 + a;
         const uint32_t buf = slot;
-        const int w0 = (m % p.tiles_w) * p.BW;
-        const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
-        const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
-        const int ow = w0 + row % p.BW;
-        const int oh = h0 + (p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH);
-        const int n = n0 + (p.halo ? (row / p.BW) % p.BNI : row / (p.BW * p.BH));
+        int w0, h0, n0;
+        tile_first_pixel(p, m, w0, h0, n0);
+        const int ow = w0 + row_w;
+        const int oh = h0 + row_h;
+        const int n = n0 + row_n;
         const bool valid = row < rows_used && ow < p.OWl && oh < p.OHl && n < p.Nimg;
         // One thread waits (bounded) for the accumulator, for the residual tile, and until the stores of
         // the previous tile have read the staging region; all epilogue threads then agree on the outcome.
@@ -598,7 +633,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         slot_phase ^= 1u << buf;
         slot = slot + 1 == (uint32_t)p.nslots ? 0 : slot + 1;
         const bool last_of_unit = a + 1 == cnt;
-        if (p.stats && last_of_unit && (t + cnt >= t_end || (t + cnt) / p.m_tiles != nt)) flush_stats(nt * p.n_tile_cols);
+        if (p.stats && last_of_unit && (t + cnt >= t_end || m0 + cnt >= p.m_tiles)) flush_stats(nt * p.n_tile_cols);
       }
       t += cnt;
     }
@@ -610,6 +645,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int row = q * 32 + lane;
     const int et = threadIdx.x - 32 * kFirstEpiWarp;
     const int rows_used = p.BW * p.BH * p.BNI;
+    // rows of a tile are ordered (w, h, image), or (w, image, h) in halo mode: this thread's place in every tile
+    const int row_w = row % p.BW;
+    const int row_h = p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH;
+    const int row_n = p.halo ? (row / p.BW) % p.BNI : row / (p.BW * p.BH);
     const int ngroups = (p.n_tile_cols + 31) >> 5;
     uint32_t slot = 0, slot_phase = 0;
     float sum_rr = 0.f, sum_kr = 0.f;    // local-loss sums of this thread (kLoss)
@@ -620,11 +659,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // waiting for DRAM.
     auto prefetch_rows = [&](const bf16* base, int tile) {
       if (tile >= t_end) return;
-      const int pntg = tile / p.m_tiles, pm = tile % p.m_tiles;
-      const int pcls = pntg / p.n_tiles, pnt = pntg % p.n_tiles;
-      const int pw = (pm % p.tiles_w) * p.BW + row % p.BW;
-      const int phh = ((pm / p.tiles_w) % p.tiles_h) * p.BH + (p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH);
-      const int pn = (pm / (p.tiles_w * p.tiles_h)) * p.BNI + (p.halo ? (row / p.BW) % p.BNI : row / (p.BW * p.BH));
+      int pntg, pm, pcls, pnt, pw, phh, pn;
+      fd_divmod(tile, p.fd_m_tiles, pntg, pm);
+      fd_divmod(pntg, p.fd_n_tiles, pcls, pnt);
+      tile_first_pixel(p, pm, pw, phh, pn);
+      pw += row_w; phh += row_h; pn += row_n;
       if (row >= rows_used || pw >= p.OWl || phh >= p.OHl || pn >= p.Nimg || grp) return;
       const long long pb =
           (((long long)pn * p.out_H + (phh * p.os + p.cls_oo_h[pcls])) * p.out_W + (pw * p.os + p.cls_oo_w[pcls])) * p.out_C +
@@ -641,10 +680,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     prefetch_addend(t_begin);
     int consts_nt = -1;                  // channel tile whose batch-norm constants are in shared memory (kBnBwd)
     for (int t = t_begin; t < t_end && !failed;) {
-      const int nt = t / p.m_tiles, m0 = t % p.m_tiles;     // nt counts (class, channel tile) pairs
-      const int cls = nt / p.n_tiles;
+      int nt, m0, cls, nt_c;                               // nt counts (class, channel tile) pairs
+      fd_divmod(t, p.fd_m_tiles, nt, m0);
+      fd_divmod(nt, p.fd_n_tiles, cls, nt_c);
       const int cnt = (p.mpair == 2 && t + 1 < t_end && m0 + 1 < p.m_tiles) ? 2 : 1;
-      const int col0 = (nt % p.n_tiles) * p.n_tile_cols;
+      const int col0 = nt_c * p.n_tile_cols;
       if constexpr (kBnBwd) {
         if (nt != consts_nt) {
           // scale, shift (the forward kernel's, for the ReLU mask), mean and rstd of this channel tile
@@ -668,13 +708,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         prefetch_addend(t + a + 1);
         const int m = m0 + a;
         const uint32_t buf = slot;
-        const int w0 = (m % p.tiles_w) * p.BW;
-        const int h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH;
-        const int n0 = (m / (p.tiles_w * p.tiles_h)) * p.BNI;
-        // rows of a tile: (w, h, image), or (w, image, h) in halo mode
-        const int ow = w0 + row % p.BW;
-        const int oh = h0 + (p.halo ? row / (p.BW * p.BNI) : (row / p.BW) % p.BH);
-        const int n = n0 + (p.halo ? (row / p.BW) % p.BNI : row / (p.BW * p.BH));
+        int w0, h0, n0;
+        tile_first_pixel(p, m, w0, h0, n0);
+        const int ow = w0 + row_w;
+        const int oh = h0 + row_h;
+        const int n = n0 + row_n;
         const bool valid = row < rows_used && ow < p.OWl && oh < p.OHl && n < p.Nimg;
         const long long obase =
             (((long long)n * p.out_H + (oh * p.os + p.cls_oo_h[cls])) * p.out_W + (ow * p.os + p.cls_oo_w[cls])) * p.out_C;
@@ -875,7 +913,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         slot = slot + 1 == (uint32_t)p.nslots ? 0 : slot + 1;
         // flush the column sums when the channel tile is about to change (or at the very end)
         const bool last_of_unit = a + 1 == cnt;
-        const bool flush = (kBnBwd || p.stats) && last_of_unit && (t + cnt >= t_end || (t + cnt) / p.m_tiles != nt);
+        const bool flush = (kBnBwd || p.stats) && last_of_unit && (t + cnt >= t_end || m0 + cnt >= p.m_tiles);
         if (flush) {
           asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
           for (int c = et; c < p.n_tile_cols; c += kEpiThreads) {

@@ -723,6 +723,9 @@ static int launch_conv_tc(lp_handle* h, const TcGemmSpec& s, int* dev_err, cudaS
     p.stage_offset = (uint32_t)(stages * p.stage_bytes);
     p.tail_offset = p.stage_offset + (uint32_t)stage_bytes;
   }
+  p.fd_tiles_w = tc::make_fastdiv(p.tiles_w); p.fd_tiles_h = tc::make_fastdiv(p.tiles_h);
+  p.fd_m_tiles = tc::make_fastdiv(p.m_tiles); p.fd_n_tiles = tc::make_fastdiv(p.n_tiles);
+  p.fd_chunks = tc::make_fastdiv(p.chunks);
   p.idesc = tc::instr_desc_bf16(128, p.n_tile_cols, 0, 0);
   p.desc_hi = tc::smem_desc_hi(16, 8 * row_bytes, tc::swizzle_code_for_row_bytes(row_bytes));
   p.out = s.out; p.addend = s.addend; p.stats = s.stats; p.err = dev_err;
