@@ -132,23 +132,41 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     // loops, one elected lane issues
     const bool do_a = warp == 0;
     uint32_t s = 0, ph = 0;
+    // Nothing in the loop divides: the pixel tile advances by one per iteration (its three coordinates are
+    // counted up), and a sub-box's channel offset and tap shift do not depend on the iteration (lane j keeps
+    // those of sub-box j and hands them to the issuing lane).  On layers of few channels the divide
+    // instructions of 8 to 16 copies per stage were what the producer spent its time on.
+    int tw, th, tn;
+    {
+      const int q1 = pt_begin / p.tiles_w;
+      tw = pt_begin - q1 * p.tiles_w;
+      tn = q1 / p.tiles_h;
+      th = q1 - tn * p.tiles_h;
+    }
+    int my_c0 = 0, my_dw = 0, my_dh = 0;
+    if (do_a && lane < p.rpt * cnt) {
+      int g = m_tile * p.rpt + lane;
+      if (g >= p.total_chunks) g = p.total_chunks - 1;  // padding rows of the last tile: any finite data
+      const int tap = g / p.cin_chunks;
+      my_c0 = (g - tap * p.cin_chunks) * p.sca;
+      const int r = tap / p.R;
+      my_dh = r - p.pad;
+      my_dw = tap - r * p.R - p.pad;
+    }
     for (int it = 0; it < n_iter; ++it) {
-      const int pt = pt_begin + it;
-      const int w0 = (pt % p.tiles_w) * p.BW;
-      const int h0 = ((pt / p.tiles_w) % p.tiles_h) * p.BH;
-      const int n0 = (pt / (p.tiles_w * p.tiles_h)) * p.BNI;
+      const int w0 = tw * p.BW, h0 = th * p.BH, n0 = tn * p.BNI;
+      if (++tw == p.tiles_w) { tw = 0; if (++th == p.tiles_h) { th = 0; ++tn; } }
       if (!mbar_wait_warp(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
       uint8_t* sa = smem + s * p.stage_bytes;
       const bool leader = elect_one();
-      if (leader && do_a) {
-        mbar_expect_tx(&tail->full[s], cnt * p.tx_a);
+      if (do_a) {
+        if (leader) mbar_expect_tx(&tail->full[s], cnt * p.tx_a);
         for (int j = 0; j < p.rpt * cnt; ++j) {
-          int g = m_tile * p.rpt + j;
-          if (g >= p.total_chunks) g = p.total_chunks - 1;  // padding rows of the last tile: any finite data
-          const int tap = g / p.cin_chunks, c0 = (g % p.cin_chunks) * p.sca;
-          const int r = tap / p.R, q = tap % p.R;
-          tma_load_4d(sa + j * p.a_sub_bytes, &tmX, &tail->full[s], c0, w0 * p.stride + q - p.pad,
-                      h0 * p.stride + r - p.pad, n0);
+          const int c0 = __shfl_sync(0xffffffffu, my_c0, j);
+          const int dw = __shfl_sync(0xffffffffu, my_dw, j);
+          const int dh = __shfl_sync(0xffffffffu, my_dh, j);
+          if (leader)
+            tma_load_4d(sa + j * p.a_sub_bytes, &tmX, &tail->full[s], c0, w0 * p.stride + dw, h0 * p.stride + dh, n0);
         }
       } else if (leader) {
         mbar_expect_tx(&tail->full[s], p.tx_b);
@@ -337,11 +355,16 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   if (warp == 0 || warp == 6) {
     const bool do_a = warp == 0;
     uint32_t s = 0, ph = 0;
+    int tw, th, tn;      // the pixel tile advances by one per iteration: its coordinates are counted up, not divided out
+    {
+      const int q1 = pt_begin / p.tiles_w;
+      tw = pt_begin - q1 * p.tiles_w;
+      tn = q1 / p.tiles_h;
+      th = q1 - tn * p.tiles_h;
+    }
     for (int it = 0; it < n_iter; ++it) {
-      const int pt = pt_begin + it;
-      const int w0 = (pt % p.tiles_w) * 8;
-      const int h0 = ((pt / p.tiles_w) % p.tiles_h) * p.BH;
-      const int n0 = (pt / (p.tiles_w * p.tiles_h)) * p.BNI;
+      const int w0 = tw * 8, h0 = th * p.BH, n0 = tn * p.BNI;
+      if (++tw == p.tiles_w) { tw = 0; if (++th == p.tiles_h) { th = 0; ++tn; } }
       if (!mbar_wait_warp(&tail->empty[s], ph ^ 1, abort_flag)) { failed = true; break; }
       uint8_t* sa = smem + s * p.stage_bytes;
       const bool leader = elect_one();
