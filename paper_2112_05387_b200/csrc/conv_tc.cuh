@@ -241,17 +241,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int t_begin = (int)(((long long)p.total_tiles * blockIdx.x) / gridDim.x);
   const int t_end = (int)(((long long)p.total_tiles * (blockIdx.x + 1)) / gridDim.x);
 
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(&tail->full[s], 1);
-      mbar_init(&tail->empty[s], 2);   // one arrival per MMA warp
-      mbar_init(&tail->full_b[s], 1);
-      mbar_init(&tail->empty_b[s], 2);
-    }
-    for (int b = 0; b < kMaxSlots; ++b) {
-      mbar_init(&tail->tmem_full[b], 1);
-      mbar_init(&tail->tmem_empty[b], kEpiThreads / 32);
-    }
+  // barrier set-up spread over the first threads (one thread doing all 57 took about a thousand cycles)
+  if (threadIdx.x < kMaxStages) {
+    const int s = threadIdx.x;
+    mbar_init(&tail->full[s], 1);
+    mbar_init(&tail->empty[s], 2);   // one arrival per MMA warp
+    mbar_init(&tail->full_b[s], 1);
+    mbar_init(&tail->empty_b[s], 2);
+    fence_barrier_init();
+  } else if (threadIdx.x >= 32 && threadIdx.x < 32 + kMaxSlots) {
+    const int b = threadIdx.x - 32;
+    mbar_init(&tail->tmem_full[b], 1);
+    mbar_init(&tail->tmem_empty[b], kEpiThreads / 32);
+    fence_barrier_init();
+  }
+  if (threadIdx.x == 64) {
     mbar_init(&tail->add_full, 1);
     tail->abort_flag = 0;
     fence_barrier_init();
