@@ -760,6 +760,7 @@ struct PackEntry {
   int cout, taps, cin;
   long long begin;       // first flat element index handled for this entry
   long long tile_begin;  // first 32x32 tile index of this entry (tiled kernel)
+  long long tile64_begin;  // first 64x64 tile index of this entry (sgd_pack_tiled64_kernel)
 };
 
 __global__ void pack_weights_kernel(const PackEntry* __restrict__ tab, int n_entries, long long total) {
@@ -882,6 +883,87 @@ __global__ void sgd_pack_tiled_kernel(const PackEntry* __restrict__ tab, int n_e
   for (int i = ty; i < 32; i += 8) {
     const int ci2 = ci0 + i, co = co0 + tx;
     if (co < e.cout && ci2 < e.cin) e.wt[((long long)ci2 * e.taps + t) * e.cout + co] = __float2bfloat16_rn(tile[tx][i]);
+  }
+}
+
+// The same update and copies on 64 (c_out) x 64 (c_in) tiles with 16-byte accesses: a thread holds four float4
+// pieces of the parameters and of the gradients (128 bytes of loads in flight instead of 32), the K-major copy
+// leaves in 8-byte pieces and the transposed one in 128-byte rows of 64 output channels.  Requires c_in % 4 == 0,
+// c_out % 2 == 0 and 16-byte aligned weight tensors inside the blobs (checked when the table is built).
+// blockDim = 256.
+__global__ void __launch_bounds__(256)
+sgd_pack_tiled64_kernel(const PackEntry* __restrict__ tab, int n_entries, float* __restrict__ p_base,
+                        const float* __restrict__ g_base, float* __restrict__ m_base, float lr, float momentum, float wd) {
+  __shared__ float tile[64][65];
+  const long long b = blockIdx.x;
+  int lo = 0, hi = n_entries - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (tab[mid].tile64_begin <= b) lo = mid; else hi = mid - 1;
+  }
+  const PackEntry e = tab[lo];
+  const long long base = e.w - p_base;
+  const int tiles_ci = (e.cin + 63) >> 6, tiles_co = (e.cout + 63) >> 6;
+  int r = (int)(b - e.tile64_begin);
+  const int ci0 = (r % tiles_ci) << 6;
+  r /= tiles_ci;
+  const int co0 = (r % tiles_co) << 6;
+  const int t = r / tiles_co;
+  const int tid = threadIdx.x;
+  const int cx = (tid & 15) << 2, ry = tid >> 4;   // four input channels of one of 16 rows per pass
+  const int ci = ci0 + cx;
+  float4 pv[4], gv[4], mv[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int co = co0 + ry + 16 * q;
+    pv[q] = gv[q] = mv[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (co < e.cout && ci < e.cin) {
+      const long long j = base + ((long long)co * e.taps + t) * e.cin + ci;
+      pv[q] = *reinterpret_cast<const float4*>(p_base + j);
+      gv[q] = *reinterpret_cast<const float4*>(g_base + j);
+      if (momentum != 0.f) mv[q] = *reinterpret_cast<const float4*>(m_base + j);
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int row = ry + 16 * q;
+    const int co = co0 + row;
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    if (co < e.cout && ci < e.cin) {
+      const long long j = ((long long)co * e.taps + t) * e.cin + ci;
+      const float pw[4] = {pv[q].x, pv[q].y, pv[q].z, pv[q].w};
+      const float gw[4] = {gv[q].x, gv[q].y, gv[q].z, gv[q].w};
+      const float mw[4] = {mv[q].x, mv[q].y, mv[q].z, mv[q].w};
+      float gi[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        gi[u] = gw[u] + wd * pw[u];
+        if (momentum != 0.f) gi[u] = momentum * mw[u] + gi[u];
+        v[u] = pw[u] - lr * gi[u];
+      }
+      if (momentum != 0.f) *reinterpret_cast<float4*>(m_base + base + j) = make_float4(gi[0], gi[1], gi[2], gi[3]);
+      *reinterpret_cast<float4*>(p_base + base + j) = make_float4(v[0], v[1], v[2], v[3]);
+      const __nv_bfloat162 lo2 = __floats2bfloat162_rn(v[0], v[1]), hi2 = __floats2bfloat162_rn(v[2], v[3]);
+      uint2 pk;
+      pk.x = *reinterpret_cast<const uint32_t*>(&lo2);
+      pk.y = *reinterpret_cast<const uint32_t*>(&hi2);
+      *reinterpret_cast<uint2*>(e.wf + j) = pk;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) tile[row][cx + u] = v[u];
+  }
+  if (!e.wt) return;
+  __syncthreads();
+  const int warp = tid >> 5, lane = tid & 31;
+  const int co = co0 + 2 * lane;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int cil = warp + 8 * i;
+    const int ci2 = ci0 + cil;
+    if (ci2 < e.cin && co < e.cout) {
+      const __nv_bfloat162 v2 = __floats2bfloat162_rn(tile[2 * lane][cil], tile[2 * lane + 1][cil]);
+      *reinterpret_cast<__nv_bfloat162*>(e.wt + ((long long)ci2 * e.taps + t) * e.cout + co) = v2;
+    }
   }
 }
 

@@ -91,6 +91,8 @@ struct ParamSet {
   SgdRange* dev_ranges = nullptr;
   long long pack_total = 0;
   long long pack_tiles = 0;
+  long long pack_tiles64 = 0;   // 64x64 tiles of the update kernel with 16-byte accesses
+  bool pack64_ok = true;        // every packed weight tensor starts on a 16-byte boundary of the blobs
   bool grads_fresh = false;
   bool momentum_used = false;
 };
@@ -1197,6 +1199,9 @@ struct Planner {
       pe.w = c.w; pe.wf = c.wf; pe.wt = c.wt; pe.cout = cout; pe.taps = R * R; pe.cin = cin;
       pe.begin = P.ps.pack_total;
       pe.tile_begin = P.ps.pack_tiles;
+      pe.tile64_begin = P.ps.pack_tiles64;
+      P.ps.pack_tiles64 += (long long)R * R * ((cin + 63) / 64) * ((cout + 63) / 64);
+      if (e->offset % 4 != 0 || cin % 4 != 0 || cout % 2 != 0) P.ps.pack64_ok = false;
       P.ps.pack_total += (long long)n;
       P.ps.pack_tiles += (long long)R * R * ((cin + 31) / 32) * ((cout + 31) / 32);
       P.ps.host_pack.push_back(pe);
@@ -1956,6 +1961,12 @@ static int sgd_update_inner(lp_handle* h, Plan& P, float lr, float momentum, flo
                                                                          momentum, weight_decay);
     h->launches++;
   }
+  const bool blobs16 = ((reinterpret_cast<uintptr_t>(P.ps.p) | reinterpret_cast<uintptr_t>(P.ps.g) |
+                         reinterpret_cast<uintptr_t>(P.ps.m)) & 15) == 0;
+  if (P.ps.pack64_ok && blobs16)
+    sgd_pack_tiled64_kernel<<<(unsigned)P.ps.pack_tiles64, 256, 0, st>>>(P.ps.dev_pack, (int)P.ps.host_pack.size(), P.ps.p,
+                                                                         P.ps.g, mom, lr, momentum, weight_decay);
+  else
   sgd_pack_tiled_kernel<<<(unsigned)P.ps.pack_tiles, dim3(32, 8), 0, st>>>(P.ps.dev_pack, (int)P.ps.host_pack.size(),
                                                                            P.ps.p, P.ps.g, mom, lr, momentum,
                                                                            weight_decay);
@@ -2721,7 +2732,7 @@ int lp_conv2d(int op, int dtype, int impl, int N, int H, int W, int Cin, int Cou
       // pack on the fly: one-entry table placed after the two weight copies is not available on the
       // device, so build it in pinned-free fashion: the table lives in the scratch tail
       PackEntry pe;
-      pe.w = c.w; pe.wf = c.wf; pe.wt = c.wt; pe.cout = Cout; pe.taps = R * R; pe.cin = Cin; pe.begin = 0; pe.tile_begin = 0;
+      pe.w = c.w; pe.wf = c.wf; pe.wt = c.wt; pe.cout = Cout; pe.taps = R * R; pe.cin = Cin; pe.begin = 0; pe.tile_begin = 0; pe.tile64_begin = 0;
       PackEntry* dpe = (PackEntry*)(sp + 256 + 2 * align_up(n * 2, 256));
       LP_CUDA_OK(cudaMemcpyAsync(dpe, &pe, sizeof(pe), cudaMemcpyHostToDevice, st));
       LP_CUDA_OK(cudaStreamSynchronize(st));
@@ -2814,7 +2825,7 @@ int lp_conv2d_fwd_noalloc(int N, int H, int W, int Cin, int Cout, int R, int str
   c.wf = (bf16*)(sp + 256);
   c.wt = nullptr;
   PackEntry pe;
-  pe.w = c.w; pe.wf = c.wf; pe.wt = nullptr; pe.cout = Cout; pe.taps = R * R; pe.cin = Cin; pe.begin = 0; pe.tile_begin = 0;
+  pe.w = c.w; pe.wf = c.wf; pe.wt = nullptr; pe.cout = Cout; pe.taps = R * R; pe.cin = Cin; pe.begin = 0; pe.tile_begin = 0; pe.tile64_begin = 0;
   PackEntry* dpe = (PackEntry*)(sp + 256 + align_up(n * 2, 256));
   LP_CUDA_OK(cudaMemsetAsync(dev_err, 0, 4, st));  // the only word that must start at zero
   LP_CUDA_OK(cudaMemcpyAsync(dpe, &pe, sizeof(pe), cudaMemcpyHostToDevice, st));
