@@ -629,6 +629,57 @@ __global__ void head_fwd_kernel(const int32_t* __restrict__ labels, const float*
   if (threadIdx.x == 0) atomicAdd(loss_acc, (double)(lse - lg[lab]) / (double)N);
 }
 
+// Heads of few classes (at most 128: the CIFAR-shaped networks) in one launch, one block of 256 threads per
+// sample: the average pool (kept in shared memory and written out for the backward pass), the logits (one warp
+// per class, the same summation order as head_logits_kernel) and, by the first warp, softmax, loss and dlogits.
+// Three dependent launches of a few microseconds of work each become one on the last module's chain.
+template <typename T>
+__global__ void __launch_bounds__(256)
+head_fused_kernel(const T* __restrict__ x, const float* __restrict__ Wt, const float* __restrict__ bias,
+                  const int32_t* __restrict__ labels, float* __restrict__ pooled, float* __restrict__ logits,
+                  float* __restrict__ dlogits, double* __restrict__ loss_acc, int N, int HW, int C, int classes) {
+  extern __shared__ float sh[];  // [C] pooled, then [classes] logits
+  float* sp = sh;
+  float* lg = sh + C;
+  const int n = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int c = threadIdx.x; c < C; c += blockDim.x) {
+    float acc = 0.f;
+    const T* p = x + (long long)n * HW * C + c;
+    for (int i = 0; i < HW; ++i) acc += to_f(p[(long long)i * C]);
+    const float v = acc / (float)HW;
+    pooled[(long long)n * C + c] = v;
+    sp[c] = v;
+  }
+  __syncthreads();
+  for (int j = warp; j < classes; j += (int)(blockDim.x >> 5)) {
+    const float* w = Wt + (long long)j * C;
+    float acc = 0.f;
+    for (int c = lane; c < C; c += 32) acc += w[c] * sp[c];
+    acc = warp_sum(acc);
+    if (lane == 0) {
+      const float v = acc + bias[j];
+      lg[j] = v;
+      logits[(long long)n * classes + j] = v;
+    }
+  }
+  __syncthreads();
+  if (warp != 0) return;
+  float mx = -INFINITY;
+  for (int j = lane; j < classes; j += 32) mx = fmaxf(mx, lg[j]);
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  float se = 0.f;
+  for (int j = lane; j < classes; j += 32) se += __expf(lg[j] - mx);
+  se = warp_sum(se);
+  const float lse = logf(se) + mx;
+  const int lab = labels[n];
+  for (int j = lane; j < classes; j += 32) {
+    const float pj = __expf(lg[j] - lse);
+    dlogits[(long long)n * classes + j] = (pj - (j == lab ? 1.f : 0.f)) / (float)N;
+  }
+  if (lane == 0) atomicAdd(loss_acc, (double)(lse - lg[lab]) / (double)N);
+}
+
 __global__ void ce_finalize_kernel(const double* __restrict__ acc, float* __restrict__ loss_out) {
   loss_out[0] = (float)acc[0];
   loss_out[1] = 0.f;

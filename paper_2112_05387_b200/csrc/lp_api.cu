@@ -1800,9 +1800,20 @@ static int run_op_t(lp_handle* h, Plan& P, const Op& op, const RunCtx& c) {
     }
     case OP_HEAD_FWD: {
       HeadDef& hd = P.head;
+      const int32_t* labels = c.labels ? c.labels : h->zero_labels;  // logits-only runs use label 0
+      if (hd.classes <= 128 && (size_t)(hd.C + hd.classes) * 4 <= 40 * 1024) {
+        head_fused_kernel<T><<<hd.N, 256, (size_t)(hd.C + hd.classes) * 4, st>>>(
+            (const T*)resolve(op.in, c), hd.W, hd.b, labels, hd.pooled, hd.logits, hd.dlogits, P.loss_acc, hd.N, hd.HW, hd.C,
+            hd.classes);
+        h->launches++;
+        if (c.loss_out) {
+          ce_finalize_kernel<<<1, 1, 0, st>>>(P.loss_acc, c.loss_out);
+          h->launches++;
+        }
+        break;
+      }
       avgpool_kernel<T><<<hd.N, 256, 0, st>>>((const T*)resolve(op.in, c), hd.pooled, hd.HW, hd.C);
       h->launches++;
-      const int32_t* labels = c.labels ? c.labels : h->zero_labels;  // logits-only runs use label 0
       head_logits_kernel<<<dim3((hd.classes + 3) / 4, (hd.N + 7) / 8), 128, 0, st>>>(hd.pooled, hd.W, hd.b, hd.logits, hd.N,
                                                                                      hd.C, hd.classes);
       head_fwd_kernel<<<hd.N, 128, (size_t)(hd.classes + 32) * 4, st>>>(labels, hd.logits, hd.dlogits, P.loss_acc, hd.N,
