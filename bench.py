@@ -561,7 +561,7 @@ def run_ours(args):
     peak_gbs = float(peaks.get("hbm_gbs", 6650.0))
     hbm_names = {"bn_apply": "bn_apply_kernel", "bn_bwd": "bn_bwd_reduce_kernel + bn_bwd_apply_kernel",
                  "bn_stats": "bn_stats_kernel", "out_loss": "module_out_loss_kernel",
-                 "update": "sgd_pack_tiled_kernel + sgd_ranges_kernel + kappa_update_kernel"}
+                 "update": "sgd_pack_tiled64_kernel + sgd_ranges_kernel + kappa_update_kernel"}
     roofline_hbm = []
     for op, kernel in hbm_names.items():
         rs = [r for r in tl_recs if r["op"] == op and r["bytes"] > 0]
