@@ -874,73 +874,13 @@ __global__ void pack_weights_tiled_kernel(const PackEntry* __restrict__ tab, int
 }
 
 // The update and the weight copies in one pass over the packed convolution weights:
-//   w <- w - lr*(g + wd*w [momentum])   then the two bf16 copies of the new w, as above.
-// `p_base` / `g_base` / `m_base` are the parameter, gradient and momentum blobs the entries point
-// into (m_base may be null when momentum is 0).
-__global__ void sgd_pack_tiled_kernel(const PackEntry* __restrict__ tab, int n_entries, float* __restrict__ p_base,
-                                      const float* __restrict__ g_base, float* __restrict__ m_base, float lr,
-                                      float momentum, float wd) {
-  __shared__ float tile[32][33];
-  const long long b = blockIdx.x;
-  int lo = 0, hi = n_entries - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (tab[mid].tile_begin <= b) lo = mid; else hi = mid - 1;
-  }
-  const PackEntry e = tab[lo];
-  const long long base = e.w - p_base;
-  const int tiles_ci = (e.cin + 31) >> 5, tiles_co = (e.cout + 31) >> 5;
-  int r = (int)(b - e.tile_begin);
-  const int ci0 = (r % tiles_ci) << 5;
-  r /= tiles_ci;
-  const int co0 = (r % tiles_co) << 5;
-  const int t = r / tiles_co;
-  const int tx = threadIdx.x, ty = threadIdx.y;
-  // all loads of the thread's four elements first (independent requests in flight), then the arithmetic and stores
-  float pv[4], gv[4], mv[4];
-  const int ci = ci0 + tx;
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int co = co0 + ty + 8 * q;
-    pv[q] = gv[q] = mv[q] = 0.f;
-    if (co < e.cout && ci < e.cin) {
-      const long long j = base + ((long long)co * e.taps + t) * e.cin + ci;
-      pv[q] = p_base[j];
-      gv[q] = g_base[j];
-      if (momentum != 0.f) mv[q] = m_base[j];
-    }
-  }
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int i = ty + 8 * q;
-    const int co = co0 + i;
-    float v = 0.f;
-    if (co < e.cout && ci < e.cin) {
-      const long long j = ((long long)co * e.taps + t) * e.cin + ci;
-      v = pv[q];
-      float gi = gv[q] + wd * v;
-      if (momentum != 0.f) {
-        gi = momentum * mv[q] + gi;
-        m_base[base + j] = gi;
-      }
-      v -= lr * gi;
-      p_base[base + j] = v;
-      e.wf[j] = __float2bfloat16_rn(v);
-    }
-    tile[i][tx] = v;
-  }
-  if (!e.wt) return;
-  __syncthreads();
-  for (int i = ty; i < 32; i += 8) {
-    const int ci2 = ci0 + i, co = co0 + tx;
-    if (co < e.cout && ci2 < e.cin) e.wt[((long long)ci2 * e.taps + t) * e.cout + co] = __float2bfloat16_rn(tile[tx][i]);
-  }
-}
-
-// The same update and copies on 64 (c_out) x 64 (c_in) tiles with 16-byte accesses: a thread holds four float4
-// pieces of the parameters and of the gradients (128 bytes of loads in flight instead of 32), the K-major copy
-// leaves in 8-byte pieces and the transposed one in 128-byte rows of 64 output channels.  Requires c_in % 4 == 0,
-// c_out % 2 == 0 and 16-byte aligned weight tensors inside the blobs (checked when the table is built).
+//   w <- w - lr*(g + wd*w [momentum])   then the two bf16 copies of the new w, as above,
+// on 64 (c_out) x 64 (c_in) tiles of one tap with 16-byte accesses: a thread holds four float4 pieces of the
+// parameters and of the gradients (128 bytes of loads in flight), the K-major copy leaves in 8-byte pieces and
+// the transposed one, through shared memory, in 128-byte rows of 64 output channels.  `p_base` / `g_base` /
+// `m_base` are the parameter, gradient and momentum blobs the entries point into (m_base may be null when
+// momentum is 0).  Requires c_in % 4 == 0, c_out % 2 == 0 and 16-byte aligned weight tensors inside the blobs
+// (checked when the table is built; otherwise the plain update and pack_weights_tiled_kernel run instead).
 // blockDim = 256.
 __global__ void __launch_bounds__(256)
 sgd_pack_tiled64_kernel(const PackEntry* __restrict__ tab, int n_entries, float* __restrict__ p_base,

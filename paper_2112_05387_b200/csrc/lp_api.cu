@@ -1967,20 +1967,28 @@ static int sgd_update_inner(lp_handle* h, Plan& P, float lr, float momentum, flo
     LP_CUDA_OK(cudaGetLastError());
     return LP_OK;
   }
+  const bool blobs16 = ((reinterpret_cast<uintptr_t>(P.ps.p) | reinterpret_cast<uintptr_t>(P.ps.g) |
+                         reinterpret_cast<uintptr_t>(P.ps.m)) & 15) == 0;
+  if (!(P.ps.pack64_ok && blobs16)) {
+    // a weight tensor off the 16-byte grid of the blobs: the plain update over everything, then the copies
+    sgd_kernel<<<grid_for((long long)P.ps.n, 256, cur_dev().sm_count, 8), 256, 0, st>>>(P.ps.p, P.ps.g, P.ps.m,
+                                                                                    (long long)P.ps.n, lr, momentum,
+                                                                                    weight_decay);
+    h->launches++;
+    LP_CUDA_OK(cudaGetLastError());
+    pack_weights_tiled_kernel<<<(unsigned)P.ps.pack_tiles, dim3(32, 8), 0, st>>>(P.ps.dev_pack,
+                                                                                (int)P.ps.host_pack.size());
+    h->launches++;
+    LP_CUDA_OK(cudaGetLastError());
+    return LP_OK;
+  }
   if (!P.ps.host_ranges.empty()) {
     sgd_ranges_kernel<<<(unsigned)P.ps.host_ranges.size(), 256, 0, st>>>(P.ps.dev_ranges, P.ps.p, P.ps.g, mom, lr,
                                                                          momentum, weight_decay);
     h->launches++;
   }
-  const bool blobs16 = ((reinterpret_cast<uintptr_t>(P.ps.p) | reinterpret_cast<uintptr_t>(P.ps.g) |
-                         reinterpret_cast<uintptr_t>(P.ps.m)) & 15) == 0;
-  if (P.ps.pack64_ok && blobs16)
-    sgd_pack_tiled64_kernel<<<(unsigned)P.ps.pack_tiles64, 256, 0, st>>>(P.ps.dev_pack, (int)P.ps.host_pack.size(), P.ps.p,
-                                                                         P.ps.g, mom, lr, momentum, weight_decay);
-  else
-  sgd_pack_tiled_kernel<<<(unsigned)P.ps.pack_tiles, dim3(32, 8), 0, st>>>(P.ps.dev_pack, (int)P.ps.host_pack.size(),
-                                                                           P.ps.p, P.ps.g, mom, lr, momentum,
-                                                                           weight_decay);
+  sgd_pack_tiled64_kernel<<<(unsigned)P.ps.pack_tiles64, 256, 0, st>>>(P.ps.dev_pack, (int)P.ps.host_pack.size(), P.ps.p,
+                                                                       P.ps.g, mom, lr, momentum, weight_decay);
   h->launches++;
   LP_CUDA_OK(cudaGetLastError());
   return LP_OK;
